@@ -1,0 +1,719 @@
+/*
+ * zc_oracle.c — TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded CPU statement of the lossless exponent /
+ * sign+mantissa Huffman codec of "Lossless Compression of Neural Network
+ * Components: Weights, Checkpoints, and K/V Caches in Low-Precision Formats"
+ * (Heilper & Singer, 2025).  It exists so that the CUDA library can be
+ * compared with something that is obviously correct.  It shares no code,
+ * header, table or constant generator with the CUDA library and must never be
+ * called from the product path: only the tests, the smoke check and the
+ * benchmark's CPU-baseline leg may load it.
+ *
+ * What the paper fixes, and where each function follows it:
+ *   - Field split (Sec. 3.1 BF16: 1 sign, 8 exponent, 7 mantissa bits;
+ *     Sec. 3.2 FP8 E4M3: 1 sign, 4 exponent, 3 mantissa bits; Sec. 3.4 / 4.4
+ *     FP4: "2 bits from each of 4 consecutive values" form a byte):
+ *     zo_split / zo_merge.
+ *   - Byte grouping of two FP8 elements' exponents and two elements'
+ *     sign+mantissa (Fig. 7 caption): zo_split.
+ *   - One Huffman code per stream per tensor (Sec. 3.1, 3.2, 4.1 "per layer
+ *     file, using standard Huffman encoding"): zo_code_lengths,
+ *     zo_canonical_codes.
+ *   - Mantissa "evaluated for entropy; Huffman if compressible, otherwise
+ *     stored uncompressed" (Sec. 3.1, 4.3): zo_choose_mode.
+ *   - "Fixed-size chunks with lightweight metadata per block, designed for
+ *     random access and parallel decoding" (Sec. 3.1, Sec. 4): zo_compress,
+ *     zo_decompress, zo_decompress_chunk.
+ *
+ * What the paper leaves open (bit positions inside a grouped byte, the length
+ * limit, every tie-break, the byte layout of the container, the RAW/HUFF
+ * threshold) is a reading chosen by this build; those readings are "parity
+ * unpinned" by the paper and pinned only by theory-level tests: round trip,
+ * Kraft equality, brute-force optimal cost, payload bits = sum freq*len,
+ * entropy bounds, format bit-pattern values and hand-worked bitstreams.
+ *
+ * Readings used here:
+ *   R1  Standard bit layouts.  BF16 little-endian u16: sign 15, exponent 14..7,
+ *       mantissa 6..0.  FP8 E4M3: sign 7, exponent 6..3, mantissa 2..0.
+ *       FP4 E2M1 packed two per byte, element 2i in bits 3..0 and 2i+1 in
+ *       bits 7..4: sign 3, exponent 2..1, mantissa 0.
+ *   R2  Every stream is a stream of 8-bit symbols; symbol k holds the fields
+ *       of elements G*k .. G*k+G-1 (G = 1, 2, 4), element G*k+i in bits
+ *       [w*i, w*i+w), w = 8/G.  Missing tail fields are zero.  Stream 0 is the
+ *       exponent field e, stream 1 is (sign << mantissa_bits) | mantissa.
+ *   R3  Code lengths: optimal prefix code with maximum length 12, obtained by
+ *       the package-merge construction on leaves sorted by (count, symbol);
+ *       at equal weight a leaf precedes a package.  One active symbol gets
+ *       length 1.
+ *   R4  Canonical codes in (length, symbol) order, emitted most significant
+ *       bit first; bit k of a chunk payload is bit 31-(k%32) of little-endian
+ *       32-bit word k/32.
+ *   R5  A chunk covers chunk_bytes of element bytes = chunk_bytes/2 symbols of
+ *       each stream, cut into 32 equal subchunks that are concatenated bit by
+ *       bit; each chunk payload starts on a 16-byte boundary.
+ *   R6  AUTO policy: a stream is Huffman-coded iff
+ *       64 * sum(count*len) <= 63 * 8 * n_syms, otherwise stored raw.
+ *
+ * Container layout (little-endian, every section 16-byte aligned):
+ *   header 128 B:
+ *     0  u32 magic 'Z','C','1','0'   4 u16 version=1   6 u8 format  7 u8 n_streams=2
+ *     8  u64 n_elems                16 u32 chunk_bytes 20 u32 n_chunks
+ *     24 u8 L_max=12  25 u8 G  26 u8 subchunks=32  27 u8 0  28 u32 0
+ *     32 u64 total_bytes  40 u64 payload_off  48 u64 payload_bytes  56 u64 0
+ *     64 + 32*s: u8 mode (0 RAW, 1 HUFF), u8[7] 0, u64 n_syms, u64 payload_bits,
+ *                u64 section_off
+ *   for each HUFF stream, in stream order, its table section:
+ *     u8  code_len[256]
+ *     u32 chunk_off16[n_chunks]        (padded with zeros to a multiple of 16 B)
+ *     u32 sub_end[n_chunks][32]        end bit of each subchunk inside its chunk
+ *   for each RAW stream, in stream order: its n_syms symbol bytes, zero padded
+ *     to a multiple of 16 B
+ *   payload area at payload_off: for chunk 0,1,..: for each HUFF stream in
+ *     stream order: that chunk's bits, zero padded to a multiple of 16 B.
+ *     chunk_off16[c] is the offset of that piece from payload_off in units
+ *     of 16 B.  payload_bytes counts the area without the guard.
+ *   16 zero guard bytes if at least one stream is HUFF.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3 };
+enum { ZO_RAW = 0, ZO_HUFF = 1 };
+enum { ZO_POLICY_AUTO = 0, ZO_POLICY_HUFF_ALL = 1, ZO_POLICY_RAW_ALL = 2 };
+enum { ZO_LMAX = 12, ZO_SUBS = 32, ZO_HEADER = 128 };
+
+/* ------------------------------------------------------------------ */
+/* Element values (used only to pin the bit layouts of reading R1)     */
+/* ------------------------------------------------------------------ */
+
+/* BF16: value = (-1)^s * 2^(e-127) * (1 + m/128); e = 0 subnormal, e = 255 inf/nan (Sec. 3.1). */
+double zo_bf16_value(uint16_t x)
+{
+    int s = x >> 15, e = (x >> 7) & 0xFF, m = x & 0x7F;
+    double v;
+    if (e == 255) v = m ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)m / 128.0, -126);
+    else v = ldexp(1.0 + (double)m / 128.0, e - 127);
+    return s ? -v : v;
+}
+
+/* FP8 E4M3 (finite-only variant): bias 7, no infinities, S.1111.111 is NaN (Sec. 3.2). */
+double zo_e4m3_value(uint8_t x)
+{
+    int s = x >> 7, e = (x >> 3) & 0xF, m = x & 7;
+    double v;
+    if (e == 15 && m == 7) v = NAN;
+    else if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* FP4 E2M1: bias 1, values 0, .5, 1, 1.5, 2, 3, 4, 6 (Sec. 3.4). */
+double zo_e2m1_value(uint8_t nib)
+{
+    int s = (nib >> 3) & 1, e = (nib >> 1) & 3, m = nib & 1;
+    double v;
+    if (e == 0) v = 0.5 * m;
+    else v = ldexp(1.0 + 0.5 * m, e - 1);
+    return s ? -v : v;
+}
+
+/* ------------------------------------------------------------------ */
+/* Geometry                                                            */
+/* ------------------------------------------------------------------ */
+
+int zo_group(int fmt)
+{
+    switch (fmt) {
+    case ZO_BF16: return 1;
+    case ZO_FP8_E4M3: return 2;
+    case ZO_FP4_E2M1: return 4;
+    default: return 0;
+    }
+}
+
+uint64_t zo_n_syms(int fmt, uint64_t n_elems)
+{
+    uint64_t g = (uint64_t)zo_group(fmt);
+    return g ? (n_elems + g - 1) / g : 0;
+}
+
+uint64_t zo_input_bytes(int fmt, uint64_t n_elems)
+{
+    switch (fmt) {
+    case ZO_BF16: return 2 * n_elems;
+    case ZO_FP8_E4M3: return n_elems;
+    case ZO_FP4_E2M1: return (n_elems + 1) / 2;
+    default: return 0;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Field split and merge (readings R1, R2)                             */
+/* ------------------------------------------------------------------ */
+
+/* Fetch the exponent field and the sign+mantissa field of element i. */
+static void element_fields(int fmt, const uint8_t *in, uint64_t i, unsigned *e, unsigned *sm)
+{
+    if (fmt == ZO_BF16) {
+        unsigned x = (unsigned)in[2 * i] | ((unsigned)in[2 * i + 1] << 8);
+        *e = (x >> 7) & 0xFF;
+        *sm = ((x >> 15) << 7) | (x & 0x7F);
+    } else if (fmt == ZO_FP8_E4M3) {
+        unsigned x = in[i];
+        *e = (x >> 3) & 0xF;
+        *sm = ((x >> 7) << 3) | (x & 7);
+    } else {
+        unsigned b = in[i / 2];
+        unsigned x = (i & 1) ? (b >> 4) : (b & 0xF);
+        *e = (x >> 1) & 3;
+        *sm = ((x >> 3) << 1) | (x & 1);
+    }
+}
+
+/* s0 and s1 receive zo_n_syms() bytes each. */
+void zo_split(int fmt, const uint8_t *in, uint64_t n_elems, uint8_t *s0, uint8_t *s1)
+{
+    int g = zo_group(fmt);
+    int w = 8 / g;
+    uint64_t ns = zo_n_syms(fmt, n_elems);
+    for (uint64_t k = 0; k < ns; ++k) {
+        unsigned a = 0, b = 0;
+        for (int i = 0; i < g; ++i) {
+            uint64_t el = (uint64_t)g * k + (uint64_t)i;
+            if (el < n_elems) {
+                unsigned e, sm;
+                element_fields(fmt, in, el, &e, &sm);
+                a |= e << (w * i);
+                b |= sm << (w * i);
+            }
+        }
+        s0[k] = (uint8_t)a;
+        s1[k] = (uint8_t)b;
+    }
+}
+
+/* Inverse of zo_split: writes zo_input_bytes() bytes. */
+void zo_merge(int fmt, const uint8_t *s0, const uint8_t *s1, uint64_t n_elems, uint8_t *out)
+{
+    int g = zo_group(fmt);
+    int w = 8 / g;
+    unsigned fmask = (1u << w) - 1u;
+    if (fmt == ZO_FP4_E2M1) memset(out, 0, (size_t)zo_input_bytes(fmt, n_elems));
+    for (uint64_t el = 0; el < n_elems; ++el) {
+        uint64_t k = el / (uint64_t)g;
+        int i = (int)(el % (uint64_t)g);
+        unsigned e = (s0[k] >> (w * i)) & fmask;
+        unsigned sm = (s1[k] >> (w * i)) & fmask;
+        if (fmt == ZO_BF16) {
+            unsigned x = ((sm >> 7) << 15) | (e << 7) | (sm & 0x7F);
+            out[2 * el] = (uint8_t)(x & 0xFF);
+            out[2 * el + 1] = (uint8_t)(x >> 8);
+        } else if (fmt == ZO_FP8_E4M3) {
+            out[el] = (uint8_t)(((sm >> 3) << 7) | (e << 3) | (sm & 7));
+        } else {
+            unsigned x = ((sm >> 1) << 3) | (e << 1) | (sm & 1);
+            out[el / 2] |= (uint8_t)((el & 1) ? (x << 4) : x);
+        }
+    }
+}
+
+void zo_histogram(const uint8_t *syms, uint64_t n, uint64_t hist[256])
+{
+    memset(hist, 0, 256 * sizeof(uint64_t));
+    for (uint64_t i = 0; i < n; ++i) hist[syms[i]]++;
+}
+
+/* ------------------------------------------------------------------ */
+/* Length-limited optimal code lengths (reading R3)                    */
+/* ------------------------------------------------------------------ */
+
+/* An item of the package-merge lists: a weight and the multiset of leaves it
+ * contains, stored as one counter per active leaf. */
+typedef struct {
+    uint64_t w;
+    int is_leaf;
+    uint16_t cnt[256];
+} zo_item;
+
+/* Returns 0 on success.  len[v] = 0 for symbols that never occur.
+ * L is the maximum code length; needs 2^L >= number of active symbols. */
+int zo_code_lengths(const uint64_t hist[256], int L, uint8_t len[256])
+{
+    int sym[256];
+    int n = 0;
+    memset(len, 0, 256);
+    for (int v = 0; v < 256; ++v)
+        if (hist[v]) sym[n++] = v;
+    if (n == 0) return 0;
+    if (n == 1) { len[sym[0]] = 1; return 0; }
+    if (L < 1 || L > 31 || (1u << L) < (unsigned)n) return -1;
+
+    /* leaves sorted ascending by (count, symbol): insertion sort, stable */
+    for (int i = 1; i < n; ++i) {
+        int s = sym[i], j = i - 1;
+        while (j >= 0 && (hist[sym[j]] > hist[s] || (hist[sym[j]] == hist[s] && sym[j] > s))) {
+            sym[j + 1] = sym[j];
+            --j;
+        }
+        sym[j + 1] = s;
+    }
+
+    zo_item *leaves = (zo_item *)calloc((size_t)n, sizeof(zo_item));
+    zo_item *cur = (zo_item *)calloc((size_t)2 * n, sizeof(zo_item));
+    zo_item *pk = (zo_item *)calloc((size_t)n, sizeof(zo_item));
+    zo_item *nxt = (zo_item *)calloc((size_t)2 * n, sizeof(zo_item));
+    if (!leaves || !cur || !pk || !nxt) { free(leaves); free(cur); free(pk); free(nxt); return -2; }
+    for (int i = 0; i < n; ++i) {
+        leaves[i].w = hist[sym[i]];
+        leaves[i].is_leaf = 1;
+        leaves[i].cnt[i] = 1;
+    }
+    int ncur = n;
+    for (int i = 0; i < n; ++i) cur[i] = leaves[i];
+
+    for (int round = 0; round < L - 1; ++round) {
+        /* package consecutive pairs; an odd last item is dropped */
+        int np = ncur / 2;
+        for (int k = 0; k < np; ++k) {
+            pk[k].w = cur[2 * k].w + cur[2 * k + 1].w;
+            pk[k].is_leaf = 0;
+            for (int i = 0; i < n; ++i) pk[k].cnt[i] = (uint16_t)(cur[2 * k].cnt[i] + cur[2 * k + 1].cnt[i]);
+        }
+        /* merge leaves and packages by weight; at equal weight the leaf goes first */
+        int a = 0, b = 0, m = 0;
+        while (a < n || b < np) {
+            if (b >= np || (a < n && leaves[a].w <= pk[b].w)) nxt[m++] = leaves[a++];
+            else nxt[m++] = pk[b++];
+        }
+        zo_item *t = cur; cur = nxt; nxt = t;
+        ncur = m;
+    }
+
+    /* the first 2n-2 items of the last list; a symbol's length is how often it occurs in them */
+    for (int k = 0; k < 2 * n - 2; ++k)
+        for (int i = 0; i < n; ++i) len[sym[i]] = (uint8_t)(len[sym[i]] + cur[k].cnt[i]);
+
+    free(leaves); free(cur); free(pk); free(nxt);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Canonical codes (reading R4)                                        */
+/* ------------------------------------------------------------------ */
+
+/* Symbols in (length, symbol) order receive consecutive code values; the
+ * value is shifted left whenever the length grows.  code[v] holds the code
+ * right-aligned in len[v] bits; unused symbols get 0. */
+void zo_canonical_codes(const uint8_t len[256], uint32_t code[256])
+{
+    uint32_t next = 0;
+    int prev = 0;
+    memset(code, 0, 256 * sizeof(uint32_t));
+    for (int l = 1; l <= 31; ++l) {
+        for (int v = 0; v < 256; ++v) {
+            if (len[v] != l) continue;
+            if (prev) next = (next + 1) << (l - prev);
+            code[v] = next;
+            prev = l;
+        }
+    }
+}
+
+/* Sum of count*len. */
+uint64_t zo_payload_bits(const uint64_t hist[256], const uint8_t len[256])
+{
+    uint64_t t = 0;
+    for (int v = 0; v < 256; ++v) t += hist[v] * (uint64_t)len[v];
+    return t;
+}
+
+/* RAW/HUFF decision of one stream (reading R6; Sec. 3.1 "if compressibility is
+ * high ... otherwise stored uncompressed"). */
+int zo_choose_mode(const uint64_t hist[256], const uint8_t len[256], int policy)
+{
+    uint64_t n = 0;
+    for (int v = 0; v < 256; ++v) n += hist[v];
+    if (n == 0) return ZO_RAW;
+    if (policy == ZO_POLICY_RAW_ALL) return ZO_RAW;
+    if (policy == ZO_POLICY_HUFF_ALL) return ZO_HUFF;
+    return (64 * zo_payload_bits(hist, len) <= 63 * 8 * n) ? ZO_HUFF : ZO_RAW;
+}
+
+/* ------------------------------------------------------------------ */
+/* Container writer                                                    */
+/* ------------------------------------------------------------------ */
+
+static uint64_t round16(uint64_t x) { return (x + 15) & ~(uint64_t)15; }
+
+static void put16(uint8_t *p, unsigned v) { p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); }
+static void put32(uint8_t *p, uint32_t v) { for (int i = 0; i < 4; ++i) p[i] = (uint8_t)(v >> (8 * i)); }
+static void put64(uint8_t *p, uint64_t v) { for (int i = 0; i < 8; ++i) p[i] = (uint8_t)(v >> (8 * i)); }
+static uint32_t get16(const uint8_t *p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8); }
+static uint32_t get32(const uint8_t *p) { uint32_t v = 0; for (int i = 0; i < 4; ++i) v |= (uint32_t)p[i] << (8 * i); return v; }
+static uint64_t get64(const uint8_t *p) { uint64_t v = 0; for (int i = 0; i < 8; ++i) v |= (uint64_t)p[i] << (8 * i); return v; }
+
+static uint32_t n_chunks_of(uint64_t n_syms, uint32_t chunk_bytes)
+{
+    uint64_t cs = chunk_bytes / 2;
+    return (uint32_t)((n_syms + cs - 1) / cs);
+}
+
+static uint64_t table_section_bytes(uint32_t n_chunks)
+{
+    return 256 + round16(4ull * n_chunks) + 128ull * n_chunks;
+}
+
+static int valid_chunk_bytes(uint32_t cb) { return cb >= 1024 && cb <= 262144 && cb % 1024 == 0; }
+
+/* Largest container any code with lengths <= 12 can produce. */
+uint64_t zo_container_bound(int fmt, uint64_t n_elems, uint32_t chunk_bytes)
+{
+    if (!zo_group(fmt) || !valid_chunk_bytes(chunk_bytes)) return 0;
+    uint64_t ns = zo_n_syms(fmt, n_elems);
+    uint32_t nc = n_chunks_of(ns, chunk_bytes);
+    uint64_t cs = chunk_bytes / 2;
+    uint64_t worst_chunk = round16((cs * ZO_LMAX + 7) / 8);
+    uint64_t huff = table_section_bytes(nc) + (uint64_t)nc * worst_chunk;
+    uint64_t raw = round16(ns);
+    return ZO_HEADER + 2 * (huff > raw ? huff : raw) + 16;
+}
+
+/* Set bit number pos (counted from the start of the chunk piece) to 1. */
+static void set_bit(uint8_t *piece, uint64_t pos)
+{
+    uint64_t word = pos / 32;
+    unsigned in_word = 31u - (unsigned)(pos % 32);      /* MSB of the 32-bit word first */
+    piece[4 * word + in_word / 8] |= (uint8_t)(1u << (in_word % 8));   /* little-endian word */
+}
+
+/* Compress one tensor.  mode[s] and len[s][256] describe the code of stream s
+ * (len ignored for RAW).  Returns the container size, or a negative error:
+ * -1 bad argument, -2 out of memory, -3 capacity too small, -4 a symbol has no code. */
+int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk_bytes,
+                    const int mode[2], const uint8_t len[2][256], uint8_t *out, uint64_t cap)
+{
+    int g = zo_group(fmt);
+    if (!g || !valid_chunk_bytes(chunk_bytes)) return -1;
+    if (fmt == ZO_FP4_E2M1 && (n_elems & 1)) return -1;
+    uint64_t ns = zo_n_syms(fmt, n_elems);
+    uint32_t nc = n_chunks_of(ns, chunk_bytes);
+    uint64_t cs = chunk_bytes / 2, sub = cs / ZO_SUBS;
+
+    uint8_t *st[2];
+    st[0] = (uint8_t *)malloc((size_t)ns + 1);
+    st[1] = (uint8_t *)malloc((size_t)ns + 1);
+    if (!st[0] || !st[1]) { free(st[0]); free(st[1]); return -2; }
+    zo_split(fmt, in, n_elems, st[0], st[1]);
+
+    uint32_t code[2][256];
+    for (int s = 0; s < 2; ++s) {
+        if (mode[s] == ZO_HUFF) {
+            zo_canonical_codes(len[s], code[s]);
+            for (uint64_t k = 0; k < ns; ++k)
+                if (len[s][st[s][k]] == 0 || len[s][st[s][k]] > ZO_LMAX) { free(st[0]); free(st[1]); return -4; }
+        }
+    }
+
+    /* section offsets */
+    uint64_t off = ZO_HEADER, sec[2] = {0, 0};
+    for (int s = 0; s < 2; ++s) if (mode[s] == ZO_HUFF) { sec[s] = off; off += table_section_bytes(nc); }
+    for (int s = 0; s < 2; ++s) if (mode[s] == ZO_RAW) { sec[s] = off; off += round16(ns); }
+    uint64_t payload_off = off;
+    int any_huff = (mode[0] == ZO_HUFF) || (mode[1] == ZO_HUFF);
+
+    if (cap < payload_off) { free(st[0]); free(st[1]); return -3; }
+    memset(out, 0, (size_t)payload_off);
+
+    for (int s = 0; s < 2; ++s) {
+        if (mode[s] == ZO_RAW) memcpy(out + sec[s], st[s], (size_t)ns);
+        else memcpy(out + sec[s], len[s], 256);
+    }
+
+    uint64_t pbits[2] = {8 * ns, 8 * ns};
+    if (mode[0] == ZO_HUFF) pbits[0] = 0;
+    if (mode[1] == ZO_HUFF) pbits[1] = 0;
+
+    uint64_t pos16 = 0;                                 /* running payload offset, 16-byte units */
+    for (uint32_t c = 0; c < nc && any_huff; ++c) {
+        uint64_t c_lo = (uint64_t)c * cs;
+        uint64_t c_hi = c_lo + cs < ns ? c_lo + cs : ns;
+        for (int s = 0; s < 2; ++s) {
+            if (mode[s] != ZO_HUFF) continue;
+            uint8_t *chunk_off = out + sec[s] + 256;
+            uint8_t *sub_end = out + sec[s] + 256 + round16(4ull * nc);
+            /* bits of this chunk */
+            uint64_t bits = 0;
+            for (uint64_t k = c_lo; k < c_hi; ++k) bits += len[s][st[s][k]];
+            uint64_t piece_bytes = round16((bits + 7) / 8);
+            uint64_t piece_off = payload_off + 16 * pos16;
+            if (cap < piece_off + piece_bytes + 16) { free(st[0]); free(st[1]); return -3; }
+            memset(out + piece_off, 0, (size_t)piece_bytes);
+            put32(chunk_off + 4ull * c, (uint32_t)pos16);
+            uint64_t bit = 0;
+            for (int j = 0; j < ZO_SUBS; ++j) {
+                uint64_t lo = c_lo + (uint64_t)j * sub, hi = lo + sub;
+                if (lo > c_hi) lo = c_hi;
+                if (hi > c_hi) hi = c_hi;
+                for (uint64_t k = lo; k < hi; ++k) {
+                    unsigned l = len[s][st[s][k]];
+                    uint32_t cw = code[s][st[s][k]];
+                    for (unsigned b = 0; b < l; ++b, ++bit)          /* most significant code bit first */
+                        if ((cw >> (l - 1 - b)) & 1) set_bit(out + piece_off, bit);
+                }
+                put32(sub_end + 128ull * c + 4ull * j, (uint32_t)bit);
+            }
+            pbits[s] += bits;
+            pos16 += piece_bytes / 16;
+        }
+    }
+    uint64_t payload_bytes = 16 * pos16;
+    uint64_t total = payload_off + payload_bytes + (any_huff ? 16 : 0);
+    if (cap < total) { free(st[0]); free(st[1]); return -3; }
+    if (any_huff) memset(out + payload_off + payload_bytes, 0, 16);
+
+    uint8_t *h = out;
+    h[0] = 'Z'; h[1] = 'C'; h[2] = '1'; h[3] = '0';
+    put16(h + 4, 1);
+    h[6] = (uint8_t)fmt; h[7] = 2;
+    put64(h + 8, n_elems);
+    put32(h + 16, chunk_bytes);
+    put32(h + 20, nc);
+    h[24] = ZO_LMAX; h[25] = (uint8_t)g; h[26] = ZO_SUBS;
+    put64(h + 32, total);
+    put64(h + 40, payload_off);
+    put64(h + 48, payload_bytes);
+    for (int s = 0; s < 2; ++s) {
+        uint8_t *d = h + 64 + 32 * s;
+        d[0] = (uint8_t)mode[s];
+        put64(d + 8, ns);
+        put64(d + 16, pbits[s]);
+        put64(d + 24, sec[s]);
+    }
+    free(st[0]); free(st[1]);
+    return (int64_t)total;
+}
+
+/* ------------------------------------------------------------------ */
+/* Container reader: bit-serial canonical decoding                     */
+/* ------------------------------------------------------------------ */
+
+typedef struct {
+    int fmt, g;
+    uint64_t n_elems, n_syms, total, payload_off, payload_bytes;
+    uint32_t chunk_bytes, n_chunks;
+    int mode[2];
+    uint64_t pbits[2], sec[2];
+} zo_header;
+
+static int parse_header(const uint8_t *c, uint64_t bytes, zo_header *h)
+{
+    if (bytes < ZO_HEADER) return -1;
+    if (c[0] != 'Z' || c[1] != 'C' || c[2] != '1' || c[3] != '0') return -1;
+    if (get16(c + 4) != 1 || c[7] != 2 || c[24] != ZO_LMAX || c[26] != ZO_SUBS) return -1;
+    h->fmt = c[6];
+    h->g = zo_group(h->fmt);
+    if (!h->g || c[25] != h->g) return -1;
+    h->n_elems = get64(c + 8);
+    h->chunk_bytes = get32(c + 16);
+    h->n_chunks = get32(c + 20);
+    if (!valid_chunk_bytes(h->chunk_bytes)) return -1;
+    h->n_syms = zo_n_syms(h->fmt, h->n_elems);
+    if (h->n_chunks != n_chunks_of(h->n_syms, h->chunk_bytes)) return -1;
+    h->total = get64(c + 32);
+    h->payload_off = get64(c + 40);
+    h->payload_bytes = get64(c + 48);
+    if (h->total > bytes || h->payload_off > h->total || h->payload_bytes > h->total - h->payload_off) return -1;
+    for (int s = 0; s < 2; ++s) {
+        const uint8_t *d = c + 64 + 32 * s;
+        h->mode[s] = d[0];
+        if (h->mode[s] != ZO_RAW && h->mode[s] != ZO_HUFF) return -1;
+        if (get64(d + 8) != h->n_syms) return -1;
+        h->pbits[s] = get64(d + 16);
+        h->sec[s] = get64(d + 24);
+        uint64_t need = h->mode[s] == ZO_HUFF ? table_section_bytes(h->n_chunks) : round16(h->n_syms);
+        if (h->sec[s] < ZO_HEADER || h->sec[s] > h->total || need > h->total - h->sec[s]) return -1;
+    }
+    return 0;
+}
+
+/* Read bit number pos of a chunk piece. */
+static unsigned get_bit(const uint8_t *piece, uint64_t pos)
+{
+    uint64_t word = pos / 32;
+    unsigned in_word = 31u - (unsigned)(pos % 32);
+    return (piece[4 * word + in_word / 8] >> (in_word % 8)) & 1u;
+}
+
+/* Tables for walking a canonical code one bit at a time: how many codes
+ * there are of each length, and the symbols in (length, symbol) order. */
+typedef struct {
+    unsigned count[ZO_LMAX + 1];
+    uint8_t order[256];
+    unsigned n;
+} zo_walk;
+
+static int make_walk(const uint8_t len[256], zo_walk *w)
+{
+    memset(w, 0, sizeof(*w));
+    for (int v = 0; v < 256; ++v) {
+        if (len[v] > ZO_LMAX) return -1;
+        if (len[v]) w->count[len[v]]++;
+    }
+    for (int l = 1; l <= ZO_LMAX; ++l)
+        for (int v = 0; v < 256; ++v)
+            if (len[v] == l) w->order[w->n++] = (uint8_t)v;
+    /* the code must not be over-subscribed */
+    uint64_t kraft = 0;
+    for (int l = 1; l <= ZO_LMAX; ++l) kraft += (uint64_t)w->count[l] << (ZO_LMAX - l);
+    if (kraft > (1ull << ZO_LMAX)) return -1;
+    return 0;
+}
+
+/* Decode one symbol starting at *pos; returns -1 if no code matches within 12 bits
+ * or the piece ends. */
+static int walk_symbol(const zo_walk *w, const uint8_t *piece, uint64_t limit_bits, uint64_t *pos)
+{
+    unsigned code = 0, first = 0, index = 0;
+    for (int l = 1; l <= ZO_LMAX; ++l) {
+        if (*pos >= limit_bits) return -1;
+        code = (code << 1) | get_bit(piece, (*pos)++);
+        unsigned cnt = w->count[l];
+        if (code < first + cnt) return w->order[index + (code - first)];
+        index += cnt;
+        first = (first + cnt) << 1;
+    }
+    return -1;
+}
+
+/* Decode the symbols of chunk c of stream s into dst (which receives the
+ * chunk's symbol count).  Returns 0, or -1 on a damaged container. */
+static int decode_chunk_stream(const uint8_t *cont, const zo_header *h, int s, uint32_t c, uint8_t *dst)
+{
+    uint64_t cs = h->chunk_bytes / 2, sub = cs / ZO_SUBS;
+    uint64_t c_lo = (uint64_t)c * cs;
+    uint64_t c_hi = c_lo + cs < h->n_syms ? c_lo + cs : h->n_syms;
+    if (h->mode[s] == ZO_RAW) {
+        memcpy(dst, cont + h->sec[s] + c_lo, (size_t)(c_hi - c_lo));
+        return 0;
+    }
+    zo_walk w;
+    if (make_walk(cont + h->sec[s], &w)) return -1;
+    const uint8_t *chunk_off = cont + h->sec[s] + 256;
+    const uint8_t *sub_end = cont + h->sec[s] + 256 + round16(4ull * h->n_chunks);
+    uint64_t off16 = get32(chunk_off + 4ull * c);
+    uint64_t chunk_bits = get32(sub_end + 128ull * c + 4 * (ZO_SUBS - 1));
+    uint64_t piece_bytes = round16((chunk_bits + 7) / 8);
+    if (16 * off16 > h->payload_bytes || piece_bytes > h->payload_bytes - 16 * off16) return -1;
+    const uint8_t *piece = cont + h->payload_off + 16 * off16;
+    uint64_t start = 0;
+    for (int j = 0; j < ZO_SUBS; ++j) {
+        uint64_t lo = c_lo + (uint64_t)j * sub, hi = lo + sub;
+        if (lo > c_hi) lo = c_hi;
+        if (hi > c_hi) hi = c_hi;
+        uint64_t end = get32(sub_end + 128ull * c + 4ull * j);
+        if (end < start || end > chunk_bits) return -1;
+        uint64_t pos = start;
+        for (uint64_t k = lo; k < hi; ++k) {
+            int v = walk_symbol(&w, piece, end, &pos);
+            if (v < 0) return -1;
+            dst[k - c_lo] = (uint8_t)v;
+        }
+        if (pos != end) return -1;                      /* a subchunk uses exactly its bits */
+        start = end;
+    }
+    return 0;
+}
+
+/* Output bytes of chunk c (all chunks but the last give chunk_bytes). */
+static uint64_t chunk_out_bytes(const zo_header *h, uint32_t c, uint64_t *byte_off)
+{
+    uint64_t cs = h->chunk_bytes / 2;
+    uint64_t el_lo = (uint64_t)c * cs * (uint64_t)h->g;
+    uint64_t el_hi = el_lo + cs * (uint64_t)h->g;
+    if (el_hi > h->n_elems) el_hi = h->n_elems;
+    *byte_off = zo_input_bytes(h->fmt, el_lo);
+    return zo_input_bytes(h->fmt, el_hi) - *byte_off;
+}
+
+/* Decode one chunk alone into out (random access, Sec. 3.1).  Returns the number of
+ * bytes written, or a negative error. */
+int64_t zo_decompress_chunk(const uint8_t *cont, uint64_t bytes, uint32_t c, uint8_t *out, uint64_t cap)
+{
+    zo_header h;
+    if (parse_header(cont, bytes, &h)) return -1;
+    if (c >= h.n_chunks) return -1;
+    uint64_t cs = h.chunk_bytes / 2;
+    uint8_t *a = (uint8_t *)calloc((size_t)cs + 1, 1), *b = (uint8_t *)calloc((size_t)cs + 1, 1);
+    if (!a || !b) { free(a); free(b); return -2; }
+    int rc = decode_chunk_stream(cont, &h, 0, c, a) || decode_chunk_stream(cont, &h, 1, c, b);
+    int64_t ret = -1;
+    if (!rc) {
+        uint64_t off, nb = chunk_out_bytes(&h, c, &off);
+        uint64_t el_lo = (uint64_t)c * cs * (uint64_t)h.g;
+        uint64_t el_hi = el_lo + cs * (uint64_t)h.g;
+        if (el_hi > h.n_elems) el_hi = h.n_elems;
+        if (nb <= cap) { zo_merge(h.fmt, a, b, el_hi - el_lo, out); ret = (int64_t)nb; }
+        else ret = -3;
+    }
+    free(a); free(b);
+    return ret;
+}
+
+/* Decode a whole container.  Returns bytes written or a negative error:
+ * -1 damaged container, -2 out of memory, -3 capacity too small. */
+int64_t zo_decompress(const uint8_t *cont, uint64_t bytes, uint8_t *out, uint64_t cap)
+{
+    zo_header h;
+    if (parse_header(cont, bytes, &h)) return -1;
+    uint64_t need = zo_input_bytes(h.fmt, h.n_elems);
+    if (cap < need) return -3;
+    uint64_t used[2] = {0, 0};
+    for (uint32_t c = 0; c < h.n_chunks; ++c) {
+        uint64_t off, nb = chunk_out_bytes(&h, c, &off);
+        int64_t r = zo_decompress_chunk(cont, bytes, c, out + off, nb);
+        if (r < 0) return r;
+        for (int s = 0; s < 2; ++s)
+            if (h.mode[s] == ZO_HUFF) {
+                const uint8_t *sub_end = cont + h.sec[s] + 256 + round16(4ull * h.n_chunks);
+                used[s] += get32(sub_end + 128ull * c + 4 * (ZO_SUBS - 1));
+            }
+    }
+    for (int s = 0; s < 2; ++s)
+        if (h.mode[s] == ZO_HUFF && used[s] != h.pbits[s]) return -1;   /* all payload bits are consumed */
+    return (int64_t)need;
+}
+
+/* ------------------------------------------------------------------ */
+/* Statistics (Sec. 4 "component-wise breakdown")                      */
+/* ------------------------------------------------------------------ */
+
+typedef struct {
+    uint64_t n_syms, raw_bits, payload_bits;
+    uint32_t mode, n_active, max_len, pad;
+    double avg_len, entropy_bits;
+} zo_stream_stats;
+
+void zo_stream_stats_of(const uint64_t hist[256], const uint8_t len[256], int mode, zo_stream_stats *o)
+{
+    memset(o, 0, sizeof(*o));
+    for (int v = 0; v < 256; ++v) o->n_syms += hist[v];
+    o->raw_bits = 8 * o->n_syms;
+    o->mode = (uint32_t)mode;
+    uint64_t bits = 0;
+    double H = 0.0;
+    for (int v = 0; v < 256; ++v) {
+        if (!hist[v]) continue;
+        o->n_active++;
+        if (len[v] > o->max_len) o->max_len = len[v];
+        bits += hist[v] * (uint64_t)len[v];
+        double p = (double)hist[v] / (double)o->n_syms;
+        H -= p * log2(p);
+    }
+    o->entropy_bits = H;
+    o->avg_len = o->n_syms ? (double)bits / (double)o->n_syms : 0.0;
+    o->payload_bits = mode == ZO_HUFF ? bits : o->raw_bits;
+}
