@@ -1,0 +1,217 @@
+/*
+ * zc.h — C ABI of the B200 lossless exponent / sign+mantissa Huffman codec.
+ *
+ * The library implements the data-parallel hot path of "Lossless Compression of
+ * Neural Network Components: Weights, Checkpoints, and K/V Caches in
+ * Low-Precision Formats" (Heilper & Singer, 2025): every BF16 / FP8 E4M3 /
+ * FP4 E2M1 element is split into an exponent field and a sign+mantissa field
+ * (Sec. 3.1, 3.2, 3.4), the fields of 1 / 2 / 4 neighbouring elements are
+ * grouped into byte symbols (Fig. 7 caption; Sec. 3.4 "2 bits from each of the
+ * 4 consecutive FP4 values"), each of the two symbol streams gets its own
+ * Huffman code or is stored raw when it does not compress (Sec. 3.1), and the
+ * result is written in fixed-size chunks that decode independently (Sec. 3.1
+ * "fixed-size chunks with lightweight metadata ... random access and parallel
+ * decoding").  Decoding restores the original bit patterns exactly.
+ *
+ * Conventions
+ *   - "d_" pointers are DEVICE pointers of the current CUDA device, "h_" pointers
+ *     are HOST pointers.  The caller owns every buffer it passes.  The library
+ *     owns plan and codebook objects until the matching *_destroy call.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Device work is enqueued on it and is asynchronous unless stated otherwise.
+ *   - The library allocates no device memory.  All device scratch is the
+ *     caller's `d_workspace` of zc_workspace_bytes() bytes (256-byte aligned);
+ *     its contents need not be initialised and are undefined afterwards.
+ *     Two calls that overlap in time on the GPU must not share a workspace.
+ *   - Device pointers d_in / d_out / d_comp / d_workspace must be 16-byte aligned.
+ *   - Every function returns a zc_status; nothing throws; out-parameters are
+ *     untouched on error.
+ *
+ * Geometry (fixed by the plan)
+ *   G            elements per symbol: 1 (BF16), 2 (FP8), 4 (FP4)
+ *   n_syms       ceil(n_elems / G) symbols in each of the two streams;
+ *                stream 0 = exponent fields, stream 1 = sign+mantissa fields;
+ *                element G*k+i sits in bits [w*i, w*i+w) of symbol k, w = 8/G;
+ *                missing tail fields are zero
+ *   chunk        chunk_bytes of element bytes = chunk_bytes/2 symbols per stream,
+ *                cut into 32 equal subchunks
+ *   code         canonical prefix code, lengths <= 12 bits, most significant bit
+ *                first inside little-endian 32-bit words
+ *
+ * Container layout (little-endian; every section starts on a 16-byte boundary)
+ *   header, 128 bytes
+ *      0 u32 magic "ZC10"   4 u16 version = 1   6 u8 format   7 u8 n_streams = 2
+ *      8 u64 n_elems       16 u32 chunk_bytes  20 u32 n_chunks
+ *     24 u8 12 (max code length)  25 u8 G  26 u8 32 (subchunks)  27 u8 0  28 u32 0
+ *     32 u64 total_bytes   40 u64 payload_off  48 u64 payload_bytes  56 u64 0
+ *     64 + 32 s : u8 mode (0 RAW, 1 HUFF), 7 zero bytes, u64 n_syms,
+ *                 u64 payload_bits, u64 section_off            (s = 0, 1)
+ *   one table section per HUFF stream (stream order):
+ *      u8  code_len[256]            0 = symbol has no code
+ *      u32 chunk_off16[n_chunks]    zero padded to a multiple of 16 bytes; offset of
+ *                                   the chunk's bits from payload_off, in 16-byte units
+ *      u32 sub_end[n_chunks][32]    end bit of every subchunk inside its chunk
+ *   one body per RAW stream (stream order): n_syms symbol bytes, zero padded to 16
+ *   payload area: for chunk 0, 1, ...: for each HUFF stream (stream order) the
+ *      chunk's bits, zero padded to a multiple of 16 bytes
+ *   16 zero guard bytes when at least one stream is HUFF
+ * The container is a pure function of (input bytes, plan, codebook).
+ */
+#ifndef ZC_H
+#define ZC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum zc_status {
+    ZC_OK = 0,
+    ZC_E_INVALID_ARG = 1,       /* null pointer, bad size, bad alignment, bad chunk size */
+    ZC_E_UNSUPPORTED = 2,       /* unknown format or policy */
+    ZC_E_BUFFER_TOO_SMALL = 3,  /* output capacity below zc_max_compressed_bytes() */
+    ZC_E_CORRUPT = 4,           /* container does not match the plan or is damaged */
+    ZC_E_CUDA = 5,              /* a CUDA runtime call failed */
+    ZC_E_NOMEM = 6,             /* host allocation failed */
+    ZC_E_DEVICE_TIMEOUT = 7,    /* a bounded wait inside a kernel gave up */
+    ZC_E_NO_CODE = 8            /* a symbol of the input has no code in the codebook */
+} zc_status;
+
+typedef enum zc_format {
+    ZC_FMT_BF16 = 1,            /* u16 little-endian: sign 15, exponent 14..7, mantissa 6..0 */
+    ZC_FMT_FP8_E4M3 = 2,        /* u8: sign 7, exponent 6..3, mantissa 2..0 */
+    ZC_FMT_FP4_E2M1 = 3         /* two per byte, element 2i in bits 3..0: sign 3, exponent 2..1, mantissa 0 */
+} zc_format;
+
+typedef enum zc_policy {
+    ZC_POLICY_AUTO = 0,         /* Huffman only for a stream that saves at least 1/64 (Sec. 3.1 rule) */
+    ZC_POLICY_HUFF_ALL = 1,     /* Huffman for every non-empty stream */
+    ZC_POLICY_RAW_ALL = 2       /* both streams stored raw (split / merge only) */
+} zc_policy;
+
+typedef enum zc_mode { ZC_MODE_RAW = 0, ZC_MODE_HUFF = 1 } zc_mode;
+
+typedef struct zc_plan_s zc_plan_t;
+typedef struct zc_codebook_s zc_codebook_t;
+
+typedef struct zc_plan_info {
+    uint32_t format, group, chunk_bytes, n_chunks;
+    uint64_t n_elems, n_syms, input_bytes;
+    uint32_t syms_per_chunk, syms_per_subchunk;
+} zc_plan_info;
+
+typedef struct zc_stream_stats {
+    uint64_t n_syms;            /* symbols in the stream */
+    uint64_t raw_bits;          /* 8 * n_syms */
+    uint64_t payload_bits;      /* sum count*len for HUFF, raw_bits for RAW */
+    uint64_t container_bytes;   /* bytes this stream occupies in the container incl. its tables
+                                   (0 when no header was given) */
+    uint32_t mode;              /* zc_mode */
+    uint32_t n_active_symbols;
+    uint32_t max_len;
+    uint32_t reserved;
+    double avg_len;             /* sum count*len / n_syms with the codebook's lengths */
+    double entropy_bits;        /* Shannon entropy of the histogram, bits per symbol */
+} zc_stream_stats;
+
+typedef struct zc_stats_t {
+    zc_stream_stats stream[2];
+    uint64_t in_bytes;          /* element bytes of the tensor */
+    uint64_t out_bytes;         /* container bytes (header's total_bytes), 0 without header */
+    double ratio_payload;       /* (payload_bits0 + payload_bits1) / (8 * in_bytes) */
+    double ratio_container;     /* out_bytes / in_bytes, 0 without header */
+} zc_stats_t;
+
+/* ---- plan: problem statement of one tensor (Sec. 4 "compression was applied per tensor
+ *      using fixed-size chunks") ------------------------------------------------------------
+ * fmt         element format
+ * n_elems     number of elements (0 is valid and gives a header-only container);
+ *             must be even for FP4
+ * chunk_bytes uncompressed element bytes per chunk: a multiple of 1024 in [1 KiB, 256 KiB]
+ * out         receives a new plan (host object; destroy with zc_plan_destroy)
+ * Errors: INVALID_ARG (null out, bad chunk_bytes, odd FP4 count, more than 2^32-1 chunks),
+ *         UNSUPPORTED (format), NOMEM. */
+zc_status zc_plan(zc_format fmt, uint64_t n_elems, uint32_t chunk_bytes, zc_plan_t** out);
+void zc_plan_destroy(zc_plan_t* plan);
+zc_status zc_plan_get_info(const zc_plan_t* plan, zc_plan_info* out);
+
+/* Capacity in bytes that d_out of zc_compress must have: the size of the container when
+ * every symbol of both streams takes a 12-bit code.  0 for a null plan. */
+size_t zc_max_compressed_bytes(const zc_plan_t* plan);
+
+/* Bytes of device scratch zc_compress / zc_decompress need.  0 for a null plan. */
+size_t zc_workspace_bytes(const zc_plan_t* plan);
+
+/* ---- split + histogram (Sec. 3.1-3.4 field split; the counts every Huffman code needs) ----
+ * d_in    device, zc_plan_info.input_bytes bytes of elements
+ * d_hist  device, uint64_t[2][256]; overwritten with the symbol counts of stream 0 and 1
+ *         over the whole tensor (tail fields of a partial last symbol count as zero)
+ * Asynchronous on cuda_stream.  Errors: INVALID_ARG, CUDA. */
+zc_status zc_histogram(const zc_plan_t* plan, const void* d_in, uint64_t* d_hist, void* cuda_stream);
+
+/* ---- codebook (Sec. 3.1 / 4.1 "standard Huffman encoding", one code per stream per tensor;
+ *      Sec. 3.3 precomputed dictionaries: any histogram may be given) ------------------------
+ * h_hist  host, uint64_t[2][256]
+ * policy  which streams are Huffman-coded
+ * out     receives a new codebook (host object, no device memory)
+ * Lengths are those of an optimal prefix code with maximum length 12 (leaves ordered by
+ * (count, symbol); leaf before package at equal weight); codes are canonical in
+ * (length, symbol) order; a stream with one active symbol gets a 1-bit code.
+ * Host-only: needs no GPU.  Errors: INVALID_ARG, UNSUPPORTED (policy), NOMEM. */
+zc_status zc_build_codebook(const zc_plan_t* plan, const uint64_t* h_hist, zc_policy policy,
+                            zc_codebook_t** out);
+void zc_codebook_destroy(zc_codebook_t* cb);
+
+/* Copy out one stream's mode, code lengths and right-aligned code values
+ * (any of the three out pointers may be null). */
+zc_status zc_codebook_get(const zc_codebook_t* cb, uint32_t stream, uint32_t* mode,
+                          uint8_t* len256, uint32_t* code256);
+
+/* ---- compress (Sec. 3.1 chunked entropy coding of both streams) ---------------------------
+ * d_in          device, the tensor's element bytes
+ * d_out         device, receives the container; out_capacity >= zc_max_compressed_bytes()
+ * d_workspace   device scratch, zc_workspace_bytes() bytes
+ * h_out_bytes   host, optional: when non-null the call synchronises cuda_stream, stores the
+ *               container size and returns the device status (NO_CODE / DEVICE_TIMEOUT
+ *               included); when null the call is asynchronous and the size is the
+ *               header's total_bytes field
+ * The codebook need not come from this tensor's histogram, but every symbol that occurs in
+ * a HUFF stream must have a code; otherwise the device status becomes ZC_E_NO_CODE and the
+ * container is invalid.
+ * Errors: INVALID_ARG, BUFFER_TOO_SMALL, CUDA, and the device status when synchronous. */
+zc_status zc_compress(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, void* d_out,
+                      size_t out_capacity, void* d_workspace, uint64_t* h_out_bytes, void* cuda_stream);
+
+/* ---- decompress (Sec. 3.1 "parallel decoding") --------------------------------------------
+ * d_comp      device, a container made for the same plan; comp_bytes = bytes available
+ * d_out       device, receives zc_plan_info.input_bytes bytes, identical to the original
+ * The header is checked on the device against the plan before anything is decoded; a
+ * mismatch or damaged table sets the device status to ZC_E_CORRUPT and nothing is written.
+ * Asynchronous; read the outcome with zc_device_status().  Errors: INVALID_ARG, CUDA. */
+zc_status zc_decompress(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes, void* d_out,
+                        void* d_workspace, void* cuda_stream);
+
+/* Synchronise cuda_stream and return the status word the last zc_compress / zc_decompress
+ * call on this workspace left on the device (ZC_OK if none was raised). */
+zc_status zc_device_status(const zc_plan_t* plan, const void* d_workspace, void* cuda_stream);
+
+/* ---- host-side checks and statistics ------------------------------------------------------
+ * zc_validate_container: structural check of a HOST copy of a container against a plan:
+ * header fields, section bounds, Kraft sum of each code-length table, monotone chunk
+ * offsets and subchunk ends, payload bit totals.  Returns ZC_OK or ZC_E_CORRUPT. */
+zc_status zc_validate_container(const zc_plan_t* plan, const void* h_container, size_t bytes);
+
+/* zc_stats (Sec. 4 "component-wise breakdown (exponent vs. mantissa)"): per-stream and total
+ * sizes and ratios from a histogram and a codebook; h_header (host copy of at least the first
+ * 128 container bytes) is optional and adds the container-inclusive figures. */
+zc_status zc_stats(const zc_plan_t* plan, const zc_codebook_t* cb, const uint64_t* h_hist,
+                   const void* h_header, zc_stats_t* out);
+
+const char* zc_strerror(zc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZC_H */

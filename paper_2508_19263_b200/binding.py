@@ -1,0 +1,240 @@
+"""Thin ctypes binding of libzc's C ABI.
+
+Argument marshalling only: every step of the codec runs in the library's CUDA kernels (or, for
+the codebook and the statistics, in its host code).  The functions have the names of the C entry
+points without the ``zc_`` prefix.  PyTorch supplies device memory and streams.
+
+The library must be present (``paper_2508_19263_b200/libzc.so``, built by ``build.build_library``);
+importing this module fails loudly when it is not — there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 1, 2, 3
+POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL = 0, 1, 2
+MODE_RAW, MODE_HUFF = 0, 1
+OK, E_INVALID_ARG, E_UNSUPPORTED, E_BUFFER_TOO_SMALL, E_CORRUPT, E_CUDA, E_NOMEM, E_DEVICE_TIMEOUT, E_NO_CODE = range(9)
+
+
+class ZcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_lib.zc_strerror(status).decode()} (status {status})")
+
+
+class PlanInfo(C.Structure):
+    _fields_ = [("format", C.c_uint32), ("group", C.c_uint32), ("chunk_bytes", C.c_uint32), ("n_chunks", C.c_uint32),
+                ("n_elems", C.c_uint64), ("n_syms", C.c_uint64), ("input_bytes", C.c_uint64),
+                ("syms_per_chunk", C.c_uint32), ("syms_per_subchunk", C.c_uint32)]
+
+
+class StreamStats(C.Structure):
+    _fields_ = [("n_syms", C.c_uint64), ("raw_bits", C.c_uint64), ("payload_bits", C.c_uint64),
+                ("container_bytes", C.c_uint64), ("mode", C.c_uint32), ("n_active_symbols", C.c_uint32),
+                ("max_len", C.c_uint32), ("reserved", C.c_uint32), ("avg_len", C.c_double),
+                ("entropy_bits", C.c_double)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("stream", StreamStats * 2), ("in_bytes", C.c_uint64), ("out_bytes", C.c_uint64),
+                ("ratio_payload", C.c_double), ("ratio_container", C.c_double)]
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: run paper_2508_19263_b200.build.build_library() "
+                          "(or __graft_entry__.build()) first; there is no fallback implementation")
+    L = C.CDLL(path)
+    vp, u64p = C.c_void_p, C.POINTER(C.c_uint64)
+    L.zc_plan.restype = C.c_int
+    L.zc_plan.argtypes = [C.c_int, C.c_uint64, C.c_uint32, C.POINTER(vp)]
+    L.zc_plan_destroy.restype = None
+    L.zc_plan_destroy.argtypes = [vp]
+    L.zc_plan_get_info.restype = C.c_int
+    L.zc_plan_get_info.argtypes = [vp, C.POINTER(PlanInfo)]
+    L.zc_max_compressed_bytes.restype = C.c_size_t
+    L.zc_max_compressed_bytes.argtypes = [vp]
+    L.zc_workspace_bytes.restype = C.c_size_t
+    L.zc_workspace_bytes.argtypes = [vp]
+    L.zc_histogram.restype = C.c_int
+    L.zc_histogram.argtypes = [vp, vp, vp, vp]
+    L.zc_build_codebook.restype = C.c_int
+    L.zc_build_codebook.argtypes = [vp, u64p, C.c_int, C.POINTER(vp)]
+    L.zc_codebook_destroy.restype = None
+    L.zc_codebook_destroy.argtypes = [vp]
+    L.zc_codebook_get.restype = C.c_int
+    L.zc_codebook_get.argtypes = [vp, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint8), C.POINTER(C.c_uint32)]
+    L.zc_compress.restype = C.c_int
+    L.zc_compress.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, u64p, vp]
+    L.zc_decompress.restype = C.c_int
+    L.zc_decompress.argtypes = [vp, vp, C.c_size_t, vp, vp, vp]
+    L.zc_device_status.restype = C.c_int
+    L.zc_device_status.argtypes = [vp, vp, vp]
+    L.zc_validate_container.restype = C.c_int
+    L.zc_validate_container.argtypes = [vp, vp, C.c_size_t]
+    L.zc_stats.restype = C.c_int
+    L.zc_stats.argtypes = [vp, vp, u64p, vp, C.POINTER(Stats)]
+    L.zc_strerror.restype = C.c_char_p
+    L.zc_strerror.argtypes = [C.c_int]
+    L.zc_test_split16.restype = C.c_int
+    L.zc_test_split16.argtypes = [C.c_int, vp, vp, vp]
+    L.zc_test_merge16.restype = C.c_int
+    L.zc_test_merge16.argtypes = [C.c_int, vp, vp, vp]
+    return L
+
+
+_lib = _load()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise ZcError(status, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def strerror(status: int) -> str:
+    return _lib.zc_strerror(status).decode()
+
+
+class Plan:
+    """zc_plan: the problem statement of one tensor (format, element count, chunk size)."""
+
+    def __init__(self, fmt: int, n_elems: int, chunk_bytes: int):
+        h = C.c_void_p()
+        _check(_lib.zc_plan(fmt, n_elems, chunk_bytes, C.byref(h)), "zc_plan")
+        self._h = h
+        info = PlanInfo()
+        _check(_lib.zc_plan_get_info(h, C.byref(info)), "zc_plan_get_info")
+        self.info = info
+        self.format, self.n_elems, self.chunk_bytes = fmt, n_elems, chunk_bytes
+        self.n_syms, self.n_chunks, self.input_bytes = info.n_syms, info.n_chunks, info.input_bytes
+        self.max_compressed_bytes = _lib.zc_max_compressed_bytes(h)
+        self.workspace_bytes = _lib.zc_workspace_bytes(h)
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h:
+            _lib.zc_plan_destroy(h)
+            self._h = None
+
+
+def plan(fmt: int, n_elems: int, chunk_bytes: int) -> Plan:
+    return Plan(fmt, n_elems, chunk_bytes)
+
+
+class Codebook:
+    """zc_build_codebook result: per stream a mode, 256 code lengths and 256 canonical code values."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    def get(self, stream_idx: int):
+        mode = C.c_uint32()
+        lens = np.zeros(256, np.uint8)
+        codes = np.zeros(256, np.uint32)
+        _check(_lib.zc_codebook_get(self._h, stream_idx, C.byref(mode), lens.ctypes.data_as(C.POINTER(C.c_uint8)),
+                                    codes.ctypes.data_as(C.POINTER(C.c_uint32))), "zc_codebook_get")
+        return mode.value, lens, codes
+
+    @property
+    def modes(self):
+        return [self.get(0)[0], self.get(1)[0]]
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h:
+            _lib.zc_codebook_destroy(h)
+            self._h = None
+
+
+def histogram(p: Plan, d_in: torch.Tensor, d_hist: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """zc_histogram: returns a device tensor uint64-as-int64 [2, 256]."""
+    assert d_in.is_cuda and d_in.is_contiguous()
+    if d_hist is None:
+        d_hist = torch.empty((2, 256), dtype=torch.int64, device=d_in.device)
+    _check(_lib.zc_histogram(p._h, d_in.data_ptr(), d_hist.data_ptr(), _stream_ptr(stream)), "zc_histogram")
+    return d_hist
+
+
+def build_codebook(p: Plan, h_hist, policy: int = POLICY_AUTO) -> Codebook:
+    """zc_build_codebook: host only.  h_hist: array-like [2, 256] of counts."""
+    h = np.ascontiguousarray(np.asarray(h_hist).astype(np.uint64)).reshape(512)
+    out = C.c_void_p()
+    _check(_lib.zc_build_codebook(p._h, h.ctypes.data_as(C.POINTER(C.c_uint64)), policy, C.byref(out)),
+           "zc_build_codebook")
+    return Codebook(out)
+
+
+def compress(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Tensor, d_workspace: torch.Tensor,
+             sync: bool = True, stream=None) -> Optional[int]:
+    """zc_compress.  With sync=True returns the container size in bytes (and raises on a device-side
+    error); with sync=False the call is asynchronous and returns None."""
+    assert d_in.is_cuda and d_out.is_cuda and d_workspace.is_cuda
+    assert d_workspace.numel() * d_workspace.element_size() >= p.workspace_bytes
+    n = C.c_uint64(0)
+    st = _lib.zc_compress(p._h, cb._h, d_in.data_ptr(), d_out.data_ptr(), d_out.numel() * d_out.element_size(),
+                          d_workspace.data_ptr(), C.byref(n) if sync else None, _stream_ptr(stream))
+    _check(st, "zc_compress")
+    return n.value if sync else None
+
+
+def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tensor, d_workspace: torch.Tensor,
+               stream=None) -> None:
+    """zc_decompress (asynchronous; call device_status() to learn the outcome)."""
+    assert d_comp.is_cuda and d_out.is_cuda and d_workspace.is_cuda
+    assert d_out.numel() * d_out.element_size() >= p.input_bytes
+    _check(_lib.zc_decompress(p._h, d_comp.data_ptr(), comp_bytes, d_out.data_ptr(), d_workspace.data_ptr(),
+                              _stream_ptr(stream)), "zc_decompress")
+
+
+def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:
+    return _lib.zc_device_status(p._h, d_workspace.data_ptr(), _stream_ptr(stream))
+
+
+def validate_container(p: Plan, h_container) -> int:
+    c = np.ascontiguousarray(h_container, np.uint8)
+    return _lib.zc_validate_container(p._h, c.ctypes.data, c.size)
+
+
+def stats(p: Plan, cb: Codebook, h_hist, h_header=None) -> Stats:
+    h = np.ascontiguousarray(np.asarray(h_hist).astype(np.uint64)).reshape(512)
+    hd = None
+    if h_header is not None:
+        hd = np.ascontiguousarray(h_header, np.uint8)
+        assert hd.size >= 128
+    out = Stats()
+    _check(_lib.zc_stats(p._h, cb._h, h.ctypes.data_as(C.POINTER(C.c_uint64)), hd.ctypes.data if hd is not None else None,
+                         C.byref(out)), "zc_stats")
+    return out
+
+
+def test_split16(fmt: int, in16: np.ndarray):
+    a = np.ascontiguousarray(in16, np.uint8)
+    e, sm = np.zeros(8, np.uint8), np.zeros(8, np.uint8)
+    _check(_lib.zc_test_split16(fmt, a.ctypes.data, e.ctypes.data, sm.ctypes.data), "zc_test_split16")
+    return e, sm
+
+
+def test_merge16(fmt: int, e8: np.ndarray, sm8: np.ndarray):
+    e, sm = np.ascontiguousarray(e8, np.uint8), np.ascontiguousarray(sm8, np.uint8)
+    out = np.zeros(16, np.uint8)
+    _check(_lib.zc_test_merge16(fmt, e.ctypes.data, sm.ctypes.data, out.ctypes.data), "zc_test_merge16")
+    return out
+
+
+test_split16.__test__ = False
+test_merge16.__test__ = False

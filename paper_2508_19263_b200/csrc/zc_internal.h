@@ -1,0 +1,84 @@
+// Internal definitions shared by the host logic and the kernels of libzc.
+#pragma once
+#include <stdint.h>
+#include <stddef.h>
+#include "zc.h"
+
+namespace zc {
+
+constexpr uint32_t kLmax = 12;            // longest code; decode table has 2^12 entries
+constexpr uint32_t kSubs = 32;            // subchunks per chunk = lanes of the decoding warp
+constexpr uint32_t kHeaderBytes = 128;
+constexpr uint32_t kMagic = 0x3031435Au;  // 'Z','C','1','0' little-endian
+
+// Byte offsets inside the 128-byte header.
+constexpr uint32_t kHdrMagic = 0, kHdrVersion = 4, kHdrFormat = 6, kHdrStreams = 7, kHdrElems = 8,
+                   kHdrChunkBytes = 16, kHdrChunks = 20, kHdrLmax = 24, kHdrGroup = 25, kHdrSubs = 26,
+                   kHdrTotal = 32, kHdrPayloadOff = 40, kHdrPayloadBytes = 48, kHdrStream0 = 64,
+                   kHdrStreamStride = 32;
+// Inside a stream descriptor.
+constexpr uint32_t kSdMode = 0, kSdSyms = 8, kSdBits = 16, kSdSection = 24;
+
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// Where things are for given modes: everything except the payload size is known before encoding.
+struct Layout {
+    uint64_t section_off[2];   // table section (HUFF) or raw body (RAW)
+    uint64_t chunk_off_tab[2]; // HUFF: offset of chunk_off16[]
+    uint64_t sub_end_tab[2];   // HUFF: offset of sub_end[][32]
+    uint64_t payload_off;
+};
+
+}  // namespace zc
+
+struct zc_plan_s {
+    uint32_t format, group, chunk_bytes, n_chunks;
+    uint64_t n_elems, n_syms, input_bytes;
+    uint32_t syms_per_chunk, syms_per_sub;
+};
+
+struct zc_codebook_s {
+    uint32_t mode[2];
+    uint8_t len[2][256];
+    uint32_t code[2][256];     // right-aligned canonical code values
+};
+
+namespace zc {
+
+inline uint64_t table_section_bytes(uint32_t n_chunks)
+{
+    return 256 + round_up(4ull * n_chunks, 16) + 128ull * n_chunks;
+}
+
+inline Layout make_layout(const zc_plan_s& p, const uint32_t mode[2])
+{
+    Layout L{};
+    uint64_t off = kHeaderBytes;
+    for (int s = 0; s < 2; ++s)
+        if (mode[s] == ZC_MODE_HUFF) {
+            L.section_off[s] = off;
+            L.chunk_off_tab[s] = off + 256;
+            L.sub_end_tab[s] = off + 256 + round_up(4ull * p.n_chunks, 16);
+            off += table_section_bytes(p.n_chunks);
+        }
+    for (int s = 0; s < 2; ++s)
+        if (mode[s] == ZC_MODE_RAW) {
+            L.section_off[s] = off;
+            off += round_up(p.n_syms, 16);
+        }
+    L.payload_off = off;
+    return L;
+}
+
+// Device workspace: a control block followed by one look-back word per chunk.
+struct Control {
+    uint32_t status;           // zc_status raised on the device (first one wins)
+    uint32_t ticket;           // next chunk to hand out
+    unsigned long long payload_bits[2];
+    unsigned long long total16;  // payload area size in 16-byte units
+    uint32_t done;             // chunks finished
+    uint32_t pad[7];
+};
+constexpr size_t kControlBytes = 256;
+
+}  // namespace zc
