@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the split + Huffman codec on B200.
+
+One *step* = one pass of the whole hot path over the whole synthetic workload: for every tensor
+split+histogram on the GPU, codebook on the host, compress on the GPU, decompress on the GPU.
+The default workload is the BF16 Llama-8B-shaped weight stack (225 tensors, 15.0 GB).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--chunk-kib C]
+
+Prints ONE JSON line (rank 0).  `value` is uncompressed GB per second through the whole path with all
+inputs resident in HBM; `decode` / `encode` / `histogram` hold the per-call throughputs and their
+fraction of the HBM roofline time (uncompressed + compressed bytes) / peak; `e2e` repeats the step with
+host buffers (pinned) and the host<->device copies inside the timed region; `cpu_baseline` times the CPU
+oracle on a bounded sample.  `--impl reference` times the CPU oracle alone (the paper ships no code).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2508_19263_b200 import workloads as wl
+
+METRIC = "decode & encode GB/s (uncompressed bytes) on 1 B200, % HBM roofline, compression ratio"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+ORACLE_SAMPLE_BYTES = 256 << 20
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+# --------------------------------------------------------------------------------------------
+# workloads
+# --------------------------------------------------------------------------------------------
+
+def workload_specs(name: str):
+    if name == "cfg2_bf16_llama8b":
+        return wl.BF16, wl.llama8b_stack(2)
+    if name == "cfg3_fp8_llama8b":
+        return wl.FP8_E4M3, wl.llama8b_stack(3)
+    if name == "cfg4_fp4_llama8b":
+        return wl.FP4_E2M1, wl.llama8b_stack(4)
+    if name == "small_bf16":
+        return wl.BF16, wl.llama8b_stack(2, n_layers=2, include_embedding=False)
+    if name == "small_fp8":
+        return wl.FP8_E4M3, wl.llama8b_stack(3, n_layers=2, include_embedding=False)
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_id: str):
+        self.rows = []
+        self.proc = None
+        self.idx = device_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2])); power.append(float(r[3]))
+                for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7), ("sw_power_cap", 8)):
+                    if r[col].lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle as baseline / reference arm
+# --------------------------------------------------------------------------------------------
+
+def oracle_sample(fmt, specs, device):
+    """The first tensors of the workload up to ORACLE_SAMPLE_BYTES, as host arrays."""
+    out, total = [], 0
+    for spec in specs:
+        t, n, _ = wl.make_weight(spec, fmt, device)
+        if total and total + t.numel() > ORACLE_SAMPLE_BYTES:
+            break
+        out.append((spec.name, t.cpu().numpy(), n))
+        total += t.numel()
+        if total >= ORACLE_SAMPLE_BYTES:
+            break
+    return out, total
+
+
+def oracle_step(fmt, sample, chunk_bytes):
+    """Whole path on the CPU oracle (single thread): histogram, codebook, compress, decompress."""
+    import oracle as zo
+    t_h = t_e = t_d = 0.0
+    cbytes = 0
+    for name, data, n in sample:
+        t0 = time.perf_counter()
+        h = zo.histogram(fmt, data, n)
+        cb = zo.build_codebook(h, zo.POLICY_AUTO)
+        t1 = time.perf_counter()
+        c = zo.compress(fmt, data, n, chunk_bytes, cb)
+        t2 = time.perf_counter()
+        back = zo.decompress(c, data.size)
+        t3 = time.perf_counter()
+        assert np.array_equal(back, data)
+        t_h += t1 - t0; t_e += t2 - t1; t_d += t3 - t2
+        cbytes += c.size
+    return t_h, t_e, t_d, cbytes
+
+
+def run_reference(args):
+    """--impl reference: the paper ships no code, so the reference arm is the CPU oracle as it stands."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    fmt, specs = workload_specs(args.workload)
+    sample, total = oracle_sample(fmt, specs, "cpu")
+    chunk_bytes = args.chunk_kib * 1024
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(fmt, sample[:1], chunk_bytes)
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        t_h, t_e, t_d, cbytes = oracle_step(fmt, sample, chunk_bytes)
+        times.append(time.perf_counter() - t0)
+    dt = float(np.mean(times))
+    value = total / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.workload, "chunk_kib": args.chunk_kib, "policy": "auto",
+                   "sample": f"first {len(sample)} tensors, {total} bytes"},
+        "decode": {"value": total / t_d / 1e9, "unit": UNIT}, "encode": {"value": total / t_e / 1e9, "unit": UNIT},
+        "compression_ratio": cbytes / total,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"first {len(sample)} tensors of {args.workload}, {total} bytes per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    from paper_2508_19263_b200 import binding as zc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    fmt, specs = workload_specs(args.workload)
+    chunk_bytes = args.chunk_kib * 1024
+    # weak scaling: every rank holds its own copy of the stack (same shapes, its own seeds)
+    for s in specs:
+        s.seed += 100000 * rank
+
+    # ---- resident inputs, plans, output buffers ----
+    tensors = []
+    for spec in specs:
+        t, n, _ = wl.make_weight(spec, fmt, dev)
+        p = zc.plan(fmt, n, chunk_bytes)
+        tensors.append({"name": spec.name, "in": t, "n": n, "plan": p,
+                        "comp": torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=dev),
+                        "out": torch.empty(p.input_bytes, dtype=torch.uint8, device=dev),
+                        "ws": torch.empty(p.workspace_bytes, dtype=torch.uint8, device=dev)})
+    n_t = len(tensors)
+    U = sum(t["plan"].input_bytes for t in tensors)
+    d_hist = torch.zeros((n_t, 2, 256), dtype=torch.int64, device=dev)
+    h_hist = torch.zeros((n_t, 2, 256), dtype=torch.int64).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def phase_hist():
+        for i, t in enumerate(tensors):
+            zc.histogram(t["plan"], t["in"], d_hist[i])
+        h_hist.copy_(d_hist, non_blocking=True)
+        stream.synchronize()
+
+    def phase_codebooks():
+        hh = h_hist.numpy()
+        for i, t in enumerate(tensors):
+            t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
+
+    def phase_compress():
+        for t in tensors:
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False)
+
+    def phase_decompress():
+        for t in tensors:
+            zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"])
+
+    def read_sizes():
+        torch.cuda.synchronize()
+        for t in tensors:
+            hdr = t["comp"][:128].cpu().numpy()
+            t["cbytes"] = int(np.frombuffer(hdr[32:40].tobytes(), "<u8")[0])
+            t["hdr"] = hdr
+
+    def step():
+        # histogram of every tensor, then codebook / compress / decompress per tensor: the host builds the
+        # next codebook while the GPU is busy with the previous tensors
+        phase_hist()
+        hh = h_hist.numpy()
+        for i, t in enumerate(tensors):
+            t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False)
+            # the decoder only needs an upper bound of the container size; the header carries the exact one
+            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"])
+
+    def timed(fn, reps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            tms = torch.tensor([ms], device=dev)
+            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+            ms = float(tms.item())
+        return ms / reps
+
+    # ---- correctness of what is timed (untimed): statuses, byte-identical round trip ----
+    step()
+    read_sizes()
+    for t in tensors:
+        st = zc.device_status(t["plan"], t["ws"])
+        if st != zc.OK:
+            raise SystemExit(f"device status {st} on {t['name']}")
+        if not torch.equal(t["out"], t["in"]):
+            raise SystemExit(f"round trip mismatch on {t['name']}")
+    C = sum(t["cbytes"] for t in tensors)
+
+    for _ in range(max(args.warmup - 1, 0)):
+        step()
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    ms_step = timed(step, args.steps)
+    # per-call throughputs: the same calls, each kind timed back to back over all tensors
+    ms_hist = timed(phase_hist, args.steps)
+    phase_codebooks()
+    t0 = time.perf_counter()
+    phase_codebooks()
+    ms_codebook = (time.perf_counter() - t0) * 1e3
+    ms_enc = timed(phase_compress, args.steps)
+    ms_dec = timed(phase_decompress, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end with host buffers: H2D of the inputs and D2H of the containers inside the timed region ----
+    e2e = None
+    try:
+        h_in = [t["in"].cpu().pin_memory() for t in tensors]
+        h_out = [torch.empty(t["cbytes"], dtype=torch.uint8).pin_memory() for t in tensors]
+
+        def e2e_step():
+            for i, t in enumerate(tensors):
+                t["in"].copy_(h_in[i], non_blocking=True)
+                zc.histogram(t["plan"], t["in"], d_hist[i])
+            h_hist.copy_(d_hist, non_blocking=True)
+            stream.synchronize()
+            hh = h_hist.numpy()
+            for i, t in enumerate(tensors):
+                cb = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
+                zc.compress(t["plan"], cb, t["in"], t["comp"], t["ws"], sync=False)
+                h_out[i].copy_(t["comp"][: t["cbytes"]], non_blocking=True)
+                zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"])
+
+        e2e_step()
+        ms_e2e = timed(e2e_step, max(1, min(args.steps, 3)))
+        e2e = {"value": world * U / ms_e2e / 1e6, "unit": UNIT, "h2d_bytes_per_step": U, "d2h_bytes_per_step": C + n_t * 4096,
+               "ms_per_step": ms_e2e,
+               "note": "host tensor -> H2D -> histogram -> codebook -> compress -> D2H container; decoded tensor stays on the device"}
+        del h_in, h_out
+    except Exception as ex:  # pinned host memory for the whole stack may be unavailable
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "error": str(ex)[:200]}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peaks()
+    gbs = lambda nbytes, ms: nbytes / ms / 1e6
+
+    def leg(ms, nbytes_alg):
+        return {"value": world * gbs(U, ms), "unit": UNIT, "ms": ms, "algorithmic_bytes": nbytes_alg,
+                "hbm_gbs": gbs(nbytes_alg, ms), "frac_of_measured_peak": gbs(nbytes_alg, ms) / peak,
+                "frac_of_nominal_8TBs": gbs(nbytes_alg, ms) / NOMINAL_HBM_GBS}
+
+    dec, enc, hist = leg(ms_dec, U + C), leg(ms_enc, U + C), leg(ms_hist, U)
+    dom_name, dom = ("decode_kernel", dec) if ms_dec >= ms_enc else ("encode_kernel", enc)
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": dom["hbm_gbs"], "peak": peak, "unit": "GB/s",
+                "frac": dom["hbm_gbs"] / peak, "peak_source": peak_src,
+                "avg_launch_ms": (ms_dec if dom_name == "decode_kernel" else ms_enc) / n_t,
+                "algorithmic_bytes_per_launch": (U + C) / n_t, "traffic": None}
+
+    # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only) ----
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        sample, total = oracle_sample(fmt, specs, dev)
+        t_h, t_e, t_d, cb_sample = oracle_step(fmt, sample, chunk_bytes)
+        cpu = {"value": total / (t_h + t_e + t_d) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {len(sample)} tensors of {args.workload}, {total} bytes",
+               "decode_gbs": total / t_d / 1e9, "encode_gbs": total / t_e / 1e9, "histogram_codebook_gbs": total / t_h / 1e9}
+
+    # compression ratios next to the paper's (context): exponent stream, sign+mantissa stream, total
+    st_bits = [0, 0]
+    for t in tensors:
+        for s in range(2):
+            st_bits[s] += int(np.frombuffer(t["hdr"][64 + 32 * s + 16: 64 + 32 * s + 24].tobytes(), "<u8")[0])
+    n_syms = sum(t["plan"].n_syms for t in tensors)
+    line = {
+        "metric": METRIC, "value": world * gbs(U, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.workload, "tensors": n_t, "uncompressed_bytes": U, "compressed_bytes": C,
+                   "chunk_kib": args.chunk_kib, "policy": "auto", "l2": "inputs larger than L2 (no flush)"},
+        "decode": dec, "encode": enc, "histogram": hist, "codebook_host_ms": ms_codebook,
+        "compression_ratio": {"total_container": C / U, "exponent_stream_payload": st_bits[0] / (8 * n_syms),
+                              "sign_mantissa_stream_payload": st_bits[1] / (8 * n_syms),
+                              "paper_context": "abstract: up to 62% (BF16) / 83% (FP8) total"},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": 4 * n_t * args.steps,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2_bf16_llama8b")
+    ap.add_argument("--chunk-kib", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -221,7 +221,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     if (blockIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
             if (P.mode[s] == ZC_MODE_HUFF) {
-                if (threadIdx.x < 256) P.out[P.lay.section_off[s] + threadIdx.x] = (uint8_t)(T.enc[s][threadIdx.x] >> 16);
+                for (uint32_t v = threadIdx.x; v < 256; v += blockDim.x) P.out[P.lay.section_off[s] + v] = (uint8_t)(T.enc[s][v] >> 16);
                 const uint32_t padded = (P.n_chunks + 3) & ~3u;
                 for (uint32_t i = P.n_chunks + threadIdx.x; i < padded; i += blockDim.x)
                     reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[i] = 0;

@@ -1,0 +1,231 @@
+"""Parity of the CUDA path with the CPU oracle: bit-exact histograms, containers and round trips.
+
+Everything goes through the C ABI (via the ctypes binding).  Integer work: no tolerance.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as zo
+from paper_2508_19263_b200 import binding as zc
+from paper_2508_19263_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1]
+DEV = "cuda"
+
+
+def _gpu_round_trip(fmt, data_np, n, chunk_bytes, policy, oracle_codebook_hist=None, check_container=True):
+    """Run histogram -> codebook -> compress -> decompress on the GPU and compare every stage with the oracle."""
+    p = zc.plan(fmt, n, chunk_bytes)
+    d_in = torch.from_numpy(data_np.copy()).to(DEV) if data_np.size else torch.zeros(16, dtype=torch.uint8, device=DEV)
+    # histogram
+    d_hist = zc.histogram(p, d_in)
+    hist = d_hist.cpu().numpy().astype(np.uint64)
+    want_hist = zo.histogram(fmt, data_np, n)
+    assert np.array_equal(hist, want_hist)
+    # codebook (possibly from another histogram: static dictionary)
+    hsrc = hist if oracle_codebook_hist is None else oracle_codebook_hist
+    cb = zc.build_codebook(p, hsrc, policy)
+    ocb = zo.build_codebook(hsrc, policy)
+    # compress
+    d_out = torch.full((p.max_compressed_bytes + 64,), 0xA5, dtype=torch.uint8, device=DEV)
+    d_ws = torch.full((p.workspace_bytes,), 0x5A, dtype=torch.uint8, device=DEV)
+    nbytes = zc.compress(p, cb, d_in, d_out[: p.max_compressed_bytes], d_ws)
+    cont = d_out[:nbytes].cpu().numpy()
+    assert (d_out[p.max_compressed_bytes:].cpu().numpy() == 0xA5).all()        # canary after the buffer
+    if check_container:
+        want = zo.compress(fmt, data_np, n, chunk_bytes, ocb)
+        assert nbytes == want.size
+        if not np.array_equal(cont, want):
+            bad = np.flatnonzero(cont != want)
+            raise AssertionError(f"container differs at {bad[:8]} of {want.size} (first: got {cont[bad[0]]:#x} want {want[bad[0]]:#x})")
+        assert zc.validate_container(p, cont) == zc.OK
+    # decompress the GPU container on the GPU
+    d_back = torch.full((p.input_bytes + 64,), 0xEE, dtype=torch.uint8, device=DEV)
+    zc.decompress(p, d_out, nbytes, d_back, d_ws)
+    assert zc.device_status(p, d_ws) == zc.OK
+    back = d_back.cpu().numpy()
+    assert np.array_equal(back[: p.input_bytes], data_np[: p.input_bytes])
+    assert (back[p.input_bytes:] == 0xEE).all()
+    # and the oracle decodes it too
+    assert np.array_equal(zo.decompress(cont, p.input_bytes), data_np[: p.input_bytes])
+    return p, cb, hist, cont
+
+
+def _weights(fmt, n, seed):
+    rng = np.random.default_rng(seed)
+    if n == 0:
+        return np.zeros(0, np.uint8)
+    if fmt == zc.FMT_BF16:
+        x = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+        return x.to(torch.bfloat16).view(torch.uint8).numpy().reshape(-1).copy()
+    if fmt == zc.FMT_FP8_E4M3:
+        x = rng.standard_normal(n).astype(np.float32)
+        x = x / (np.abs(x).max() / 448.0)
+        return torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(-1).copy()
+    v = rng.choice(16, size=n, p=np.array([6, 5, 4, 3, 2, 1, 1, 1, 6, 5, 4, 3, 2, 1, 1, 1]) / 46.0).astype(np.uint8)
+    return (v[0::2] | (v[1::2] << 4)).astype(np.uint8)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("policy", [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL])
+@pytest.mark.parametrize("chunk_bytes", [1024, 2048, 3072, 8192, 16384, 65536])
+def test_round_trip_several_chunks_and_ragged_tail(fmt, policy, chunk_bytes):
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    n = (5 * cs + cs // 3 + 11) * G
+    if fmt == zc.FMT_FP4_E2M1:
+        n -= n % 2
+    _gpu_round_trip(fmt, _weights(fmt, n, chunk_bytes + fmt), n, chunk_bytes, policy)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_edge_sizes(fmt):
+    G = zo.group(fmt)
+    chunk_bytes = 1024
+    cs = chunk_bytes // 2
+    sizes = {0, 1, G - 1, G, G + 1, 2 * G, 7 * G, 8 * G, 9 * G, cs * G - 1, cs * G, cs * G + 1, cs * G + G,
+             2 * cs * G, 33 * cs * G + 5 * G, 16 * G - 1, 16 * G + 1}
+    for n in sorted(sizes):
+        if n < 0 or (fmt == zc.FMT_FP4_E2M1 and n % 2):
+            continue
+        for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL):
+            _gpu_round_trip(fmt, _weights(fmt, n, 100 + n), n, chunk_bytes, policy)
+
+
+def test_special_bit_patterns():
+    z = np.zeros(20000, np.uint16).view(np.uint8)                     # one active symbol per stream
+    _gpu_round_trip(zc.FMT_BF16, z, 20000, 4096, zc.POLICY_HUFF_ALL)
+    pats = np.array([0x7FC0, 0xFFC1, 0x7F80, 0xFF80, 0x8000, 0x0001, 0x807F, 0x7FFF] * 3000, np.uint16).view(np.uint8)
+    _gpu_round_trip(zc.FMT_BF16, pats, 24000, 4096, zc.POLICY_HUFF_ALL)
+    allb = np.tile(np.arange(256, dtype=np.uint8), 100)
+    _gpu_round_trip(zc.FMT_FP8_E4M3, allb, allb.size, 2048, zc.POLICY_HUFF_ALL)
+    _gpu_round_trip(zc.FMT_FP4_E2M1, allb, 2 * allb.size, 2048, zc.POLICY_HUFF_ALL)
+    rng = np.random.default_rng(1)
+    uni = rng.integers(0, 256, 1 << 18, dtype=np.uint8)               # incompressible: every code length near 8
+    _gpu_round_trip(zc.FMT_BF16, uni, 1 << 17, 8192, zc.POLICY_HUFF_ALL)
+
+
+def test_long_codes_and_skew():
+    """Exponentially skewed exponents: the 12-bit limit binds and codes of every length occur."""
+    rng = np.random.default_rng(5)
+    n = 300000
+    e = np.minimum(rng.geometric(0.45, n) + 100, 254).astype(np.uint16)
+    m = rng.integers(0, 128, n).astype(np.uint16)
+    s = rng.integers(0, 2, n).astype(np.uint16)
+    data = ((s << 15) | (e << 7) | m).astype(np.uint16).view(np.uint8)
+    p, cb, hist, cont = _gpu_round_trip(zc.FMT_BF16, data, n, 16384, zc.POLICY_AUTO)
+    assert cb.get(0)[1].max() == 12
+
+
+def test_static_dictionary_and_missing_code():
+    a = _weights(zc.FMT_BF16, 50000, 1)
+    b = _weights(zc.FMT_BF16, 50000, 2)
+    ha = zo.histogram(zo.BF16, a, 50000)
+    _gpu_round_trip(zc.FMT_BF16, b, 50000, 8192, zc.POLICY_HUFF_ALL, oracle_codebook_hist=ha + 1)
+    # a symbol without a code: the device reports it
+    p = zc.plan(zc.FMT_BF16, 50000, 8192)
+    cb = zc.build_codebook(p, ha, zc.POLICY_HUFF_ALL)
+    missing = int(np.flatnonzero(ha[0] == 0)[0])
+    bad = b.copy().view(np.uint16); bad[777] = missing << 7
+    d_in = torch.from_numpy(bad.view(np.uint8)).to(DEV)
+    d_out = torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=DEV)
+    d_ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress(p, cb, d_in, d_out, d_ws)
+    assert e.value.status == zc.E_NO_CODE
+
+
+def test_decoder_accepts_oracle_containers_and_flags_damage():
+    n = 70000
+    data = _weights(zc.FMT_BF16, n, 3)
+    hist = zo.histogram(zo.BF16, data, n)
+    for policy in (zo.POLICY_AUTO, zo.POLICY_HUFF_ALL):
+        cont = zo.compress(zo.BF16, data, n, 8192, zo.build_codebook(hist, policy))
+        p = zc.plan(zc.FMT_BF16, n, 8192)
+        d_ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+        d_back = torch.zeros(p.input_bytes, dtype=torch.uint8, device=DEV)
+        d_c = torch.from_numpy(cont).to(DEV)
+        zc.decompress(p, d_c, cont.size, d_back, d_ws)
+        assert zc.device_status(p, d_ws) == zc.OK
+        assert np.array_equal(d_back.cpu().numpy(), data)
+        # header damage and table damage are reported, never trapped on
+        hd = zo.parse_header(cont)
+        sec = hd["streams"][0]["section_off"]
+        used = int(np.flatnonzero(cont[sec:sec + 256])[0])
+        tab = sec + 256 + ((4 * hd["n_chunks"] + 15) // 16) * 16
+        for off, val in ((0, 0x58), (6, 2), (8, 1), (17, 0x40), (64, 7), (sec + used, 13), (tab + 4 * 31 + 2, 0xFF)):
+            bad = cont.copy(); bad[off] = val
+            zc.decompress(p, torch.from_numpy(bad).to(DEV), bad.size, d_back, d_ws)
+            assert zc.device_status(p, d_ws) == zc.E_CORRUPT, off
+        # a plan that does not match
+        p2 = zc.plan(zc.FMT_BF16, n + 1, 8192)
+        d_ws2 = torch.empty(p2.workspace_bytes, dtype=torch.uint8, device=DEV)
+        d_back2 = torch.zeros(p2.input_bytes, dtype=torch.uint8, device=DEV)
+        zc.decompress(p2, d_c, cont.size, d_back2, d_ws2)
+        assert zc.device_status(p2, d_ws2) == zc.E_CORRUPT
+
+
+def test_argument_checks():
+    p = zc.plan(zc.FMT_BF16, 1000, 1024)
+    d = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    ws = torch.zeros(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+    cb = zc.build_codebook(p, np.ones((2, 256)), zc.POLICY_AUTO)
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress(p, cb, d, d[:100], ws)
+    assert e.value.status == zc.E_BUFFER_TOO_SMALL
+    big = torch.zeros(p.max_compressed_bytes + 16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress(p, cb, d[1:], big, ws)                            # misaligned input
+    assert e.value.status == zc.E_INVALID_ARG
+
+
+def test_small_versions_of_the_five_configurations():
+    for name, fmt, t, n in wl.small_cases(DEV):
+        data = t.cpu().numpy()
+        for chunk_bytes in (8192, 65536):
+            for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL):
+                _gpu_round_trip(fmt, data, n, chunk_bytes, policy)
+
+
+def test_config1_exact():
+    """Config 1 in full: 1024x1024 FP8 E4M3, N(0, 0.02), per-tensor scale, seed 0, 64 KiB chunks."""
+    t, n = wl.config1_tensor(DEV)
+    data = t.cpu().numpy()
+    p, cb, hist, cont = _gpu_round_trip(zc.FMT_FP8_E4M3, data, n, 65536, zc.POLICY_AUTO)
+    assert p.n_chunks == 16
+    assert cb.modes == [zc.MODE_HUFF, zc.MODE_RAW]
+    st = zc.stats(p, cb, hist, cont[:128])
+    assert 0.78 < st.ratio_container < 0.86                       # the paper's abstract quotes "up to 83%" for FP8
+
+
+def test_large_tensor_sampled_chunks():
+    """A tensor of bench size class (64 Mi BF16 elements, 16 KiB chunks): the oracle checks sampled chunks
+    one by one, properties cover the rest."""
+    n = 1 << 26
+    g = torch.Generator(device=DEV); g.manual_seed(123)
+    x = (torch.randn(n, generator=g, device=DEV) * 0.02).to(torch.bfloat16)
+    d_in = x.view(torch.uint8)
+    chunk_bytes = 16384
+    p = zc.plan(zc.FMT_BF16, n, chunk_bytes)
+    hist = zc.histogram(p, d_in).cpu().numpy().astype(np.uint64)
+    assert int(hist[0].sum()) == n and int(hist[1].sum()) == n
+    cb = zc.build_codebook(p, hist, zc.POLICY_AUTO)
+    d_out = torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=DEV)
+    d_ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+    nbytes = zc.compress(p, cb, d_in, d_out, d_ws)
+    cont = d_out[:nbytes].cpu().numpy()
+    assert zc.validate_container(p, cont) == zc.OK
+    hd = zo.parse_header(cont)
+    mode0, lens0, _ = cb.get(0)
+    assert hd["streams"][0]["payload_bits"] == int((hist[0].astype(np.int64) * lens0).sum())
+    data = d_in.cpu().numpy()
+    rng = np.random.default_rng(0)
+    for c in [0, 1, p.n_chunks - 1] + [int(v) for v in rng.integers(0, p.n_chunks, 12)]:
+        got = zo.decompress_chunk(cont, c, chunk_bytes)
+        assert np.array_equal(got, data[c * chunk_bytes:(c + 1) * chunk_bytes])
+    d_back = torch.empty(p.input_bytes, dtype=torch.uint8, device=DEV)
+    zc.decompress(p, d_out, nbytes, d_back, d_ws)
+    assert zc.device_status(p, d_ws) == zc.OK
+    assert torch.equal(d_back, d_in)
