@@ -316,6 +316,8 @@ def run_ours(args):
     # ---- end to end with host buffers: H2D of the inputs and D2H of the containers inside the timed region ----
     e2e = None
     try:
+        if args.no_e2e:
+            raise RuntimeError("skipped (--no-e2e)")
         h_in = [t["in"].cpu().pin_memory() for t in tensors]
         h_out = [torch.empty(t["cbytes"], dtype=torch.uint8).pin_memory() for t in tensors]
 
@@ -403,6 +405,7 @@ def main():
     ap.add_argument("--workload", default="cfg2_bf16_llama8b")
     ap.add_argument("--chunk-kib", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

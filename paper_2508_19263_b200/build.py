@@ -8,8 +8,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libzc.so")
-SOURCES = ["zc_host.cpp", "zc_kernels.cu"]
-HEADERS = ["zc_internal.h", "zc_bits.cuh"]
+SOURCES = ["zc_host.cpp", "zc_hist.cu", "zc_encode.cu", "zc_decode.cu"]
+HEADERS = ["zc_internal.h", "zc_bits.cuh", "zc_device.cuh"]
 
 
 def _nvcc() -> str:

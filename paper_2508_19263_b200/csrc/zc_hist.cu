@@ -1,0 +1,89 @@
+// Split + histogram kernel and zc_histogram.
+#include "zc_device.cuh"
+
+namespace zc {
+
+constexpr int kHistThreads = 256;
+
+// ------------------------------------------------------------------------------------------------
+// split + histogram
+// ------------------------------------------------------------------------------------------------
+// Each lane of a warp owns its own copy of every bin (bins[stream][symbol][lane]): the bank of an
+// update is the lane number, so updates of one warp never collide, however skewed the exponent
+// distribution is.  The 64 KiB of bins are shared by the warps of the block through shared atomics.
+
+template <int FMT>
+__global__ void __launch_bounds__(kHistThreads)
+hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_syms, unsigned long long* __restrict__ hist)
+{
+    extern __shared__ uint32_t bins[];           // [2][256][32]
+    const uint32_t lane = threadIdx.x & 31;
+    for (uint32_t i = threadIdx.x; i < 2 * 256 * 32; i += kHistThreads) bins[i] = 0;
+    __syncthreads();
+
+    const uint64_t n_vec = (n_syms + 7) / 8;     // 16 input bytes = 8 symbols of each stream
+    for (uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x; v < n_vec; v += (uint64_t)gridDim.x * kHistThreads) {
+        const uint4 x = load16_guarded(in, 16 * v, input_bytes);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+        uint32_t e[2], sm[2];
+        split16<FMT>(w, e, sm);
+        const uint64_t left = n_syms - 8 * v;
+        const uint32_t nv = left < 8 ? (uint32_t)left : 8u;
+        if (nv == 8) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t a = (e[i >> 2] >> (8 * (i & 3))) & 0xFF;
+                const uint32_t b = (sm[i >> 2] >> (8 * (i & 3))) & 0xFF;
+                atomicAdd(&bins[a * 32 + lane], 1u);
+                atomicAdd(&bins[(256 + b) * 32 + lane], 1u);
+            }
+        } else {
+            for (uint32_t i = 0; i < nv; ++i) {
+                const uint32_t a = (e[i >> 2] >> (8 * (i & 3))) & 0xFF;
+                const uint32_t b = (sm[i >> 2] >> (8 * (i & 3))) & 0xFF;
+                atomicAdd(&bins[a * 32 + lane], 1u);
+                atomicAdd(&bins[(256 + b) * 32 + lane], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < 512; b += kHistThreads) {
+        uint32_t sum = 0;
+#pragma unroll 8
+        for (uint32_t i = 0; i < 32; ++i) sum += bins[b * 32 + ((i + lane) & 31)];
+        if (sum) atomicAdd(&hist[b], (unsigned long long)sum);
+    }
+}
+
+}  // namespace zc
+
+using namespace zc;
+
+extern "C" {
+
+zc_status zc_histogram(const zc_plan_t* p, const void* d_in, uint64_t* d_hist, void* cuda_stream)
+{
+    if (!p || !d_hist || (!d_in && p->n_elems) || !aligned16(d_in)) return ZC_E_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(d_hist, 0, 2 * 256 * sizeof(uint64_t), st) != cudaSuccess) return ZC_E_CUDA;
+    if (p->n_syms == 0) return ZC_OK;
+    const size_t smem = 2 * 256 * 32 * sizeof(uint32_t);
+    const uint64_t n_vec = (p->n_syms + 7) / 8;
+    const uint64_t want = (n_vec + kHistThreads * 8 - 1) / (kHistThreads * 8);
+    const uint32_t grid = (uint32_t)std::min<uint64_t>(std::max<uint64_t>(want, 1), (uint64_t)sm_count() * 3);
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kern) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return;
+        kern<<<grid, kHistThreads, smem, st>>>((const uint8_t*)d_in, p->input_bytes, p->n_syms, (unsigned long long*)d_hist);
+        e = cudaGetLastError();
+    };
+    switch (p->format) {
+    case ZC_FMT_BF16: launch(hist_kernel<ZC_FMT_BF16>); break;
+    case ZC_FMT_FP8_E4M3: launch(hist_kernel<ZC_FMT_FP8_E4M3>); break;
+    default: launch(hist_kernel<ZC_FMT_FP4_E2M1>); break;
+    }
+    return e == cudaSuccess ? ZC_OK : ZC_E_CUDA;
+}
+
+}  // extern "C"
