@@ -115,6 +115,20 @@ ZC_HD void split16(const uint32_t in[4], uint32_t e[2], uint32_t sm[2])
 template <int FMT>
 ZC_HD void merge16(const uint32_t e[2], const uint32_t sm[2], uint32_t out[4])
 {
+    if (FMT == ZC_FMT_BF16) {
+        // element = sign | exponent << 7 | mantissa.  The exponent byte goes to bits 14..7 (placed in byte 1
+        // and shifted right by one); the sign+mantissa byte is duplicated into both bytes so that its bit 7
+        // lands on bit 15 and its bits 6..0 on bits 6..0; one select picks each bit from the right source.
+        const uint32_t m = 0x7F807F80u;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t xl = byte_perm(e[h], 0, 0x1404) >> 1, yl = byte_perm(sm[h], 0, 0x1100);
+            const uint32_t xh = byte_perm(e[h], 0, 0x3424) >> 1, yh = byte_perm(sm[h], 0, 0x3322);
+            out[2 * h] = (xl & m) | (yl & ~m);
+            out[2 * h + 1] = (xh & m) | (yh & ~m);
+        }
+        return;
+    }
     out[0] = Fields<FMT>::merge_word(spread_lo(e[0]), spread_lo(sm[0]));
     out[1] = Fields<FMT>::merge_word(spread_hi(e[0]), spread_hi(sm[0]));
     out[2] = Fields<FMT>::merge_word(spread_lo(e[1]), spread_lo(sm[1]));

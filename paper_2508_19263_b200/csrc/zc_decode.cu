@@ -19,21 +19,22 @@ struct DecParams {
     uint32_t pool_bytes;     // per-warp shared memory: symbol rows first, the rest stages compressed pieces
 };
 
-constexpr uint32_t kWideLutBytes = kLutEntries * 8;   // stream 0: up to 4 symbols per lookup
-constexpr uint32_t kNarrowLutBytes = kLutEntries * 4; // stream 1: up to 2 symbols per lookup
+constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
 constexpr uint32_t kScratchBytes = 1024;
-constexpr uint32_t kDecFixedSmem = kWideLutBytes + kNarrowLutBytes + kScratchBytes;
+constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
+constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
 
-__device__ __forceinline__ uint2 lds64(uint32_t addr)
+__device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void sts8_if(bool p, uint32_t addr, uint32_t v)
-{
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u8 [%0], %1;\n\t}"
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}"
                  :: "r"(addr), "r"(v), "r"((uint32_t)p) : "memory");
+}
+__device__ __forceinline__ uint32_t lds32_if(bool p, uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\tmov.u32 %0, 0;\n\t@q ld.shared.u32 %0, [%1];\n\t}"
+                 : "=r"(v) : "r"(addr), "r"((uint32_t)p));
+    return v;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -71,12 +72,18 @@ __device__ __forceinline__ uint32_t walk_code(uint32_t window12, const CodeBook&
     return 0;
 }
 
-// Fills the table of one stream.  WIDE: 8-byte entries {symbols (up to 4, low byte first), len | cnt << 8};
-// otherwise 4-byte entries len | cnt << 8 | sym1 << 16 | sym2 << 24.  `single` is a 4096 x u16 scratch table.
-// Every entry yields at least one symbol, so a decoding lane always advances.  Returns false to all
-// threads if the lengths are not a complete prefix code (or the one-symbol code).
-template <bool WIDE>
-__device__ bool build_lut(const uint8_t* __restrict__ code_len, uint8_t* lut, uint16_t* single, uint32_t* scratch)
+// Fills the table of one stream and decides how many symbols every lookup yields (returned in *per_lookup).
+//   entry bits  7..0  bits the lookup consumes      15..8 first symbol     23..16 second symbol
+//              27..24 length of the first code       31   "only the first symbol is valid" (2-symbol mode)
+// Two-symbol mode: a lookup normally yields the two symbols whose codes start the 12-bit window; when the two
+// codes together are longer than 12 bits the entry carries the first one and bit 31, and the decoder fetches
+// the second with one more lookup.  That mode is chosen when such pairs are rare (estimated from the code
+// lengths with p(symbol) = 2^-length); otherwise every lookup yields exactly one symbol.  A fixed number of
+// symbols per lookup lets a lane assemble words of 4 symbols in registers without any bookkeeping.
+// `single` is a 4096 x u16 scratch table.  Returns false to all threads if the lengths are not a complete
+// prefix code (or the one-symbol code).
+__device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, uint16_t* single, uint32_t* scratch,
+                          uint32_t* per_lookup)
 {
     const CodeBook b = codebook_views(scratch);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -111,8 +118,15 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint8_t* lut, ui
         const bool complete = kraft == (1ull << kLmax);
         const bool one = active == 1 && b.count[1] == 1;
         if (!(complete || one || active == 0)) *b.ok = 0;
+        // probability (in units of 2^-24) that two consecutive codes need more than 12 bits
+        uint64_t long_pairs = 0;
+        for (uint32_t l1 = 1; l1 <= kLmax; ++l1)
+            for (uint32_t l2 = kLmax + 1 - l1; l2 <= kLmax; ++l2)
+                long_pairs += ((uint64_t)b.count[l1] << (kLmax - l1)) * ((uint64_t)b.count[l2] << (kLmax - l2));
+        b.ok[1] = long_pairs <= (1ull << 24) / 32 ? 2u : 1u;
     }
     __syncthreads();
+    const uint32_t mode = b.ok[1];
     if (tid < 256 && my_len) b.sorted[b.offset[my_len] + b.wcount[warp * 16 + my_len] + my_rank] = (uint8_t)tid;
     __syncthreads();
     // one symbol per window; a window no code matches (possible only for the one-symbol code) reads as
@@ -124,21 +138,19 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint8_t* lut, ui
     }
     __syncthreads();
     for (uint32_t idx = tid; idx < kLutEntries; idx += blockDim.x) {
-        uint32_t rest = idx, total = 0, cnt = 0, syms = 0;
-#pragma unroll
-        for (int k = 0; k < (WIDE ? 4 : 2); ++k) {
-            const uint32_t e = single[rest];
-            const uint32_t l = e >> 8;
-            if (k > 0 && total + l > kLmax) break;
-            syms |= (e & 0xFF) << (8 * k);
-            total += l;
-            ++cnt;
-            rest = (rest << l) & (kLutEntries - 1);
+        const uint32_t e1 = single[idx];
+        const uint32_t l1 = e1 >> 8, s1 = e1 & 0xFF;
+        uint32_t e = l1 | (s1 << 8) | (l1 << 24);
+        if (mode == 2) {
+            const uint32_t e2 = single[(idx << l1) & (kLutEntries - 1)];
+            const uint32_t l2 = e2 >> 8, s2 = e2 & 0xFF;
+            if (l1 + l2 <= kLmax) e = (l1 + l2) | (s1 << 8) | (s2 << 16) | (l1 << 24);
+            else e |= 0x80000000u;
         }
-        if (WIDE) reinterpret_cast<uint2*>(lut)[idx] = make_uint2(syms, total | (cnt << 8));
-        else reinterpret_cast<uint32_t*>(lut)[idx] = total | (cnt << 8) | (syms << 16);
+        lut[idx] = e;
     }
     __syncthreads();
+    if (tid == 0) *per_lookup = mode;
     return *b.ok != 0;
 }
 
@@ -147,64 +159,94 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint8_t* lut, ui
 // ------------------------------------------------------------------------------------------------
 
 struct LaneStream {
-    uint32_t pos;         // next bit of my subchunk, counted from the start of the chunk's piece
-    uint32_t carry_n;     // symbols already decoded beyond the previous round (0..3)
-    uint32_t carry_syms;  // those symbols, first one in the low byte
+    uint32_t hi, lo;        // bit buffer: the next bit is the top bit of hi; bits below `valid` are zero
+    uint32_t valid;         // number of valid bits in the buffer
+    uint32_t ptr_s;         // shared address of the next payload word (piece staged in shared memory)
+    const uint32_t* ptr_g;  // or its global address (piece read from global memory)
 };
 
-// Decode until `target` symbols sit in the lane's row.  Each pass loads a 32-bit window at the current
-// bit and does two table lookups (a lookup consumes at most 12 bits); all symbol bytes of an entry are
-// stored and the write position advances by the number that is valid.
-template <bool WIDE, bool STAGED>
-__device__ __forceinline__ void decode_round(LaneStream& st, uint32_t pay_s, const uint32_t* __restrict__ pay_g,
-                                             uint32_t lut_s, uint32_t row_s, uint32_t target)
+// Point the lane at bit `start` of the chunk's piece.
+template <bool STAGED>
+__device__ __forceinline__ void lane_begin(LaneStream& st, uint32_t pay_s, const uint32_t* __restrict__ pay_g, uint32_t start)
 {
-    uint32_t out = st.carry_n;
-    if (out) sts32(row_s, st.carry_syms);
-    uint32_t pos = st.pos;
-    uint32_t last_syms = 0, last_meta = 0;
-    while (out < target) {
-        const uint32_t w = pos >> 5;
-        uint32_t hi, lo;
-        if (STAGED) { hi = lds32(pay_s + 4 * w); lo = lds32(pay_s + 4 * w + 4); }
-        else { hi = __ldg(pay_g + w); lo = __ldg(pay_g + w + 1); }
-        uint32_t win = __funnelshift_l(lo, hi, pos);
-        uint32_t syms, meta;
-        if (WIDE) {
-            const uint2 e = lds64(lut_s + ((win >> (29 - kLmax)) & (8 * kLutEntries - 8)));
-            syms = e.x; meta = e.y;
-        } else {
-            const uint32_t e = lds32(lut_s + ((win >> (30 - kLmax)) & (4 * kLutEntries - 4)));
-            syms = e >> 16; meta = e & 0xFFFF;
-        }
-        const uint32_t a = row_s + out;
-        sts8(a, syms); sts8(a + 1, syms >> 8);
-        if (WIDE) { sts8(a + 2, syms >> 16); sts8(a + 3, syms >> 24); }
-        out += meta >> 8;
-        win = __funnelshift_l(0, win, meta);               // shift count = low 5 bits = bits consumed
-        uint32_t used = meta;
-        last_syms = syms; last_meta = meta;
-        const bool more = out < target;
-        {
-            uint32_t syms2, meta2;
-            if (WIDE) {
-                const uint2 e = lds64(lut_s + ((win >> (29 - kLmax)) & (8 * kLutEntries - 8)));
-                syms2 = e.x; meta2 = e.y;
-            } else {
-                const uint32_t e = lds32(lut_s + ((win >> (30 - kLmax)) & (4 * kLutEntries - 4)));
-                syms2 = e >> 16; meta2 = e & 0xFFFF;
+    const uint32_t w = start >> 5;
+    uint32_t w0, w1;
+    if (STAGED) { w0 = lds32(pay_s + 4 * w); w1 = lds32(pay_s + 4 * w + 4); st.ptr_s = pay_s + 4 * w + 8; }
+    else { w0 = __ldg(pay_g + w); w1 = __ldg(pay_g + w + 1); st.ptr_g = pay_g + w + 2; }
+    st.hi = __funnelshift_l(w1, w0, start);
+    st.lo = __funnelshift_l(0, w1, start);
+    st.valid = 64 - (start & 31);
+}
+
+// Top the 64-bit buffer up with one word when 32 bits or fewer are left: at least 33 are valid afterwards,
+// enough for two lookups of at most 12 bits each.
+template <bool STAGED>
+__device__ __forceinline__ void lane_refill(LaneStream& st)
+{
+    const bool need = st.valid <= 32;
+    uint32_t word = 0;
+    if (STAGED) { if (need) word = lds32(st.ptr_s); st.ptr_s += need ? 4 : 0; }
+    else { if (need) word = __ldg(st.ptr_g); st.ptr_g += need ? 1 : 0; }
+    st.hi |= __funnelshift_rc(word, 0, st.valid);               // word >> valid (0 when valid == 32)
+    st.lo |= __funnelshift_rc(0, word, st.valid);               // word << (32 - valid)
+    st.valid += need ? 32 : 0;
+}
+
+__device__ __forceinline__ uint32_t lane_peek(const LaneStream& st, uint32_t lut_s)
+{
+    return lds32(lut_s + ((st.hi >> (30 - kLmax)) & (4 * kLutEntries - 4)));
+}
+__device__ __forceinline__ void lane_consume(LaneStream& st, uint32_t n)    // n < 32 in its low 5 bits
+{
+    st.hi = __funnelshift_l(st.lo, st.hi, n);
+    st.lo = __funnelshift_l(0, st.lo, n);
+}
+
+// Decode n_words words of 4 symbols into the lane's row.  K = symbols per lookup (1 or 2).
+// One-symbol mode: top up, two lookups, top up, two lookups.  Two-symbol mode: top up, two lookups; a lookup
+// whose second code did not fit the window (bit 31 of the entry, rare by construction of the mode) tops up
+// again and takes the second symbol from the next window.
+template <int K, bool STAGED>
+__device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+{
+    for (uint32_t i = 0; i < n_words; ++i) {
+        uint32_t word;
+        if (K == 2) {
+            lane_refill<STAGED>(st);
+            uint32_t pair[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t e = lane_peek(st, lut_s);
+                lane_consume(st, e);
+                st.valid -= e & 0xFF;
+                if ((int)e < 0) {
+                    lane_refill<STAGED>(st);
+                    const uint32_t f = lane_peek(st, lut_s);
+                    const uint32_t l = (f >> 24) & 15;
+                    lane_consume(st, l);
+                    st.valid -= l;
+                    e = (e & 0xFF00u) | ((f & 0xFF00u) << 8);
+                }
+                pair[h] = e;
             }
-            const uint32_t a2 = row_s + out;
-            sts8_if(more, a2, syms2); sts8_if(more, a2 + 1, syms2 >> 8);
-            if (WIDE) { sts8_if(more, a2 + 2, syms2 >> 16); sts8_if(more, a2 + 3, syms2 >> 24); }
-            if (more) { out += meta2 >> 8; used += meta2; last_syms = syms2; last_meta = meta2; }
+            word = __byte_perm(pair[0], pair[1], 0x6521);
+        } else {
+            lane_refill<STAGED>(st);
+            const uint32_t a = lane_peek(st, lut_s);
+            lane_consume(st, a);
+            const uint32_t b = lane_peek(st, lut_s);
+            lane_consume(st, b);
+            st.valid -= (a + b) & 0xFF;
+            lane_refill<STAGED>(st);
+            const uint32_t c = lane_peek(st, lut_s);
+            lane_consume(st, c);
+            const uint32_t d = lane_peek(st, lut_s);
+            lane_consume(st, d);
+            st.valid -= (c + d) & 0xFF;
+            word = __byte_perm(__byte_perm(a, b, 0x0051), __byte_perm(c, d, 0x0051), 0x5410);
         }
-        pos += used & 0xFF;
+        sts32(row_s + 4 * i, word);
     }
-    st.pos = pos;
-    const uint32_t extra = out - target;                     // symbols of the last entry that belong to the next round
-    st.carry_n = extra;
-    st.carry_syms = extra ? last_syms >> (8 * ((last_meta >> 8) - extra)) : 0u;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -213,7 +255,7 @@ __device__ __forceinline__ void decode_round(LaneStream& st, uint32_t pay_s, con
 // PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
 
 template <int FMT, int PPL>
-__global__ void __launch_bounds__(1024, 1)
+__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
 decode_kernel(const __grid_constant__ DecParams P)
 {
     constexpr uint32_t R = 16 * PPL;
@@ -222,16 +264,16 @@ decode_kernel(const __grid_constant__ DecParams P)
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
 
-    uint8_t* lut0 = smem;                                      // wide table of stream 0
-    uint8_t* lut1 = smem + kWideLutBytes;                      // narrow table of stream 1
-    uint32_t* scratch = reinterpret_cast<uint32_t*>(smem + kWideLutBytes + kNarrowLutBytes);
+    uint32_t* lut0 = reinterpret_cast<uint32_t*>(smem);                 // decode table of stream 0
+    uint32_t* lut1 = reinterpret_cast<uint32_t*>(smem + kLutBytes);     // decode table of stream 1
+    uint32_t* scratch = reinterpret_cast<uint32_t*>(smem + 2 * kLutBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecFixedSmem);
     uint8_t* pools = reinterpret_cast<uint8_t*>(bars + 2 * n_warps);
     uint8_t* pool = pools + (size_t)warp * P.pool_bytes;
     uint64_t* bar = bars + 2 * warp;
 
     // ---- header check against the plan ----
-    __shared__ uint32_t s_mode[2];
+    __shared__ uint32_t s_mode[2], s_per_lookup[2];
     __shared__ uint32_t s_ok;
     __shared__ unsigned long long s_payload_off, s_payload_bytes, s_sec[2];
     if (threadIdx.x == 0) {
@@ -275,8 +317,9 @@ decode_kernel(const __grid_constant__ DecParams P)
         // the warps' pools are free until the main loop: 8 KiB of them hold the one-symbol scratch table
         uint16_t* single = reinterpret_cast<uint16_t*>(pools);
         bool tables_ok = true;
-        if (huff0) tables_ok = build_lut<true>(P.comp + s_sec[0], lut0, single, scratch) && tables_ok;
-        if (huff1) tables_ok = build_lut<false>(P.comp + s_sec[1], lut1, single, scratch) && tables_ok;
+        if (huff0) tables_ok = build_lut(P.comp + s_sec[0], lut0, single, scratch, &s_per_lookup[0]) && tables_ok;
+        if (huff1) tables_ok = build_lut(P.comp + s_sec[1], lut1, single, scratch, &s_per_lookup[1]) && tables_ok;
+        __syncthreads();
         if (!tables_ok) { if (threadIdx.x == 0) raise_status(P.ctl, ZC_E_CORRUPT); return; }
     }
 
@@ -295,6 +338,7 @@ decode_kernel(const __grid_constant__ DecParams P)
     const uint32_t slot1_s = slot0_s + (huff0 ? slot_bytes : 0);
     const uint32_t rows0_s = smem_u32(pool + rows0_off), rows1_s = smem_u32(pool + rows1_off);
     const uint32_t lut0_s = smem_u32(lut0), lut1_s = smem_u32(lut1);
+    const bool pairs0 = huff0 && s_per_lookup[0] == 2, pairs1 = huff1 && s_per_lookup[1] == 2;
     const uint32_t step = gridDim.x * n_warps;
     uint32_t parity0 = 0, parity1 = 0;
     uint32_t err = 0;
@@ -319,7 +363,8 @@ decode_kernel(const __grid_constant__ DecParams P)
         const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
 
         // ---- where my subchunk starts and where the chunk's pieces are; check, then stage ----
-        LaneStream st0{0, 0, 0}, st1{0, 0, 0};
+        LaneStream st0{0, 0, 0, 0, nullptr}, st1{0, 0, 0, 0, nullptr};
+        uint32_t start0 = 0, start1 = 0;
         const uint32_t* pay0_g = nullptr;
         const uint32_t* pay1_g = nullptr;
         bool staged0 = false, staged1 = false;
@@ -333,7 +378,7 @@ decode_kernel(const __grid_constant__ DecParams P)
             piece0 = ((chunk_bits + 127) / 128) * 16;
             ok = ok && start <= my_end && my_end <= chunk_bits && my_end - start <= n_my * kLmax &&
                  16ull * off16 + piece0 <= payload_bytes;
-            st0.pos = start;
+            start0 = start;
             pay0_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
         }
         if (huff1) {
@@ -344,7 +389,7 @@ decode_kernel(const __grid_constant__ DecParams P)
             piece1 = ((chunk_bits + 127) / 128) * 16;
             ok = ok && start <= my_end && my_end <= chunk_bits && my_end - start <= n_my * kLmax &&
                  16ull * off16 + piece1 <= payload_bytes;
-            st1.pos = start;
+            start1 = start;
             pay1_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
         }
         if (!__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; break; }
@@ -402,20 +447,25 @@ decode_kernel(const __grid_constant__ DecParams P)
                     parity1 ^= 1;
                 }
                 if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                if (n_my) {
+                    if (huff0) { if (staged0) lane_begin<true>(st0, slot0_s, nullptr, start0); else lane_begin<false>(st0, 0, pay0_g, start0); }
+                    if (huff1) { if (staged1) lane_begin<true>(st1, slot1_s, nullptr, start1); else lane_begin<false>(st1, 0, pay1_g, start1); }
+                }
             }
             // ---- every lane decodes R symbols of its subchunk ----
             const uint32_t done = r * R;
             const uint32_t target = n_my > done ? min(R, n_my - done) : 0u;
-            if (target) {
+            const uint32_t n_words = (target + 3) / 4;          // a ragged last word decodes up to 3 symbols too many
+            if (n_words) {
                 if (huff0) {
                     const uint32_t row_s = rows0_s + lane * kRowStride;
-                    if (staged0) decode_round<true, true>(st0, slot0_s, nullptr, lut0_s, row_s, target);
-                    else decode_round<true, false>(st0, 0, pay0_g, lut0_s, row_s, target);
+                    if (staged0) { if (pairs0) decode_words<2, true>(st0, lut0_s, row_s, n_words); else decode_words<1, true>(st0, lut0_s, row_s, n_words); }
+                    else { if (pairs0) decode_words<2, false>(st0, lut0_s, row_s, n_words); else decode_words<1, false>(st0, lut0_s, row_s, n_words); }
                 }
                 if (huff1) {
                     const uint32_t row_s = rows1_s + lane * kRowStride;
-                    if (staged1) decode_round<false, true>(st1, slot1_s, nullptr, lut1_s, row_s, target);
-                    else decode_round<false, false>(st1, 0, pay1_g, lut1_s, row_s, target);
+                    if (staged1) { if (pairs1) decode_words<2, true>(st1, lut1_s, row_s, n_words); else decode_words<1, true>(st1, lut1_s, row_s, n_words); }
+                    else { if (pairs1) decode_words<2, false>(st1, lut1_s, row_s, n_words); else decode_words<1, false>(st1, lut1_s, row_s, n_words); }
                 }
             }
             __syncwarp();
@@ -444,8 +494,7 @@ decode_kernel(const __grid_constant__ DecParams P)
                 const uint32_t byte = 2 * k;
                 uint8_t* dst = P.out + out_lo + byte;
                 if (byte + 32 <= out_bytes) {
-                    st_cs_v4(dst, make_uint4(o[0], o[1], o[2], o[3]));
-                    st_cs_v4(dst + 16, make_uint4(o[4], o[5], o[6], o[7]));
+                    st_cs_v8(dst, o);
                 } else {
 #pragma unroll
                     for (int t = 0; t < 32; ++t)
@@ -495,15 +544,15 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     P.pool_bytes = std::max<uint32_t>(rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32, 2 * rows_bytes);
     const size_t fixed = kDecFixedSmem + 64 /* static shared */;
     size_t per_warp = 16 + P.pool_bytes;
-    uint32_t warps = (uint32_t)std::min<size_t>(32, (kMaxSmem - fixed - 1024) / per_warp);
+    uint32_t warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     if (warps < 8) {                 // large chunks: stage less
         P.pool_bytes = std::max<uint32_t>(rows_bytes + 4096 + 32, 2 * rows_bytes);
         per_warp = 16 + P.pool_bytes;
-        warps = (uint32_t)std::min<size_t>(32, (kMaxSmem - fixed - 1024) / per_warp);
+        warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     }
     // the table build uses 8 KiB of the pools and 256 threads
     while (warps * (size_t)P.pool_bytes < 8192) ++warps;
-    if (warps < 8 || warps > 32) return ZC_E_UNSUPPORTED;
+    if (warps < 8 || warps > kDecMaxWarps) return ZC_E_UNSUPPORTED;
     const size_t smem = kDecFixedSmem + warps * per_warp;
     // at least one block even for an empty tensor: the header is still checked
     const uint32_t want = std::max<uint32_t>((p->n_chunks + warps - 1) / warps, 1);

@@ -7,7 +7,8 @@ namespace zc {
 // encoder
 // ------------------------------------------------------------------------------------------------
 
-struct EncTables { uint32_t enc[2][256]; };     // (length << 16) | code value; 0 = symbol has no code
+// Per symbol: the code left-aligned in bits 31..20 and its length in bits 3..0; a symbol without a code is 16.
+struct EncTables { uint32_t enc[2][256]; };
 
 struct EncParams {
     const uint8_t* in;
@@ -19,7 +20,8 @@ struct EncParams {
     uint32_t mode[2];
     uint32_t format, group;
     Layout lay;
-    uint32_t stage_stride;                       // bytes of one stream's symbol staging per warp
+    uint32_t stage_stride;                       // bytes of one coded stream's lane regions per warp
+    uint32_t region_bytes;                       // one lane region: 1.5 * sub + 4
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
 };
 
@@ -76,11 +78,28 @@ __device__ bool lookback_exclusive(unsigned long long* flags, uint32_t c, uint32
     return true;
 }
 
-// Symbol k of a chunk is staged at byte k + 4 * (k / sub): subchunk regions are padded by 4 bytes
-// so that lanes walking their own regions hit different banks.
+// Per-warp shared memory of one coded stream: 32 lane regions of 1.5 * sub bytes (+4 bytes of padding, which
+// also makes the region stride an odd number of words so that lanes walking their regions hit different
+// banks).  A region first holds the subchunk's symbols in its upper two thirds; the lane then packs the codes
+// into the same region from its start.  Codes are at most 12 bits, so after k symbols at most 1.5 k bytes are
+// written while the read position is 0.5 * sub + k: the write position never passes unread symbols.
+
+// Append `len` bits (given left-aligned in `code`, zero below them) to a lane's bit accumulator and write a
+// full 32-bit word to the region when one is complete.  hi holds the nb (< 32) pending bits left-aligned.
+__device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& hi, uint32_t& nb, uint32_t& waddr)
+{
+    hi |= code >> nb;
+    const uint32_t lo = __funnelshift_r(0, code, nb);           // the bits that do not fit: code << (32 - nb), 0 if nb == 0
+    const uint32_t n = nb + len;
+    const bool full = n >= 32;
+    if (full) sts32(waddr, hi);
+    waddr += full ? 4 : 0;
+    hi = full ? lo : hi;
+    nb = n & 31;
+}
 
 template <int FMT>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(1024, 1)
 encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTables T)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -88,19 +107,19 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     const bool huff0 = P.mode[0] == ZC_MODE_HUFF, huff1 = P.mode[1] == ZC_MODE_HUFF;
     const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
 
-    // shared: enc[2][256] | per warp: sub_bits[2][32] | per warp: staging[n_huff][stage_stride]
+    // shared: enc[2][256] | per warp: regions[n_huff][stage_stride]
     uint32_t* enc = reinterpret_cast<uint32_t*>(smem);
-    uint32_t* sub_bits_all = enc + 512;
-    uint8_t* stage_all = reinterpret_cast<uint8_t*>(sub_bits_all + 64 * n_warps);
+    uint8_t* stage_all = smem + 2048;
     for (uint32_t i = threadIdx.x; i < 512; i += blockDim.x) enc[i] = T.enc[i >> 8][i & 255];
-    uint32_t* sub_bits = sub_bits_all + 64 * warp;
     uint8_t* stage = stage_all + (size_t)warp * n_huff * P.stage_stride;
+    const uint32_t region = P.region_bytes;                     // 1.5 * sub + 4
+    const uint32_t sym_off = P.sub / 2;                         // symbols sit at this offset inside a region
 
     // block 0 writes the static parts of the table sections and the tail padding of raw bodies
     if (blockIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
             if (P.mode[s] == ZC_MODE_HUFF) {
-                for (uint32_t v = threadIdx.x; v < 256; v += blockDim.x) P.out[P.lay.section_off[s] + v] = (uint8_t)(T.enc[s][v] >> 16);
+                for (uint32_t v = threadIdx.x; v < 256; v += blockDim.x) P.out[P.lay.section_off[s] + v] = (uint8_t)(T.enc[s][v] & 15);
                 const uint32_t padded = (P.n_chunks + 3) & ~3u;
                 for (uint32_t i = P.n_chunks + threadIdx.x; i < padded; i += blockDim.x)
                     reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[i] = 0;
@@ -112,7 +131,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     }
     __syncthreads();
 
-    uint32_t first_bad = 0;
+    uint32_t bad = 0;
     while (true) {
         uint32_t c = 0;
         if (lane == 0) c = atomicAdd(&P.ctl->ticket, 1u);
@@ -121,11 +140,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         const uint64_t c_lo = (uint64_t)c * P.cs;
         const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
 
-        sub_bits[lane] = 0;
-        sub_bits[32 + lane] = 0;
-        __syncwarp();
-
-        // ---- phase A: coalesced load, split, raw stores, symbol staging, code-length sums ----
+        // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
         const uint32_t n_vec = (c_syms + 7) / 8;
         for (uint32_t it = lane; it < n_vec; it += 32) {
             const uint32_t k = it * 8;
@@ -133,26 +148,14 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
             uint32_t sy[2][2];
             split16<FMT>(w, sy[0], sy[1]);
-            const uint32_t nv = min(8u, c_syms - k);
             uint32_t hs = 0;
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] == ZC_MODE_RAW) {
                     st_cs_v2(P.out + P.lay.section_off[s] + c_lo + k, make_uint2(sy[s][0], sy[s][1]));
                 } else {
-                    uint32_t acc = 0, bad = 0;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint32_t v = (sy[s][i >> 2] >> (8 * (i & 3))) & 0xFF;
-                        const uint32_t e = (uint32_t)i < nv ? enc[256 * s + v] : 0x10000u;
-                        bad |= (e == 0);
-                        acc += e;
-                    }
-                    if (bad) first_bad = ZC_E_NO_CODE;
-                    const uint32_t bits = (acc >> 16) - (8 - nv);       // codes < 2^12: their sum stays below bit 16
                     const uint32_t j = __umulhi(k, P.sub_magic);          // subchunk of these 8 symbols
-                    atomicAdd(&sub_bits[32 * hs + j], bits);
-                    uint32_t* st = reinterpret_cast<uint32_t*>(stage + hs * P.stage_stride + k + 4 * j);
+                    uint32_t* st = reinterpret_cast<uint32_t*>(stage + hs * P.stage_stride + j * region + sym_off + (k - j * P.sub));
                     st[0] = sy[s][0];
                     st[1] = sy[s][1];
                     ++hs;
@@ -161,21 +164,60 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         }
         __syncwarp();
 
-        // ---- phase B: subchunk end bits, piece sizes, position of the chunk in the payload area ----
-        uint32_t my_bits[2] = {0, 0}, my_end[2] = {0, 0}, piece16[2] = {0, 0};
+        // ---- phase B: every lane packs the codes of its subchunk into its own region, from bit 0 ----
+        const uint32_t lo_sym = lane * P.sub;
+        const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
+        uint32_t my_bits[2] = {0, 0};
+        {
+            uint32_t hs = 0;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                if (P.mode[s] != ZC_MODE_HUFF) continue;
+                const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
+                const uint32_t tab_s = smem_u32(enc + 256 * s);
+                uint32_t hi = 0, nb = 0, waddr = reg_s, seen = 0;
+                const uint32_t src = reg_s + sym_off;
+                const uint32_t full_words = n_my / 4;
+                for (uint32_t i = 0; i < full_words; ++i) {
+                    const uint32_t four = lds32(src + 4 * i);
+                    const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
+                    const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
+                    const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
+                    const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
+                    seen |= e0 | e1 | e2 | e3;
+                    // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
+                    // first entry = its length); the length fields end up below bit 8 and are masked off
+                    const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
+                    put_bits(ca, (e0 + e1) & 31, hi, nb, waddr);
+                    const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
+                    put_bits(cb, (e2 + e3) & 31, hi, nb, waddr);
+                }
+                for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
+                    const uint32_t four = lds32(src + (i & ~3u));
+                    const uint32_t e = lds32(tab_s + (((four >> (8 * (i & 3))) & 0xFF) << 2));
+                    seen |= e;
+                    put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr);
+                }
+                sts32(waddr, hi);                                       // pending bits (or zero)
+                my_bits[hs] = 8 * (waddr - reg_s) + nb;
+                bad |= seen & 16;                                       // an entry without a code carries bit 4
+                ++hs;
+            }
+        }
+
+        // ---- phase C: subchunk end bits, piece sizes, position of the chunk in the payload area ----
+        uint32_t my_end[2] = {0, 0}, piece16[2] = {0, 0};
         uint64_t tot16 = 0;
         {
             uint32_t hs = 0;
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
-                const uint32_t b = sub_bits[32 * hs + lane];
-                uint32_t inc = b;
+                uint32_t inc = my_bits[hs];
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
                     if (lane >= (uint32_t)o) inc += t;
                 }
-                my_bits[hs] = b;
                 my_end[hs] = inc;
                 reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * c)[lane] = inc;
                 const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
@@ -193,7 +235,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
             }
         }
 
-        // ---- phase C: each lane packs its subchunk at its final bit position ----
+        // ---- phase D: every lane moves its bits to their final position in the chunk's piece ----
         {
             uint32_t hs = 0;
             uint64_t piece_off16 = off16;
@@ -202,7 +244,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                 if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[c] = (uint32_t)piece_off16;
                 uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
                 const uint32_t piece_words = 4 * piece16[hs];
-                const uint32_t end = my_end[hs], start = end - my_bits[hs];
+                const uint32_t end = my_end[hs], bits = my_bits[hs], start = end - bits;
                 const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
                 // words shared between neighbours (and the padding) start from zero and are OR-ed into
                 if ((start >> 5) < piece_words) piece[start >> 5] = 0;
@@ -212,49 +254,31 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                     if (32ull * w >= chunk_bits) piece[w] = 0;
                 }
                 __syncwarp();
-
-                const uint32_t lo_sym = lane * P.sub;
-                const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
-                const uint8_t* src = stage + hs * P.stage_stride + lo_sym + 4 * lane;
-                const uint32_t* tab = enc + 256 * s;
-                uint64_t acc = 0;
-                uint32_t nb = start & 31, wi = start >> 5;
-                bool first = true;
-                for (uint32_t i = 0; i < n_my; i += 4) {
-                    const uint32_t four = *reinterpret_cast<const uint32_t*>(src + i);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (i + q < n_my) {
-                            const uint32_t e = tab[(four >> (8 * q)) & 0xFF];
-                            const uint32_t l = e >> 16;
-                            acc = (acc << l) | (e & 0xFFFF);
-                            nb += l;
-                        }
-                        if ((q & 1) && nb >= 32) {            // two codes add at most 24 bits to at most 31 pending
-                            const uint32_t word = (uint32_t)(acc >> (nb - 32));
-                            if (first) { atomicOr(&piece[wi], word); first = false; }
-                            else piece[wi] = word;
-                            ++wi;
-                            nb -= 32;
-                        }
+                if (bits) {
+                    const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
+                    const uint32_t sh = start & 31, d0 = start >> 5;
+                    const uint32_t n_dst = (sh + bits + 31) / 32;         // destination words I touch
+                    const uint32_t n_src = (bits + 31) / 32;
+                    uint32_t prev = 0;
+                    for (uint32_t i = 0; i < n_dst; ++i) {
+                        const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
+                        const uint32_t v = __funnelshift_r(cur, prev, sh);  // (prev:cur) >> sh, low word
+                        prev = cur;
+                        // the first word may hold the previous lane's bits, a ragged last word the next lane's
+                        const bool shared_word = i == 0 || (i == n_dst - 1 && ((sh + bits) & 31) != 0);
+                        if (shared_word) atomicOr(&piece[d0 + i], v);
+                        else piece[d0 + i] = v;
                     }
                 }
-                if (nb >= 32) {                                // cannot happen (flushed after every pair), kept for safety
-                    const uint32_t word = (uint32_t)(acc >> (nb - 32));
-                    atomicOr(&piece[wi], word);
-                    ++wi; nb -= 32;
-                }
-                if (nb && my_bits[hs]) atomicOr(&piece[wi], (uint32_t)(acc << (32 - nb)));
                 piece_off16 += piece16[hs];
                 ++hs;
             }
         }
         __syncwarp();
-
         // the warp that owns the last chunk knows the size of the whole payload area
         if (lane == 0 && c == P.n_chunks - 1) P.ctl->total16 = off16 + tot16;
     }
-    if (first_bad) raise_status(P.ctl, first_bad);
+    if (bad) raise_status(P.ctl, ZC_E_NO_CODE);
 }
 
 // Writes the 128-byte header and the guard once every chunk is in place (stream order guarantees it).
@@ -320,20 +344,22 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         n_huff += P.mode[s] == ZC_MODE_HUFF;
     }
     P.lay = make_layout(*p, P.mode);
-    P.stage_stride = p->syms_per_chunk + 4 * kSubs;
+    P.region_bytes = p->syms_per_sub + p->syms_per_sub / 2 + 4;
+    P.stage_stride = kSubs * P.region_bytes;
     P.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
 
     EncTables T;
     for (int s = 0; s < 2; ++s)
-        for (int v = 0; v < 256; ++v) T.enc[s][v] = cb->len[s][v] ? ((uint32_t)cb->len[s][v] << 16) | cb->code[s][v] : 0u;
+        for (int v = 0; v < 256; ++v)
+            T.enc[s][v] = cb->len[s][v] ? (cb->code[s][v] << (32 - cb->len[s][v])) | cb->len[s][v] : 16u;
 
     if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * p->n_chunks, st) != cudaSuccess) return ZC_E_CUDA;
 
     cudaError_t e = cudaSuccess;
     if (p->n_chunks) {
         const size_t fixed = 512 * sizeof(uint32_t);
-        const size_t per_warp = 64 * sizeof(uint32_t) + (size_t)n_huff * P.stage_stride;
-        uint32_t warps = (uint32_t)std::min<size_t>(16, (kMaxSmem - fixed - 1024) / per_warp);
+        const size_t per_warp = std::max<size_t>((size_t)n_huff * P.stage_stride, 16);
+        uint32_t warps = (uint32_t)std::min<size_t>(32, (kMaxSmem - fixed - 1024) / per_warp);
         if (warps == 0) return ZC_E_UNSUPPORTED;
         const size_t smem = fixed + warps * per_warp;
         // resident blocks per SM by shared memory (leave 1 KiB per block for the system) and threads
