@@ -76,7 +76,8 @@ typedef enum zc_status {
     ZC_E_CUDA = 5,              /* a CUDA runtime call failed */
     ZC_E_NOMEM = 6,             /* host allocation failed */
     ZC_E_DEVICE_TIMEOUT = 7,    /* a bounded wait inside a kernel gave up */
-    ZC_E_NO_CODE = 8            /* a symbol of the input has no code in the codebook */
+    ZC_E_NO_CODE = 8,           /* a symbol of the input has no code in the codebook */
+    ZC_E_TOO_LARGE = 9          /* the tensor needs more built-in scratch than zc_compress_noalloc has */
 } zc_status;
 
 typedef enum zc_format {
@@ -183,6 +184,38 @@ zc_status zc_codebook_get(const zc_codebook_t* cb, uint32_t stream, uint32_t* mo
  * Errors: INVALID_ARG, BUFFER_TOO_SMALL, CUDA, and the device status when synchronous. */
 zc_status zc_compress(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, void* d_out,
                       size_t out_capacity, void* d_workspace, uint64_t* h_out_bytes, void* cuda_stream);
+
+/* ---- compress without a caller-supplied workspace ------------------------------------------
+ * (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ *
+ * Same operation and same result, byte for byte, as zc_compress, but the device scratch that
+ * zc_compress takes as `d_workspace` lives inside the library: a fixed array in device memory
+ * of ZC_NOALLOC_SCRATCH_BYTES bytes that every GPU loading the library holds until the process
+ * exits.  It is meant for code that runs where cudaMalloc is off limits or unaffordable: inside
+ * a memory pool that has handed out all of its budget, in a latency-critical serving loop that
+ * must not touch the allocator, or in a plugin that is only given input and output buffers.
+ * The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ * d_in, d_out, out_capacity, h_out_bytes, cuda_stream: exactly as for zc_compress (the caller
+ * still owns and passes input and output).
+ *
+ * Limit: the plan may have at most ZC_NOALLOC_MAX_CHUNKS chunks (n_chunks of zc_plan_info);
+ * larger tensors are refused with ZC_E_TOO_LARGE and nothing is launched.  Use a larger
+ * chunk_bytes, split the tensor, or call zc_compress with your own workspace.
+ *
+ * First call on a device: the library looks up the device address of its scratch array once
+ * per device (with that device current) and remembers it.  Make that first call outside of
+ * any stream capture.
+ *
+ * Sharing: all calls on one device use the same scratch array.  Each call clears the part it
+ * needs before use, so stale contents of an earlier call never matter, but two calls whose
+ * GPU work overlaps in time (different streams, or different host threads) race on it and
+ * corrupt each other's containers.  Serialise such calls on one stream.
+ * Errors: as zc_compress, plus ZC_E_TOO_LARGE. */
+#define ZC_NOALLOC_MAX_CHUNKS 65536u
+#define ZC_NOALLOC_SCRATCH_BYTES (256u + 8u * ZC_NOALLOC_MAX_CHUNKS)
+zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, void* d_out,
+                              size_t out_capacity, uint64_t* h_out_bytes, void* cuda_stream);
 
 /* ---- decompress (Sec. 3.1 "parallel decoding") --------------------------------------------
  * d_comp      device, a container made for the same plan; comp_bytes = bytes available

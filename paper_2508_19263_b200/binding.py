@@ -21,7 +21,9 @@ from . import build as _build
 FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 1, 2, 3
 POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL = 0, 1, 2
 MODE_RAW, MODE_HUFF = 0, 1
-OK, E_INVALID_ARG, E_UNSUPPORTED, E_BUFFER_TOO_SMALL, E_CORRUPT, E_CUDA, E_NOMEM, E_DEVICE_TIMEOUT, E_NO_CODE = range(9)
+(OK, E_INVALID_ARG, E_UNSUPPORTED, E_BUFFER_TOO_SMALL, E_CORRUPT, E_CUDA, E_NOMEM, E_DEVICE_TIMEOUT, E_NO_CODE,
+ E_TOO_LARGE) = range(10)
+NOALLOC_MAX_CHUNKS = 65536
 
 
 class ZcError(RuntimeError):
@@ -75,6 +77,8 @@ def _load():
     L.zc_codebook_get.argtypes = [vp, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint8), C.POINTER(C.c_uint32)]
     L.zc_compress.restype = C.c_int
     L.zc_compress.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, u64p, vp]
+    L.zc_compress_noalloc.restype = C.c_int
+    L.zc_compress_noalloc.argtypes = [vp, vp, vp, vp, C.c_size_t, u64p, vp]
     L.zc_decompress.restype = C.c_int
     L.zc_decompress.argtypes = [vp, vp, C.c_size_t, vp, vp, vp]
     L.zc_device_status.restype = C.c_int
@@ -189,6 +193,19 @@ def compress(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Tensor, d_w
     st = _lib.zc_compress(p._h, cb._h, d_in.data_ptr(), d_out.data_ptr(), d_out.numel() * d_out.element_size(),
                           d_workspace.data_ptr(), C.byref(n) if sync else None, _stream_ptr(stream))
     _check(st, "zc_compress")
+    return n.value if sync else None
+
+
+def compress_noalloc(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Tensor, sync: bool = True,
+                     stream=None) -> Optional[int]:
+    """zc_compress_noalloc: like compress() but without a workspace argument.  The scratch is a fixed array
+    inside the library (at most NOALLOC_MAX_CHUNKS chunks; larger plans raise E_TOO_LARGE).  For callers that
+    may not allocate device memory.  Calls that overlap on the GPU must not be issued: they share the scratch."""
+    assert d_in.is_cuda and d_out.is_cuda
+    n = C.c_uint64(0)
+    st = _lib.zc_compress_noalloc(p._h, cb._h, d_in.data_ptr(), d_out.data_ptr(), d_out.numel() * d_out.element_size(),
+                                  C.byref(n) if sync else None, _stream_ptr(stream))
+    _check(st, "zc_compress_noalloc")
     return n.value if sync else None
 
 

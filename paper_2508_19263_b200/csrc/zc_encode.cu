@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(1024, 1)
 encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTables T)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool huff0 = P.mode[0] == ZC_MODE_HUFF, huff1 = P.mode[1] == ZC_MODE_HUFF;
     const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
 
@@ -391,6 +391,44 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         *h_out_bytes = h.total16;
     }
     return ZC_OK;
+}
+
+// ---- compression without a caller-supplied workspace ---------------------------------------------
+// The scratch zc_compress needs (control block + one look-back word per chunk) for up to
+// ZC_NOALLOC_MAX_CHUNKS chunks, resident in every GPU that loads the library.  Host code must not pass
+// this symbol to a kernel: on the host its name is only a stand-in, the device address comes from
+// cudaGetSymbolAddress and differs per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ZC_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device; looked up once per device.
+zc_status noalloc_scratch(void** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ZC_E_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return ZC_E_CUDA;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return ZC_OK;
+}
+}  // namespace
+
+zc_status zc_compress_noalloc(const zc_plan_t* p, const zc_codebook_t* cb, const void* d_in, void* d_out,
+                              size_t out_capacity, uint64_t* h_out_bytes, void* cuda_stream)
+{
+    if (!p) return ZC_E_INVALID_ARG;
+    if (p->n_chunks > ZC_NOALLOC_MAX_CHUNKS || zc_workspace_bytes(p) > ZC_NOALLOC_SCRATCH_BYTES) return ZC_E_TOO_LARGE;
+    void* scratch = nullptr;
+    const zc_status st = noalloc_scratch(&scratch);
+    if (st != ZC_OK) return st;
+    // zc_compress clears the control block and the look-back words it uses before launching
+    return zc_compress(p, cb, d_in, d_out, out_capacity, scratch, h_out_bytes, cuda_stream);
 }
 
 zc_status zc_device_status(const zc_plan_t* p, const void* d_workspace, void* cuda_stream)

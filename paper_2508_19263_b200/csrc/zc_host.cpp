@@ -353,6 +353,7 @@ const char* zc_strerror(zc_status s)
     case ZC_E_NOMEM: return "out of host memory";
     case ZC_E_DEVICE_TIMEOUT: return "a bounded wait on the device gave up";
     case ZC_E_NO_CODE: return "an input symbol has no code in the codebook";
+    case ZC_E_TOO_LARGE: return "tensor has more chunks than the built-in scratch of zc_compress_noalloc covers";
     default: return "unknown status";
     }
 }
