@@ -228,10 +228,22 @@ def run_ours(args):
     d_hist = torch.zeros((n_t, 2, 256), dtype=torch.int64, device=dev)
     h_hist = torch.zeros((n_t, 2, 256), dtype=torch.int64).pin_memory()
     stream = torch.cuda.current_stream()
+    side = [torch.cuda.Stream(device=dev) for _ in range(max(args.streams - 1, 0))]
+    lanes = [stream] + side                      # per-tensor calls go round robin over these streams
+
+    def fork():
+        for s in side:
+            s.wait_stream(stream)
+
+    def join():
+        for s in side:
+            stream.wait_stream(s)
 
     def phase_hist():
+        fork()
         for i, t in enumerate(tensors):
-            zc.histogram(t["plan"], t["in"], d_hist[i])
+            zc.histogram(t["plan"], t["in"], d_hist[i], stream=lanes[i % len(lanes)])
+        join()
         h_hist.copy_(d_hist, non_blocking=True)
         stream.synchronize()
 
@@ -241,12 +253,16 @@ def run_ours(args):
             t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
 
     def phase_compress():
-        for t in tensors:
-            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False)
+        fork()
+        for i, t in enumerate(tensors):
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=lanes[i % len(lanes)])
+        join()
 
     def phase_decompress():
-        for t in tensors:
-            zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"])
+        fork()
+        for i, t in enumerate(tensors):
+            zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"], stream=lanes[i % len(lanes)])
+        join()
 
     def read_sizes():
         torch.cuda.synchronize()
@@ -260,11 +276,14 @@ def run_ours(args):
         # next codebook while the GPU is busy with the previous tensors
         phase_hist()
         hh = h_hist.numpy()
+        fork()
         for i, t in enumerate(tensors):
+            ln = lanes[i % len(lanes)]
             t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
-            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False)
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=ln)
             # the decoder only needs an upper bound of the container size; the header carries the exact one
-            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"])
+            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], stream=ln)
+        join()
 
     def timed(fn, reps):
         barrier()
@@ -383,7 +402,8 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.workload, "tensors": n_t, "uncompressed_bytes": U, "compressed_bytes": C,
-                   "chunk_kib": args.chunk_kib, "policy": "auto", "l2": "inputs larger than L2 (no flush)"},
+                   "chunk_kib": args.chunk_kib, "policy": "auto", "streams": args.streams,
+                   "l2": "inputs larger than L2 (no flush)"},
         "decode": dec, "encode": enc, "histogram": hist, "codebook_host_ms": ms_codebook,
         "compression_ratio": {"total_container": C / U, "exponent_stream_payload": st_bits[0] / (8 * n_syms),
                               "sign_mantissa_stream_payload": st_bits[1] / (8 * n_syms),
@@ -404,6 +424,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_bf16_llama8b")
     ap.add_argument("--chunk-kib", type=int, default=16)
+    ap.add_argument("--streams", type=int, default=1,
+                    help="CUDA streams the per-tensor calls are spread over (tails of one tensor's kernels overlap the next)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used for profiler captures)")
     args = ap.parse_args()

@@ -100,6 +100,18 @@ template <> struct Fields<ZC_FMT_FP4_E2M1> {
 template <int FMT>
 ZC_HD void split16(const uint32_t in[4], uint32_t e[2], uint32_t sm[2])
 {
+    if (FMT == ZC_FMT_BF16) {
+        // gather the four high bytes (sign, exponent bits 7..1) and the four low bytes (exponent bit 0,
+        // mantissa) of four elements, then recombine per byte lane
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t hb = byte_perm(in[2 * h], in[2 * h + 1], 0x7531);
+            const uint32_t lb = byte_perm(in[2 * h], in[2 * h + 1], 0x6420);
+            sm[h] = (lb & 0x7F7F7F7Fu) | (hb & 0x80808080u);
+            e[h] = ((hb << 1) & 0xFEFEFEFEu) | ((lb >> 7) & 0x01010101u);
+        }
+        return;
+    }
     uint32_t ea, sa, eb, sb;
     Fields<FMT>::split_word(in[0], ea, sa);
     Fields<FMT>::split_word(in[1], eb, sb);

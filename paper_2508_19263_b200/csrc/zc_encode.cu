@@ -141,10 +141,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
 
         // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
-        const uint32_t n_vec = (c_syms + 7) / 8;
-        for (uint32_t it = lane; it < n_vec; it += 32) {
-            const uint32_t k = it * 8;
-            const uint4 x = load16_guarded(P.in, 2 * (c_lo + k), P.input_bytes);
+        auto stage_group = [&](const uint4 x, const uint32_t k) {
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
             uint32_t sy[2][2];
             split16<FMT>(w, sy[0], sy[1]);
@@ -161,6 +158,24 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                     ++hs;
                 }
             }
+        };
+        const uint32_t n_vec = (c_syms + 7) / 8;
+        const uint8_t* src_c = P.in + 2 * c_lo;
+        uint32_t it = lane;
+        if (2 * (c_lo + 8ull * n_vec) <= P.input_bytes) {           // every group of this chunk is complete
+            for (; it + 96 < n_vec; it += 128) {                        // four loads in flight per lane
+                const uint4 x0 = ld_nc_v4(src_c + 16 * it);
+                const uint4 x1 = ld_nc_v4(src_c + 16 * (it + 32));
+                const uint4 x2 = ld_nc_v4(src_c + 16 * (it + 64));
+                const uint4 x3 = ld_nc_v4(src_c + 16 * (it + 96));
+                stage_group(x0, 8 * it);
+                stage_group(x1, 8 * (it + 32));
+                stage_group(x2, 8 * (it + 64));
+                stage_group(x3, 8 * (it + 96));
+            }
+            for (; it < n_vec; it += 32) stage_group(ld_nc_v4(src_c + 16 * it), 8 * it);
+        } else {
+            for (; it < n_vec; it += 32) stage_group(load16_guarded(P.in, 2 * (c_lo + 8ull * it), P.input_bytes), 8 * it);
         }
         __syncwarp();
 

@@ -12,6 +12,31 @@ constexpr int kHistThreads = 256;
 // update is the lane number, so updates of one warp never collide, however skewed the exponent
 // distribution is.  The 64 KiB of bins are shared by the warps of the block through shared atomics.
 
+__device__ __forceinline__ void red_add1(uint32_t addr)
+{
+    asm volatile("red.shared.add.u32 [%0], 1;" :: "r"(addr) : "memory");
+}
+
+// Count the 8 + 8 symbols of one 16-byte group.  lane_bins = shared address of bins[0][0][lane];
+// a symbol's counter is 128 bytes further per symbol value, stream 1 starts 32 KiB later.
+template <int FMT>
+__device__ __forceinline__ void count16(const uint4 x, uint32_t lane_bins)
+{
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    uint32_t e[2], sm[2];
+    split16<FMT>(w, e, sm);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t a = __byte_perm(e[h], 0, 0x4440 + q);
+            const uint32_t b = __byte_perm(sm[h], 0, 0x4440 + q);
+            red_add1(lane_bins + a * 128u);
+            red_add1(lane_bins + 32768u + b * 128u);
+        }
+    }
+}
+
 template <int FMT>
 __global__ void __launch_bounds__(kHistThreads)
 hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_syms, unsigned long long* __restrict__ hist)
@@ -20,30 +45,35 @@ hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_sym
     const uint32_t lane = threadIdx.x & 31;
     for (uint32_t i = threadIdx.x; i < 2 * 256 * 32; i += kHistThreads) bins[i] = 0;
     __syncthreads();
+    const uint32_t lane_bins = smem_u32(bins) + 4 * lane;
 
-    const uint64_t n_vec = (n_syms + 7) / 8;     // 16 input bytes = 8 symbols of each stream
-    for (uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x; v < n_vec; v += (uint64_t)gridDim.x * kHistThreads) {
-        const uint4 x = load16_guarded(in, 16 * v, input_bytes);
+    // groups of 16 input bytes = 8 symbols of each stream; complete groups first, four loads in flight
+    const uint64_t n_full = n_syms / 8 < input_bytes / 16 ? n_syms / 8 : input_bytes / 16;
+    const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
+    uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x;
+    for (; v + 3 * stride < n_full; v += 4 * stride) {
+        const uint4 x0 = ld_nc_v4(in + 16 * v);
+        const uint4 x1 = ld_nc_v4(in + 16 * (v + stride));
+        const uint4 x2 = ld_nc_v4(in + 16 * (v + 2 * stride));
+        const uint4 x3 = ld_nc_v4(in + 16 * (v + 3 * stride));
+        count16<FMT>(x0, lane_bins);
+        count16<FMT>(x1, lane_bins);
+        count16<FMT>(x2, lane_bins);
+        count16<FMT>(x3, lane_bins);
+    }
+    for (; v < n_full; v += stride) count16<FMT>(ld_nc_v4(in + 16 * v), lane_bins);
+    // the ragged last group (fewer than 8 symbols, or input bytes that end inside the group)
+    if (blockIdx.x == 0 && threadIdx.x == 0 && 8 * n_full < n_syms) {
+        const uint4 x = load16_guarded(in, 16 * n_full, input_bytes);
         const uint32_t w[4] = {x.x, x.y, x.z, x.w};
         uint32_t e[2], sm[2];
         split16<FMT>(w, e, sm);
-        const uint64_t left = n_syms - 8 * v;
-        const uint32_t nv = left < 8 ? (uint32_t)left : 8u;
-        if (nv == 8) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t a = (e[i >> 2] >> (8 * (i & 3))) & 0xFF;
-                const uint32_t b = (sm[i >> 2] >> (8 * (i & 3))) & 0xFF;
-                atomicAdd(&bins[a * 32 + lane], 1u);
-                atomicAdd(&bins[(256 + b) * 32 + lane], 1u);
-            }
-        } else {
-            for (uint32_t i = 0; i < nv; ++i) {
-                const uint32_t a = (e[i >> 2] >> (8 * (i & 3))) & 0xFF;
-                const uint32_t b = (sm[i >> 2] >> (8 * (i & 3))) & 0xFF;
-                atomicAdd(&bins[a * 32 + lane], 1u);
-                atomicAdd(&bins[(256 + b) * 32 + lane], 1u);
-            }
+        const uint32_t nv = (uint32_t)(n_syms - 8 * n_full);
+        for (uint32_t i = 0; i < nv && i < 8; ++i) {
+            const uint32_t a = (e[i >> 2] >> (8 * (i & 3))) & 0xFF;
+            const uint32_t b = (sm[i >> 2] >> (8 * (i & 3))) & 0xFF;
+            atomicAdd(&bins[a * 32 + lane], 1u);
+            atomicAdd(&bins[(256 + b) * 32 + lane], 1u);
         }
     }
     __syncthreads();
