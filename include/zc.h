@@ -42,7 +42,7 @@
  *   header, 128 bytes
  *      0 u32 magic "ZC10"   4 u16 version = 1   6 u8 format   7 u8 n_streams = 2
  *      8 u64 n_elems       16 u32 chunk_bytes  20 u32 n_chunks
- *     24 u8 12 (max code length)  25 u8 G  26 u8 32 (subchunks)  27 u8 0  28 u32 0
+ *     24 u8 12 (max code length)  25 u8 G  26 u8 32 (subchunks)  27 u8 bytes per sub_end entry  28 u32 0
  *     32 u64 total_bytes   40 u64 payload_off  48 u64 payload_bytes  56 u64 0
  *     64 + 32 s : u8 mode (0 RAW, 1 HUFF), 7 zero bytes, u64 n_syms,
  *                 u64 payload_bits, u64 section_off            (s = 0, 1)
@@ -50,7 +50,8 @@
  *      u8  code_len[256]            0 = symbol has no code
  *      u32 chunk_off16[n_chunks]    zero padded to a multiple of 16 bytes; offset of
  *                                   the chunk's bits from payload_off, in 16-byte units
- *      u32 sub_end[n_chunks][32]    end bit of every subchunk inside its chunk
+ *      sub_end[n_chunks][32]        end bit of every subchunk inside its chunk; u16 entries when
+ *                                   chunk_bytes <= 8192 (a chunk then holds < 65536 bits), else u32
  *   one body per RAW stream (stream order): n_syms symbol bytes, zero padded to 16
  *   payload area: for chunk 0, 1, ...: for each HUFF stream (stream order) the
  *      chunk's bits, zero padded to a multiple of 16 bytes

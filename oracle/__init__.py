@@ -258,12 +258,23 @@ def stream_stats(hist, lengths, mode: int) -> dict:
     return {k: getattr(st, k) for k, _ in _StreamStats._fields_ if k != "pad"}
 
 
+def read_tables(container, stream: int):
+    """chunk_off16[n_chunks] and sub_end[n_chunks][32] of a HUFF stream as int64 arrays (plain unpacking)."""
+    hd = parse_header(container)
+    c = np.ascontiguousarray(container, np.uint8)
+    sec, nc, w = hd["streams"][stream]["section_off"], hd["n_chunks"], hd["sub_end_bytes"]
+    off16 = np.frombuffer(c[sec + 256: sec + 256 + 4 * nc].tobytes(), "<u4").astype(np.int64)
+    tab = sec + 256 + ((4 * nc + 15) // 16) * 16
+    sub_end = np.frombuffer(c[tab: tab + 32 * w * nc].tobytes(), "<u2" if w == 2 else "<u4").reshape(nc, 32).astype(np.int64)
+    return off16, sub_end, tab
+
+
 def parse_header(container) -> dict:
     """Decode the 128-byte header into a dict (plain struct unpacking, for tests and reports)."""
     import struct
     b = bytes(np.ascontiguousarray(container, np.uint8)[:128])
-    magic, version, fmt, n_streams, n_elems, chunk_bytes, n_chunks, lmax, g, subs = struct.unpack_from(
-        "<4sHBBQIIBBB", b, 0)
+    magic, version, fmt, n_streams, n_elems, chunk_bytes, n_chunks, lmax, g, subs, sub_w = struct.unpack_from(
+        "<4sHBBQIIBBBB", b, 0)
     total, payload_off, payload_bytes = struct.unpack_from("<QQQ", b, 32)
     streams = []
     for s in range(2):
@@ -271,5 +282,5 @@ def parse_header(container) -> dict:
         ns, pbits, sec = struct.unpack_from("<QQQ", b, 64 + 32 * s + 8)
         streams.append(dict(mode=mode, n_syms=ns, payload_bits=pbits, section_off=sec))
     return dict(magic=magic, version=version, format=fmt, n_streams=n_streams, n_elems=n_elems,
-                chunk_bytes=chunk_bytes, n_chunks=n_chunks, l_max=lmax, group=g, subchunks=subs,
+                chunk_bytes=chunk_bytes, n_chunks=n_chunks, l_max=lmax, group=g, subchunks=subs, sub_end_bytes=sub_w,
                 total_bytes=total, payload_off=payload_off, payload_bytes=payload_bytes, streams=streams)

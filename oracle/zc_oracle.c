@@ -59,14 +59,15 @@
  *   header 128 B:
  *     0  u32 magic 'Z','C','1','0'   4 u16 version=1   6 u8 format  7 u8 n_streams=2
  *     8  u64 n_elems                16 u32 chunk_bytes 20 u32 n_chunks
- *     24 u8 L_max=12  25 u8 G  26 u8 subchunks=32  27 u8 0  28 u32 0
+ *     24 u8 L_max=12  25 u8 G  26 u8 subchunks=32  27 u8 bytes per sub_end entry (2 or 4)  28 u32 0
  *     32 u64 total_bytes  40 u64 payload_off  48 u64 payload_bytes  56 u64 0
  *     64 + 32*s: u8 mode (0 RAW, 1 HUFF), u8[7] 0, u64 n_syms, u64 payload_bits,
  *                u64 section_off
  *   for each HUFF stream, in stream order, its table section:
  *     u8  code_len[256]
  *     u32 chunk_off16[n_chunks]        (padded with zeros to a multiple of 16 B)
- *     u32 sub_end[n_chunks][32]        end bit of each subchunk inside its chunk
+ *     u16 or u32 sub_end[n_chunks][32] end bit of each subchunk inside its chunk; u16 when chunk_bytes <= 8192
+ *                                      (a chunk then has at most 4096 * 12 < 65536 bits), else u32
  *   for each RAW stream, in stream order: its n_syms symbol bytes, zero padded
  *     to a multiple of 16 B
  *   payload area at payload_off: for chunk 0,1,..: for each HUFF stream in
@@ -362,9 +363,23 @@ static uint32_t n_chunks_of(uint64_t n_syms, uint32_t chunk_bytes)
     return (uint32_t)((n_syms + cs - 1) / cs);
 }
 
-static uint64_t table_section_bytes(uint32_t n_chunks)
+/* bytes of one sub_end entry (reading R5: small chunks get the narrow table) */
+static uint32_t sub_end_width(uint32_t chunk_bytes) { return chunk_bytes <= 8192 ? 2u : 4u; }
+
+static uint64_t table_section_bytes(uint32_t n_chunks, uint32_t chunk_bytes)
 {
-    return 256 + round16(4ull * n_chunks) + 128ull * n_chunks;
+    return 256 + round16(4ull * n_chunks) + 32ull * sub_end_width(chunk_bytes) * n_chunks;
+}
+
+static void put_sub_end(uint8_t *tab, uint32_t width, uint32_t chunk, int j, uint32_t v)
+{
+    if (width == 2) put16(tab + 64ull * chunk + 2ull * j, v);
+    else put32(tab + 128ull * chunk + 4ull * j, v);
+}
+
+static uint32_t get_sub_end(const uint8_t *tab, uint32_t width, uint32_t chunk, int j)
+{
+    return width == 2 ? get16(tab + 64ull * chunk + 2ull * j) : get32(tab + 128ull * chunk + 4ull * j);
 }
 
 static int valid_chunk_bytes(uint32_t cb) { return cb >= 1024 && cb <= 262144 && cb % 1024 == 0; }
@@ -377,7 +392,7 @@ uint64_t zo_container_bound(int fmt, uint64_t n_elems, uint32_t chunk_bytes)
     uint32_t nc = n_chunks_of(ns, chunk_bytes);
     uint64_t cs = chunk_bytes / 2;
     uint64_t worst_chunk = round16((cs * ZO_LMAX + 7) / 8);
-    uint64_t huff = table_section_bytes(nc) + (uint64_t)nc * worst_chunk;
+    uint64_t huff = table_section_bytes(nc, chunk_bytes) + (uint64_t)nc * worst_chunk;
     uint64_t raw = round16(ns);
     return ZO_HEADER + 2 * (huff > raw ? huff : raw) + 16;
 }
@@ -420,7 +435,7 @@ int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk
 
     /* section offsets */
     uint64_t off = ZO_HEADER, sec[2] = {0, 0};
-    for (int s = 0; s < 2; ++s) if (mode[s] == ZO_HUFF) { sec[s] = off; off += table_section_bytes(nc); }
+    for (int s = 0; s < 2; ++s) if (mode[s] == ZO_HUFF) { sec[s] = off; off += table_section_bytes(nc, chunk_bytes); }
     for (int s = 0; s < 2; ++s) if (mode[s] == ZO_RAW) { sec[s] = off; off += round16(ns); }
     uint64_t payload_off = off;
     int any_huff = (mode[0] == ZO_HUFF) || (mode[1] == ZO_HUFF);
@@ -464,7 +479,7 @@ int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk
                     for (unsigned b = 0; b < l; ++b, ++bit)          /* most significant code bit first */
                         if ((cw >> (l - 1 - b)) & 1) set_bit(out + piece_off, bit);
                 }
-                put32(sub_end + 128ull * c + 4ull * j, (uint32_t)bit);
+                put_sub_end(sub_end, sub_end_width(chunk_bytes), c, j, (uint32_t)bit);
             }
             pbits[s] += bits;
             pos16 += piece_bytes / 16;
@@ -482,7 +497,7 @@ int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk
     put64(h + 8, n_elems);
     put32(h + 16, chunk_bytes);
     put32(h + 20, nc);
-    h[24] = ZO_LMAX; h[25] = (uint8_t)g; h[26] = ZO_SUBS;
+    h[24] = ZO_LMAX; h[25] = (uint8_t)g; h[26] = ZO_SUBS; h[27] = (uint8_t)sub_end_width(chunk_bytes);
     put64(h + 32, total);
     put64(h + 40, payload_off);
     put64(h + 48, payload_bytes);
@@ -521,6 +536,7 @@ static int parse_header(const uint8_t *c, uint64_t bytes, zo_header *h)
     h->chunk_bytes = get32(c + 16);
     h->n_chunks = get32(c + 20);
     if (!valid_chunk_bytes(h->chunk_bytes)) return -1;
+    if (c[27] != sub_end_width(h->chunk_bytes)) return -1;
     h->n_syms = zo_n_syms(h->fmt, h->n_elems);
     if (h->n_chunks != n_chunks_of(h->n_syms, h->chunk_bytes)) return -1;
     h->total = get64(c + 32);
@@ -534,7 +550,7 @@ static int parse_header(const uint8_t *c, uint64_t bytes, zo_header *h)
         if (get64(d + 8) != h->n_syms) return -1;
         h->pbits[s] = get64(d + 16);
         h->sec[s] = get64(d + 24);
-        uint64_t need = h->mode[s] == ZO_HUFF ? table_section_bytes(h->n_chunks) : round16(h->n_syms);
+        uint64_t need = h->mode[s] == ZO_HUFF ? table_section_bytes(h->n_chunks, h->chunk_bytes) : round16(h->n_syms);
         if (h->sec[s] < ZO_HEADER || h->sec[s] > h->total || need > h->total - h->sec[s]) return -1;
     }
     return 0;
@@ -605,7 +621,8 @@ static int decode_chunk_stream(const uint8_t *cont, const zo_header *h, int s, u
     const uint8_t *chunk_off = cont + h->sec[s] + 256;
     const uint8_t *sub_end = cont + h->sec[s] + 256 + round16(4ull * h->n_chunks);
     uint64_t off16 = get32(chunk_off + 4ull * c);
-    uint64_t chunk_bits = get32(sub_end + 128ull * c + 4 * (ZO_SUBS - 1));
+    const uint32_t sw = sub_end_width(h->chunk_bytes);
+    uint64_t chunk_bits = get_sub_end(sub_end, sw, c, ZO_SUBS - 1);
     uint64_t piece_bytes = round16((chunk_bits + 7) / 8);
     if (16 * off16 > h->payload_bytes || piece_bytes > h->payload_bytes - 16 * off16) return -1;
     const uint8_t *piece = cont + h->payload_off + 16 * off16;
@@ -614,7 +631,7 @@ static int decode_chunk_stream(const uint8_t *cont, const zo_header *h, int s, u
         uint64_t lo = c_lo + (uint64_t)j * sub, hi = lo + sub;
         if (lo > c_hi) lo = c_hi;
         if (hi > c_hi) hi = c_hi;
-        uint64_t end = get32(sub_end + 128ull * c + 4ull * j);
+        uint64_t end = get_sub_end(sub_end, sw, c, j);
         if (end < start || end > chunk_bits) return -1;
         uint64_t pos = start;
         for (uint64_t k = lo; k < hi; ++k) {
@@ -679,7 +696,7 @@ int64_t zo_decompress(const uint8_t *cont, uint64_t bytes, uint8_t *out, uint64_
         for (int s = 0; s < 2; ++s)
             if (h.mode[s] == ZO_HUFF) {
                 const uint8_t *sub_end = cont + h.sec[s] + 256 + round16(4ull * h.n_chunks);
-                used[s] += get32(sub_end + 128ull * c + 4 * (ZO_SUBS - 1));
+                used[s] += get_sub_end(sub_end, sub_end_width(h.chunk_bytes), c, ZO_SUBS - 1);
             }
     }
     for (int s = 0; s < 2; ++s)

@@ -158,6 +158,12 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, u
 // per-lane decoding of one round
 // ------------------------------------------------------------------------------------------------
 
+__device__ __forceinline__ uint32_t load_sub_end(const uint8_t* tab, uint32_t width, uint32_t chunk, uint32_t lane)
+{
+    if (width == 2) return reinterpret_cast<const uint16_t*>(tab + 64ull * chunk)[lane];
+    return reinterpret_cast<const uint32_t*>(tab + 128ull * chunk)[lane];
+}
+
 struct LaneStream {
     uint32_t hi, lo;        // bit buffer: the next bit is the top bit of hi; bits below `valid` are zero
     uint32_t valid;         // number of valid bits in the buffer
@@ -272,6 +278,7 @@ decode_kernel(const __grid_constant__ DecParams P)
     uint8_t* pool = pools + (size_t)warp * P.pool_bytes;
     uint64_t* bar = bars + 2 * warp;
 
+    const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;     // bytes per sub_end entry
     // ---- header check against the plan ----
     __shared__ uint32_t s_mode[2], s_per_lookup[2];
     __shared__ uint32_t s_ok;
@@ -282,7 +289,8 @@ decode_kernel(const __grid_constant__ DecParams P)
         const unsigned long long* h64 = reinterpret_cast<const unsigned long long*>(h);
         bool ok = h32[0] == kMagic && h[kHdrVersion] == 1 && h[kHdrVersion + 1] == 0 && h[kHdrFormat] == P.format &&
                   h[kHdrStreams] == 2 && h64[kHdrElems / 8] == P.n_elems && h32[kHdrChunkBytes / 4] == P.chunk_bytes &&
-                  h32[kHdrChunks / 4] == P.n_chunks && h[kHdrLmax] == kLmax && h[kHdrGroup] == P.group && h[kHdrSubs] == kSubs;
+                  h32[kHdrChunks / 4] == P.n_chunks && h[kHdrLmax] == kLmax && h[kHdrGroup] == P.group && h[kHdrSubs] == kSubs &&
+                  h[kHdrSubWidth] == sub_w;
         uint32_t mode[2] = {0, 0};
         for (int s = 0; s < 2 && ok; ++s) {
             const uint8_t* d = h + kHdrStream0 + kHdrStreamStride * s;
@@ -292,7 +300,7 @@ decode_kernel(const __grid_constant__ DecParams P)
         if (ok) {
             // recompute where everything must be and compare with what the header says
             uint64_t off = kHeaderBytes, sec[2] = {0, 0};
-            const uint64_t tab = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 128ull * P.n_chunks;
+            const uint64_t tab = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * sub_w * P.n_chunks;
             for (int s = 0; s < 2; ++s) if (mode[s] == ZC_MODE_HUFF) { sec[s] = off; off += tab; }
             for (int s = 0; s < 2; ++s) if (mode[s] == ZC_MODE_RAW) { sec[s] = off; off += (P.n_syms + 15) & ~15ull; }
             const bool any_huff = mode[0] == ZC_MODE_HUFF || mode[1] == ZC_MODE_HUFF;
@@ -348,9 +356,9 @@ decode_kernel(const __grid_constant__ DecParams P)
     uint32_t c = blockIdx.x * n_warps + warp;
     uint32_t nx_end0 = 0, nx_off0 = 0, nx_end1 = 0, nx_off1 = 0;
     if (c < P.n_chunks) {
-        if (huff0) { nx_end0 = reinterpret_cast<const uint32_t*>(sec0 + tab_sub + 128ull * c)[lane];
+        if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, c, lane);
                      nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[c]; }
-        if (huff1) { nx_end1 = reinterpret_cast<const uint32_t*>(sec1 + tab_sub + 128ull * c)[lane];
+        if (huff1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, c, lane);
                      nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c]; }
     }
 
@@ -414,9 +422,9 @@ decode_kernel(const __grid_constant__ DecParams P)
         {
             const uint32_t cn = c + step;
             if (cn < P.n_chunks) {
-                if (huff0) { nx_end0 = reinterpret_cast<const uint32_t*>(sec0 + tab_sub + 128ull * cn)[lane];
+                if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
                              nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
-                if (huff1) { nx_end1 = reinterpret_cast<const uint32_t*>(sec1 + tab_sub + 128ull * cn)[lane];
+                if (huff1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
                              nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[cn]; }
             }
         }

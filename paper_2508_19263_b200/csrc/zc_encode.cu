@@ -22,6 +22,7 @@ struct EncParams {
     Layout lay;
     uint32_t stage_stride;                       // bytes of one coded stream's lane regions per warp
     uint32_t region_bytes;                       // one lane region: 1.5 * sub + 4
+    uint32_t sub_width;                          // bytes per sub_end entry (2 or 4)
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
 };
 
@@ -234,7 +235,8 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                     if (lane >= (uint32_t)o) inc += t;
                 }
                 my_end[hs] = inc;
-                reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * c)[lane] = inc;
+                if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * c)[lane] = (uint16_t)inc;
+                else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * c)[lane] = inc;
                 const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
                 piece16[hs] = (chunk_bits + 127) / 128;
                 tot16 += piece16[hs];
@@ -311,7 +313,7 @@ __global__ void finish_kernel(const EncParams P)
     h64[kHdrElems / 8] = P.n_elems;
     h32[kHdrChunkBytes / 4] = P.chunk_bytes;
     h32[kHdrChunks / 4] = P.n_chunks;
-    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)P.group; h[kHdrSubs] = kSubs;
+    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)P.group; h[kHdrSubs] = kSubs; h[kHdrSubWidth] = (uint8_t)P.sub_width;
     const uint64_t total = P.lay.payload_off + payload_bytes + (any_huff ? 16 : 0);
     h64[kHdrTotal / 8] = total;
     h64[kHdrPayloadOff / 8] = P.lay.payload_off;
@@ -360,6 +362,7 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
     }
     P.lay = make_layout(*p, P.mode);
     P.region_bytes = p->syms_per_sub + p->syms_per_sub / 2 + 4;
+    P.sub_width = sub_end_width(p->chunk_bytes);
     P.stage_stride = kSubs * P.region_bytes;
     P.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
 

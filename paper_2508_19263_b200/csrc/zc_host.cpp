@@ -149,7 +149,7 @@ size_t zc_max_compressed_bytes(const zc_plan_t* p)
 {
     if (!p) return 0;
     const uint64_t worst_piece = round_up(((uint64_t)p->syms_per_chunk * kLmax + 7) / 8, 16);
-    const uint64_t huff = table_section_bytes(p->n_chunks) + (uint64_t)p->n_chunks * worst_piece;
+    const uint64_t huff = table_section_bytes(p->n_chunks, p->chunk_bytes) + (uint64_t)p->n_chunks * worst_piece;
     const uint64_t raw = round_up(p->n_syms, 16);
     return (size_t)(kHeaderBytes + 2 * std::max(huff, raw) + 16);
 }
@@ -199,7 +199,8 @@ zc_status zc_validate_container(const zc_plan_t* p, const void* h_container, siz
     const uint8_t* c = (const uint8_t*)h_container;
     if (bytes < kHeaderBytes) return ZC_E_CORRUPT;
     if (rd(c + kHdrMagic, 4) != kMagic || rd(c + kHdrVersion, 2) != 1 || c[kHdrStreams] != 2) return ZC_E_CORRUPT;
-    if (c[kHdrFormat] != p->format || c[kHdrGroup] != p->group || c[kHdrLmax] != kLmax || c[kHdrSubs] != kSubs)
+    if (c[kHdrFormat] != p->format || c[kHdrGroup] != p->group || c[kHdrLmax] != kLmax || c[kHdrSubs] != kSubs ||
+        c[kHdrSubWidth] != sub_end_width(p->chunk_bytes))
         return ZC_E_CORRUPT;
     if (rd(c + kHdrElems, 8) != p->n_elems || rd(c + kHdrChunkBytes, 4) != p->chunk_bytes ||
         rd(c + kHdrChunks, 4) != p->n_chunks)
@@ -235,10 +236,11 @@ zc_status zc_validate_container(const zc_plan_t* p, const void* h_container, siz
         for (int s = 0; s < 2; ++s) {
             if (mode[s] != ZC_MODE_HUFF) continue;
             if (rd(c + L.chunk_off_tab[s] + 4ull * ch, 4) != pos16) return ZC_E_CORRUPT;
-            const uint8_t* se = c + L.sub_end_tab[s] + 128ull * ch;
+            const uint32_t sw = sub_end_width(p->chunk_bytes);
+            const uint8_t* se = c + L.sub_end_tab[s] + 32ull * sw * ch;
             uint64_t prev = 0;
             for (uint32_t j = 0; j < kSubs; ++j) {
-                const uint64_t e = rd(se + 4 * j, 4);
+                const uint64_t e = rd(se + sw * j, (int)sw);
                 if (e < prev || e - prev > (uint64_t)p->syms_per_sub * kLmax) return ZC_E_CORRUPT;
                 prev = e;
             }
@@ -290,7 +292,7 @@ zc_status zc_stats(const zc_plan_t* p, const zc_codebook_t* cb, const uint64_t* 
             const uint8_t* d = hd + kHdrStream0 + kHdrStreamStride * s;
             if (d[kSdMode] != o.mode) return ZC_E_CORRUPT;
             const uint64_t hb = rd(d + kSdBits, 8);
-            o.container_bytes = o.mode == ZC_MODE_HUFF ? table_section_bytes(p->n_chunks)
+            o.container_bytes = o.mode == ZC_MODE_HUFF ? table_section_bytes(p->n_chunks, p->chunk_bytes)
                                                        : round_up(p->n_syms, 16);
             if (o.mode == ZC_MODE_HUFF) {
                 // this stream's share of the payload area: its bits, pieces rounded to 16 bytes are

@@ -13,7 +13,7 @@ constexpr uint32_t kMagic = 0x3031435Au;  // 'Z','C','1','0' little-endian
 
 // Byte offsets inside the 128-byte header.
 constexpr uint32_t kHdrMagic = 0, kHdrVersion = 4, kHdrFormat = 6, kHdrStreams = 7, kHdrElems = 8,
-                   kHdrChunkBytes = 16, kHdrChunks = 20, kHdrLmax = 24, kHdrGroup = 25, kHdrSubs = 26,
+                   kHdrChunkBytes = 16, kHdrChunks = 20, kHdrLmax = 24, kHdrGroup = 25, kHdrSubs = 26, kHdrSubWidth = 27,
                    kHdrTotal = 32, kHdrPayloadOff = 40, kHdrPayloadBytes = 48, kHdrStream0 = 64,
                    kHdrStreamStride = 32;
 // Inside a stream descriptor.
@@ -45,9 +45,12 @@ struct zc_codebook_s {
 
 namespace zc {
 
-inline uint64_t table_section_bytes(uint32_t n_chunks)
+// Bytes of one sub_end entry: chunks of at most 8 KiB hold fewer than 65536 bits, so 16 bits are enough.
+inline uint32_t sub_end_width(uint32_t chunk_bytes) { return chunk_bytes <= 8192 ? 2u : 4u; }
+
+inline uint64_t table_section_bytes(uint32_t n_chunks, uint32_t chunk_bytes)
 {
-    return 256 + round_up(4ull * n_chunks, 16) + 128ull * n_chunks;
+    return 256 + round_up(4ull * n_chunks, 16) + 32ull * sub_end_width(chunk_bytes) * n_chunks;
 }
 
 inline Layout make_layout(const zc_plan_s& p, const uint32_t mode[2])
@@ -59,7 +62,7 @@ inline Layout make_layout(const zc_plan_s& p, const uint32_t mode[2])
             L.section_off[s] = off;
             L.chunk_off_tab[s] = off + 256;
             L.sub_end_tab[s] = off + 256 + round_up(4ull * p.n_chunks, 16);
-            off += table_section_bytes(p.n_chunks);
+            off += table_section_bytes(p.n_chunks, p.chunk_bytes);
         }
     for (int s = 0; s < 2; ++s)
         if (mode[s] == ZC_MODE_RAW) {

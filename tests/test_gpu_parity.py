@@ -154,8 +154,9 @@ def test_decoder_accepts_oracle_containers_and_flags_damage():
         hd = zo.parse_header(cont)
         sec = hd["streams"][0]["section_off"]
         used = int(np.flatnonzero(cont[sec:sec + 256])[0])
-        tab = sec + 256 + ((4 * hd["n_chunks"] + 15) // 16) * 16
-        for off, val in ((0, 0x58), (6, 2), (8, 1), (17, 0x40), (64, 7), (sec + used, 13), (tab + 4 * 31 + 2, 0xFF)):
+        _, _, tab = zo.read_tables(cont, 0)
+        w = hd["sub_end_bytes"]
+        for off, val in ((0, 0x58), (6, 2), (8, 1), (17, 0x40), (27, 3), (64, 7), (sec + used, 13), (tab + w * 31 + w - 1, 0xFF)):
             bad = cont.copy(); bad[off] = val
             zc.decompress(p, torch.from_numpy(bad).to(DEV), bad.size, d_back, d_ws)
             assert zc.device_status(p, d_ws) == zc.E_CORRUPT, off

@@ -168,18 +168,19 @@ def _container(fmt, n, chunk_bytes, policy, seed=0):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("policy", [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL])
-def test_validate_accepts_oracle_containers_and_rejects_damage(fmt, policy):
-    n = 5 * 1024 + 36
-    data, hist, cb, cont = _container(fmt, n, 2048, policy)
-    p = zc.plan(fmt, n, 2048)
+@pytest.mark.parametrize("cbytes", [2048, 16384])
+def test_validate_accepts_oracle_containers_and_rejects_damage(fmt, policy, cbytes):
+    n = 5 * (cbytes // 2) + 36
+    data, hist, cb, cont = _container(fmt, n, cbytes, policy)
+    p = zc.plan(fmt, n, cbytes)
     assert zc.validate_container(p, cont) == zc.OK
     assert cont.size <= p.max_compressed_bytes
     # a plan with other parameters does not accept it
-    assert zc.validate_container(zc.plan(fmt, n + 2, 2048), cont) == zc.E_CORRUPT
-    assert zc.validate_container(zc.plan(fmt, n, 4096), cont) == zc.E_CORRUPT
+    assert zc.validate_container(zc.plan(fmt, n + 2, cbytes), cont) == zc.E_CORRUPT
+    assert zc.validate_container(zc.plan(fmt, n, 2 * cbytes), cont) == zc.E_CORRUPT
     assert zc.validate_container(p, cont[:-1]) == zc.E_CORRUPT
     hd = zo.parse_header(cont)
-    for off in (0, 4, 6, 7, 8, 16, 20, 24, 25, 26, 32, 40, 48, 64, 72, 80, 88, 96, 104, 112, 120):
+    for off in (0, 4, 6, 7, 8, 16, 20, 24, 25, 26, 27, 32, 40, 48, 64, 72, 80, 88, 96, 104, 112, 120):
         bad = cont.copy(); bad[off] ^= 0x01
         assert zc.validate_container(p, bad) == zc.E_CORRUPT, off
     for s in range(2):
@@ -191,8 +192,8 @@ def test_validate_accepts_oracle_containers_and_rejects_damage(fmt, policy):
         assert zc.validate_container(p, bad) == zc.E_CORRUPT
         bad = cont.copy(); bad[sec + 256] ^= 1                        # first chunk offset
         assert zc.validate_container(p, bad) == zc.E_CORRUPT
-        tab = sec + 256 + ((4 * hd["n_chunks"] + 15) // 16) * 16
-        bad = cont.copy(); bad[tab + 4 * 7 + 1] ^= 0x40               # a subchunk end jumps
+        _, _, tab = zo.read_tables(cont, s)
+        bad = cont.copy(); bad[tab + hd["sub_end_bytes"] * 7 + 1] ^= 0x40   # a subchunk end jumps
         assert zc.validate_container(p, bad) == zc.E_CORRUPT
         bad = cont.copy(); bad[-3] = 1                                # guard not zero
         assert zc.validate_container(p, bad) == zc.E_CORRUPT

@@ -383,7 +383,8 @@ def test_golden_message_bitstream():
     assert _bits_of_piece(cont[p:p + 16], 15) == bits
     sec = hd["streams"][0]["section_off"]
     assert np.array_equal(cont[sec:sec + 256], cb.lengths[0])
-    sub_end = np.frombuffer(cont[sec + 256 + 16: sec + 256 + 16 + 128].tobytes(), "<u4")
+    assert hd["sub_end_bytes"] == 2                       # 1 KiB chunks use the narrow table
+    sub_end = np.frombuffer(cont[sec + 256 + 16: sec + 256 + 16 + 64].tobytes(), "<u2")
     assert list(sub_end) == [15] * 32                     # 9 symbols all fall in subchunk 0 (16 symbols each)
     assert np.array_equal(zo.decompress(cont, elems.size * 2), elems.view(np.uint8))
 
@@ -405,8 +406,8 @@ def _random_tensor(fmt, n, seed, skew=True):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("policy", [zo.POLICY_AUTO, zo.POLICY_HUFF_ALL, zo.POLICY_RAW_ALL])
-def test_container_invariants_and_independent_decode(fmt, policy):
-    chunk_bytes = 2048
+@pytest.mark.parametrize("chunk_bytes", [2048, 16384])
+def test_container_invariants_and_independent_decode(fmt, policy, chunk_bytes):
     G = zo.group(fmt)
     cs = chunk_bytes // 2
     n = (3 * cs + cs // 2 + 37) * G                       # 3 full chunks + a ragged one
@@ -436,9 +437,8 @@ def test_container_invariants_and_independent_decode(fmt, policy):
         assert st["payload_bits"] == int((hist[s].astype(np.int64) * lens).sum())
         sec = st["section_off"]
         nc = hd["n_chunks"]
-        off16 = np.frombuffer(cont[sec + 256: sec + 256 + 4 * nc].tobytes(), "<u4").astype(np.int64)
-        tab = sec + 256 + ((4 * nc + 15) // 16) * 16
-        sub_end = np.frombuffer(cont[tab: tab + 128 * nc].tobytes(), "<u4").reshape(nc, 32).astype(np.int64)
+        off16, sub_end, _ = zo.read_tables(cont, s)
+        assert hd["sub_end_bytes"] == (2 if chunk_bytes <= 8192 else 4)
         code_str = {v: format(int(cb.codes[s][v]), f"0{int(lens[v])}b") for v in range(256) if lens[v]}
         total_bits = 0
         for c in range(nc):
@@ -536,10 +536,9 @@ def test_damaged_container_is_rejected():
         bad = cont.copy(); bad[off] = val
         with pytest.raises(ValueError):
             zo.decompress(bad, data.size)
-    sec = hd["streams"][0]["section_off"]
     bad = cont.copy()
-    tab = sec + 256 + ((4 * hd["n_chunks"] + 15) // 16) * 16
-    bad[tab + 4 * 5] ^= 0x10                               # a subchunk boundary moves
+    _, _, tab = zo.read_tables(cont, 0)
+    bad[tab + hd["sub_end_bytes"] * 5] ^= 0x10             # a subchunk boundary moves
     with pytest.raises(ValueError):
         zo.decompress(bad, data.size)
 
