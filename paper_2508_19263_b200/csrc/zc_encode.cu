@@ -85,6 +85,12 @@ __device__ bool lookback_exclusive(unsigned long long* flags, uint32_t c, uint32
 // into the same region from its start.  Codes are at most 12 bits, so after k symbols at most 1.5 k bytes are
 // written while the read position is 0.5 * sub + k: the write position never passes unread symbols.
 
+__device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}"
+                 :: "r"(addr), "r"(v), "r"((uint32_t)p) : "memory");
+}
+
 // Append `len` bits (given left-aligned in `code`, zero below them) to a lane's bit accumulator and write a
 // full 32-bit word to the region when one is complete.  hi holds the nb (< 32) pending bits left-aligned.
 __device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& hi, uint32_t& nb, uint32_t& waddr)
@@ -93,14 +99,14 @@ __device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& 
     const uint32_t lo = __funnelshift_r(0, code, nb);           // the bits that do not fit: code << (32 - nb), 0 if nb == 0
     const uint32_t n = nb + len;
     const bool full = n >= 32;
-    if (full) sts32(waddr, hi);
+    sts32_if(full, waddr, hi);
     waddr += full ? 4 : 0;
     hi = full ? lo : hi;
     nb = n & 31;
 }
 
 template <int FMT>
-__global__ void __launch_bounds__(1024, 1)
+__global__ void __launch_bounds__(256, 4)
 encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTables T)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -132,14 +138,24 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     }
     __syncthreads();
 
+    // The block takes batches of n_warps consecutive chunks (one ticket per batch), one chunk per warp.
+    // Piece positions need the sizes of all earlier chunks: the warps of a batch add up their sizes in
+    // shared memory and warp 0 alone does the look-back over the per-batch words, so few warps ever spin.
+    __shared__ uint32_t s_base;
+    __shared__ unsigned long long s_tot[32], s_off[32];
+    __shared__ uint32_t s_fail;
+    const uint32_t n_warps = blockDim.x >> 5;
+    if (threadIdx.x == 0) s_fail = 0;
     uint32_t bad = 0;
     while (true) {
-        uint32_t c = 0;
-        if (lane == 0) c = atomicAdd(&P.ctl->ticket, 1u);
-        c = __shfl_sync(0xFFFFFFFFu, c, 0);
-        if (c >= P.n_chunks) break;
-        const uint64_t c_lo = (uint64_t)c * P.cs;
-        const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
+        if (threadIdx.x == 0) s_base = atomicAdd(&P.ctl->ticket, n_warps);
+        __syncthreads();
+        const uint32_t base = s_base;
+        if (base >= P.n_chunks) break;
+        const uint32_t c = base + warp;
+        const bool active = c < P.n_chunks;
+        const uint64_t c_lo = (uint64_t)(active ? c : 0) * P.cs;
+        const uint32_t c_syms = active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
 
         // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
         auto stage_group = [&](const uint4 x, const uint32_t k) {
@@ -235,6 +251,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                     if (lane >= (uint32_t)o) inc += t;
                 }
                 my_end[hs] = inc;
+                if (!active) { ++hs; continue; }
                 if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * c)[lane] = (uint16_t)inc;
                 else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * c)[lane] = inc;
                 const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
@@ -246,10 +263,27 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         }
         uint64_t off16 = 0;
         if (n_huff) {
-            if (!lookback_exclusive(P.flags, c, lane, tot16, off16)) {
-                raise_status(P.ctl, ZC_E_DEVICE_TIMEOUT);
+            if (lane == 0) s_tot[warp] = tot16;
+            __syncthreads();
+            if (warp == 0) {
+                unsigned long long v = lane < n_warps ? s_tot[lane] : 0ull, inc = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= (uint32_t)o) inc += t;
+                }
+                const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                uint64_t batch_off = 0;
+                const bool ok = lookback_exclusive(P.flags, base / n_warps, lane, batch_total, batch_off);
+                s_off[lane] = batch_off + inc - v;
+                if (!ok && lane == 0) s_fail = 1;
+            }
+            __syncthreads();
+            if (s_fail) {
+                if (threadIdx.x == 0) raise_status(P.ctl, ZC_E_DEVICE_TIMEOUT);
                 break;
             }
+            off16 = s_off[warp];
         }
 
         // ---- phase D: every lane moves its bits to their final position in the chunk's piece ----
@@ -258,6 +292,7 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
             uint64_t piece_off16 = off16;
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
+                if (!active) { ++hs; continue; }
                 if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[c] = (uint32_t)piece_off16;
                 uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
                 const uint32_t piece_words = 4 * piece16[hs];
@@ -293,7 +328,8 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         }
         __syncwarp();
         // the warp that owns the last chunk knows the size of the whole payload area
-        if (lane == 0 && c == P.n_chunks - 1) P.ctl->total16 = off16 + tot16;
+        if (lane == 0 && active && c == P.n_chunks - 1) P.ctl->total16 = off16 + tot16;
+        __syncthreads();                                        // s_base is rewritten at the top of the loop
     }
     if (bad) raise_status(P.ctl, ZC_E_NO_CODE);
 }
@@ -377,11 +413,12 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
     if (p->n_chunks) {
         const size_t fixed = 512 * sizeof(uint32_t);
         const size_t per_warp = std::max<size_t>((size_t)n_huff * P.stage_stride, 16);
-        uint32_t warps = (uint32_t)std::min<size_t>(32, (kMaxSmem - fixed - 1024) / per_warp);
+        // blocks of up to 8 warps (a batch of 8 consecutive chunks); several blocks per SM so that loading,
+        // packing and copy-out phases of different blocks overlap
+        uint32_t warps = (uint32_t)std::min<size_t>(8, (kMaxSmem - fixed - 1024) / per_warp);
         if (warps == 0) return ZC_E_UNSUPPORTED;
         const size_t smem = fixed + warps * per_warp;
-        // resident blocks per SM by shared memory (leave 1 KiB per block for the system) and threads
-        uint32_t per_sm = (uint32_t)std::min<size_t>(kMaxSmem / (smem + 1024), 2048 / (warps * 32));
+        uint32_t per_sm = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (smem + 1024 + 1024), 4);
         per_sm = std::max(per_sm, 1u);
         const uint32_t want = (p->n_chunks + warps - 1) / warps;
         const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * per_sm);
