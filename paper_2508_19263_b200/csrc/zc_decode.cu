@@ -20,7 +20,7 @@ struct DecParams {
 };
 
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
-constexpr uint32_t kScratchBytes = 1024;
+constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
 constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
 constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
 
@@ -40,36 +40,27 @@ __device__ __forceinline__ uint32_t lds32_if(bool p, uint32_t addr)
 // ------------------------------------------------------------------------------------------------
 // decode tables, built by every block from the container's code-length table
 // ------------------------------------------------------------------------------------------------
-// Canonical-code bookkeeping in shared memory: for each length the first code value, the number of
-// codes and the offset of its symbols in the (length, symbol)-sorted list.
-
+// Canonical-code bookkeeping in shared memory, per code length l = 1..12:
+//   count[l]  codes of that length            first[l]  value of the first one
+//   offset[l] position of its symbols in the (length, symbol)-sorted list
+//   limit[l]  windows below this value start with a code of length <= l
 struct CodeBook {
     uint32_t* count;   // [16]
     uint32_t* first;   // [16]
     uint32_t* offset;  // [16]
+    uint32_t* limit;   // [16]
     uint32_t* wcount;  // [8][16] per-warp counts, then exclusive prefix over warps
     uint8_t* sorted;   // [256]
-    uint32_t* ok;
+    uint32_t* ok;      // [0] lengths usable, [1] symbols per lookup
 };
 
 __device__ __forceinline__ CodeBook codebook_views(uint32_t* scratch)
 {
     CodeBook b;
-    b.count = scratch; b.first = scratch + 16; b.offset = scratch + 32; b.wcount = scratch + 48;
-    b.sorted = reinterpret_cast<uint8_t*>(scratch + 48 + 128);
-    b.ok = scratch + 48 + 128 + 64;
+    b.count = scratch; b.first = scratch + 16; b.offset = scratch + 32; b.limit = scratch + 48; b.wcount = scratch + 64;
+    b.sorted = reinterpret_cast<uint8_t*>(scratch + 64 + 128);
+    b.ok = scratch + 64 + 128 + 64;
     return b;
-}
-
-// One symbol from the top bits of a 12-bit window: (len << 8) | symbol, or 0 if no code matches.
-__device__ __forceinline__ uint32_t walk_code(uint32_t window12, const CodeBook& b)
-{
-    for (uint32_t l = 1; l <= kLmax; ++l) {
-        const uint32_t code = window12 >> (kLmax - l);
-        const uint32_t rel = code - b.first[l];
-        if (code >= b.first[l] && rel < b.count[l]) return (l << 8) | b.sorted[b.offset[l] + rel];
-    }
-    return 0;
 }
 
 // Fills the table of one stream and decides how many symbols every lookup yields (returned in *per_lookup).
@@ -80,20 +71,20 @@ __device__ __forceinline__ uint32_t walk_code(uint32_t window12, const CodeBook&
 // the second with one more lookup.  That mode is chosen when such pairs are rare (estimated from the code
 // lengths with p(symbol) = 2^-length); otherwise every lookup yields exactly one symbol.  A fixed number of
 // symbols per lookup lets a lane assemble words of 4 symbols in registers without any bookkeeping.
-// `single` is a 4096 x u16 scratch table.  Returns false to all threads if the lengths are not a complete
-// prefix code (or the one-symbol code).
+// `single` is a 4096 x u16 scratch table (length << 8 | symbol of the first code of every window).
+// Returns false to all threads if the lengths are not a complete prefix code (or the one-symbol code).
 __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, uint16_t* single, uint32_t* scratch,
                           uint32_t* per_lookup)
 {
     const CodeBook b = codebook_views(scratch);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid < 48 + 128) scratch[tid] = 0;
-    if (tid == 0) *b.ok = 1;
-    __syncthreads();
     uint32_t my_len = 0, my_rank = 0;
+    if (tid < 256) my_len = code_len[tid];                       // issued before the barrier below
+    if (tid < 64 + 128) scratch[tid] = 0;
+    if (tid == 0) b.ok[0] = 1;
+    __syncthreads();
     if (tid < 256) {
-        my_len = code_len[tid];
-        if (my_len > kLmax) { *b.ok = 0; my_len = 0; }
+        if (my_len > kLmax) { b.ok[0] = 0; my_len = 0; }
         for (uint32_t l = 1; l <= kLmax; ++l) {
             const uint32_t m = __ballot_sync(0xFFFFFFFFu, my_len == l);
             if (my_len == l) my_rank = __popc(m & ((1u << lane) - 1));
@@ -101,40 +92,53 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, u
         }
     }
     __syncthreads();
+    if (tid >= 1 && tid <= kLmax) {                              // thread l adds up length l over the 8 warps
+        uint32_t cnt = 0;
+        for (uint32_t w = 0; w < 8; ++w) { const uint32_t t = b.wcount[w * 16 + tid]; b.wcount[w * 16 + tid] = cnt; cnt += t; }
+        b.count[tid] = cnt;
+    }
+    __syncthreads();
     if (tid == 0) {
         uint32_t code = 0, off = 0, active = 0;
-        uint64_t kraft = 0;
+        uint32_t p[kLmax + 2];                                    // weight of length l in units of 2^-12
         for (uint32_t l = 1; l <= kLmax; ++l) {
-            uint32_t cnt = 0;
-            for (uint32_t w = 0; w < 8; ++w) { const uint32_t t = b.wcount[w * 16 + l]; b.wcount[w * 16 + l] = cnt; cnt += t; }
-            b.count[l] = cnt;
+            const uint32_t cnt = b.count[l];
             code = (code + b.count[l - 1]) << 1;
             b.first[l] = code;
             b.offset[l] = off;
+            b.limit[l] = (code + cnt) << (kLmax - l);
             off += cnt;
             active += cnt;
-            kraft += (uint64_t)cnt << (kLmax - l);
+            p[l] = cnt << (kLmax - l);
         }
-        const bool complete = kraft == (1ull << kLmax);
+        const bool complete = b.limit[kLmax] == kLutEntries;      // Kraft sum is exactly one
         const bool one = active == 1 && b.count[1] == 1;
-        if (!(complete || one || active == 0)) *b.ok = 0;
-        // probability (in units of 2^-24) that two consecutive codes need more than 12 bits
+        if (!(complete || one || active == 0)) b.ok[0] = 0;
+        // probability (units of 2^-24) that two consecutive codes need more than 12 bits
         uint64_t long_pairs = 0;
-        for (uint32_t l1 = 1; l1 <= kLmax; ++l1)
-            for (uint32_t l2 = kLmax + 1 - l1; l2 <= kLmax; ++l2)
-                long_pairs += ((uint64_t)b.count[l1] << (kLmax - l1)) * ((uint64_t)b.count[l2] << (kLmax - l2));
+        uint32_t tail = 0;                                        // sum of p[l2] for l2 >= 13 - l1
+        for (uint32_t l1 = 1; l1 <= kLmax; ++l1) {
+            tail += p[kLmax + 1 - l1];
+            long_pairs += (uint64_t)p[l1] * tail;
+        }
         b.ok[1] = long_pairs <= (1ull << 24) / 32 ? 2u : 1u;
+        if (one) b.limit[1] = kLutEntries;                        // the unused half of the windows reads as the one symbol
     }
     __syncthreads();
     const uint32_t mode = b.ok[1];
     if (tid < 256 && my_len) b.sorted[b.offset[my_len] + b.wcount[warp * 16 + my_len] + my_rank] = (uint8_t)tid;
+    uint32_t lim[kLmax + 1];
+#pragma unroll
+    for (uint32_t l = 1; l <= kLmax; ++l) lim[l] = b.limit[l];
     __syncthreads();
-    // one symbol per window; a window no code matches (possible only for the one-symbol code) reads as
-    // that list's first symbol with length 1
+    // first code of every window: its length is the number of limits at or below the window value, plus one
     for (uint32_t idx = tid; idx < kLutEntries; idx += blockDim.x) {
-        uint32_t e = walk_code(idx, b);
-        if (e == 0) e = (1u << 8) | b.sorted[0];
-        single[idx] = (uint16_t)e;
+        uint32_t l = 1;
+#pragma unroll
+        for (uint32_t k = 1; k < kLmax; ++k) l += idx >= lim[k] ? 1u : 0u;
+        uint32_t rel = (idx >> (kLmax - l)) - b.first[l];
+        if (rel >= b.count[l]) rel = 0;                           // only reachable with damaged or one-symbol tables
+        single[idx] = (uint16_t)((l << 8) | b.sorted[b.offset[l] + rel]);
     }
     __syncthreads();
     for (uint32_t idx = tid; idx < kLutEntries; idx += blockDim.x) {
@@ -151,7 +155,7 @@ __device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, u
     }
     __syncthreads();
     if (tid == 0) *per_lookup = mode;
-    return *b.ok != 0;
+    return b.ok[0] != 0;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -283,10 +287,15 @@ decode_kernel(const __grid_constant__ DecParams P)
     __shared__ uint32_t s_mode[2], s_per_lookup[2];
     __shared__ uint32_t s_ok;
     __shared__ unsigned long long s_payload_off, s_payload_bytes, s_sec[2];
+    __shared__ __align__(16) uint32_t s_hdr[32];
+    if (warp == 0) {
+        s_hdr[lane] = reinterpret_cast<const uint32_t*>(P.comp)[lane];      // the 128-byte header in one request
+        __syncwarp();
+    }
     if (threadIdx.x == 0) {
-        const uint8_t* h = P.comp;
-        const uint32_t* h32 = reinterpret_cast<const uint32_t*>(h);
-        const unsigned long long* h64 = reinterpret_cast<const unsigned long long*>(h);
+        const uint8_t* h = reinterpret_cast<const uint8_t*>(s_hdr);
+        const uint32_t* h32 = s_hdr;
+        const unsigned long long* h64 = reinterpret_cast<const unsigned long long*>(s_hdr);
         bool ok = h32[0] == kMagic && h[kHdrVersion] == 1 && h[kHdrVersion + 1] == 0 && h[kHdrFormat] == P.format &&
                   h[kHdrStreams] == 2 && h64[kHdrElems / 8] == P.n_elems && h32[kHdrChunkBytes / 4] == P.chunk_bytes &&
                   h32[kHdrChunks / 4] == P.n_chunks && h[kHdrLmax] == kLmax && h[kHdrGroup] == P.group && h[kHdrSubs] == kSubs &&
@@ -550,7 +559,7 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     // per warp: one stream's rows plus room to stage a piece as large as the raw chunk stream; pieces that
     // do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
     P.pool_bytes = std::max<uint32_t>(rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32, 2 * rows_bytes);
-    const size_t fixed = kDecFixedSmem + 64 /* static shared */;
+    const size_t fixed = kDecFixedSmem + 512 /* static shared */;
     size_t per_warp = 16 + P.pool_bytes;
     uint32_t warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     if (warps < 8) {                 // large chunks: stage less
