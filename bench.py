@@ -409,7 +409,7 @@ def run_ours(args):
                               "sign_mantissa_stream_payload": st_bits[1] / (8 * n_syms),
                               "paper_context": "abstract: up to 62% (BF16) / 83% (FP8) total"},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": 4 * n_t * args.steps,
+        "gpu_launches": 3 * n_t * args.steps,
     }
     print(json.dumps(line))
     if dist is not None:

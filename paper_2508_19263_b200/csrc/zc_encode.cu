@@ -23,6 +23,7 @@ struct EncParams {
     uint32_t stage_stride;                       // bytes of one coded stream's lane regions per warp
     uint32_t region_bytes;                       // one lane region: 1.5 * sub + 4
     uint32_t sub_width;                          // bytes per sub_end entry (2 or 4)
+    uint32_t deep;                               // lane regions have two pack slots (see encode_kernel)
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
 };
 
@@ -79,11 +80,17 @@ __device__ bool lookback_exclusive(unsigned long long* flags, uint32_t c, uint32
     return true;
 }
 
-// Per-warp shared memory of one coded stream: 32 lane regions of 1.5 * sub bytes (+4 bytes of padding, which
-// also makes the region stride an odd number of words so that lanes walking their regions hit different
-// banks).  A region first holds the subchunk's symbols in its upper two thirds; the lane then packs the codes
-// into the same region from its start.  Codes are at most 12 bits, so after k symbols at most 1.5 k bytes are
-// written while the read position is 0.5 * sub + k: the write position never passes unread symbols.
+// Per-warp shared memory of one coded stream: 32 lane regions (+4 bytes of padding each, which also makes
+// the region stride an odd number of words so that lanes walking their regions hit different banks).
+// A region is cut into slots of `sub` bytes.  Two layouts:
+//   plain  [pack | symbols]           the lane packs its codes in place: codes are at most 12 bits, so after k
+//                                     symbols at most 1.5 k bytes are written while the read position is
+//                                     sub + k, and the writer never passes unread symbols
+//   deep   [pack A | pack B | symbols] packing alternates between A and B, so the packed bits of the previous
+//                                     batch survive the packing of the next one and their copy-out can wait a
+//                                     whole iteration for the batch's position in the payload area
+// The packed bits of a subchunk normally stay within one slot (8 bits per symbol); a batch in which some lane
+// needs more is finished on a slow path before anything else is staged.
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
@@ -92,35 +99,101 @@ __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 }
 
 // Append `len` bits (given left-aligned in `code`, zero below them) to a lane's bit accumulator and write a
-// full 32-bit word to the region when one is complete.  hi holds the nb (< 32) pending bits left-aligned.
-__device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& hi, uint32_t& nb, uint32_t& waddr)
+// full 32-bit word to the region when one is complete and lies below `limit`.  hi holds the nb (< 32)
+// pending bits left-aligned.
+__device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& hi, uint32_t& nb, uint32_t& waddr, uint32_t limit)
 {
     hi |= code >> nb;
     const uint32_t lo = __funnelshift_r(0, code, nb);           // the bits that do not fit: code << (32 - nb), 0 if nb == 0
     const uint32_t n = nb + len;
     const bool full = n >= 32;
-    sts32_if(full, waddr, hi);
+    sts32_if(full && waddr < limit, waddr, hi);
     waddr += full ? 4 : 0;
     hi = full ? lo : hi;
     nb = n & 31;
 }
 
+__device__ __forceinline__ unsigned long long ld_ctl(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Writes the 128-byte header and the guard; called by one thread once every chunk is in place.
+__device__ void write_header(const EncParams& P)
+{
+    const bool any_huff = P.mode[0] == ZC_MODE_HUFF || P.mode[1] == ZC_MODE_HUFF;
+    const uint64_t payload_bytes = any_huff ? 16ull * ld_ctl(&P.ctl->total16) : 0;
+    uint8_t* h = P.out;
+    uint32_t* h32 = reinterpret_cast<uint32_t*>(h);
+    unsigned long long* h64 = reinterpret_cast<unsigned long long*>(h);
+    for (int i = 0; i < 32; ++i) h32[i] = 0;
+    h32[0] = kMagic;
+    h[kHdrVersion] = 1; h[kHdrFormat] = (uint8_t)P.format; h[kHdrStreams] = 2;
+    h64[kHdrElems / 8] = P.n_elems;
+    h32[kHdrChunkBytes / 4] = P.chunk_bytes;
+    h32[kHdrChunks / 4] = P.n_chunks;
+    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)P.group; h[kHdrSubs] = kSubs; h[kHdrSubWidth] = (uint8_t)P.sub_width;
+    const uint64_t total = P.lay.payload_off + payload_bytes + (any_huff ? 16 : 0);
+    h64[kHdrTotal / 8] = total;
+    h64[kHdrPayloadOff / 8] = P.lay.payload_off;
+    h64[kHdrPayloadBytes / 8] = payload_bytes;
+    for (int s = 0; s < 2; ++s) {
+        uint8_t* d = h + kHdrStream0 + kHdrStreamStride * s;
+        d[kSdMode] = (uint8_t)P.mode[s];
+        reinterpret_cast<unsigned long long*>(d)[1] = P.n_syms;
+        reinterpret_cast<unsigned long long*>(d)[2] = P.mode[s] == ZC_MODE_HUFF ? ld_ctl(&P.ctl->payload_bits[s]) : 8 * P.n_syms;
+        reinterpret_cast<unsigned long long*>(d)[3] = P.lay.section_off[s];
+    }
+    if (any_huff) {
+        uint32_t* g = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + payload_bytes);
+        g[0] = g[1] = g[2] = g[3] = 0;
+    }
+    P.ctl->total16 = total;                      // the host reads the container size from here
+}
+
+
+// For an empty tensor no encoder block runs: the header is all there is.
+__global__ void finish_kernel(const EncParams P)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) write_header(P);
+}
+
+constexpr uint32_t kEncMaxWorkers = 8;       // worker warps per block = chunks per batch; one more warp does the look-back
+
+// What a worker warp keeps about a chunk between packing it and copying it out.
+struct PackedChunk {
+    uint32_t c;                 // chunk index
+    bool active;                // this warp has a chunk in the batch
+    uint32_t slot;              // byte offset of the pack slot inside the lane regions
+    uint32_t bits[2];           // my subchunk's bit count per stream
+    uint32_t end[2];            // inclusive scan of it over the lanes = the sub_end entry
+};
+
 template <int FMT>
-__global__ void __launch_bounds__(256, 4)
+__global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, 3)
 encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTables T)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t n_workers = (blockDim.x >> 5) - 1;
+    const bool scanner = warp == n_workers;                     // the last warp only does the look-back
     const bool huff0 = P.mode[0] == ZC_MODE_HUFF, huff1 = P.mode[1] == ZC_MODE_HUFF;
     const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
+    const bool deep = P.deep != 0;
 
-    // shared: enc[2][256] | per warp: regions[n_huff][stage_stride]
+    // shared: enc[2][256] | per worker warp: regions[n_huff][stage_stride]
     uint32_t* enc = reinterpret_cast<uint32_t*>(smem);
     uint8_t* stage_all = smem + 2048;
     for (uint32_t i = threadIdx.x; i < 512; i += blockDim.x) enc[i] = T.enc[i >> 8][i & 255];
-    uint8_t* stage = stage_all + (size_t)warp * n_huff * P.stage_stride;
-    const uint32_t region = P.region_bytes;                     // 1.5 * sub + 4
-    const uint32_t sym_off = P.sub / 2;                         // symbols sit at this offset inside a region
+    uint8_t* stage = stage_all + (size_t)(scanner ? 0 : warp) * n_huff * P.stage_stride;
+    const uint32_t region = P.region_bytes;                     // (2 or 3) * sub + 4
+    const uint32_t sym_off = deep ? 2 * P.sub : P.sub;          // symbols sit at this offset inside a region
+
+    __shared__ uint32_t s_base[2];
+    __shared__ unsigned long long s_tot[32], s_off[32];
+    __shared__ uint32_t s_fail, s_slow;
 
     // block 0 writes the static parts of the table sections and the tail padding of raw bodies
     if (blockIdx.x == 0) {
@@ -136,26 +209,94 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
             }
         }
     }
+    if (threadIdx.x == 0) {
+        s_fail = 0; s_slow = 0;
+        s_base[0] = atomicAdd(&P.ctl->ticket, n_workers);       // batches of n_workers consecutive chunks
+    }
     __syncthreads();
 
-    // The block takes batches of n_warps consecutive chunks (one ticket per batch), one chunk per warp.
-    // Piece positions need the sizes of all earlier chunks: the warps of a batch add up their sizes in
-    // shared memory and warp 0 alone does the look-back over the per-batch words, so few warps ever spin.
-    __shared__ uint32_t s_base;
-    __shared__ unsigned long long s_tot[32], s_off[32];
-    __shared__ uint32_t s_fail;
-    const uint32_t n_warps = blockDim.x >> 5;
-    if (threadIdx.x == 0) s_fail = 0;
+    // ---- copy-out of a packed chunk: every lane moves its bits to their final position in the piece ----
+    auto copy_out = [&](const PackedChunk& pc, const uint64_t off16) {
+        uint32_t hs = 0;
+        uint64_t piece_off16 = off16;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            if (P.mode[s] != ZC_MODE_HUFF) continue;
+            const uint32_t end = pc.end[s], bits = pc.bits[s], start = end - bits;
+            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
+            const uint32_t piece16 = (chunk_bits + 127) / 128;
+            if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[pc.c] = (uint32_t)piece_off16;
+            uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
+            const uint32_t piece_words = 4 * piece16;
+            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region) + pc.slot;
+            const uint32_t sh = start & 31, d0 = start >> 5;
+            const uint32_t n_dst = (sh + bits + 31) / 32;             // destination words I touch
+            const uint32_t n_src = (bits + 31) / 32;
+            if (__all_sync(0xFFFFFFFFu, bits >= 32)) {
+                // every lane spans a word boundary, so a destination word is shared by at most two neighbouring
+                // lanes: a lane hands its ragged last word to the next lane, which merges it into its first word
+                const bool ragged = ((sh + bits) & 31) != 0;
+                const uint32_t il = n_dst - 1;
+                const uint32_t lc = il < n_src ? lds32(reg_s + 4 * il) : 0u;
+                const uint32_t lp = il >= 1 ? lds32(reg_s + 4 * (il - 1)) : 0u;
+                const uint32_t tail = ragged ? __funnelshift_r(lc, lp, sh) : 0u;
+                uint32_t head = __shfl_up_sync(0xFFFFFFFFu, tail, 1);
+                if (lane == 0) head = 0;
+                const uint32_t n_mine = n_dst - ((ragged && lane != 31) ? 1u : 0u);
+                uint32_t prev = 0;
+                for (uint32_t i = 0; i < n_mine; ++i) {
+                    const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
+                    uint32_t v = __funnelshift_r(cur, prev, sh);      // (prev:cur) >> sh, low word
+                    prev = cur;
+                    if (i == 0) v |= head;
+                    piece[d0 + i] = v;
+                }
+                if (lane < 4 && piece_words) {                        // zero padding up to the 16-byte boundary
+                    const uint32_t w = piece_words - 4 + lane;
+                    if (32ull * w >= chunk_bits) piece[w] = 0;
+                }
+            } else {
+                // general case (short or empty subchunks): words shared between neighbours (and the padding)
+                // start from zero and are OR-ed into
+                if ((start >> 5) < piece_words) piece[start >> 5] = 0;
+                if (lane == 31 && (end >> 5) < piece_words) piece[end >> 5] = 0;
+                if (lane < 4 && piece_words) {
+                    const uint32_t w = piece_words - 4 + lane;
+                    if (32ull * w >= chunk_bits) piece[w] = 0;
+                }
+                __syncwarp();
+                if (bits) {
+                    uint32_t prev = 0;
+                    for (uint32_t i = 0; i < n_dst; ++i) {
+                        const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
+                        const uint32_t v = __funnelshift_r(cur, prev, sh);
+                        prev = cur;
+                        // the first word may hold the previous lane's bits, a ragged last word the next lane's
+                        const bool shared_word = i == 0 || (i == n_dst - 1 && ((sh + bits) & 31) != 0);
+                        if (shared_word) atomicOr(&piece[d0 + i], v);
+                        else piece[d0 + i] = v;
+                    }
+                }
+            }
+            piece_off16 += piece16;
+            ++hs;
+        }
+        // the warp that owns the last chunk knows the size of the whole payload area
+        if (lane == 0 && pc.c == P.n_chunks - 1) P.ctl->total16 = piece_off16;
+        __syncwarp();
+    };
+
     uint32_t bad = 0;
-    while (true) {
-        if (threadIdx.x == 0) s_base = atomicAdd(&P.ctl->ticket, n_warps);
-        __syncthreads();
-        const uint32_t base = s_base;
-        if (base >= P.n_chunks) break;
-        const uint32_t c = base + warp;
-        const bool active = c < P.n_chunks;
-        const uint64_t c_lo = (uint64_t)(active ? c : 0) * P.cs;
-        const uint32_t c_syms = active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
+    PackedChunk prev{0, false, 0, {0, 0}, {0, 0}};
+    bool pending = false;                                       // a packed batch still waits for its copy-out
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t base = s_base[it & 1];
+        const bool have = base < P.n_chunks;
+        if (!have && !pending) break;
+
+        PackedChunk cur{base + warp, have && !scanner && base + warp < P.n_chunks, deep ? (it & 1) * P.sub : 0u, {0, 0}, {0, 0}};
+        const uint64_t c_lo = (uint64_t)(cur.active ? cur.c : 0) * P.cs;
+        const uint32_t c_syms = cur.active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
 
         // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
         auto stage_group = [&](const uint4 x, const uint32_t k) {
@@ -178,194 +319,170 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         };
         const uint32_t n_vec = (c_syms + 7) / 8;
         const uint8_t* src_c = P.in + 2 * c_lo;
-        uint32_t it = lane;
+        uint32_t g = lane;
         if (2 * (c_lo + 8ull * n_vec) <= P.input_bytes) {           // every group of this chunk is complete
-            for (; it + 96 < n_vec; it += 128) {                        // four loads in flight per lane
-                const uint4 x0 = ld_nc_v4(src_c + 16 * it);
-                const uint4 x1 = ld_nc_v4(src_c + 16 * (it + 32));
-                const uint4 x2 = ld_nc_v4(src_c + 16 * (it + 64));
-                const uint4 x3 = ld_nc_v4(src_c + 16 * (it + 96));
-                stage_group(x0, 8 * it);
-                stage_group(x1, 8 * (it + 32));
-                stage_group(x2, 8 * (it + 64));
-                stage_group(x3, 8 * (it + 96));
+            for (; g + 96 < n_vec; g += 128) {                          // four loads in flight per lane
+                const uint4 x0 = ld_nc_v4(src_c + 16 * g);
+                const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32));
+                const uint4 x2 = ld_nc_v4(src_c + 16 * (g + 64));
+                const uint4 x3 = ld_nc_v4(src_c + 16 * (g + 96));
+                stage_group(x0, 8 * g);
+                stage_group(x1, 8 * (g + 32));
+                stage_group(x2, 8 * (g + 64));
+                stage_group(x3, 8 * (g + 96));
             }
-            for (; it < n_vec; it += 32) stage_group(ld_nc_v4(src_c + 16 * it), 8 * it);
+            for (; g < n_vec; g += 32) stage_group(ld_nc_v4(src_c + 16 * g), 8 * g);
         } else {
-            for (; it < n_vec; it += 32) stage_group(load16_guarded(P.in, 2 * (c_lo + 8ull * it), P.input_bytes), 8 * it);
+            for (; g < n_vec; g += 32) stage_group(load16_guarded(P.in, 2 * (c_lo + 8ull * g), P.input_bytes), 8 * g);
         }
         __syncwarp();
 
-        // ---- phase B: every lane packs the codes of its subchunk into its own region, from bit 0 ----
+        // plain layout: the previous batch must leave its slot before this batch is packed into it; its
+        // look-back ran while this batch was loaded
+        if (!deep) {
+            __syncthreads();
+            if (s_fail) break;
+            if (pending && prev.active && n_huff) copy_out(prev, s_off[warp]);
+        }
+
+        // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
         const uint32_t lo_sym = lane * P.sub;
         const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
-        uint32_t my_bits[2] = {0, 0};
+        // returns the bit count; stores stop at `room` bytes (the count goes on)
+        auto pack = [&](const int s, const uint32_t hs, const uint32_t slot, const uint32_t room) -> uint32_t {
+            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
+            const uint32_t tab_s = smem_u32(enc + 256 * s);
+            const uint32_t w0 = reg_s + slot, limit = w0 + room;
+            uint32_t hi = 0, nb = 0, waddr = w0, seen = 0;
+            const uint32_t src = reg_s + sym_off;
+            const uint32_t full_words = n_my / 4;
+            for (uint32_t i = 0; i < full_words; ++i) {
+                const uint32_t four = lds32(src + 4 * i);
+                const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
+                const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
+                const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
+                const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
+                seen |= e0 | e1 | e2 | e3;
+                // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
+                // first entry = its length); the length fields end up below bit 8 and are masked off
+                const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
+                put_bits(ca, (e0 + e1) & 31, hi, nb, waddr, limit);
+                const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
+                put_bits(cb, (e2 + e3) & 31, hi, nb, waddr, limit);
+            }
+            for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
+                const uint32_t four = lds32(src + (i & ~3u));
+                const uint32_t e = lds32(tab_s + (((four >> (8 * (i & 3))) & 0xFF) << 2));
+                seen |= e;
+                put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr, limit);
+            }
+            if (cur.active && waddr < limit) sts32(waddr, hi);      // pending bits (or zero)
+            bad |= seen & 16;                                       // an entry without a code carries bit 4
+            return 8 * (waddr - w0) + nb;
+        };
         {
             uint32_t hs = 0;
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
-                const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
-                const uint32_t tab_s = smem_u32(enc + 256 * s);
-                uint32_t hi = 0, nb = 0, waddr = reg_s, seen = 0;
-                const uint32_t src = reg_s + sym_off;
-                const uint32_t full_words = n_my / 4;
-                for (uint32_t i = 0; i < full_words; ++i) {
-                    const uint32_t four = lds32(src + 4 * i);
-                    const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
-                    const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
-                    const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
-                    const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
-                    seen |= e0 | e1 | e2 | e3;
-                    // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
-                    // first entry = its length); the length fields end up below bit 8 and are masked off
-                    const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
-                    put_bits(ca, (e0 + e1) & 31, hi, nb, waddr);
-                    const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
-                    put_bits(cb, (e2 + e3) & 31, hi, nb, waddr);
-                }
-                for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
-                    const uint32_t four = lds32(src + (i & ~3u));
-                    const uint32_t e = lds32(tab_s + (((four >> (8 * (i & 3))) & 0xFF) << 2));
-                    seen |= e;
-                    put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr);
-                }
-                sts32(waddr, hi);                                       // pending bits (or zero)
-                my_bits[hs] = 8 * (waddr - reg_s) + nb;
-                bad |= seen & 16;                                       // an entry without a code carries bit 4
+                // deep layout, slot A: anything beyond the slot would overwrite the previous batch in slot B
+                const uint32_t room = (deep && cur.slot == 0) ? P.sub : 3 * P.sub;
+                cur.bits[s] = pack(s, hs, cur.slot, room);
+                // more than 8 bits per symbol: the bits beyond the slot do not survive the next staging
+                if (cur.bits[s] > 8 * P.sub) s_slow = 1;
                 ++hs;
             }
         }
 
-        // ---- phase C: subchunk end bits, piece sizes, position of the chunk in the payload area ----
-        uint32_t my_end[2] = {0, 0}, piece16[2] = {0, 0};
+        // deep layout: the previous batch sits in the other pack slot; its look-back had this whole packing time
+        if (deep) {
+            __syncthreads();
+            if (s_fail) break;
+            if (pending && prev.active && n_huff) copy_out(prev, s_off[warp]);
+        }
+
+        // the ticket of the next batch is taken as late as possible (batches must start in the order they
+        // were handed out, or the look-back of other blocks waits for a batch that is not even begun); its
+        // latency hides behind phase C
+        uint32_t next_base = base;
+        if (threadIdx.x == 0 && have) next_base = atomicAdd(&P.ctl->ticket, n_workers);
+
+        // ---- phase C: subchunk end bits and the chunk's size in the payload area ----
         uint64_t tot16 = 0;
         {
-            uint32_t hs = 0;
+#pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
-                uint32_t inc = my_bits[hs];
+                uint32_t inc = cur.bits[s];
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
                     if (lane >= (uint32_t)o) inc += t;
                 }
-                my_end[hs] = inc;
-                if (!active) { ++hs; continue; }
-                if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * c)[lane] = (uint16_t)inc;
-                else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * c)[lane] = inc;
-                const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                piece16[hs] = (chunk_bits + 127) / 128;
-                tot16 += piece16[hs];
-                if (lane == 0) atomicAdd(&P.ctl->payload_bits[s], (unsigned long long)chunk_bits);
-                ++hs;
-            }
-        }
-        uint64_t off16 = 0;
-        if (n_huff) {
-            if (lane == 0) s_tot[warp] = tot16;
-            __syncthreads();
-            if (warp == 0) {
-                unsigned long long v = lane < n_warps ? s_tot[lane] : 0ull, inc = v;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= (uint32_t)o) inc += t;
+                cur.end[s] = inc;
+                if (cur.active) {
+                    if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * cur.c)[lane] = (uint16_t)inc;
+                    else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * cur.c)[lane] = inc;
+                    const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                    tot16 += (chunk_bits + 127) / 128;
+                    if (lane == 0) atomicAdd(&P.ctl->payload_bits[s], (unsigned long long)chunk_bits);
                 }
-                const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                uint64_t batch_off = 0;
-                const bool ok = lookback_exclusive(P.flags, base / n_warps, lane, batch_total, batch_off);
-                s_off[lane] = batch_off + inc - v;
-                if (!ok && lane == 0) s_fail = 1;
             }
-            __syncthreads();
-            if (s_fail) {
-                if (threadIdx.x == 0) raise_status(P.ctl, ZC_E_DEVICE_TIMEOUT);
-                break;
-            }
-            off16 = s_off[warp];
         }
+        if (lane == 0) s_tot[warp] = tot16;
+        if (threadIdx.x == 0) s_base[(it + 1) & 1] = next_base;
+        __syncthreads();
 
-        // ---- phase D: every lane moves its bits to their final position in the chunk's piece ----
-        {
-            uint32_t hs = 0;
-            uint64_t piece_off16 = off16;
-            for (int s = 0; s < 2; ++s) {
-                if (P.mode[s] != ZC_MODE_HUFF) continue;
-                if (!active) { ++hs; continue; }
-                if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[c] = (uint32_t)piece_off16;
-                uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
-                const uint32_t piece_words = 4 * piece16[hs];
-                const uint32_t end = my_end[hs], bits = my_bits[hs], start = end - bits;
-                const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
-                // words shared between neighbours (and the padding) start from zero and are OR-ed into
-                if ((start >> 5) < piece_words) piece[start >> 5] = 0;
-                if (lane == 31 && (end >> 5) < piece_words) piece[end >> 5] = 0;
-                if (lane < 4 && piece_words) {
-                    const uint32_t w = piece_words - 4 + lane;
-                    if (32ull * w >= chunk_bits) piece[w] = 0;
+        // ---- the look-back warp places the batch; the workers go on with the next batch meanwhile ----
+        const bool slow = s_slow != 0;
+        if (scanner && have && n_huff) {
+            unsigned long long v = lane < n_workers ? s_tot[lane] : 0ull, inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= (uint32_t)o) inc += t;
+            }
+            const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint64_t batch_off = 0;
+            const bool ok = lookback_exclusive(P.flags, base / n_workers, lane, batch_total, batch_off);
+            s_off[lane] = batch_off + inc - v;
+            if (!ok && lane == 0) s_fail = 1;
+        }
+        if (slow) {
+            // some subchunk needs more than 8 bits per symbol: finish this batch before anything else is staged.
+            // In the deep layout the other slot is free by now, so a clipped packing into slot A is redone.
+            if (deep && cur.slot == 0) {
+                uint32_t hs = 0;
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    if (P.mode[s] != ZC_MODE_HUFF) continue;
+                    pack(s, hs, 0, 3 * P.sub);
+                    ++hs;
                 }
                 __syncwarp();
-                if (bits) {
-                    const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
-                    const uint32_t sh = start & 31, d0 = start >> 5;
-                    const uint32_t n_dst = (sh + bits + 31) / 32;         // destination words I touch
-                    const uint32_t n_src = (bits + 31) / 32;
-                    uint32_t prev = 0;
-                    for (uint32_t i = 0; i < n_dst; ++i) {
-                        const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
-                        const uint32_t v = __funnelshift_r(cur, prev, sh);  // (prev:cur) >> sh, low word
-                        prev = cur;
-                        // the first word may hold the previous lane's bits, a ragged last word the next lane's
-                        const bool shared_word = i == 0 || (i == n_dst - 1 && ((sh + bits) & 31) != 0);
-                        if (shared_word) atomicOr(&piece[d0 + i], v);
-                        else piece[d0 + i] = v;
-                    }
-                }
-                piece_off16 += piece16[hs];
-                ++hs;
             }
+            __syncthreads();
+            if (s_fail) break;
+            if (cur.active && n_huff) copy_out(cur, s_off[warp]);
+            __syncthreads();
+            if (threadIdx.x == 0) s_slow = 0;
+            pending = false;
+        } else {
+            prev = cur;
+            pending = have;
         }
-        __syncwarp();
-        // the warp that owns the last chunk knows the size of the whole payload area
-        if (lane == 0 && active && c == P.n_chunks - 1) P.ctl->total16 = off16 + tot16;
-        __syncthreads();                                        // s_base is rewritten at the top of the loop
     }
+    if (s_fail && threadIdx.x == 0) raise_status(P.ctl, ZC_E_DEVICE_TIMEOUT);
     if (bad) raise_status(P.ctl, ZC_E_NO_CODE);
-}
-
-// Writes the 128-byte header and the guard once every chunk is in place (stream order guarantees it).
-__global__ void finish_kernel(const EncParams P)
-{
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    const bool any_huff = P.mode[0] == ZC_MODE_HUFF || P.mode[1] == ZC_MODE_HUFF;
-    const uint64_t payload_bytes = any_huff ? 16ull * P.ctl->total16 : 0;
-    uint8_t* h = P.out;
-    uint32_t* h32 = reinterpret_cast<uint32_t*>(h);
-    unsigned long long* h64 = reinterpret_cast<unsigned long long*>(h);
-    for (int i = 0; i < 32; ++i) h32[i] = 0;
-    h32[0] = kMagic;
-    h[kHdrVersion] = 1; h[kHdrFormat] = (uint8_t)P.format; h[kHdrStreams] = 2;
-    h64[kHdrElems / 8] = P.n_elems;
-    h32[kHdrChunkBytes / 4] = P.chunk_bytes;
-    h32[kHdrChunks / 4] = P.n_chunks;
-    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)P.group; h[kHdrSubs] = kSubs; h[kHdrSubWidth] = (uint8_t)P.sub_width;
-    const uint64_t total = P.lay.payload_off + payload_bytes + (any_huff ? 16 : 0);
-    h64[kHdrTotal / 8] = total;
-    h64[kHdrPayloadOff / 8] = P.lay.payload_off;
-    h64[kHdrPayloadBytes / 8] = payload_bytes;
-    for (int s = 0; s < 2; ++s) {
-        uint8_t* d = h + kHdrStream0 + kHdrStreamStride * s;
-        d[kSdMode] = (uint8_t)P.mode[s];
-        reinterpret_cast<unsigned long long*>(d)[1] = P.n_syms;
-        reinterpret_cast<unsigned long long*>(d)[2] = P.mode[s] == ZC_MODE_HUFF ? P.ctl->payload_bits[s] : 8 * P.n_syms;
-        reinterpret_cast<unsigned long long*>(d)[3] = P.lay.section_off[s];
+    // the block that finishes last writes the header (every block's results are fenced before its count)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&P.ctl->done, 1u) == gridDim.x - 1) {
+            __threadfence();
+            write_header(P);
+        }
     }
-    if (any_huff) {
-        uint32_t* g = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + payload_bytes);
-        g[0] = g[1] = g[2] = g[3] = 0;
-    }
-    P.ctl->total16 = total;                      // the host reads the container size from here
 }
 
 }  // namespace zc
@@ -397,7 +514,9 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         n_huff += P.mode[s] == ZC_MODE_HUFF;
     }
     P.lay = make_layout(*p, P.mode);
-    P.region_bytes = p->syms_per_sub + p->syms_per_sub / 2 + 4;
+    // two pack slots per lane region when the chunks are small enough to keep three blocks per SM resident
+    P.deep = p->chunk_bytes <= 4096 ? 1u : 0u;
+    P.region_bytes = (P.deep ? 3 : 2) * p->syms_per_sub + 4;
     P.sub_width = sub_end_width(p->chunk_bytes);
     P.stage_stride = kSubs * P.region_bytes;
     P.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
@@ -413,14 +532,15 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
     if (p->n_chunks) {
         const size_t fixed = 512 * sizeof(uint32_t);
         const size_t per_warp = std::max<size_t>((size_t)n_huff * P.stage_stride, 16);
-        // blocks of up to 8 warps (a batch of 8 consecutive chunks); several blocks per SM so that loading,
-        // packing and copy-out phases of different blocks overlap
-        uint32_t warps = (uint32_t)std::min<size_t>(8, (kMaxSmem - fixed - 1024) / per_warp);
-        if (warps == 0) return ZC_E_UNSUPPORTED;
-        const size_t smem = fixed + warps * per_warp;
-        uint32_t per_sm = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (smem + 1024 + 1024), 4);
+        // blocks of up to 8 worker warps (a batch of 8 consecutive chunks) plus the look-back warp; several
+        // blocks per SM so that loading, packing and copy-out phases of different blocks overlap
+        const uint32_t workers = (uint32_t)std::min<size_t>(kEncMaxWorkers, (kMaxSmem - fixed - 1024) / per_warp);
+        if (workers == 0) return ZC_E_UNSUPPORTED;
+        const uint32_t warps = workers + 1;
+        const size_t smem = fixed + workers * per_warp;
+        uint32_t per_sm = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (smem + 1024 + 1024), 3);
         per_sm = std::max(per_sm, 1u);
-        const uint32_t want = (p->n_chunks + warps - 1) / warps;
+        const uint32_t want = (p->n_chunks + workers - 1) / workers;
         const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * per_sm);
         auto launch = [&](auto kern) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -435,8 +555,10 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         }
         if (e != cudaSuccess) return ZC_E_CUDA;
     }
-    finish_kernel<<<1, 32, 0, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return ZC_E_CUDA;
+    if (p->n_chunks == 0) {
+        finish_kernel<<<1, 32, 0, st>>>(P);
+        if (cudaGetLastError() != cudaSuccess) return ZC_E_CUDA;
+    }
 
     if (h_out_bytes) {
         Control h;
