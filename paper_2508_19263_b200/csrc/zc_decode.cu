@@ -8,6 +8,9 @@
 // DRAM latency hides behind the table lookups.
 #include "zc_device.cuh"
 
+#include <atomic>
+#include <chrono>
+
 namespace zc {
 
 struct DecParams {
@@ -17,6 +20,8 @@ struct DecParams {
     uint64_t comp_bytes, input_bytes, n_syms, n_elems;
     uint32_t n_chunks, cs, sub, chunk_bytes, format, group;
     uint32_t pool_bytes;     // per-warp shared memory: symbol rows first, the rest stages compressed pieces
+    uint32_t spec;           // the container is long enough to read stream 0's tables before the header is checked
+    unsigned long long call_id;
 };
 
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
@@ -73,13 +78,11 @@ __device__ __forceinline__ CodeBook codebook_views(uint32_t* scratch)
 // symbols per lookup lets a lane assemble words of 4 symbols in registers without any bookkeeping.
 // `single` is a 4096 x u16 scratch table (length << 8 | symbol of the first code of every window).
 // Returns false to all threads if the lengths are not a complete prefix code (or the one-symbol code).
-__device__ bool build_lut(const uint8_t* __restrict__ code_len, uint32_t* lut, uint16_t* single, uint32_t* scratch,
-                          uint32_t* per_lookup)
+__device__ bool build_lut(uint32_t my_len, uint32_t* lut, uint16_t* single, uint32_t* scratch, uint32_t* per_lookup)
 {
     const CodeBook b = codebook_views(scratch);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t my_len = 0, my_rank = 0;
-    if (tid < 256) my_len = code_len[tid];                       // issued before the barrier below
+    uint32_t my_rank = 0;                                        // my_len: length of symbol tid's code (threads < 256)
     if (tid < 64 + 128) scratch[tid] = 0;
     if (tid == 0) b.ok[0] = 1;
     __syncthreads();
@@ -283,6 +286,20 @@ decode_kernel(const __grid_constant__ DecParams P)
     uint64_t* bar = bars + 2 * warp;
 
     const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;     // bytes per sub_end entry
+    const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
+    // Nearly every container has stream 0 coded, its table section right behind the header.  Its code lengths
+    // and this warp's first table entries are requested now, together with the header, and thrown away if the
+    // header says otherwise.
+    uint32_t spec_len = 0, spec_end = 0, spec_off = 0;
+    if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
+    if (P.spec) {
+        if (threadIdx.x < 256) spec_len = P.comp[kHeaderBytes + threadIdx.x];
+        const uint32_t c0 = blockIdx.x * n_warps + warp;
+        if (c0 < P.n_chunks) {
+            spec_end = load_sub_end(P.comp + kHeaderBytes + tab_sub, sub_w, c0, lane);
+            spec_off = reinterpret_cast<const uint32_t*>(P.comp + kHeaderBytes + tab_chunk)[c0];
+        }
+    }
     // ---- header check against the plan ----
     __shared__ uint32_t s_mode[2], s_per_lookup[2];
     __shared__ uint32_t s_ok;
@@ -327,20 +344,27 @@ decode_kernel(const __grid_constant__ DecParams P)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    if (!s_ok) { if (threadIdx.x == 0) raise_status(P.ctl, ZC_E_CORRUPT); return; }
+    if (!s_ok) { if (threadIdx.x == 0) raise_status(P.ctl, P.call_id, ZC_E_CORRUPT); return; }
 
     const bool huff0 = s_mode[0] == ZC_MODE_HUFF, huff1 = s_mode[1] == ZC_MODE_HUFF;
     {
         // the warps' pools are free until the main loop: 8 KiB of them hold the one-symbol scratch table
         uint16_t* single = reinterpret_cast<uint16_t*>(pools);
         bool tables_ok = true;
-        if (huff0) tables_ok = build_lut(P.comp + s_sec[0], lut0, single, scratch, &s_per_lookup[0]) && tables_ok;
-        if (huff1) tables_ok = build_lut(P.comp + s_sec[1], lut1, single, scratch, &s_per_lookup[1]) && tables_ok;
+        if (huff0) {
+            uint32_t len = spec_len;                             // stream 0's section always starts behind the header
+            if (!P.spec && threadIdx.x < 256) len = P.comp[s_sec[0] + threadIdx.x];
+            tables_ok = build_lut(len, lut0, single, scratch, &s_per_lookup[0]) && tables_ok;
+        }
+        if (huff1) {
+            uint32_t len = 0;
+            if (threadIdx.x < 256) len = P.comp[s_sec[1] + threadIdx.x];
+            tables_ok = build_lut(len, lut1, single, scratch, &s_per_lookup[1]) && tables_ok;
+        }
         __syncthreads();
-        if (!tables_ok) { if (threadIdx.x == 0) raise_status(P.ctl, ZC_E_CORRUPT); return; }
+        if (!tables_ok) { if (threadIdx.x == 0) raise_status(P.ctl, P.call_id, ZC_E_CORRUPT); return; }
     }
 
-    const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
     const uint8_t* payload = P.comp + s_payload_off;
     const unsigned long long payload_bytes = s_payload_bytes;
     const uint8_t* sec0 = P.comp + s_sec[0];
@@ -365,8 +389,9 @@ decode_kernel(const __grid_constant__ DecParams P)
     uint32_t c = blockIdx.x * n_warps + warp;
     uint32_t nx_end0 = 0, nx_off0 = 0, nx_end1 = 0, nx_off1 = 0;
     if (c < P.n_chunks) {
-        if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, c, lane);
-                     nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[c]; }
+        if (huff0 && P.spec) { nx_end0 = spec_end; nx_off0 = spec_off; }
+        else if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, c, lane);
+                          nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[c]; }
         if (huff1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, c, lane);
                      nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c]; }
     }
@@ -527,7 +552,7 @@ decode_kernel(const __grid_constant__ DecParams P)
         for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0 ^ 1); ++spins) {}
         for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1 ^ 1); ++spins) {}
     }
-    if (err) raise_status(P.ctl, err);
+    if (err) raise_status(P.ctl, P.call_id, err);
 }
 
 }  // namespace zc
@@ -543,8 +568,6 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     if (!aligned16(d_comp) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (comp_bytes < kHeaderBytes) return ZC_E_CORRUPT;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemsetAsync(d_workspace, 0, kControlBytes, st) != cudaSuccess) return ZC_E_CUDA;
-
     DecParams P{};
     P.comp = (const uint8_t*)d_comp;
     P.out = (uint8_t*)d_out;
@@ -552,6 +575,10 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     P.comp_bytes = comp_bytes; P.input_bytes = p->input_bytes; P.n_syms = p->n_syms; P.n_elems = p->n_elems;
     P.n_chunks = p->n_chunks; P.cs = p->syms_per_chunk; P.sub = p->syms_per_sub; P.chunk_bytes = p->chunk_bytes;
     P.format = p->format; P.group = p->group;
+    // no clearing of the workspace: errors are tagged with the id of the call that raised them
+    static std::atomic<unsigned long long> next_call{(unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count()};
+    P.call_id = (next_call.fetch_add(1) & ((1ull << 56) - 1)) | 1ull << 55;
+    P.spec = comp_bytes >= kHeaderBytes + table_section_bytes(p->n_chunks, p->chunk_bytes) ? 1u : 0u;
 
     // symbols per round and lane: the largest of 64 / 32 / 16 that divides the subchunk length
     const uint32_t ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;

@@ -472,8 +472,8 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
             pending = have;
         }
     }
-    if (s_fail && threadIdx.x == 0) raise_status(P.ctl, ZC_E_DEVICE_TIMEOUT);
-    if (bad) raise_status(P.ctl, ZC_E_NO_CODE);
+    if (s_fail && threadIdx.x == 0) raise_status(P.ctl, 0, ZC_E_DEVICE_TIMEOUT);
+    if (bad) raise_status(P.ctl, 0, ZC_E_NO_CODE);
     // the block that finishes last writes the header (every block's results are fenced before its count)
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -564,7 +564,7 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         Control h;
         if (cudaMemcpyAsync(&h, d_workspace, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
-        if (h.status) return (zc_status)h.status;
+        if (h.status & 0xFF) return (zc_status)(h.status & 0xFF);
         *h_out_bytes = h.total16;
     }
     return ZC_OK;
@@ -612,10 +612,11 @@ zc_status zc_device_status(const zc_plan_t* p, const void* d_workspace, void* cu
 {
     if (!p || !d_workspace) return ZC_E_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    uint32_t status = 0;
-    if (cudaMemcpyAsync(&status, d_workspace, sizeof(status), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
+    unsigned long long word[2] = {0, 0};            // status, call id
+    if (cudaMemcpyAsync(word, d_workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
-    return (zc_status)status;
+    // an error word left by an earlier call carries that call's id and does not count
+    return (word[0] >> 8) == word[1] ? (zc_status)(word[0] & 0xFF) : ZC_OK;
 }
 
 }  // extern "C"

@@ -75,12 +75,14 @@ inline Layout make_layout(const zc_plan_s& p, const uint32_t mode[2])
 
 // Device workspace: a control block followed by one look-back word per chunk.
 struct Control {
-    uint32_t status;           // zc_status raised on the device (first one wins)
-    uint32_t ticket;           // next chunk to hand out
+    unsigned long long status;   // (call id << 8) | zc_status raised on the device; first error of a call wins
+    unsigned long long call_id;  // id of the call that last used the block; a status with another id is stale.
+                                 // zc_compress clears the whole block and uses id 0.
+    uint32_t ticket;             // next batch of chunks to hand out
+    uint32_t done;               // encoder blocks finished
     unsigned long long payload_bits[2];
-    unsigned long long total16;  // payload area size in 16-byte units
-    uint32_t done;             // chunks finished
-    uint32_t pad[7];
+    unsigned long long total16;  // payload area size in 16-byte units; finally the container size in bytes
+    uint32_t pad[4];
 };
 constexpr size_t kControlBytes = 256;
 
