@@ -215,17 +215,18 @@ __device__ __forceinline__ void lane_consume(LaneStream& st, uint32_t n)    // n
     st.lo = __funnelshift_l(0, st.lo, n);
 }
 
-// Decode n_words words of 4 symbols into the lane's row.  K = symbols per lookup (1 or 2).
+// Decode n_words words of 4 symbols into the lane's row from a piece staged in shared memory.
+// K = symbols per lookup (1 or 2).
 // One-symbol mode: top up, two lookups, top up, two lookups.  Two-symbol mode: top up, two lookups; a lookup
 // whose second code did not fit the window (bit 31 of the entry, rare by construction of the mode) tops up
 // again and takes the second symbol from the next window.
-template <int K, bool STAGED>
+template <int K>
 __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uint32_t row_s, uint32_t n_words)
 {
     for (uint32_t i = 0; i < n_words; ++i) {
         uint32_t word;
         if (K == 2) {
-            lane_refill<STAGED>(st);
+            lane_refill<true>(st);
             uint32_t pair[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -233,7 +234,7 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
                 lane_consume(st, e);
                 st.valid -= e & 0xFF;
                 if ((int)e < 0) {
-                    lane_refill<STAGED>(st);
+                    lane_refill<true>(st);
                     const uint32_t f = lane_peek(st, lut_s);
                     const uint32_t l = (f >> 24) & 15;
                     lane_consume(st, l);
@@ -244,13 +245,13 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
             }
             word = __byte_perm(pair[0], pair[1], 0x6521);
         } else {
-            lane_refill<STAGED>(st);
+            lane_refill<true>(st);
             const uint32_t a = lane_peek(st, lut_s);
             lane_consume(st, a);
             const uint32_t b = lane_peek(st, lut_s);
             lane_consume(st, b);
             st.valid -= (a + b) & 0xFF;
-            lane_refill<STAGED>(st);
+            lane_refill<true>(st);
             const uint32_t c = lane_peek(st, lut_s);
             lane_consume(st, c);
             const uint32_t d = lane_peek(st, lut_s);
@@ -262,6 +263,229 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
     }
 }
 
+// The same result one symbol at a time, from the first-code fields every table entry carries whatever the
+// table's mode (symbol in bits 15..8, length in bits 27..24).  Small and slow on purpose: it serves pieces
+// that were too long to stage (read from global memory) and the rarely coded sign+mantissa stream.
+template <bool STAGED>
+__device__ __forceinline__ void decode_words_plain(LaneStream& st, uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+{
+    for (uint32_t i = 0; i < n_words; ++i) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if ((k & 1) == 0) lane_refill<STAGED>(st);
+            const uint32_t e = lane_peek(st, lut_s);
+            const uint32_t l = (e >> 24) & 15;
+            lane_consume(st, l);
+            st.valid -= l;
+            word |= ((e >> 8) & 0xFF) << (8 * k);
+        }
+        sts32(row_s + 4 * i, word);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// chunk loop of one warp, specialised for which streams are Huffman-coded
+// ------------------------------------------------------------------------------------------------
+
+struct DecShared {                   // what the block's prologue leaves for the chunk loop
+    uint32_t lut0_s, lut1_s;         // shared addresses of the decode tables
+    uint32_t pairs0;                 // stream 0's table yields two symbols per lookup
+    unsigned long long sec0, sec1;   // byte offsets of the streams' sections
+    unsigned long long payload_off, payload_bytes;
+};
+
+// PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
+template <int FMT, int PPL, bool H0, bool H1>
+__device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShared& S, uint8_t* pool, uint64_t* bar,
+                                               uint32_t first_end0, uint32_t first_off0)
+{
+    constexpr uint32_t R = 16 * PPL;
+    constexpr uint32_t kRowStride = R + 4;                     // bytes; the padding spreads the lanes' rows over the banks
+    constexpr uint32_t kRowsBytes = 32 * kRowStride;           // one stream's rows of a warp (multiple of 16)
+    constexpr uint32_t kHuff = (H0 ? 1u : 0u) + (H1 ? 1u : 0u);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;
+    const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
+    const uint8_t* sec0 = P.comp + S.sec0;
+    const uint8_t* sec1 = P.comp + S.sec1;
+    const uint8_t* payload = P.comp + S.payload_off;
+
+    // pool: rows of stream 0 (if coded), rows of stream 1 (if coded), then one staging slot per coded stream
+    constexpr uint32_t rows1_off = H0 ? kRowsBytes : 0;
+    constexpr uint32_t slots_off = rows1_off + (H1 ? kRowsBytes : 0);
+    const uint32_t slot_room = P.pool_bytes > slots_off ? P.pool_bytes - slots_off : 0u;
+    const uint32_t slot_bytes = kHuff ? (slot_room / (kHuff ? kHuff : 1)) & ~15u : 0u;
+    const uint32_t rows0_s = smem_u32(pool), rows1_s = rows0_s + rows1_off;
+    const uint32_t slot0_s = rows0_s + slots_off, slot1_s = slot0_s + (H0 ? slot_bytes : 0);
+    const uint32_t step = gridDim.x * n_warps;
+    uint32_t parity0 = 0, parity1 = 0, err = 0;
+
+    // this lane's parts of a round: part i covers symbols k_lane + i * k_step (+ round offset) of the chunk
+    const uint32_t k_lane = (lane / PPL) * P.sub + (lane % PPL) * 16, k_step = (32 / PPL) * P.sub;
+    const uint32_t row_lane = (lane / PPL) * kRowStride + (lane % PPL) * 16, row_step = (32 / PPL) * kRowStride;
+
+    uint32_t c = blockIdx.x * n_warps + warp;
+    uint32_t nx_end0 = first_end0, nx_off0 = first_off0, nx_end1 = 0, nx_off1 = 0;
+    if (H1 && c < P.n_chunks) {
+        nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, c, lane);
+        nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c];
+    }
+
+    for (; c < P.n_chunks; c += step) {
+        const uint64_t c_lo = (uint64_t)c * P.cs;
+        const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
+        const uint64_t out_lo = 2 * c_lo;                       // two element bytes per symbol in every format
+        const uint32_t out_bytes = (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - out_lo);
+        const uint32_t lo_sym = lane * P.sub;
+        const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
+
+        // ---- where my subchunk starts and where the chunk's pieces are; check, then stage ----
+        LaneStream st0{0, 0, 0, 0, nullptr}, st1{0, 0, 0, 0, nullptr};
+        uint32_t start0 = 0, start1 = 0, piece0 = 0, piece1 = 0;
+        const uint32_t* pay0_g = nullptr;
+        const uint32_t* pay1_g = nullptr;
+        bool staged0 = false, staged1 = false, ok = true;
+        if (H0) {
+            const uint32_t my_end = nx_end0, off16 = nx_off0;
+            start0 = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
+            if (lane == 0) start0 = 0;
+            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
+            piece0 = ((chunk_bits + 127) / 128) * 16;
+            ok = ok && start0 <= my_end && my_end - start0 <= n_my * kLmax && 16ull * off16 + piece0 <= S.payload_bytes;
+            pay0_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
+        }
+        if (H1) {
+            const uint32_t my_end = nx_end1, off16 = nx_off1;
+            start1 = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
+            if (lane == 0) start1 = 0;
+            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
+            piece1 = ((chunk_bits + 127) / 128) * 16;
+            ok = ok && start1 <= my_end && my_end - start1 <= n_my * kLmax && 16ull * off16 + piece1 <= S.payload_bytes;
+            pay1_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
+        }
+        if (kHuff && !__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; break; }
+        // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
+        if (H0 && piece0 + 16 <= slot_bytes) {
+            staged0 = true;
+            if (lane == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(&bar[0], piece0 + 16);
+                bulk_g2s(pool + slots_off, pay0_g, piece0 + 16, &bar[0]);
+            }
+        }
+        if (H1 && piece1 + 16 <= slot_bytes) {
+            staged1 = true;
+            if (lane == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(&bar[1], piece1 + 16);
+                bulk_g2s(pool + slots_off + (H0 ? slot_bytes : 0), pay1_g, piece1 + 16, &bar[1]);
+            }
+        }
+        // request the next chunk's table entries now; they are consumed in the next iteration
+        {
+            const uint32_t cn = c + step;
+            if (cn < P.n_chunks) {
+                if (H0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
+                          nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
+                if (H1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
+                          nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[cn]; }
+            }
+        }
+
+        const uint8_t* raw0 = sec0 + c_lo + k_lane;             // my first part's bytes in a raw stream
+        const uint8_t* raw1 = sec1 + c_lo + k_lane;
+        uint8_t* dst_lane = P.out + out_lo + 2 * k_lane;
+        const uint32_t n_rounds = P.sub / R;
+        bool waited = false;
+        for (uint32_t r = 0; r < n_rounds; ++r) {
+            if (r * R >= c_syms) break;                          // lane 0 has the most symbols; nothing left
+            // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
+            uint4 pre[PPL];
+#pragma unroll
+            for (int i = 0; i < PPL; ++i) {
+                pre[i] = make_uint4(0, 0, 0, 0);
+                if (!H1 && k_lane + i * k_step + r * R < c_syms) pre[i] = ld_nc_v4(raw1 + i * k_step + r * R);
+            }
+            if (kHuff && !waited) {
+                waited = true;
+                if (H0 && staged0) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&bar[0], parity0)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                    parity0 ^= 1;
+                }
+                if (H1 && staged1) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&bar[1], parity1)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                    parity1 ^= 1;
+                }
+                if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                if (n_my) {
+                    if (H0) { if (staged0) lane_begin<true>(st0, slot0_s, nullptr, start0); else lane_begin<false>(st0, 0, pay0_g, start0); }
+                    if (H1) { if (staged1) lane_begin<true>(st1, slot1_s, nullptr, start1); else lane_begin<false>(st1, 0, pay1_g, start1); }
+                }
+            }
+            // ---- every lane decodes R symbols of its subchunk ----
+            if (kHuff) {
+                const uint32_t done = r * R;
+                const uint32_t target = n_my > done ? min(R, n_my - done) : 0u;
+                const uint32_t n_words = (target + 3) / 4;      // a ragged last word decodes up to 3 symbols too many
+                if (n_words) {
+                    if (H0) {
+                        const uint32_t row_s = rows0_s + lane * kRowStride;
+                        if (!staged0) decode_words_plain<false>(st0, S.lut0_s, row_s, n_words);
+                        else if (S.pairs0) decode_words<2>(st0, S.lut0_s, row_s, n_words);
+                        else decode_words<1>(st0, S.lut0_s, row_s, n_words);
+                    }
+                    if (H1) {
+                        const uint32_t row_s = rows1_s + lane * kRowStride;
+                        if (staged1) decode_words_plain<true>(st1, S.lut1_s, row_s, n_words);
+                        else decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
+                    }
+                }
+                __syncwarp();
+            }
+            // ---- cooperative merge: a part covers 16 symbols = 32 output bytes ----
+#pragma unroll
+            for (int i = 0; i < PPL; ++i) {
+                const uint32_t k = k_lane + i * k_step + r * R;
+                if (k >= c_syms) continue;
+                uint32_t e[4], m[4];
+                if (H0) {
+                    const uint32_t a = rows0_s + row_lane + i * row_step;
+                    e[0] = lds32(a); e[1] = lds32(a + 4); e[2] = lds32(a + 8); e[3] = lds32(a + 12);
+                } else {
+                    const uint4 v = ld_nc_v4(raw0 + i * k_step + r * R);
+                    e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
+                }
+                if (H1) {
+                    const uint32_t a = rows1_s + row_lane + i * row_step;
+                    m[0] = lds32(a); m[1] = lds32(a + 4); m[2] = lds32(a + 8); m[3] = lds32(a + 12);
+                } else { m[0] = pre[i].x; m[1] = pre[i].y; m[2] = pre[i].z; m[3] = pre[i].w; }
+                uint32_t o[8];
+                merge16<FMT>(e, m, o);
+                merge16<FMT>(e + 2, m + 2, o + 4);
+                uint8_t* dst = dst_lane + 2 * (i * k_step + r * R);
+                if (2 * k + 32 <= out_bytes) {
+                    st_cs_v8(dst, o);
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 32; ++t)
+                        if (2 * k + t < out_bytes) dst[t] = (uint8_t)(o[t >> 2] >> (8 * (t & 3)));
+                }
+            }
+            if (kHuff) __syncwarp();
+        }
+        if (err) break;
+    }
+    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) {
+        // give copies in flight one more bounded chance to land before the block leaves
+        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0 ^ 1); ++spins) {}
+        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1 ^ 1); ++spins) {}
+    }
+    return err;
+}
+
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
@@ -271,9 +495,6 @@ template <int FMT, int PPL>
 __global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
 decode_kernel(const __grid_constant__ DecParams P)
 {
-    constexpr uint32_t R = 16 * PPL;
-    constexpr uint32_t kRowStride = R + 4;                     // bytes; the padding spreads the lanes' rows over the banks
-    constexpr uint32_t kRowsBytes = 32 * kRowStride;           // one stream's rows of a warp (multiple of 16)
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
 
@@ -365,193 +586,24 @@ decode_kernel(const __grid_constant__ DecParams P)
         if (!tables_ok) { if (threadIdx.x == 0) raise_status(P.ctl, P.call_id, ZC_E_CORRUPT); return; }
     }
 
-    const uint8_t* payload = P.comp + s_payload_off;
-    const unsigned long long payload_bytes = s_payload_bytes;
-    const uint8_t* sec0 = P.comp + s_sec[0];
-    const uint8_t* sec1 = P.comp + s_sec[1];
-    // pool: rows of stream 0 (if coded), rows of stream 1 (if coded), then one staging slot per coded stream
-    const uint32_t rows0_off = 0, rows1_off = huff0 ? kRowsBytes : 0;
-    const uint32_t slots_off = rows1_off + (huff1 ? kRowsBytes : 0);
-    const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
-    const uint32_t slot_room = P.pool_bytes > slots_off ? P.pool_bytes - slots_off : 0u;
-    const uint32_t slot_bytes = n_huff ? (slot_room / n_huff) & ~15u : 0u;
-    const uint32_t slot0_s = smem_u32(pool + slots_off);
-    const uint32_t slot1_s = slot0_s + (huff0 ? slot_bytes : 0);
-    const uint32_t rows0_s = smem_u32(pool + rows0_off), rows1_s = smem_u32(pool + rows1_off);
-    const uint32_t lut0_s = smem_u32(lut0), lut1_s = smem_u32(lut1);
-    const bool pairs0 = huff0 && s_per_lookup[0] == 2, pairs1 = huff1 && s_per_lookup[1] == 2;
-    const uint32_t step = gridDim.x * n_warps;
-    uint32_t parity0 = 0, parity1 = 0;
-    uint32_t err = 0;
-
-    // subchunk end bits and piece offsets of the first chunk; those of the following chunk are
-    // requested while the current one is decoded
-    uint32_t c = blockIdx.x * n_warps + warp;
-    uint32_t nx_end0 = 0, nx_off0 = 0, nx_end1 = 0, nx_off1 = 0;
-    if (c < P.n_chunks) {
-        if (huff0 && P.spec) { nx_end0 = spec_end; nx_off0 = spec_off; }
-        else if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, c, lane);
-                          nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[c]; }
-        if (huff1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, c, lane);
-                     nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c]; }
+    DecShared S;
+    S.lut0_s = smem_u32(lut0); S.lut1_s = smem_u32(lut1);
+    S.pairs0 = huff0 && s_per_lookup[0] == 2;
+    S.sec0 = s_sec[0]; S.sec1 = s_sec[1];
+    S.payload_off = s_payload_off; S.payload_bytes = s_payload_bytes;
+    uint32_t first_end0 = spec_end, first_off0 = spec_off;
+    if (huff0 && !P.spec) {
+        const uint32_t c0 = blockIdx.x * n_warps + warp;
+        if (c0 < P.n_chunks) {
+            first_end0 = load_sub_end(P.comp + S.sec0 + tab_sub, sub_w, c0, lane);
+            first_off0 = reinterpret_cast<const uint32_t*>(P.comp + S.sec0 + tab_chunk)[c0];
+        }
     }
-
-    for (; c < P.n_chunks; c += step) {
-        const uint64_t c_lo = (uint64_t)c * P.cs;
-        const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
-        const uint64_t out_lo = 2 * c_lo;                       // two element bytes per symbol in every format
-        const uint32_t out_bytes = (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - out_lo);
-        const uint32_t lo_sym = lane * P.sub;
-        const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
-
-        // ---- where my subchunk starts and where the chunk's pieces are; check, then stage ----
-        LaneStream st0{0, 0, 0, 0, nullptr}, st1{0, 0, 0, 0, nullptr};
-        uint32_t start0 = 0, start1 = 0;
-        const uint32_t* pay0_g = nullptr;
-        const uint32_t* pay1_g = nullptr;
-        bool staged0 = false, staged1 = false;
-        uint32_t piece0 = 0, piece1 = 0;
-        bool ok = true;
-        if (huff0) {
-            const uint32_t my_end = nx_end0, off16 = nx_off0;
-            uint32_t start = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
-            if (lane == 0) start = 0;
-            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
-            piece0 = ((chunk_bits + 127) / 128) * 16;
-            ok = ok && start <= my_end && my_end <= chunk_bits && my_end - start <= n_my * kLmax &&
-                 16ull * off16 + piece0 <= payload_bytes;
-            start0 = start;
-            pay0_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
-        }
-        if (huff1) {
-            const uint32_t my_end = nx_end1, off16 = nx_off1;
-            uint32_t start = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
-            if (lane == 0) start = 0;
-            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
-            piece1 = ((chunk_bits + 127) / 128) * 16;
-            ok = ok && start <= my_end && my_end <= chunk_bits && my_end - start <= n_my * kLmax &&
-                 16ull * off16 + piece1 <= payload_bytes;
-            start1 = start;
-            pay1_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
-        }
-        if (!__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; break; }
-        // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
-        if (huff0 && piece0 + 16 <= slot_bytes) {
-            staged0 = true;
-            if (lane == 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_expect_tx(&bar[0], piece0 + 16);
-                bulk_g2s(pool + slots_off, pay0_g, piece0 + 16, &bar[0]);
-            }
-        }
-        if (huff1 && piece1 + 16 <= slot_bytes) {
-            staged1 = true;
-            if (lane == 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_expect_tx(&bar[1], piece1 + 16);
-                bulk_g2s(pool + slots_off + (huff0 ? slot_bytes : 0), pay1_g, piece1 + 16, &bar[1]);
-            }
-        }
-        // request the next chunk's tables now; they are consumed in the next iteration
-        {
-            const uint32_t cn = c + step;
-            if (cn < P.n_chunks) {
-                if (huff0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
-                             nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
-                if (huff1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
-                             nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[cn]; }
-            }
-        }
-
-        const uint32_t n_rounds = P.sub / R;
-        bool waited = false;
-        for (uint32_t r = 0; r < n_rounds; ++r) {
-            if (r * R >= c_syms) break;                          // lane 0 has the most symbols; nothing left
-            // ---- raw stream bytes of this round go to registers before the decoding starts ----
-            uint4 raw1[PPL];
-#pragma unroll
-            for (int i = 0; i < PPL; ++i) {
-                const uint32_t q = i * 32 + lane;
-                const uint32_t k = (q / PPL) * P.sub + r * R + (q % PPL) * 16;   // symbol index inside the chunk
-                raw1[i] = make_uint4(0, 0, 0, 0);
-                if (k < c_syms && !huff1) raw1[i] = ld_nc_v4(sec1 + c_lo + k);
-            }
-            if (!waited) {
-                waited = true;
-                if (staged0) {
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait(&bar[0], parity0)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                    parity0 ^= 1;
-                }
-                if (staged1) {
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait(&bar[1], parity1)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                    parity1 ^= 1;
-                }
-                if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                if (n_my) {
-                    if (huff0) { if (staged0) lane_begin<true>(st0, slot0_s, nullptr, start0); else lane_begin<false>(st0, 0, pay0_g, start0); }
-                    if (huff1) { if (staged1) lane_begin<true>(st1, slot1_s, nullptr, start1); else lane_begin<false>(st1, 0, pay1_g, start1); }
-                }
-            }
-            // ---- every lane decodes R symbols of its subchunk ----
-            const uint32_t done = r * R;
-            const uint32_t target = n_my > done ? min(R, n_my - done) : 0u;
-            const uint32_t n_words = (target + 3) / 4;          // a ragged last word decodes up to 3 symbols too many
-            if (n_words) {
-                if (huff0) {
-                    const uint32_t row_s = rows0_s + lane * kRowStride;
-                    if (staged0) { if (pairs0) decode_words<2, true>(st0, lut0_s, row_s, n_words); else decode_words<1, true>(st0, lut0_s, row_s, n_words); }
-                    else { if (pairs0) decode_words<2, false>(st0, lut0_s, row_s, n_words); else decode_words<1, false>(st0, lut0_s, row_s, n_words); }
-                }
-                if (huff1) {
-                    const uint32_t row_s = rows1_s + lane * kRowStride;
-                    if (staged1) { if (pairs1) decode_words<2, true>(st1, lut1_s, row_s, n_words); else decode_words<1, true>(st1, lut1_s, row_s, n_words); }
-                    else { if (pairs1) decode_words<2, false>(st1, lut1_s, row_s, n_words); else decode_words<1, false>(st1, lut1_s, row_s, n_words); }
-                }
-            }
-            __syncwarp();
-            // ---- cooperative merge: part q covers 16 symbols = 32 output bytes ----
-#pragma unroll
-            for (int i = 0; i < PPL; ++i) {
-                const uint32_t q = i * 32 + lane;
-                const uint32_t j = q / PPL, p = q % PPL;
-                const uint32_t k = j * P.sub + r * R + p * 16;
-                if (k >= c_syms) continue;
-                uint32_t e[4], s[4];
-                if (huff0) {
-                    const uint32_t a = rows0_s + j * kRowStride + p * 16;
-                    e[0] = lds32(a); e[1] = lds32(a + 4); e[2] = lds32(a + 8); e[3] = lds32(a + 12);
-                } else {
-                    const uint4 v = ld_nc_v4(sec0 + c_lo + k);
-                    e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
-                }
-                if (huff1) {
-                    const uint32_t a = rows1_s + j * kRowStride + p * 16;
-                    s[0] = lds32(a); s[1] = lds32(a + 4); s[2] = lds32(a + 8); s[3] = lds32(a + 12);
-                } else { s[0] = raw1[i].x; s[1] = raw1[i].y; s[2] = raw1[i].z; s[3] = raw1[i].w; }
-                uint32_t o[8];
-                merge16<FMT>(e, s, o);
-                merge16<FMT>(e + 2, s + 2, o + 4);
-                const uint32_t byte = 2 * k;
-                uint8_t* dst = P.out + out_lo + byte;
-                if (byte + 32 <= out_bytes) {
-                    st_cs_v8(dst, o);
-                } else {
-#pragma unroll
-                    for (int t = 0; t < 32; ++t)
-                        if (byte + t < out_bytes) dst[t] = (uint8_t)(o[t >> 2] >> (8 * (t & 3)));
-                }
-            }
-            __syncwarp();
-        }
-        if (err) break;
-    }
-    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) {
-        // give copies in flight one more bounded chance to land before the block leaves
-        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0 ^ 1); ++spins) {}
-        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1 ^ 1); ++spins) {}
-    }
+    uint32_t err;
+    if (huff0 && !huff1) err = run_chunks<FMT, PPL, true, false>(P, S, pool, bar, first_end0, first_off0);
+    else if (!huff0 && !huff1) err = run_chunks<FMT, PPL, false, false>(P, S, pool, bar, 0, 0);
+    else if (huff0) err = run_chunks<FMT, PPL, true, true>(P, S, pool, bar, first_end0, first_off0);
+    else err = run_chunks<FMT, PPL, false, true>(P, S, pool, bar, 0, 0);
     if (err) raise_status(P.ctl, P.call_id, err);
 }
 
