@@ -32,6 +32,18 @@ ZC_HD uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel)
 #endif
 }
 
+// x * 128 as a multiply-add, so that it does not compete with the shifts and logic ops for the integer pipe
+ZC_HD uint32_t mul128(uint32_t x)
+{
+#if defined(__CUDA_ARCH__)
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, 128, 0;" : "=r"(r) : "r"(x));
+    return r;
+#else
+    return x * 128u;
+#endif
+}
+
 // two spread pairs -> 4 packed symbols (bytes 0,2 of a then bytes 0,2 of b)
 ZC_HD uint32_t pack_spread(uint32_t a, uint32_t b) { return byte_perm(a, b, 0x6420); }
 // 4 packed symbols -> spread pair of symbols 0,1 / of symbols 2,3 (bytes 1 and 3 are zero)
@@ -128,14 +140,14 @@ template <int FMT>
 ZC_HD void merge16(const uint32_t e[2], const uint32_t sm[2], uint32_t out[4])
 {
     if (FMT == ZC_FMT_BF16) {
-        // element = sign | exponent << 7 | mantissa.  The exponent byte goes to bits 14..7 (placed in byte 1
-        // and shifted right by one); the sign+mantissa byte is duplicated into both bytes so that its bit 7
+        // element = sign | exponent << 7 | mantissa.  The exponent byte goes to bits 14..7 (placed in byte 0
+        // and multiplied by 128 on the multiply-add pipe); the sign+mantissa byte is duplicated into both bytes so that its bit 7
         // lands on bit 15 and its bits 6..0 on bits 6..0; one select picks each bit from the right source.
         const uint32_t m = 0x7F807F80u;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint32_t xl = byte_perm(e[h], 0, 0x1404) >> 1, yl = byte_perm(sm[h], 0, 0x1100);
-            const uint32_t xh = byte_perm(e[h], 0, 0x3424) >> 1, yh = byte_perm(sm[h], 0, 0x3322);
+            const uint32_t xl = mul128(byte_perm(e[h], 0, 0x4140)), yl = byte_perm(sm[h], 0, 0x1100);
+            const uint32_t xh = mul128(byte_perm(e[h], 0, 0x4342)), yh = byte_perm(sm[h], 0, 0x3322);
             out[2 * h] = (xl & m) | (yl & ~m);
             out[2 * h + 1] = (xh & m) | (yh & ~m);
         }

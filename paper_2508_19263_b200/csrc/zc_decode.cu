@@ -228,12 +228,15 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
         if (K == 2) {
             lane_refill<true>(st);
             uint32_t pair[2];
+            uint32_t used = 0;                                    // bits consumed since the last update of st.valid
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t e = lane_peek(st, lut_s);
                 lane_consume(st, e);
-                st.valid -= e & 0xFF;
+                used += e;                                        // low byte = bits; the sum of two stays below 256
                 if ((int)e < 0) {
+                    st.valid -= used & 0xFF;
+                    used = 0;
                     lane_refill<true>(st);
                     const uint32_t f = lane_peek(st, lut_s);
                     const uint32_t l = (f >> 24) & 15;
@@ -243,6 +246,7 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
                 }
                 pair[h] = e;
             }
+            st.valid -= used & 0xFF;
             word = __byte_perm(pair[0], pair[1], 0x6521);
         } else {
             lane_refill<true>(st);
