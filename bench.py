@@ -423,8 +423,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_bf16_llama8b")
-    ap.add_argument("--chunk-kib", type=int, default=16)
-    ap.add_argument("--streams", type=int, default=1,
+    ap.add_argument("--chunk-kib", type=int, default=4)
+    ap.add_argument("--streams", type=int, default=4,
                     help="CUDA streams the per-tensor calls are spread over (tails of one tensor's kernels overlap the next)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used for profiler captures)")

@@ -131,7 +131,7 @@ class Plan:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h:
+        if h and _lib is not None:
             _lib.zc_plan_destroy(h)
             self._h = None
 
@@ -160,7 +160,7 @@ class Codebook:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h:
+        if h and _lib is not None:
             _lib.zc_codebook_destroy(h)
             self._h = None
 
@@ -176,9 +176,14 @@ def histogram(p: Plan, d_in: torch.Tensor, d_hist: Optional[torch.Tensor] = None
 
 def build_codebook(p: Plan, h_hist, policy: int = POLICY_AUTO) -> Codebook:
     """zc_build_codebook: host only.  h_hist: array-like [2, 256] of counts."""
-    h = np.ascontiguousarray(np.asarray(h_hist).astype(np.uint64)).reshape(512)
+    h = np.asarray(h_hist)
+    if h.dtype == np.int64 and h.flags.c_contiguous:
+        h = h.view(np.uint64)                    # counts as produced by histogram(): no copy
+    elif h.dtype != np.uint64 or not h.flags.c_contiguous:
+        h = np.ascontiguousarray(h.astype(np.uint64))
+    assert h.size == 512
     out = C.c_void_p()
-    _check(_lib.zc_build_codebook(p._h, h.ctypes.data_as(C.POINTER(C.c_uint64)), policy, C.byref(out)),
+    _check(_lib.zc_build_codebook(p._h, C.cast(h.ctypes.data, C.POINTER(C.c_uint64)), policy, C.byref(out)),
            "zc_build_codebook")
     return Codebook(out)
 

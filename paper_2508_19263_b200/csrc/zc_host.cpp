@@ -41,43 +41,46 @@ uint64_t rd(const uint8_t* p, int n)
 bool limited_lengths(const uint64_t hist[256], uint32_t L, uint8_t len[256])
 {
     std::memset(len, 0, 256);
-    std::vector<int> order;
+    int order[256];
+    size_t n = 0;
     for (int v = 0; v < 256; ++v)
-        if (hist[v]) order.push_back(v);
-    const size_t n = order.size();
+        if (hist[v]) order[n++] = v;
     if (n == 0) return true;
     if (n == 1) { len[order[0]] = 1; return true; }
-    if ((1ull << L) < n) return false;
-    std::sort(order.begin(), order.end(), [&](int a, int b) {
+    if (L > kLmax || (1ull << L) < n) return false;
+    std::sort(order, order + n, [&](int a, int b) {
         return hist[a] != hist[b] ? hist[a] < hist[b] : a < b;
     });
+    uint64_t leaf_w[256];
+    for (size_t i = 0; i < n; ++i) leaf_w[i] = hist[order[i]];
 
-    struct Level { std::vector<uint64_t> w; std::vector<uint8_t> leaf; };
-    std::vector<Level> lv(L);
-    lv[0].w.resize(n);
-    lv[0].leaf.assign(n, 1);
-    for (size_t i = 0; i < n; ++i) lv[0].w[i] = hist[order[i]];
+    // level r: merged list of the n leaves and the packages made of pairs of level r-1; a list never has
+    // more than 2n - 1 items.  Only the weights are needed to build the next level, only the flags afterwards.
+    static thread_local uint64_t w[2][512];
+    static thread_local uint8_t leaf[kLmax][512];
+    size_t size[kLmax];
+    for (size_t i = 0; i < n; ++i) { w[0][i] = leaf_w[i]; leaf[0][i] = 1; }
+    size[0] = n;
     for (uint32_t r = 1; r < L; ++r) {
-        const Level& prev = lv[r - 1];
-        const size_t np = prev.w.size() / 2;
-        Level& cur = lv[r];
-        cur.w.reserve(n + np);
-        cur.leaf.reserve(n + np);
-        size_t a = 0, b = 0;
-        while (a < n || b < np) {
-            const uint64_t pw = b < np ? prev.w[2 * b] + prev.w[2 * b + 1] : 0;
-            if (b >= np || (a < n && hist[order[a]] <= pw)) {
-                cur.w.push_back(hist[order[a]]); cur.leaf.push_back(1); ++a;
-            } else {
-                cur.w.push_back(pw); cur.leaf.push_back(0); ++b;
-            }
+        const uint64_t* pw = w[(r - 1) & 1];
+        uint64_t* cw = w[r & 1];
+        uint8_t* cf = leaf[r];
+        const size_t np = size[r - 1] / 2;
+        size_t a = 0, b = 0, m = 0;
+        while (a < n && b < np) {
+            const uint64_t pk = pw[2 * b] + pw[2 * b + 1];
+            if (leaf_w[a] <= pk) { cw[m] = leaf_w[a++]; cf[m++] = 1; }
+            else { cw[m] = pk; cf[m++] = 0; ++b; }
         }
+        for (; a < n; ++a) { cw[m] = leaf_w[a]; cf[m++] = 1; }
+        for (; b < np; ++b) { cw[m] = pw[2 * b] + pw[2 * b + 1]; cf[m++] = 0; }
+        size[r] = m;
     }
     size_t take = 2 * n - 2;
     for (int r = (int)L - 1; r >= 0 && take > 0; --r) {
-        if (take > lv[r].w.size()) return false;
+        if (take > size[r]) return false;
         size_t leaves = 0;
-        for (size_t k = 0; k < take; ++k) leaves += lv[r].leaf[k];
+        for (size_t k = 0; k < take; ++k) leaves += leaf[r][k];
         for (size_t i = 0; i < leaves; ++i) len[order[i]]++;
         take = 2 * (take - leaves);
     }
