@@ -64,6 +64,10 @@ def workload_specs(name: str):
         return wl.FP8_E4M3, wl.llama8b_stack(3)
     if name == "cfg4_fp4_llama8b":
         return wl.FP4_E2M1, wl.llama8b_stack(4)
+    if name in ("cfg5_kv_bf16", "cfg5_kv_fp8"):
+        # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers)
+        fmt = wl.BF16 if name.endswith("bf16") else wl.FP8_E4M3
+        return fmt, [wl.TensorSpec(f"kv.{l}.{'kv'[w]}", (8, 8, 32768, 128), 0.0, 10 * l + w) for l in range(4) for w in range(2)]
     if name == "small_bf16":
         return wl.BF16, wl.llama8b_stack(2, n_layers=2, include_embedding=False)
     if name == "small_fp8":
@@ -126,7 +130,10 @@ def oracle_sample(fmt, specs, device):
     """The first tensors of the workload up to ORACLE_SAMPLE_BYTES, as host arrays."""
     out, total = [], 0
     for spec in specs:
-        t, n, _ = wl.make_weight(spec, fmt, device)
+        if spec.name.startswith("kv."):
+            t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, device)
+        else:
+            t, n, _ = wl.make_weight(spec, fmt, device)
         if total and total + t.numel() > ORACLE_SAMPLE_BYTES:
             break
         out.append((spec.name, t.cpu().numpy(), n))
@@ -222,7 +229,10 @@ def run_ours(args):
     # ---- resident inputs, plans, output buffers ----
     tensors = []
     for spec in specs:
-        t, n, _ = wl.make_weight(spec, fmt, dev)
+        if spec.name.startswith("kv."):
+            t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, dev)
+        else:
+            t, n, _ = wl.make_weight(spec, fmt, dev)
         p = zc.plan(fmt, n, chunk_bytes)
         tensors.append({"name": spec.name, "in": t, "n": n, "plan": p,
                         "comp": torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=dev),

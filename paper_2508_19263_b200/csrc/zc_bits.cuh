@@ -124,6 +124,20 @@ ZC_HD void split16(const uint32_t in[4], uint32_t e[2], uint32_t sm[2])
         }
         return;
     }
+    if (FMT == ZC_FMT_FP8_E4M3) {
+        // gather the even elements (low nibbles of the symbols) and the odd ones (high nibbles) of eight bytes,
+        // then build four symbols of each stream with per-byte-lane logic
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t ev = byte_perm(in[2 * h], in[2 * h + 1], 0x6420);
+            const uint32_t od = byte_perm(in[2 * h], in[2 * h + 1], 0x7531);
+            e[h] = ((ev >> 3) & 0x0F0F0F0Fu) | ((od << 1) & 0xF0F0F0F0u);
+            const uint32_t lo = ((ev >> 4) & 0x08080808u) | (ev & 0x07070707u);
+            const uint32_t hi = (od & 0x80808080u) | ((od << 4) & 0x70707070u);
+            sm[h] = lo | hi;
+        }
+        return;
+    }
     uint32_t ea, sa, eb, sb;
     Fields<FMT>::split_word(in[0], ea, sa);
     Fields<FMT>::split_word(in[1], eb, sb);
@@ -150,6 +164,18 @@ ZC_HD void merge16(const uint32_t e[2], const uint32_t sm[2], uint32_t out[4])
             const uint32_t xh = mul128(byte_perm(e[h], 0, 0x4342)), yh = byte_perm(sm[h], 0, 0x3322);
             out[2 * h] = (xl & m) | (yl & ~m);
             out[2 * h + 1] = (xh & m) | (yh & ~m);
+        }
+        return;
+    }
+    if (FMT == ZC_FMT_FP8_E4M3) {
+        // element = sign << 7 | exponent << 3 | mantissa: the even elements come from the low nibbles of four
+        // symbols, the odd ones from the high nibbles; then the two byte vectors are interleaved
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t ev = ((e[h] << 3) & 0x78787878u) | (sm[h] & 0x07070707u) | ((sm[h] << 4) & 0x80808080u);
+            const uint32_t od = ((e[h] >> 1) & 0x78787878u) | ((sm[h] >> 4) & 0x07070707u) | (sm[h] & 0x80808080u);
+            out[2 * h] = byte_perm(ev, od, 0x5140);
+            out[2 * h + 1] = byte_perm(ev, od, 0x7362);
         }
         return;
     }
