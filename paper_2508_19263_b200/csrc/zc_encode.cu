@@ -21,9 +21,9 @@ struct EncParams {
     uint32_t format, group;
     Layout lay;
     uint32_t stage_stride;                       // bytes of one coded stream's lane regions per warp
-    uint32_t region_bytes;                       // one lane region: 1.5 * sub + 4
+    uint32_t region_bytes;                       // one lane region: (n_slots + 1) * sub + 4
     uint32_t sub_width;                          // bytes per sub_end entry (2 or 4)
-    uint32_t deep;                               // lane regions have two pack slots (see encode_kernel)
+    uint32_t n_slots;                            // pack slots per lane region (1..3, see encode_kernel)
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
 };
 
@@ -82,15 +82,17 @@ __device__ bool lookback_exclusive(unsigned long long* flags, uint32_t c, uint32
 
 // Per-warp shared memory of one coded stream: 32 lane regions (+4 bytes of padding each, which also makes
 // the region stride an odd number of words so that lanes walking their regions hit different banks).
-// A region is cut into slots of `sub` bytes.  Two layouts:
-//   plain  [pack | symbols]           the lane packs its codes in place: codes are at most 12 bits, so after k
-//                                     symbols at most 1.5 k bytes are written while the read position is
-//                                     sub + k, and the writer never passes unread symbols
-//   deep   [pack A | pack B | symbols] packing alternates between A and B, so the packed bits of the previous
-//                                     batch survive the packing of the next one and their copy-out can wait a
-//                                     whole iteration for the batch's position in the payload area
-// The packed bits of a subchunk normally stay within one slot (8 bits per symbol); a batch in which some lane
-// needs more is finished on a slow path before anything else is staged.
+// A region is cut into slots of `sub` bytes: n_slots pack slots followed by the symbols,
+//   [pack 0 | .. | pack n_slots-1 | symbols].
+// A lane packs the codes of its subchunk into pack slot (batch index mod n_slots), so the packed bits of the
+// last n_slots batches are alive at the same time and the copy-out of a batch can wait up to n_slots
+// iterations for the batch's position in the payload area (which comes from a look-back over other blocks).
+// Packing into the last slot may run on into the symbols behind it: codes are at most 12 bits, so after k
+// symbols at most 1.5 k bytes are written while the read position is sub + k, and the writer never passes
+// unread symbols.  Packing into any other slot stops at the slot's end.  The packed bits of a subchunk
+// normally fit one slot (8 bits per symbol); a chunk in which some lane needs more is finished on a slow
+// path (everything older is copied out, then the chunk is packed again from slot 0 with the whole region
+// as room) before anything else is staged.
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
@@ -164,12 +166,10 @@ constexpr uint32_t kEncMaxWorkers = 8;       // worker warps per block = chunks 
 
 // What a worker warp keeps about a chunk between packing it and copying it out.
 struct PackedChunk {
-    uint32_t c;                 // chunk index
-    bool active;                // this warp has a chunk in the batch
-    uint32_t slot;              // byte offset of the pack slot inside the lane regions
-    uint32_t bits[2];           // my subchunk's bit count per stream
-    uint32_t end[2];            // inclusive scan of it over the lanes = the sub_end entry
+    uint32_t c;                 // chunk index; kNoChunk: this warp had no chunk in the batch
+    uint32_t end[2];            // per stream: inclusive scan of the subchunks' bit counts over the lanes (= sub_end)
 };
+constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
 
 template <int FMT>
 __global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, 3)
@@ -181,19 +181,25 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     const bool scanner = warp == n_workers;                     // the last warp only does the look-back
     const bool huff0 = P.mode[0] == ZC_MODE_HUFF, huff1 = P.mode[1] == ZC_MODE_HUFF;
     const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
-    const bool deep = P.deep != 0;
+    const uint32_t n_slots = P.n_slots;
 
     // shared: enc[2][256] | per worker warp: regions[n_huff][stage_stride]
     uint32_t* enc = reinterpret_cast<uint32_t*>(smem);
     uint8_t* stage_all = smem + 2048;
     for (uint32_t i = threadIdx.x; i < 512; i += blockDim.x) enc[i] = T.enc[i >> 8][i & 255];
     uint8_t* stage = stage_all + (size_t)(scanner ? 0 : warp) * n_huff * P.stage_stride;
-    const uint32_t region = P.region_bytes;                     // (2 or 3) * sub + 4
-    const uint32_t sym_off = deep ? 2 * P.sub : P.sub;          // symbols sit at this offset inside a region
+    const uint32_t region = P.region_bytes;                     // (n_slots + 1) * sub + 4
+    const uint32_t sym_off = n_slots * P.sub;                   // symbols sit at this offset inside a region
 
-    __shared__ uint32_t s_base[2];
-    __shared__ unsigned long long s_tot[32], s_off[32];
-    __shared__ uint32_t s_fail, s_slow;
+    // The warps of a block are coupled only through these words (no block barrier inside the loop):
+    //   s_base[it & 3], s_base_seq   first chunk of the block's batch `it`; seq = batches handed out so far
+    //   s_tot[it & 3][w], s_cnt[..]  payload size of worker w's chunk; cnt = workers that have posted it
+    //   s_off[it & 3][w], s_off_seq  position of that chunk in the payload area; seq = batches placed so far
+    // A worker has consumed the position of batch `it - n_slots` (n_slots <= 3) before it posts a size for
+    // batch `it`, and the look-back warp places a batch only after every worker has posted, so no warp is more
+    // than three batches away from any other and four copies of each word are enough.
+    __shared__ uint32_t s_base[4], s_base_seq, s_cnt[4], s_off_seq, s_fail;
+    __shared__ unsigned long long s_tot[4][kEncMaxWorkers], s_off[4][kEncMaxWorkers];
 
     // block 0 writes the static parts of the table sections and the tail padding of raw bodies
     if (blockIdx.x == 0) {
@@ -210,25 +216,43 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         }
     }
     if (threadIdx.x == 0) {
-        s_fail = 0; s_slow = 0;
+        s_fail = 0; s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; s_cnt[3] = 0; s_off_seq = 0;
         s_base[0] = atomicAdd(&P.ctl->ticket, n_workers);       // batches of n_workers consecutive chunks
+        s_base_seq = 1;
     }
     __syncthreads();
 
+    // Bounded wait of a whole warp until a sequence word reaches `target`; false on a failure flag or when
+    // the wait gives up (the caller then raises the failure flag itself).
+    auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
+        bool ok = false;
+        for (uint32_t n = 0; n < kSpinLimit; ++n) {
+            if (*reinterpret_cast<const volatile uint32_t*>(word) >= target) { ok = true; break; }
+            if (*reinterpret_cast<const volatile uint32_t*>(&s_fail)) break;
+            if (n > 64) __nanosleep(40);
+        }
+        __syncwarp();
+        __threadfence_block();
+        return ok;
+    };
+
     // ---- copy-out of a packed chunk: every lane moves its bits to their final position in the piece ----
-    auto copy_out = [&](const PackedChunk& pc, const uint64_t off16) {
+    auto copy_out = [&](const PackedChunk& pc, const uint32_t slot, const uint64_t off16) {
         uint32_t hs = 0;
         uint64_t piece_off16 = off16;
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
             if (P.mode[s] != ZC_MODE_HUFF) continue;
-            const uint32_t end = pc.end[s], bits = pc.bits[s], start = end - bits;
+            const uint32_t end = pc.end[s];
+            uint32_t start = __shfl_up_sync(0xFFFFFFFFu, end, 1);
+            if (lane == 0) start = 0;
+            const uint32_t bits = end - start;
             const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
             const uint32_t piece16 = (chunk_bits + 127) / 128;
             if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[pc.c] = (uint32_t)piece_off16;
             uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
             const uint32_t piece_words = 4 * piece16;
-            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region) + pc.slot;
+            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region) + slot;
             const uint32_t sh = start & 31, d0 = start >> 5;
             const uint32_t n_dst = (sh + bits + 31) / 32;             // destination words I touch
             const uint32_t n_src = (bits + 31) / 32;
@@ -287,16 +311,74 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
     };
 
     uint32_t bad = 0;
-    PackedChunk prev{0, false, 0, {0, 0}, {0, 0}};
-    bool pending = false;                                       // a packed batch still waits for its copy-out
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t base = s_base[it & 1];
-        const bool have = base < P.n_chunks;
-        if (!have && !pending) break;
 
-        PackedChunk cur{base + warp, have && !scanner && base + warp < P.n_chunks, deep ? (it & 1) * P.sub : 0u, {0, 0}, {0, 0}};
-        const uint64_t c_lo = (uint64_t)(cur.active ? cur.c : 0) * P.cs;
-        const uint32_t c_syms = cur.active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
+    if (scanner) {
+        // ---- the look-back warp places batch after batch; the workers are a batch ahead of it ----
+        for (uint32_t it = 0; n_huff; ++it) {
+            if (!wait_seq(&s_base_seq, it + 1)) { s_fail = 1; break; }
+            const uint32_t base = *reinterpret_cast<const volatile uint32_t*>(&s_base[it & 3]);
+            if (base >= P.n_chunks) break;
+            bool ok = false;
+            for (uint32_t n = 0; n < kSpinLimit; ++n) {             // every worker posts a size (0 without a chunk)
+                if (*reinterpret_cast<const volatile uint32_t*>(&s_cnt[it & 3]) == n_workers) { ok = true; break; }
+                if (*reinterpret_cast<const volatile uint32_t*>(&s_fail)) break;
+                __nanosleep(40);
+            }
+            __syncwarp();
+            __threadfence_block();
+            if (!ok) { s_fail = 1; break; }
+            if (lane == 0) s_cnt[it & 3] = 0;
+            unsigned long long v = lane < n_workers ? *reinterpret_cast<const volatile unsigned long long*>(&s_tot[it & 3][lane]) : 0ull, inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= (uint32_t)o) inc += t;
+            }
+            const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint64_t batch_off = 0;
+            ok = lookback_exclusive(P.flags, base / n_workers, lane, batch_total, batch_off);
+            if (lane < n_workers) s_off[it & 3][lane] = batch_off + inc - v;
+            __threadfence_block();
+            __syncwarp();
+            if (!ok) { s_fail = 1; break; }
+            if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = it + 1;
+        }
+    } else {
+    // packed chunks that wait for their copy-out, newest first: q0 is batch it - 1, q1 batch it - 2, ...
+    PackedChunk q0{kNoChunk, {0, 0}}, q1 = q0, q2 = q0;
+    uint32_t n_pend = 0;
+    uint32_t slot_idx = 0;                                      // pack slot of batch `it`: it mod n_slots
+    // waits until the oldest pending batch is placed and copies this warp's chunk of it out
+    auto flush_oldest = [&](const uint32_t it) -> bool {
+        const uint32_t j = it - n_pend;                         // the batch in question
+        if (n_huff) {
+            if (!wait_seq(&s_off_seq, j + 1)) return false;
+            PackedChunk pc;
+            pc.c = n_pend == 1 ? q0.c : n_pend == 2 ? q1.c : q2.c;
+            pc.end[0] = n_pend == 1 ? q0.end[0] : n_pend == 2 ? q1.end[0] : q2.end[0];
+            pc.end[1] = n_pend == 1 ? q0.end[1] : n_pend == 2 ? q1.end[1] : q2.end[1];
+            // its slot: the slots are used round-robin, so it lies n_pend steps behind the current one
+            const uint32_t sl = (slot_idx + n_slots * 4 - n_pend) % n_slots;
+            if (pc.c != kNoChunk) copy_out(pc, sl * P.sub, *reinterpret_cast<const volatile unsigned long long*>(&s_off[j & 3][warp]));
+        }
+        --n_pend;
+        return true;
+    };
+    bool failed = false;
+    for (uint32_t it = 0;; ++it) {
+        if (!wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
+        const uint32_t base = *reinterpret_cast<const volatile uint32_t*>(&s_base[it & 3]);
+        const bool have = base < P.n_chunks;
+        if (!have) {
+            while (n_pend && !failed) failed = !flush_oldest(it);
+            break;
+        }
+
+        const bool active = base + warp < P.n_chunks;
+        PackedChunk cur{active ? base + warp : kNoChunk, {0, 0}};
+        const uint32_t slot = slot_idx * P.sub;
+        const uint64_t c_lo = (uint64_t)(active ? cur.c : 0) * P.cs;
+        const uint32_t c_syms = active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
 
         // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
         auto stage_group = [&](const uint4 x, const uint32_t k) {
@@ -337,13 +419,8 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
         }
         __syncwarp();
 
-        // plain layout: the previous batch must leave its slot before this batch is packed into it; its
-        // look-back ran while this batch was loaded
-        if (!deep) {
-            __syncthreads();
-            if (s_fail) break;
-            if (pending && prev.active && n_huff) copy_out(prev, s_off[warp]);
-        }
+        // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
+        if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
 
         // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
         const uint32_t lo_sym = lane * P.sub;
@@ -376,36 +453,31 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                 seen |= e;
                 put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr, limit);
             }
-            if (cur.active && waddr < limit) sts32(waddr, hi);      // pending bits (or zero)
+            if (active && waddr < limit) sts32(waddr, hi);          // pending bits (or zero)
             bad |= seen & 16;                                       // an entry without a code carries bit 4
             return 8 * (waddr - w0) + nb;
         };
+        bool oversize = false;
+        uint32_t my_bits[2] = {0, 0};
+        const bool last_slot = slot_idx + 1 == n_slots;
         {
             uint32_t hs = 0;
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
-                // deep layout, slot A: anything beyond the slot would overwrite the previous batch in slot B
-                const uint32_t room = (deep && cur.slot == 0) ? P.sub : 3 * P.sub;
-                cur.bits[s] = pack(s, hs, cur.slot, room);
+                // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
+                my_bits[s] = pack(s, hs, slot, last_slot ? 2 * P.sub : P.sub);
                 // more than 8 bits per symbol: the bits beyond the slot do not survive the next staging
-                if (cur.bits[s] > 8 * P.sub) s_slow = 1;
+                oversize |= my_bits[s] > 8 * P.sub;
                 ++hs;
             }
-        }
-
-        // deep layout: the previous batch sits in the other pack slot; its look-back had this whole packing time
-        if (deep) {
-            __syncthreads();
-            if (s_fail) break;
-            if (pending && prev.active && n_huff) copy_out(prev, s_off[warp]);
         }
 
         // the ticket of the next batch is taken as late as possible (batches must start in the order they
         // were handed out, or the look-back of other blocks waits for a batch that is not even begun); its
         // latency hides behind phase C
-        uint32_t next_base = base;
-        if (threadIdx.x == 0 && have) next_base = atomicAdd(&P.ctl->ticket, n_workers);
+        uint32_t next_base = 0;
+        if (threadIdx.x == 0) next_base = atomicAdd(&P.ctl->ticket, n_workers);
 
         // ---- phase C: subchunk end bits and the chunk's size in the payload area ----
         uint64_t tot16 = 0;
@@ -413,14 +485,14 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (P.mode[s] != ZC_MODE_HUFF) continue;
-                uint32_t inc = cur.bits[s];
+                uint32_t inc = my_bits[s];
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
                     if (lane >= (uint32_t)o) inc += t;
                 }
                 cur.end[s] = inc;
-                if (cur.active) {
+                if (active) {
                     if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * cur.c)[lane] = (uint16_t)inc;
                     else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * cur.c)[lane] = inc;
                     const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
@@ -429,48 +501,42 @@ encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTa
                 }
             }
         }
-        if (lane == 0) s_tot[warp] = tot16;
-        if (threadIdx.x == 0) s_base[(it + 1) & 1] = next_base;
-        __syncthreads();
-
-        // ---- the look-back warp places the batch; the workers go on with the next batch meanwhile ----
-        const bool slow = s_slow != 0;
-        if (scanner && have && n_huff) {
-            unsigned long long v = lane < n_workers ? s_tot[lane] : 0ull, inc = v;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                if (lane >= (uint32_t)o) inc += t;
-            }
-            const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            uint64_t batch_off = 0;
-            const bool ok = lookback_exclusive(P.flags, base / n_workers, lane, batch_total, batch_off);
-            s_off[lane] = batch_off + inc - v;
-            if (!ok && lane == 0) s_fail = 1;
+        if (lane == 0 && n_huff) {
+            s_tot[it & 3][warp] = tot16;
+            __threadfence_block();
+            atomicAdd(&s_cnt[it & 3], 1u);
         }
-        if (slow) {
-            // some subchunk needs more than 8 bits per symbol: finish this batch before anything else is staged.
-            // In the deep layout the other slot is free by now, so a clipped packing into slot A is redone.
-            if (deep && cur.slot == 0) {
+        if (threadIdx.x == 0) {
+            s_base[(it + 1) & 3] = next_base;
+            __threadfence_block();
+            *reinterpret_cast<volatile uint32_t*>(&s_base_seq) = it + 2;
+        }
+
+        q2 = q1; q1 = q0; q0 = cur;
+        ++n_pend;
+        slot_idx = last_slot ? 0 : slot_idx + 1;
+        if (__any_sync(0xFFFFFFFFu, oversize)) {
+            // some subchunk needs more than 8 bits per symbol: finish this chunk before anything else is staged.
+            // Once everything older has left, a packing that was clipped at the end of its slot is redone from
+            // slot 0 with the rest of the region as room.
+            while (n_pend > 1 && !failed) failed = !flush_oldest(it + 1);
+            if (failed) break;
+            if (!last_slot) {
                 uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     if (P.mode[s] != ZC_MODE_HUFF) continue;
-                    pack(s, hs, 0, 3 * P.sub);
+                    pack(s, hs, 0, 2 * P.sub);
                     ++hs;
                 }
                 __syncwarp();
+                slot_idx = 1;                                   // the chunk now sits in slot 0, one behind
             }
-            __syncthreads();
-            if (s_fail) break;
-            if (cur.active && n_huff) copy_out(cur, s_off[warp]);
-            __syncthreads();
-            if (threadIdx.x == 0) s_slow = 0;
-            pending = false;
-        } else {
-            prev = cur;
-            pending = have;
+            if (!flush_oldest(it + 1)) { failed = true; break; }
+            slot_idx = 0;                                       // nothing is pending: start over with slot 0
         }
+    }
+    if (failed) s_fail = 1;
     }
     if (s_fail && threadIdx.x == 0) raise_status(P.ctl, 0, ZC_E_DEVICE_TIMEOUT);
     if (bad) raise_status(P.ctl, 0, ZC_E_NO_CODE);
@@ -514,9 +580,13 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
         n_huff += P.mode[s] == ZC_MODE_HUFF;
     }
     P.lay = make_layout(*p, P.mode);
-    // two pack slots per lane region when the chunks are small enough to keep three blocks per SM resident
-    P.deep = p->chunk_bytes <= 4096 ? 1u : 0u;
-    P.region_bytes = (P.deep ? 3 : 2) * p->syms_per_sub + 4;
+    // as many pack slots per lane region (up to 3) as still leave three blocks of 8 worker warps per SM
+    P.n_slots = 1;
+    for (uint32_t ns = 3; ns > 1; --ns) {
+        const size_t block = 2048 + (size_t)kEncMaxWorkers * std::max<uint32_t>(n_huff, 1) * kSubs * ((ns + 1) * p->syms_per_sub + 4);
+        if (3 * (block + 1024) <= kMaxSmem + 1024) { P.n_slots = ns; break; }
+    }
+    P.region_bytes = (P.n_slots + 1) * p->syms_per_sub + 4;
     P.sub_width = sub_end_width(p->chunk_bytes);
     P.stage_stride = kSubs * P.region_bytes;
     P.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);

@@ -119,6 +119,36 @@ def test_long_codes_and_skew():
     assert cb.get(0)[1].max() == 12
 
 
+@pytest.mark.parametrize("policy", [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL])
+@pytest.mark.parametrize("chunk_bytes", [1024, 4096, 6144, 8192, 32768])
+def test_subchunks_above_eight_bits_per_symbol(chunk_bytes, policy):
+    """A static dictionary meets runs of its rarest symbols: some subchunks need 12 bits per symbol, more than
+    the staging slot of the encoder holds, in the first, the last, neighbouring and isolated chunks (the chunk
+    sizes and the number of coded streams cover every staging layout of the encoder)."""
+    rng = np.random.default_rng(chunk_bytes)
+    cs = chunk_bytes // 2
+    n = 41 * cs + cs // 2 + 3
+    common = rng.choice([120, 121, 122, 123], size=n, p=[0.5, 0.25, 0.15, 0.1]).astype(np.uint16)
+    e = common.copy()
+    rare = np.arange(10, 74, dtype=np.uint16)                      # 64 exponents the dictionary barely knows
+    for c in (0, 1, 2, 7, 9, 10, 11, 12, 20, 33, 40, 41):
+        lo = c * cs + int(rng.integers(0, cs // 2))
+        hi = min(n, lo + int(rng.integers(cs // 16, cs)))
+        e[lo:hi] = rare[rng.integers(0, rare.size, hi - lo)]
+    m = rng.integers(0, 128, n).astype(np.uint16)
+    sgn = rng.integers(0, 2, n).astype(np.uint16)
+    data = ((sgn << 15) | (e << 7) | m).astype(np.uint16).view(np.uint8)
+    dict_hist = np.zeros((2, 256), np.uint64)
+    dict_hist[0, 120:124] = [500000, 250000, 150000, 100000]
+    dict_hist[0, rare] = 1
+    dict_hist[1] = zo.histogram(zo.BF16, data, n)[1]
+    p, cb, hist, cont = _gpu_round_trip(zc.FMT_BF16, data, n, chunk_bytes, policy, oracle_codebook_hist=dict_hist)
+    assert cb.get(0)[1][rare].min() > 8
+    off16, sub_end, _ = zo.read_tables(cont, 0)
+    sub_bits = np.diff(np.concatenate([np.zeros((sub_end.shape[0], 1), np.int64), sub_end.astype(np.int64)], axis=1), axis=1)
+    assert (sub_bits > 8 * (cs // 32)).any()                       # the case this test is about did occur
+
+
 def test_static_dictionary_and_missing_code():
     a = _weights(zc.FMT_BF16, 50000, 1)
     b = _weights(zc.FMT_BF16, 50000, 2)
