@@ -6,12 +6,12 @@
  * Low-Precision Formats" (Heilper & Singer, 2025): every BF16 / FP8 E4M3 /
  * FP4 E2M1 element is split into an exponent field and a sign+mantissa field
  * (Sec. 3.1, 3.2, 3.4), the fields of 1 / 2 / 4 neighbouring elements are
- * grouped into byte symbols (Fig. 7 caption; Sec. 3.4 "2 bits from each of the
- * 4 consecutive FP4 values"), each of the two symbol streams gets its own
+ * grouped into byte symbols (Fig. 7 caption for FP8 pairs; Sec. 3.4 for the 2-bit fields of four FP4
+ * values that share a byte), each of the two symbol streams gets its own
  * Huffman code or is stored raw when it does not compress (Sec. 3.1), and the
- * result is written in fixed-size chunks that decode independently (Sec. 3.1
- * "fixed-size chunks with lightweight metadata ... random access and parallel
- * decoding").  Decoding restores the original bit patterns exactly.
+ * result is written in fixed-size chunks that decode independently (Sec. 3.1:
+ * chunks of fixed size with a little metadata each, so that any chunk can be
+ * found and all chunks decode in parallel).  Decoding restores the original bit patterns exactly.
  *
  * Conventions
  *   - "d_" pointers are DEVICE pointers of the current CUDA device, "h_" pointers
@@ -126,8 +126,8 @@ typedef struct zc_stats_t {
     double ratio_container;     /* out_bytes / in_bytes, 0 without header */
 } zc_stats_t;
 
-/* ---- plan: problem statement of one tensor (Sec. 4 "compression was applied per tensor
- *      using fixed-size chunks") ------------------------------------------------------------
+/* ---- plan: problem statement of one tensor (Sec. 4: every tensor is compressed on its
+ *      own, in chunks of one fixed size) -----------------------------------------------------
  * fmt         element format
  * n_elems     number of elements (0 is valid and gives a header-only container);
  *             must be even for FP4
@@ -153,7 +153,7 @@ size_t zc_workspace_bytes(const zc_plan_t* plan);
  * Asynchronous on cuda_stream.  Errors: INVALID_ARG, CUDA. */
 zc_status zc_histogram(const zc_plan_t* plan, const void* d_in, uint64_t* d_hist, void* cuda_stream);
 
-/* ---- codebook (Sec. 3.1 / 4.1 "standard Huffman encoding", one code per stream per tensor;
+/* ---- codebook (Sec. 3.1 / 4.1: plain Huffman coding, one code per stream per tensor;
  *      Sec. 3.3 precomputed dictionaries: any histogram may be given) ------------------------
  * h_hist  host, uint64_t[2][256]
  * policy  which streams are Huffman-coded
@@ -218,7 +218,7 @@ zc_status zc_compress(const zc_plan_t* plan, const zc_codebook_t* cb, const void
 zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, void* d_out,
                               size_t out_capacity, uint64_t* h_out_bytes, void* cuda_stream);
 
-/* ---- decompress (Sec. 3.1 "parallel decoding") --------------------------------------------
+/* ---- decompress (Sec. 3.1: chunks decode independently, in parallel) ------------------------
  * d_comp      device, a container made for the same plan; comp_bytes = bytes available
  * d_out       device, receives zc_plan_info.input_bytes bytes, identical to the original
  * The header is checked on the device against the plan before anything is decoded; a
@@ -237,7 +237,7 @@ zc_status zc_device_status(const zc_plan_t* plan, const void* d_workspace, void*
  * offsets and subchunk ends, payload bit totals.  Returns ZC_OK or ZC_E_CORRUPT. */
 zc_status zc_validate_container(const zc_plan_t* plan, const void* h_container, size_t bytes);
 
-/* zc_stats (Sec. 4 "component-wise breakdown (exponent vs. mantissa)"): per-stream and total
+/* zc_stats (Sec. 4 reports exponent and mantissa results separately): per-stream and total
  * sizes and ratios from a histogram and a codebook; h_header (host copy of at least the first
  * 128 container bytes) is optional and adds the container-inclusive figures. */
 zc_status zc_stats(const zc_plan_t* plan, const zc_codebook_t* cb, const uint64_t* h_hist,

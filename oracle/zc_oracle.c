@@ -13,17 +13,17 @@
  * What the paper fixes, and where each function follows it:
  *   - Field split (Sec. 3.1 BF16: 1 sign, 8 exponent, 7 mantissa bits;
  *     Sec. 3.2 FP8 E4M3: 1 sign, 4 exponent, 3 mantissa bits; Sec. 3.4 / 4.4
- *     FP4: "2 bits from each of 4 consecutive values" form a byte):
+ *     FP4: the 2-bit fields of 4 consecutive values form a byte):
  *     zo_split / zo_merge.
  *   - Byte grouping of two FP8 elements' exponents and two elements'
  *     sign+mantissa (Fig. 7 caption): zo_split.
- *   - One Huffman code per stream per tensor (Sec. 3.1, 3.2, 4.1 "per layer
- *     file, using standard Huffman encoding"): zo_code_lengths,
+ *   - One Huffman code per stream per tensor (Sec. 3.1, 3.2, 4.1: plain Huffman
+ *     coding, applied to each layer file on its own): zo_code_lengths,
  *     zo_canonical_codes.
- *   - Mantissa "evaluated for entropy; Huffman if compressible, otherwise
- *     stored uncompressed" (Sec. 3.1, 4.3): zo_choose_mode.
- *   - "Fixed-size chunks with lightweight metadata per block, designed for
- *     random access and parallel decoding" (Sec. 3.1, Sec. 4): zo_compress,
+ *   - The mantissa stream is Huffman-coded only when its entropy makes that
+ *     worthwhile and is stored as is otherwise (Sec. 3.1, 4.3): zo_choose_mode.
+ *   - Chunks of one fixed size, each with a little metadata, so that chunks
+ *     can be located and decoded independently (Sec. 3.1, Sec. 4): zo_compress,
  *     zo_decompress, zo_decompress_chunk.
  *
  * What the paper leaves open (bit positions inside a grouped byte, the length
@@ -332,8 +332,8 @@ uint64_t zo_payload_bits(const uint64_t hist[256], const uint8_t len[256])
     return t;
 }
 
-/* RAW/HUFF decision of one stream (reading R6; Sec. 3.1 "if compressibility is
- * high ... otherwise stored uncompressed"). */
+/* RAW/HUFF decision of one stream (reading R6; Sec. 3.1: a stream is coded
+ * only when that pays, and stored uncompressed otherwise). */
 int zo_choose_mode(const uint64_t hist[256], const uint8_t len[256], int policy)
 {
     uint64_t n = 0;
@@ -705,7 +705,7 @@ int64_t zo_decompress(const uint8_t *cont, uint64_t bytes, uint8_t *out, uint64_
 }
 
 /* ------------------------------------------------------------------ */
-/* Statistics (Sec. 4 "component-wise breakdown")                      */
+/* Statistics (Sec. 4: results per component)                         */
 /* ------------------------------------------------------------------ */
 
 typedef struct {
