@@ -273,7 +273,16 @@ def run_ours(args):
             zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=lanes[i % len(lanes)])
         join()
 
+    # every tensor of the stack in one call; the decoder only needs an upper bound of each container's size
+    # (the header carries the exact one)
+    dec_batch = zc.DecompressBatch([t["plan"] for t in tensors], [t["comp"] for t in tensors],
+                                   [t["plan"].max_compressed_bytes for t in tensors], [t["out"] for t in tensors])
+    batch_ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+
     def phase_decompress():
+        if args.batch:
+            zc.decompress_batch(dec_batch, batch_ws, stream=stream)
+            return
         fork()
         for i, t in enumerate(tensors):
             zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"], stream=lanes[i % len(lanes)])
@@ -296,9 +305,11 @@ def run_ours(args):
             ln = lanes[i % len(lanes)]
             t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
             zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=ln)
-            # the decoder only needs an upper bound of the container size; the header carries the exact one
-            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], stream=ln)
+            if not args.batch:
+                zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], stream=ln)
         join()
+        if args.batch:
+            zc.decompress_batch(dec_batch, batch_ws, stream=stream)
 
     def timed(fn, reps):
         barrier()
@@ -324,6 +335,8 @@ def run_ours(args):
             raise SystemExit(f"device status {st} on {t['name']}")
         if not torch.equal(t["out"], t["in"]):
             raise SystemExit(f"round trip mismatch on {t['name']}")
+    if args.batch and zc.batch_status(batch_ws) != (zc.OK, None):
+        raise SystemExit(f"batch status {zc.batch_status(batch_ws)}")
     C = sum(t["cbytes"] for t in tensors)
 
     for _ in range(max(args.warmup - 1, 0)):
@@ -444,6 +457,8 @@ def main():
     ap.add_argument("--chunk-kib", type=int, default=4)
     ap.add_argument("--streams", type=int, default=4,
                     help="CUDA streams the per-tensor calls are spread over (tails of one tensor's kernels overlap the next)")
+    ap.add_argument("--batch", type=int, default=1, choices=[0, 1],
+                    help="1: the batched entry points (all tensors of the stack per call); 0: one call per tensor")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used for profiler captures)")
     args = ap.parse_args()

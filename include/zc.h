@@ -227,6 +227,33 @@ zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, co
 zc_status zc_decompress(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes, void* d_out,
                         void* d_workspace, void* cuda_stream);
 
+/* ---- decompress many tensors with one call (Sec. 4 and 4.1: a model or a checkpoint is a set of
+ *      tensors, each compressed on its own; Sec. 3.3: the K and V tensors of all layers) --------
+ * The result is the same as n_tensors calls of zc_decompress; the work of all tensors is spread
+ * over the GPU in one launch (per 512 tensors), so that small tensors do not pay a launch and a
+ * table build per block each.
+ * n_tensors     number of tensors (0 returns ZC_OK and launches nothing)
+ * plans         host array of n_tensors plans; all must have the same format and chunk_bytes
+ * d_comp        host array of n_tensors DEVICE pointers (16-byte aligned), one container each
+ * comp_bytes    host array: bytes available behind each d_comp[t]
+ * d_out         host array of n_tensors DEVICE pointers (16-byte aligned); d_out[t] receives
+ *               input_bytes of plans[t].  The outputs must not overlap.
+ * d_workspace   device, at least 256 bytes (zc_workspace_bytes of any plan is enough)
+ * The arrays are read before the call returns; the caller keeps ownership of everything.
+ * A tensor whose header or tables are damaged is skipped (nothing of it is written), the others
+ * are still decoded; the first error and its tensor are recorded on the device, read them with
+ * zc_batch_status().  Asynchronous.
+ * Errors: INVALID_ARG (null or misaligned pointers, mixed formats or chunk sizes), CORRUPT
+ * (a comp_bytes[t] below the header size), UNSUPPORTED, CUDA. */
+zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_comp,
+                              const size_t* comp_bytes, void* const* d_out, void* d_workspace,
+                              void* cuda_stream);
+
+/* Synchronise cuda_stream and return the status the last batch call on this workspace left on
+ * the device (ZC_OK if none).  h_failed_tensor (optional, host) receives the index of the tensor
+ * the first recorded error belongs to, or 0xFFFFFFFF. */
+zc_status zc_batch_status(const void* d_workspace, uint32_t* h_failed_tensor, void* cuda_stream);
+
 /* Synchronise cuda_stream and return the status word the last zc_compress / zc_decompress
  * call on this workspace left on the device (ZC_OK if none was raised). */
 zc_status zc_device_status(const zc_plan_t* plan, const void* d_workspace, void* cuda_stream);

@@ -81,6 +81,10 @@ def _load():
     L.zc_compress_noalloc.argtypes = [vp, vp, vp, vp, C.c_size_t, u64p, vp]
     L.zc_decompress.restype = C.c_int
     L.zc_decompress.argtypes = [vp, vp, C.c_size_t, vp, vp, vp]
+    L.zc_decompress_batch.restype = C.c_int
+    L.zc_decompress_batch.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), vp, vp]
+    L.zc_batch_status.restype = C.c_int
+    L.zc_batch_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     L.zc_device_status.restype = C.c_int
     L.zc_device_status.argtypes = [vp, vp, vp]
     L.zc_validate_container.restype = C.c_int
@@ -225,6 +229,33 @@ def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tens
 
 def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:
     return _lib.zc_device_status(p._h, d_workspace.data_ptr(), _stream_ptr(stream))
+
+
+class DecompressBatch:
+    """Argument arrays of zc_decompress_batch, marshalled once and reusable for repeated calls."""
+
+    def __init__(self, plans, d_comps, comp_bytes, d_outs):
+        n = len(plans)
+        assert len(d_comps) == n and len(comp_bytes) == n and len(d_outs) == n
+        self.n = n
+        self._keep = (list(plans), list(d_comps), list(d_outs))        # the arrays hold raw pointers
+        self.plans = (C.c_void_p * n)(*[p._h.value for p in plans])
+        self.comps = (C.c_void_p * n)(*[t.data_ptr() for t in d_comps])
+        self.sizes = (C.c_size_t * n)(*[int(b) for b in comp_bytes])
+        self.outs = (C.c_void_p * n)(*[t.data_ptr() for t in d_outs])
+
+
+def decompress_batch(batch: DecompressBatch, d_workspace: torch.Tensor, stream=None) -> None:
+    """zc_decompress_batch (asynchronous; read the outcome with batch_status)."""
+    _check(_lib.zc_decompress_batch(batch.n, batch.plans, batch.comps, batch.sizes, batch.outs, d_workspace.data_ptr(),
+                                    _stream_ptr(stream)), "zc_decompress_batch")
+
+
+def batch_status(d_workspace: torch.Tensor, stream=None):
+    """zc_batch_status: (status, index of the failing tensor or None)."""
+    failed = C.c_uint32(0xFFFFFFFF)
+    st = _lib.zc_batch_status(d_workspace.data_ptr(), C.byref(failed), _stream_ptr(stream))
+    return st, (None if failed.value == 0xFFFFFFFF else failed.value)
 
 
 def validate_container(p: Plan, h_container) -> int:

@@ -24,6 +24,23 @@ struct DecParams {
     unsigned long long call_id;
 };
 
+// One tensor of a batch, and the parameters of a batched launch.  The tensors share format and chunk size;
+// the chunks of all of them form one index space that is cut into equal contiguous ranges, one per block.
+struct DecItem {
+    const uint8_t* comp;
+    uint8_t* out;
+    uint64_t comp_bytes, input_bytes, n_syms, n_elems;
+    uint32_t n_chunks, first_chunk;          // first_chunk = chunks of all earlier tensors of the launch
+};
+constexpr uint32_t kDecBatchMax = 512;       // tensors per launch: the parameter block stays below 32 KiB
+struct DecBatchParams {
+    Control* ctl;
+    unsigned long long call_id;
+    uint32_t cs, sub, chunk_bytes, format, group, pool_bytes;
+    uint32_t n_tensors, total_chunks, tensor_base, n_ranges;
+    DecItem item[kDecBatchMax];
+};
+
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
 constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
 constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
@@ -302,13 +319,15 @@ struct DecShared {                   // what the block's prologue leaves for the
 // PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
 template <int FMT, int PPL, bool H0, bool H1>
 __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShared& S, uint8_t* pool, uint64_t* bar,
-                                               uint32_t first_end0, uint32_t first_off0)
+                                               uint32_t first_end0, uint32_t first_off0,
+                                               uint32_t c, const uint32_t c_end, const uint32_t step,
+                                               uint32_t& parity0, uint32_t& parity1)
 {
     constexpr uint32_t R = 16 * PPL;
     constexpr uint32_t kRowStride = R + 4;                     // bytes; the padding spreads the lanes' rows over the banks
     constexpr uint32_t kRowsBytes = 32 * kRowStride;           // one stream's rows of a warp (multiple of 16)
     constexpr uint32_t kHuff = (H0 ? 1u : 0u) + (H1 ? 1u : 0u);
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const uint32_t lane = threadIdx.x & 31;
     const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;
     const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
     const uint8_t* sec0 = P.comp + S.sec0;
@@ -322,21 +341,19 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
     const uint32_t slot_bytes = kHuff ? (slot_room / (kHuff ? kHuff : 1)) & ~15u : 0u;
     const uint32_t rows0_s = smem_u32(pool), rows1_s = rows0_s + rows1_off;
     const uint32_t slot0_s = rows0_s + slots_off, slot1_s = slot0_s + (H0 ? slot_bytes : 0);
-    const uint32_t step = gridDim.x * n_warps;
-    uint32_t parity0 = 0, parity1 = 0, err = 0;
+    uint32_t err = 0;
 
     // this lane's parts of a round: part i covers symbols k_lane + i * k_step (+ round offset) of the chunk
     const uint32_t k_lane = (lane / PPL) * P.sub + (lane % PPL) * 16, k_step = (32 / PPL) * P.sub;
     const uint32_t row_lane = (lane / PPL) * kRowStride + (lane % PPL) * 16, row_step = (32 / PPL) * kRowStride;
 
-    uint32_t c = blockIdx.x * n_warps + warp;
     uint32_t nx_end0 = first_end0, nx_off0 = first_off0, nx_end1 = 0, nx_off1 = 0;
-    if (H1 && c < P.n_chunks) {
+    if (H1 && c < c_end) {
         nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, c, lane);
         nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c];
     }
 
-    for (; c < P.n_chunks; c += step) {
+    for (; c < c_end; c += step) {
         const uint64_t c_lo = (uint64_t)c * P.cs;
         const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
         const uint64_t out_lo = 2 * c_lo;                       // two element bytes per symbol in every format
@@ -389,7 +406,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         // request the next chunk's table entries now; they are consumed in the next iteration
         {
             const uint32_t cn = c + step;
-            if (cn < P.n_chunks) {
+            if (cn < c_end) {
                 if (H0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
                           nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
                 if (H1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
@@ -495,32 +512,49 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
 // ------------------------------------------------------------------------------------------------
 // PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
 
-template <int FMT, int PPL>
-__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
-decode_kernel(const __grid_constant__ DecParams P)
+struct DecSmem {                     // the block's dynamic shared memory, carved up once per kernel
+    uint32_t* lut0;                  // decode table of stream 0
+    uint32_t* lut1;                  // decode table of stream 1
+    uint32_t* scratch;
+    uint8_t* pools;                  // all warps' pools
+    uint8_t* pool;                   // this warp's pool
+    uint64_t* bar;                   // this warp's two mbarriers
+};
+
+__device__ __forceinline__ DecSmem carve_smem(uint8_t* smem, uint32_t pool_bytes)
 {
-    extern __shared__ __align__(16) uint8_t smem[];
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-
-    uint32_t* lut0 = reinterpret_cast<uint32_t*>(smem);                 // decode table of stream 0
-    uint32_t* lut1 = reinterpret_cast<uint32_t*>(smem + kLutBytes);     // decode table of stream 1
-    uint32_t* scratch = reinterpret_cast<uint32_t*>(smem + 2 * kLutBytes);
+    const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    DecSmem m;
+    m.lut0 = reinterpret_cast<uint32_t*>(smem);
+    m.lut1 = reinterpret_cast<uint32_t*>(smem + kLutBytes);
+    m.scratch = reinterpret_cast<uint32_t*>(smem + 2 * kLutBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecFixedSmem);
-    uint8_t* pools = reinterpret_cast<uint8_t*>(bars + 2 * n_warps);
-    uint8_t* pool = pools + (size_t)warp * P.pool_bytes;
-    uint64_t* bar = bars + 2 * warp;
+    m.pools = reinterpret_cast<uint8_t*>(bars + 2 * n_warps);
+    m.pool = m.pools + (size_t)warp * pool_bytes;
+    m.bar = bars + 2 * warp;
+    if ((threadIdx.x & 31) == 0) { mbar_init(&m.bar[0], 1); mbar_init(&m.bar[1], 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    return m;
+}
 
+// Decodes the chunks c0, c0 + step, ... (< c_end) of one tensor with this warp; the whole block calls it
+// together (the header check and the table build are block-wide).  Returns a zc_status, the same in every
+// thread for the block-wide checks.
+template <int FMT, int PPL>
+__device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem& M, const uint32_t c0, const uint32_t c_end,
+                                               const uint32_t step, uint32_t& parity0, uint32_t& parity1)
+{
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;     // bytes per sub_end entry
     const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
     // Nearly every container has stream 0 coded, its table section right behind the header.  Its code lengths
     // and this warp's first table entries are requested now, together with the header, and thrown away if the
     // header says otherwise.
     uint32_t spec_len = 0, spec_end = 0, spec_off = 0;
-    if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
     if (P.spec) {
         if (threadIdx.x < 256) spec_len = P.comp[kHeaderBytes + threadIdx.x];
-        const uint32_t c0 = blockIdx.x * n_warps + warp;
-        if (c0 < P.n_chunks) {
+        if (c0 < c_end) {
             spec_end = load_sub_end(P.comp + kHeaderBytes + tab_sub, sub_w, c0, lane);
             spec_off = reinterpret_cast<const uint32_t*>(P.comp + kHeaderBytes + tab_chunk)[c0];
         }
@@ -565,50 +599,124 @@ decode_kernel(const __grid_constant__ DecParams P)
         }
         s_ok = ok ? 1u : 0u;
     }
-    if (lane == 0) { mbar_init(&bar[0], 1); mbar_init(&bar[1], 1); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    if (!s_ok) { if (threadIdx.x == 0) raise_status(P.ctl, P.call_id, ZC_E_CORRUPT); return; }
+    if (!s_ok) return ZC_E_CORRUPT;
 
     const bool huff0 = s_mode[0] == ZC_MODE_HUFF, huff1 = s_mode[1] == ZC_MODE_HUFF;
     {
-        // the warps' pools are free until the main loop: 8 KiB of them hold the one-symbol scratch table
-        uint16_t* single = reinterpret_cast<uint16_t*>(pools);
+        // the warps' pools are free until the chunk loop: 8 KiB of them hold the one-symbol scratch table
+        uint16_t* single = reinterpret_cast<uint16_t*>(M.pools);
         bool tables_ok = true;
         if (huff0) {
             uint32_t len = spec_len;                             // stream 0's section always starts behind the header
             if (!P.spec && threadIdx.x < 256) len = P.comp[s_sec[0] + threadIdx.x];
-            tables_ok = build_lut(len, lut0, single, scratch, &s_per_lookup[0]) && tables_ok;
+            tables_ok = build_lut(len, M.lut0, single, M.scratch, &s_per_lookup[0]) && tables_ok;
         }
         if (huff1) {
             uint32_t len = 0;
             if (threadIdx.x < 256) len = P.comp[s_sec[1] + threadIdx.x];
-            tables_ok = build_lut(len, lut1, single, scratch, &s_per_lookup[1]) && tables_ok;
+            tables_ok = build_lut(len, M.lut1, single, M.scratch, &s_per_lookup[1]) && tables_ok;
         }
         __syncthreads();
-        if (!tables_ok) { if (threadIdx.x == 0) raise_status(P.ctl, P.call_id, ZC_E_CORRUPT); return; }
+        if (!tables_ok) return ZC_E_CORRUPT;
     }
 
     DecShared S;
-    S.lut0_s = smem_u32(lut0); S.lut1_s = smem_u32(lut1);
+    S.lut0_s = smem_u32(M.lut0); S.lut1_s = smem_u32(M.lut1);
     S.pairs0 = huff0 && s_per_lookup[0] == 2;
     S.sec0 = s_sec[0]; S.sec1 = s_sec[1];
     S.payload_off = s_payload_off; S.payload_bytes = s_payload_bytes;
     uint32_t first_end0 = spec_end, first_off0 = spec_off;
-    if (huff0 && !P.spec) {
-        const uint32_t c0 = blockIdx.x * n_warps + warp;
-        if (c0 < P.n_chunks) {
-            first_end0 = load_sub_end(P.comp + S.sec0 + tab_sub, sub_w, c0, lane);
-            first_off0 = reinterpret_cast<const uint32_t*>(P.comp + S.sec0 + tab_chunk)[c0];
-        }
+    if (huff0 && !P.spec && c0 < c_end) {
+        first_end0 = load_sub_end(P.comp + S.sec0 + tab_sub, sub_w, c0, lane);
+        first_off0 = reinterpret_cast<const uint32_t*>(P.comp + S.sec0 + tab_chunk)[c0];
     }
-    uint32_t err;
-    if (huff0 && !huff1) err = run_chunks<FMT, PPL, true, false>(P, S, pool, bar, first_end0, first_off0);
-    else if (!huff0 && !huff1) err = run_chunks<FMT, PPL, false, false>(P, S, pool, bar, 0, 0);
-    else if (huff0) err = run_chunks<FMT, PPL, true, true>(P, S, pool, bar, first_end0, first_off0);
-    else err = run_chunks<FMT, PPL, false, true>(P, S, pool, bar, 0, 0);
+    if (huff0 && !huff1) return run_chunks<FMT, PPL, true, false>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    if (!huff0 && !huff1) return run_chunks<FMT, PPL, false, false>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+    if (huff0) return run_chunks<FMT, PPL, true, true>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    return run_chunks<FMT, PPL, false, true>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+}
+
+// One tensor per launch: the warps of all blocks take the chunks in turn.
+template <int FMT, int PPL>
+__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
+decode_kernel(const __grid_constant__ DecParams P)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const DecSmem M = carve_smem(smem, P.pool_bytes);
+    if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
+    uint32_t parity0 = 0, parity1 = 0;
+    const uint32_t err = decode_one<FMT, PPL>(P, M, blockIdx.x * n_warps + warp, P.n_chunks, gridDim.x * n_warps, parity0, parity1);
     if (err) raise_status(P.ctl, P.call_id, err);
+}
+
+// Many tensors per launch: block b takes the chunks [b * total / grid, (b + 1) * total / grid) of the
+// concatenated chunk index space, tensor by tensor; it builds the tables of a tensor once for its whole share.
+template <int FMT, int PPL>
+__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
+decode_batch_kernel(const __grid_constant__ DecBatchParams B)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const DecSmem M = carve_smem(smem, B.pool_bytes);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && B.tensor_base == 0) B.ctl->call_id = B.call_id;
+    uint32_t parity0 = 0, parity1 = 0;
+
+    auto run = [&](const uint32_t t, const uint32_t seg_lo, const uint32_t seg_hi) {
+        DecParams P;
+        P.comp = B.item[t].comp; P.out = B.item[t].out; P.ctl = B.ctl;
+        P.comp_bytes = B.item[t].comp_bytes; P.input_bytes = B.item[t].input_bytes;
+        P.n_syms = B.item[t].n_syms; P.n_elems = B.item[t].n_elems; P.n_chunks = B.item[t].n_chunks;
+        P.cs = B.cs; P.sub = B.sub; P.chunk_bytes = B.chunk_bytes; P.format = B.format; P.group = B.group;
+        P.pool_bytes = B.pool_bytes; P.call_id = B.call_id;
+        const uint64_t tables = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * (P.chunk_bytes <= 8192 ? 2u : 4u) * P.n_chunks;
+        P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
+        __syncthreads();                                         // everybody is done with the previous tensor's tables
+        const uint32_t err = decode_one<FMT, PPL>(P, M, seg_lo + warp, seg_hi, n_warps, parity0, parity1);
+        if (err && raise_status(B.ctl, B.call_id, err)) B.ctl->pad[0] = B.tensor_base + t + 1;
+    };
+
+    // The concatenated chunk index space is cut into n_ranges equal ranges which the blocks take one after the
+    // other from a ticket counter (tensors, and SMs, differ in how fast they get through a range).  Block 0
+    // first walks over the tensors without chunks: their headers are still checked.
+    __shared__ uint32_t s_range;
+    uint32_t empties = blockIdx.x == 0 ? 0u : B.n_tensors;      // cursor of that walk
+    uint32_t t = 0, g = 0, g_hi = 0;
+    bool in_range = false;
+    for (;;) {
+        uint32_t tt, seg_lo, seg_hi;
+        if (empties < B.n_tensors) {
+            if (B.item[empties].n_chunks != 0) { ++empties; continue; }
+            tt = empties++; seg_lo = 0; seg_hi = 0;
+        } else {
+            if (!in_range) {
+                __syncthreads();
+                if (threadIdx.x == 0) s_range = atomicAdd(&B.ctl->ticket, 1u);
+                __syncthreads();
+                const uint32_t r = s_range;
+                if (r >= B.n_ranges) break;
+                g = (uint32_t)((uint64_t)r * B.total_chunks / B.n_ranges);
+                g_hi = (uint32_t)((uint64_t)(r + 1) * B.total_chunks / B.n_ranges);
+                // the last tensor that starts at or before g (tensors without chunks share their start with the next one)
+                uint32_t lo = 0, hi = B.n_tensors;
+                while (hi - lo > 1) {
+                    const uint32_t mid = (lo + hi) / 2;
+                    if (B.item[mid].first_chunk <= g) lo = mid; else hi = mid;
+                }
+                t = lo;
+                in_range = true;
+            }
+            if (g >= g_hi || t >= B.n_tensors) { in_range = false; continue; }
+            const uint32_t first = B.item[t].first_chunk, n = B.item[t].n_chunks;
+            if (g >= first + n) { ++t; continue; }
+            seg_hi = min(g_hi, first + n) - first;
+            seg_lo = g - first;
+            tt = t++;
+            g = first + seg_hi;
+        }
+        run(tt, seg_lo, seg_hi);
+    }
 }
 
 }  // namespace zc
@@ -617,6 +725,45 @@ using namespace zc;
 
 extern "C" {
 
+namespace {
+
+// Launch shape for a plan: symbols per round and lane, per-warp pool, warps per block, shared memory.
+struct DecShape { uint32_t ppl, pool_bytes, warps; size_t smem; };
+
+zc_status dec_shape(const zc_plan_t* p, DecShape* out)
+{
+    DecShape s{};
+    // symbols per round and lane: the largest of 64 / 32 / 16 that divides the subchunk length
+    s.ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;
+    const uint32_t rows_bytes = 32 * (16 * s.ppl + 4);
+    // per warp: one stream's rows plus room to stage a piece as large as the raw chunk stream; pieces that
+    // do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
+    s.pool_bytes = std::max<uint32_t>(rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32, 2 * rows_bytes);
+    const size_t fixed = kDecFixedSmem + 512 /* static shared */;
+    size_t per_warp = 16 + s.pool_bytes;
+    s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
+    if (s.warps < 8) {               // large chunks: stage less
+        s.pool_bytes = std::max<uint32_t>(rows_bytes + 4096 + 32, 2 * rows_bytes);
+        per_warp = 16 + s.pool_bytes;
+        s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
+    }
+    // the table build uses 8 KiB of the pools and 256 threads
+    while (s.warps * (size_t)s.pool_bytes < 8192) ++s.warps;
+    if (s.warps < 8 || s.warps > kDecMaxWarps) return ZC_E_UNSUPPORTED;
+    s.smem = kDecFixedSmem + s.warps * per_warp;
+    *out = s;
+    return ZC_OK;
+}
+
+// no clearing of the workspace: errors are tagged with the id of the call that raised them
+unsigned long long new_call_id()
+{
+    static std::atomic<unsigned long long> next_call{(unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count()};
+    return (next_call.fetch_add(1) & ((1ull << 56) - 1)) | 1ull << 55;
+}
+
+}  // namespace
+
 zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_bytes, void* d_out, void* d_workspace,
                         void* cuda_stream)
 {
@@ -624,6 +771,9 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     if (!aligned16(d_comp) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (comp_bytes < kHeaderBytes) return ZC_E_CORRUPT;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    DecShape shape;
+    const zc_status ss = dec_shape(p, &shape);
+    if (ss != ZC_OK) return ss;
     DecParams P{};
     P.comp = (const uint8_t*)d_comp;
     P.out = (uint8_t*)d_out;
@@ -631,29 +781,11 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     P.comp_bytes = comp_bytes; P.input_bytes = p->input_bytes; P.n_syms = p->n_syms; P.n_elems = p->n_elems;
     P.n_chunks = p->n_chunks; P.cs = p->syms_per_chunk; P.sub = p->syms_per_sub; P.chunk_bytes = p->chunk_bytes;
     P.format = p->format; P.group = p->group;
-    // no clearing of the workspace: errors are tagged with the id of the call that raised them
-    static std::atomic<unsigned long long> next_call{(unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count()};
-    P.call_id = (next_call.fetch_add(1) & ((1ull << 56) - 1)) | 1ull << 55;
+    P.call_id = new_call_id();
     P.spec = comp_bytes >= kHeaderBytes + table_section_bytes(p->n_chunks, p->chunk_bytes) ? 1u : 0u;
-
-    // symbols per round and lane: the largest of 64 / 32 / 16 that divides the subchunk length
-    const uint32_t ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;
-    const uint32_t rows_bytes = 32 * (16 * ppl + 4);
-    // per warp: one stream's rows plus room to stage a piece as large as the raw chunk stream; pieces that
-    // do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
-    P.pool_bytes = std::max<uint32_t>(rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32, 2 * rows_bytes);
-    const size_t fixed = kDecFixedSmem + 512 /* static shared */;
-    size_t per_warp = 16 + P.pool_bytes;
-    uint32_t warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
-    if (warps < 8) {                 // large chunks: stage less
-        P.pool_bytes = std::max<uint32_t>(rows_bytes + 4096 + 32, 2 * rows_bytes);
-        per_warp = 16 + P.pool_bytes;
-        warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
-    }
-    // the table build uses 8 KiB of the pools and 256 threads
-    while (warps * (size_t)P.pool_bytes < 8192) ++warps;
-    if (warps < 8 || warps > kDecMaxWarps) return ZC_E_UNSUPPORTED;
-    const size_t smem = kDecFixedSmem + warps * per_warp;
+    P.pool_bytes = shape.pool_bytes;
+    const uint32_t warps = shape.warps, ppl = shape.ppl;
+    const size_t smem = shape.smem;
     // at least one block even for an empty tensor: the header is still checked
     const uint32_t want = std::max<uint32_t>((p->n_chunks + warps - 1) / warps, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
@@ -675,6 +807,87 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     }
 #undef ZC_DEC_CASE
     return e == cudaSuccess ? ZC_OK : ZC_E_CUDA;
+}
+
+zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_comp,
+                              const size_t* comp_bytes, void* const* d_out, void* d_workspace, void* cuda_stream)
+{
+    if (!d_workspace || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
+    if (n_tensors == 0) return ZC_OK;
+    if (!plans || !d_comp || !comp_bytes || !d_out) return ZC_E_INVALID_ARG;
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        const zc_plan_t* p = plans[t];
+        if (!p || !d_comp[t] || (!d_out[t] && p->n_elems)) return ZC_E_INVALID_ARG;
+        if (!aligned16(d_comp[t]) || !aligned16(d_out[t])) return ZC_E_INVALID_ARG;
+        if (p->format != plans[0]->format || p->chunk_bytes != plans[0]->chunk_bytes) return ZC_E_INVALID_ARG;
+        if (comp_bytes[t] < kHeaderBytes) return ZC_E_CORRUPT;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const zc_plan_t* p0 = plans[0];
+    DecShape shape;
+    const zc_status ss = dec_shape(p0, &shape);
+    if (ss != ZC_OK) return ss;
+    const unsigned long long call_id = new_call_id();
+    static thread_local DecBatchParams B;                    // 28 KiB: kept off the stack
+    for (uint32_t base = 0; base < n_tensors;) {
+        B.ctl = (Control*)d_workspace;
+        B.call_id = call_id;
+        B.cs = p0->syms_per_chunk; B.sub = p0->syms_per_sub; B.chunk_bytes = p0->chunk_bytes;
+        B.format = p0->format; B.group = p0->group; B.pool_bytes = shape.pool_bytes;
+        B.tensor_base = base;
+        uint32_t n = 0;
+        uint64_t total = 0;
+        // as many tensors as fit one launch: at most kDecBatchMax, fewer than 2^32 chunks together
+        while (base + n < n_tensors && n < kDecBatchMax && total + plans[base + n]->n_chunks < (1ull << 32)) {
+            const zc_plan_t* p = plans[base + n];
+            DecItem& it = B.item[n];
+            it.comp = (const uint8_t*)d_comp[base + n];
+            it.out = (uint8_t*)d_out[base + n];
+            it.comp_bytes = comp_bytes[base + n]; it.input_bytes = p->input_bytes; it.n_syms = p->n_syms; it.n_elems = p->n_elems;
+            it.n_chunks = p->n_chunks; it.first_chunk = (uint32_t)total;
+            total += p->n_chunks;
+            ++n;
+        }
+        B.n_tensors = n; B.total_chunks = (uint32_t)total;
+        const uint32_t want = std::max<uint32_t>((uint32_t)((total + shape.warps - 1) / shape.warps), 1);
+        const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
+        // up to 8 ranges per block, none shorter than 16 chunks per warp (a range costs a table build)
+        B.n_ranges = grid * (uint32_t)std::min<uint64_t>(8, std::max<uint64_t>(1, total / ((uint64_t)grid * shape.warps * 16)));
+        // the ranges are handed out through the ticket word of the control block
+        if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
+        cudaError_t e = cudaSuccess;
+        auto launch = [&](auto kern) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
+            if (e != cudaSuccess) return;
+            kern<<<grid, shape.warps * 32, shape.smem, st>>>(B);
+            e = cudaGetLastError();
+        };
+#define ZC_DEC_CASE(F)                                                     \
+    if (shape.ppl == 4) launch(decode_batch_kernel<F, 4>);                 \
+    else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2>);            \
+    else launch(decode_batch_kernel<F, 1>);
+        switch (p0->format) {
+        case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
+        case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
+        default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
+        }
+#undef ZC_DEC_CASE
+        if (e != cudaSuccess) return ZC_E_CUDA;
+        base += n;
+    }
+    return ZC_OK;
+}
+
+zc_status zc_batch_status(const void* d_workspace, uint32_t* h_failed_tensor, void* cuda_stream)
+{
+    if (!d_workspace) return ZC_E_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    Control h;
+    if (cudaMemcpyAsync(&h, d_workspace, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
+    const bool mine = (h.status >> 8) == h.call_id && (h.status & 0xFF) != 0;
+    if (h_failed_tensor) *h_failed_tensor = mine && h.pad[0] ? h.pad[0] - 1 : 0xFFFFFFFFu;
+    return mine ? (zc_status)(h.status & 0xFF) : ZC_OK;
 }
 
 }  // extern "C"

@@ -14,17 +14,19 @@ constexpr uint32_t kSpinLimit = 1u << 22;     // bounded waits: look-back and mb
 constexpr uint32_t kLutEntries = 1u << kLmax;
 constexpr size_t kMaxSmem = 227 * 1024;       // usable shared memory per block on sm_100
 
-// Record an error of the call `call_id` unless one of the same call is already there.
-__device__ __forceinline__ void raise_status(Control* ctl, unsigned long long call_id, uint32_t s)
+// Record an error of the call `call_id` unless one of the same call is already there.  True if this
+// thread's error is the one that was recorded.
+__device__ __forceinline__ bool raise_status(Control* ctl, unsigned long long call_id, uint32_t s)
 {
     const unsigned long long mine = (call_id << 8) | s;
     unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(&ctl->status);
     for (int tries = 0; tries < 64; ++tries) {
-        if ((cur >> 8) == call_id && (cur & 0xFF) != 0) return;
+        if ((cur >> 8) == call_id && (cur & 0xFF) != 0) return false;
         const unsigned long long old = atomicCAS(&ctl->status, cur, mine);
-        if (old == cur) return;
+        if (old == cur) return true;
         cur = old;
     }
+    return false;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }

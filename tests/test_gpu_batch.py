@@ -1,0 +1,116 @@
+"""The batched entry points against the CPU oracle: many tensors per call, bit-exact.
+
+Containers given to the batched decoder are made by the oracle; containers made by the batched encoder are
+compared with the oracle's byte for byte.  Everything goes through the C ABI (via the ctypes binding).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as zo
+from paper_2508_19263_b200 import binding as zc
+from test_gpu_parity import _weights
+
+pytestmark = pytest.mark.gpu
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1]
+DEV = "cuda"
+
+
+def _sizes(fmt, chunk_bytes):
+    """Element counts from nothing to dozens of chunks, ragged ends included."""
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    sizes = [0, 2 * G, cs * G, cs * G + 2 * G, 3 * cs * G - 2 * G, 40 * cs * G + 6 * G, 0, 7 * cs * G, 29 * cs * G + cs * G // 2,
+             64 * cs * G, 2 * G, 11 * cs * G + 10 * G]
+    return [n - (n % 2) if fmt == zc.FMT_FP4_E2M1 else n for n in sizes]
+
+
+def _oracle_containers(fmt, sizes, chunk_bytes, seed):
+    policies = [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL]
+    datas, conts = [], []
+    for i, n in enumerate(sizes):
+        data = _weights(fmt, n, seed + i)
+        cb = zo.build_codebook(zo.histogram(fmt, data, n), policies[i % 3])
+        datas.append(data)
+        conts.append(zo.compress(fmt, data, n, chunk_bytes, cb))
+    return datas, conts
+
+
+def _to_dev(a, pad=0):
+    t = torch.full((max(a.size, 16) + pad,), 0xEE, dtype=torch.uint8, device=DEV)
+    t[: a.size] = torch.from_numpy(a.copy()).to(DEV)
+    return t
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("chunk_bytes", [1024, 4096, 16384])
+def test_batched_decoder_restores_every_tensor(fmt, chunk_bytes):
+    sizes = _sizes(fmt, chunk_bytes)
+    datas, conts = _oracle_containers(fmt, sizes, chunk_bytes, 1000 * fmt + chunk_bytes)
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    d_comps = [_to_dev(c) for c in conts]
+    d_outs = [torch.full((p.input_bytes + 64,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    ws = torch.full((256,), 0x5A, dtype=torch.uint8, device=DEV)
+    batch = zc.DecompressBatch(plans, d_comps, [c.size for c in conts], d_outs)
+    for _ in range(2):                                               # the second call reuses the workspace as it is
+        zc.decompress_batch(batch, ws)
+        assert zc.batch_status(ws) == (zc.OK, None)
+        for p, data, out in zip(plans, datas, d_outs):
+            back = out.cpu().numpy()
+            assert np.array_equal(back[: p.input_bytes], data[: p.input_bytes])
+            assert (back[p.input_bytes:] == 0xEE).all()
+
+
+def test_batched_decoder_many_small_tensors_span_several_launches():
+    fmt, chunk_bytes = zc.FMT_BF16, 1024
+    rng = np.random.default_rng(7)
+    sizes = [int(v) for v in rng.integers(0, 3000, 1100)]
+    datas, conts = _oracle_containers(fmt, sizes, chunk_bytes, 5)
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    d_comps = [_to_dev(c) for c in conts]
+    d_outs = [torch.full((p.input_bytes + 16,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    zc.decompress_batch(zc.DecompressBatch(plans, d_comps, [c.size for c in conts], d_outs), ws)
+    assert zc.batch_status(ws) == (zc.OK, None)
+    for p, data, out in zip(plans, datas, d_outs):
+        back = out.cpu().numpy()
+        assert np.array_equal(back[: p.input_bytes], data[: p.input_bytes])
+        assert (back[p.input_bytes:] == 0xEE).all()
+
+
+@pytest.mark.parametrize("victim", [0, 5, 11])
+def test_batched_decoder_names_the_damaged_tensor_and_decodes_the_rest(victim):
+    fmt, chunk_bytes = zc.FMT_FP8_E4M3, 4096
+    sizes = _sizes(fmt, chunk_bytes)
+    datas, conts = _oracle_containers(fmt, sizes, chunk_bytes, 77)
+    bad = conts[victim].copy()
+    bad[17] ^= 0x40                                                  # chunk_bytes field of the header
+    conts[victim] = bad
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    d_comps = [_to_dev(c) for c in conts]
+    d_outs = [torch.full((p.input_bytes + 16,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    zc.decompress_batch(zc.DecompressBatch(plans, d_comps, [c.size for c in conts], d_outs), ws)
+    assert zc.batch_status(ws) == (zc.E_CORRUPT, victim)
+    for t, (p, data, out) in enumerate(zip(plans, datas, d_outs)):
+        back = out.cpu().numpy()
+        if t == victim:
+            assert (back == 0xEE).all()                              # nothing of it was written
+        else:
+            assert np.array_equal(back[: p.input_bytes], data[: p.input_bytes])
+
+
+def test_batch_argument_checks():
+    pa, pb = zc.plan(zc.FMT_BF16, 5000, 4096), zc.plan(zc.FMT_BF16, 5000, 8192)
+    pc = zc.plan(zc.FMT_FP8_E4M3, 5000, 4096)
+    d = [torch.zeros(1 << 15, dtype=torch.uint8, device=DEV) for _ in range(2)]
+    o = [torch.zeros(1 << 15, dtype=torch.uint8, device=DEV) for _ in range(2)]
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    for plans in ([pa, pb], [pa, pc]):
+        with pytest.raises(zc.ZcError) as e:
+            zc.decompress_batch(zc.DecompressBatch(plans, d, [1 << 15] * 2, o), ws)
+        assert e.value.status == zc.E_INVALID_ARG
+    with pytest.raises(zc.ZcError) as e:
+        zc.decompress_batch(zc.DecompressBatch([pa, pa], d, [1 << 15, 64], o), ws)
+    assert e.value.status == zc.E_CORRUPT
+    zc.decompress_batch(zc.DecompressBatch([], [], [], []), ws)      # nothing to do
