@@ -164,6 +164,15 @@ zc_status zc_histogram(const zc_plan_t* plan, const void* d_in, uint64_t* d_hist
  * Host-only: needs no GPU.  Errors: INVALID_ARG, UNSUPPORTED (policy), NOMEM. */
 zc_status zc_build_codebook(const zc_plan_t* plan, const uint64_t* h_hist, zc_policy policy,
                             zc_codebook_t** out);
+/* The codebooks of many tensors with one call, built on several host threads.
+ * h_hists    host, uint64_t[n_tensors][2][256]
+ * n_threads  host threads to use (0: as many as the machine has, at most 16, at least 8
+ *            tensors per thread)
+ * out        host array of n_tensors pointers; receives new codebooks, identical to those of
+ *            zc_build_codebook; untouched on error
+ * Errors: as zc_build_codebook. */
+zc_status zc_build_codebooks(uint32_t n_tensors, const zc_plan_t* const* plans, const uint64_t* h_hists,
+                             zc_policy policy, uint32_t n_threads, zc_codebook_t** out);
 void zc_codebook_destroy(zc_codebook_t* cb);
 
 /* Copy out one stream's mode, code lengths and right-aligned code values
@@ -226,6 +235,33 @@ zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, co
  * Asynchronous; read the outcome with zc_device_status().  Errors: INVALID_ARG, CUDA. */
 zc_status zc_decompress(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes, void* d_out,
                         void* d_workspace, void* cuda_stream);
+
+/* ---- compress many tensors with one call (Sec. 4 and 4.1: a model or a checkpoint is a set of
+ *      tensors, each compressed on its own with its own codes; Sec. 3.3: K and V of all layers) -
+ * The containers are byte for byte those of n_tensors calls of zc_compress; the chunks of all
+ * tensors are handed out through one ticket counter, so that small tensors do not pay a launch
+ * each (one launch per combination of stream modes that occurs and per 256 tensors of it).
+ * n_tensors        number of tensors (0 returns ZC_OK and launches nothing)
+ * plans            host array of n_tensors plans; all must have the same format and chunk_bytes
+ * codebooks        host array, one codebook per tensor
+ * d_in             host array of DEVICE pointers (16-byte aligned): the tensors' element bytes
+ * d_out            host array of DEVICE pointers (16-byte aligned): d_out[t] receives container t
+ * out_capacity     host array: out_capacity[t] >= zc_max_compressed_bytes(plans[t])
+ * d_workspace      device scratch of workspace_bytes >= zc_compress_batch_workspace_bytes()
+ *                  bytes (256-byte aligned); contents need not be initialised
+ * h_out_bytes      host array of n_tensors sizes, optional: when non-null the call synchronises
+ *                  cuda_stream, stores the container sizes and returns the device status; when
+ *                  null the call is asynchronous (sizes are in the headers; status via
+ *                  zc_batch_status)
+ * The arrays are read before the call returns; the caller keeps ownership of everything.
+ * Errors: INVALID_ARG (null or misaligned pointers, mixed formats or chunk sizes),
+ * BUFFER_TOO_SMALL (an output or the workspace), UNSUPPORTED, CUDA, and the device status
+ * (NO_CODE, DEVICE_TIMEOUT) when synchronous. */
+size_t zc_compress_batch_workspace_bytes(uint32_t n_tensors, const zc_plan_t* const* plans);
+zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
+                            const zc_codebook_t* const* codebooks, const void* const* d_in,
+                            void* const* d_out, const size_t* out_capacity, void* d_workspace,
+                            size_t workspace_bytes, uint64_t* h_out_bytes, void* cuda_stream);
 
 /* ---- decompress many tensors with one call (Sec. 4 and 4.1: a model or a checkpoint is a set of
  *      tensors, each compressed on its own; Sec. 3.3: the K and V tensors of all layers) --------

@@ -71,6 +71,8 @@ def _load():
     L.zc_histogram.argtypes = [vp, vp, vp, vp]
     L.zc_build_codebook.restype = C.c_int
     L.zc_build_codebook.argtypes = [vp, u64p, C.c_int, C.POINTER(vp)]
+    L.zc_build_codebooks.restype = C.c_int
+    L.zc_build_codebooks.argtypes = [C.c_uint32, C.POINTER(vp), u64p, C.c_int, C.c_uint32, C.POINTER(vp)]
     L.zc_codebook_destroy.restype = None
     L.zc_codebook_destroy.argtypes = [vp]
     L.zc_codebook_get.restype = C.c_int
@@ -81,6 +83,11 @@ def _load():
     L.zc_compress_noalloc.argtypes = [vp, vp, vp, vp, C.c_size_t, u64p, vp]
     L.zc_decompress.restype = C.c_int
     L.zc_decompress.argtypes = [vp, vp, C.c_size_t, vp, vp, vp]
+    L.zc_compress_batch_workspace_bytes.restype = C.c_size_t
+    L.zc_compress_batch_workspace_bytes.argtypes = [C.c_uint32, C.POINTER(vp)]
+    L.zc_compress_batch.restype = C.c_int
+    L.zc_compress_batch.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t),
+                                    vp, C.c_size_t, u64p, vp]
     L.zc_decompress_batch.restype = C.c_int
     L.zc_decompress_batch.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), vp, vp]
     L.zc_batch_status.restype = C.c_int
@@ -192,6 +199,23 @@ def build_codebook(p: Plan, h_hist, policy: int = POLICY_AUTO) -> Codebook:
     return Codebook(out)
 
 
+def build_codebooks(plans, h_hists, policy: int = POLICY_AUTO, n_threads: int = 0):
+    """zc_build_codebooks: the codebooks of many tensors, built on several host threads.
+    h_hists: array-like [n, 2, 256] of counts."""
+    n = len(plans)
+    h = np.asarray(h_hists)
+    if h.dtype == np.int64 and h.flags.c_contiguous:
+        h = h.view(np.uint64)
+    elif h.dtype != np.uint64 or not h.flags.c_contiguous:
+        h = np.ascontiguousarray(h.astype(np.uint64))
+    assert h.size == 512 * n
+    handles = (C.c_void_p * max(n, 1))()
+    plan_arr = (C.c_void_p * max(n, 1))(*[p._h.value for p in plans])
+    _check(_lib.zc_build_codebooks(n, plan_arr, C.cast(h.ctypes.data, C.POINTER(C.c_uint64)), policy, n_threads, handles),
+           "zc_build_codebooks")
+    return [Codebook(C.c_void_p(handles[i])) for i in range(n)]
+
+
 def compress(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Tensor, d_workspace: torch.Tensor,
              sync: bool = True, stream=None) -> Optional[int]:
     """zc_compress.  With sync=True returns the container size in bytes (and raises on a device-side
@@ -229,6 +253,37 @@ def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tens
 
 def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:
     return _lib.zc_device_status(p._h, d_workspace.data_ptr(), _stream_ptr(stream))
+
+
+class CompressBatch:
+    """Argument arrays of zc_compress_batch, marshalled once; set_codebooks() swaps in new codebooks."""
+
+    def __init__(self, plans, d_ins, d_outs):
+        n = len(plans)
+        assert len(d_ins) == n and len(d_outs) == n
+        self.n = n
+        self._keep = (list(plans), list(d_ins), list(d_outs))          # the arrays hold raw pointers
+        self.plans = (C.c_void_p * n)(*[p._h.value for p in plans])
+        self.ins = (C.c_void_p * n)(*[t.data_ptr() for t in d_ins])
+        self.outs = (C.c_void_p * n)(*[t.data_ptr() for t in d_outs])
+        self.caps = (C.c_size_t * n)(*[t.numel() for t in d_outs])
+        self.cbs = (C.c_void_p * n)()
+        self._cbs = None
+        self.workspace_bytes = _lib.zc_compress_batch_workspace_bytes(n, self.plans)
+
+    def set_codebooks(self, codebooks):
+        assert len(codebooks) == self.n
+        self._cbs = list(codebooks)
+        for i, cb in enumerate(codebooks):
+            self.cbs[i] = cb._h.value
+
+
+def compress_batch(batch: CompressBatch, d_workspace: torch.Tensor, sync: bool = True, stream=None):
+    """zc_compress_batch.  Returns the list of container sizes (sync=True) or None (asynchronous)."""
+    sizes = (C.c_uint64 * max(batch.n, 1))()
+    _check(_lib.zc_compress_batch(batch.n, batch.plans, batch.cbs, batch.ins, batch.outs, batch.caps, d_workspace.data_ptr(),
+                                  d_workspace.numel(), sizes if sync else None, _stream_ptr(stream)), "zc_compress_batch")
+    return [int(v) for v in sizes[: batch.n]] if sync else None
 
 
 class DecompressBatch:

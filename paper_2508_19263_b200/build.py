@@ -34,7 +34,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         return LIB
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-I", INCLUDE, "-shared", "-Xcompiler", "-fPIC", "-o", tmp]
+           "-I", INCLUDE, "-shared", "-Xcompiler", "-fPIC,-pthread", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, f) for f in SOURCES]

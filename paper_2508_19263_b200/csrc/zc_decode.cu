@@ -674,7 +674,7 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
         P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
         __syncthreads();                                         // everybody is done with the previous tensor's tables
         const uint32_t err = decode_one<FMT, PPL>(P, M, seg_lo + warp, seg_hi, n_warps, parity0, parity1);
-        if (err && raise_status(B.ctl, B.call_id, err)) B.ctl->pad[0] = B.tensor_base + t + 1;
+        if (err && raise_status(B.ctl, B.call_id, err)) B.ctl->failed = B.tensor_base + t + 1;
     };
 
     // The concatenated chunk index space is cut into n_ranges equal ranges which the blocks take one after the
@@ -886,7 +886,7 @@ zc_status zc_batch_status(const void* d_workspace, uint32_t* h_failed_tensor, vo
     if (cudaMemcpyAsync(&h, d_workspace, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
     const bool mine = (h.status >> 8) == h.call_id && (h.status & 0xFF) != 0;
-    if (h_failed_tensor) *h_failed_tensor = mine && h.pad[0] ? h.pad[0] - 1 : 0xFFFFFFFFu;
+    if (h_failed_tensor) *h_failed_tensor = mine && h.failed ? h.failed - 1 : 0xFFFFFFFFu;
     return mine ? (zc_status)(h.status & 0xFF) : ZC_OK;
 }
 

@@ -1,31 +1,63 @@
-// Encoder kernels (split, code-length scan, bit packing) and zc_compress / zc_device_status.
+// Encoder kernel (split, bit packing, placement of the chunks by a look-back scan) and zc_compress,
+// zc_compress_batch, zc_compress_noalloc, zc_device_status.
 #include "zc_device.cuh"
+
+#include <vector>
 
 namespace zc {
 
 // ------------------------------------------------------------------------------------------------
-// encoder
+// parameters
 // ------------------------------------------------------------------------------------------------
 
 // Per symbol: the code left-aligned in bits 31..20 and its length in bits 3..0; a symbol without a code is 16.
 struct EncTables { uint32_t enc[2][256]; };
 
-struct EncParams {
+// One tensor of a launch.
+struct EncItem {
     const uint8_t* in;
     uint8_t* out;
-    Control* ctl;
-    unsigned long long* flags;                   // one look-back word per chunk
     uint64_t input_bytes, n_syms, n_elems;
-    uint32_t n_chunks, cs, sub, chunk_bytes;     // symbols per chunk / per subchunk
-    uint32_t mode[2];
-    uint32_t format, group;
+    uint32_t n_chunks;
+    uint32_t first_batch;                        // batches of all earlier tensors of the launch
+    uint32_t index;                              // position in the caller's arrays (counters, tables, error reports)
+    uint32_t pad;
     Layout lay;
+};
+
+// A launch covers N_ITEMS tensors at most (1: zc_compress, its table travels in the parameters;
+// kEncBatchMax: zc_compress_batch, tables in global memory).  All tensors of a launch share format, chunk
+// size and the modes of the two streams.
+constexpr uint32_t kEncBatchMax = 256;           // keeps the parameter block below 32 KiB
+
+struct EncCommon {
+    Control* ctl;
+    TensorCounters* counters;                    // indexed by EncItem::index
+    unsigned long long* flags;                   // one look-back word per batch of the launch
+    const EncTables* tables;                     // indexed by EncItem::index (batched launches)
+    uint32_t cs, sub, chunk_bytes;               // symbols per chunk / per subchunk
+    uint32_t format, group;
+    uint32_t mode[2];
     uint32_t stage_stride;                       // bytes of one coded stream's lane regions per warp
-    uint32_t region_bytes;                       // one lane region: (n_slots + 1) * sub + 4
+    uint32_t region_bytes;                       // one lane region: n_slots * slot_bytes + sub + 4
+    uint32_t slot_bytes;                         // one pack slot: sub (8 bits per symbol) or 1.5 * sub (12 bits)
     uint32_t sub_width;                          // bytes per sub_end entry (2 or 4)
     uint32_t n_slots;                            // pack slots per lane region (1..3, see encode_kernel)
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
+    uint32_t n_tensors, total_batches;
 };
+
+template <int N_ITEMS> struct EncParamsT;
+template <> struct EncParamsT<1> {
+    EncCommon c;
+    EncTables table;
+    EncItem item[1];
+};
+template <> struct EncParamsT<(int)kEncBatchMax> {
+    EncCommon c;
+    EncItem item[kEncBatchMax];
+};
+static_assert(sizeof(EncParamsT<(int)kEncBatchMax>) < 32764, "kernel parameters are limited to 32764 bytes");
 
 constexpr unsigned long long kFlagAggregate = 1ull << 62, kFlagPrefix = 2ull << 62, kFlagValue = (1ull << 62) - 1;
 
@@ -40,59 +72,24 @@ __device__ __forceinline__ void st_flag(unsigned long long* p, unsigned long lon
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
 }
 
-// Sum of the sizes (16-byte units) of all chunks before chunk c: single-pass look-back over the
-// per-chunk words that earlier chunks publish.  Chunks are handed out in increasing order by a
-// ticket, so every predecessor is already running or finished.  Returns false if a wait gave up.
-__device__ bool lookback_exclusive(unsigned long long* flags, uint32_t c, uint32_t lane, uint64_t own, uint64_t& excl)
-{
-    if (c == 0) {
-        if (lane == 0) st_flag(&flags[0], kFlagPrefix | own);
-        excl = 0;
-        return true;
-    }
-    if (lane == 0) st_flag(&flags[c], kFlagAggregate | own);
-    uint64_t sum = 0;
-    int64_t base = (int64_t)c - 1;               // lane i looks at chunk base - i
-    uint32_t spins = 0;
-    while (true) {
-        const int64_t idx = base - lane;
-        unsigned long long f = kFlagPrefix;      // before chunk 0: prefix 0
-        if (idx >= 0) f = ld_flag(&flags[idx]);
-        const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (f >> 62) != 0);
-        const uint32_t prefix = __ballot_sync(0xFFFFFFFFu, (f >> 62) == 2);
-        // usable lanes: from lane 0 up to the first one holding a prefix, all of them ready
-        const uint32_t first_prefix = prefix ? (uint32_t)__ffs(prefix) - 1 : 32u;
-        const uint32_t need = first_prefix == 32 ? 0xFFFFFFFFu : (0xFFFFFFFFu >> (31 - first_prefix));
-        if ((ready & need) != need) {
-            if (++spins > kSpinLimit) return false;
-            __nanosleep(64);
-            continue;
-        }
-        uint64_t v = (lane <= first_prefix || first_prefix == 32) ? (f & kFlagValue) : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        sum += v;
-        if (first_prefix != 32) break;
-        base -= 32;
-    }
-    excl = sum;
-    if (lane == 0) st_flag(&flags[c], kFlagPrefix | (sum + own));
-    return true;
-}
-
 // Per-warp shared memory of one coded stream: 32 lane regions (+4 bytes of padding each, which also makes
 // the region stride an odd number of words so that lanes walking their regions hit different banks).
-// A region is cut into slots of `sub` bytes: n_slots pack slots followed by the symbols,
+// A region is n_slots pack slots of slot_bytes each, followed by the sub symbols of the lane's subchunk,
 //   [pack 0 | .. | pack n_slots-1 | symbols].
 // A lane packs the codes of its subchunk into pack slot (batch index mod n_slots), so the packed bits of the
 // last n_slots batches are alive at the same time and the copy-out of a batch can wait up to n_slots
 // iterations for the batch's position in the payload area (which comes from a look-back over other blocks).
-// Packing into the last slot may run on into the symbols behind it: codes are at most 12 bits, so after k
-// symbols at most 1.5 k bytes are written while the read position is sub + k, and the writer never passes
-// unread symbols.  Packing into any other slot stops at the slot's end.  The packed bits of a subchunk
-// normally fit one slot (8 bits per symbol); a chunk in which some lane needs more is finished on a slow
-// path (everything older is copied out, then the chunk is packed again from slot 0 with the whole region
-// as room) before anything else is staged.
+// Two slot sizes:
+//   slot_bytes = 1.5 * sub  holds any subchunk (codes are at most 12 bits).
+//   slot_bytes = sub        holds 8 bits per symbol, which is plenty for streams that compress well and leaves
+//                           room for one more slot.  Packing into the last slot may still run on into the
+//                           symbols behind it (after k symbols at most 1.5 k bytes are written while the read
+//                           position is sub + k, so the writer never passes unread symbols); packing into any
+//                           other slot stops at the slot's end.  A chunk in which some lane needs more than its
+//                           slot is finished on a slow path (everything older is copied out, then the chunk is
+//                           packed again from slot 0 with the rest of the region as room) before anything else
+//                           is staged.  That path waits for the chunk's own look-back, so the host picks this
+//                           size only for code tables whose expected code length is well below 8 bits.
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
@@ -122,438 +119,728 @@ __device__ __forceinline__ unsigned long long ld_ctl(const unsigned long long* p
     return v;
 }
 
-// Writes the 128-byte header and the guard; called by one thread once every chunk is in place.
-__device__ void write_header(const EncParams& P)
+// Writes the 128-byte header and the guard of one tensor; called by one thread once every chunk is in place.
+__device__ void write_header(const EncCommon& C, const EncItem& I, TensorCounters* tc)
 {
-    const bool any_huff = P.mode[0] == ZC_MODE_HUFF || P.mode[1] == ZC_MODE_HUFF;
-    const uint64_t payload_bytes = any_huff ? 16ull * ld_ctl(&P.ctl->total16) : 0;
-    uint8_t* h = P.out;
+    const bool any_huff = C.mode[0] == ZC_MODE_HUFF || C.mode[1] == ZC_MODE_HUFF;
+    const uint64_t payload_bytes = any_huff ? 16ull * ld_ctl(&tc->total16) : 0;
+    uint8_t* h = I.out;
     uint32_t* h32 = reinterpret_cast<uint32_t*>(h);
     unsigned long long* h64 = reinterpret_cast<unsigned long long*>(h);
     for (int i = 0; i < 32; ++i) h32[i] = 0;
     h32[0] = kMagic;
-    h[kHdrVersion] = 1; h[kHdrFormat] = (uint8_t)P.format; h[kHdrStreams] = 2;
-    h64[kHdrElems / 8] = P.n_elems;
-    h32[kHdrChunkBytes / 4] = P.chunk_bytes;
-    h32[kHdrChunks / 4] = P.n_chunks;
-    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)P.group; h[kHdrSubs] = kSubs; h[kHdrSubWidth] = (uint8_t)P.sub_width;
-    const uint64_t total = P.lay.payload_off + payload_bytes + (any_huff ? 16 : 0);
+    h[kHdrVersion] = 1; h[kHdrFormat] = (uint8_t)C.format; h[kHdrStreams] = 2;
+    h64[kHdrElems / 8] = I.n_elems;
+    h32[kHdrChunkBytes / 4] = C.chunk_bytes;
+    h32[kHdrChunks / 4] = I.n_chunks;
+    h[kHdrLmax] = kLmax; h[kHdrGroup] = (uint8_t)C.group; h[kHdrSubs] = kSubs; h[kHdrSubWidth] = (uint8_t)C.sub_width;
+    const uint64_t total = I.lay.payload_off + payload_bytes + (any_huff ? 16 : 0);
     h64[kHdrTotal / 8] = total;
-    h64[kHdrPayloadOff / 8] = P.lay.payload_off;
+    h64[kHdrPayloadOff / 8] = I.lay.payload_off;
     h64[kHdrPayloadBytes / 8] = payload_bytes;
     for (int s = 0; s < 2; ++s) {
         uint8_t* d = h + kHdrStream0 + kHdrStreamStride * s;
-        d[kSdMode] = (uint8_t)P.mode[s];
-        reinterpret_cast<unsigned long long*>(d)[1] = P.n_syms;
-        reinterpret_cast<unsigned long long*>(d)[2] = P.mode[s] == ZC_MODE_HUFF ? ld_ctl(&P.ctl->payload_bits[s]) : 8 * P.n_syms;
-        reinterpret_cast<unsigned long long*>(d)[3] = P.lay.section_off[s];
+        d[kSdMode] = (uint8_t)C.mode[s];
+        reinterpret_cast<unsigned long long*>(d)[1] = I.n_syms;
+        reinterpret_cast<unsigned long long*>(d)[2] = C.mode[s] == ZC_MODE_HUFF ? ld_ctl(&tc->payload_bits[s]) : 8 * I.n_syms;
+        reinterpret_cast<unsigned long long*>(d)[3] = I.lay.section_off[s];
     }
-    if (any_huff) {
-        uint32_t* g = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + payload_bytes);
+    if (any_huff) {                              // 16 zero bytes behind the payload: decoders may peek past the last piece
+        uint32_t* g = reinterpret_cast<uint32_t*>(I.out + I.lay.payload_off + payload_bytes);
         g[0] = g[1] = g[2] = g[3] = 0;
     }
-    P.ctl->total16 = total;                      // the host reads the container size from here
+    tc->total16 = total;                         // the host reads the container size from here
 }
 
-
-// For an empty tensor no encoder block runs: the header is all there is.
-__global__ void finish_kernel(const EncParams P)
-{
-    if (threadIdx.x == 0 && blockIdx.x == 0) write_header(P);
-}
-
-constexpr uint32_t kEncMaxWorkers = 8;       // worker warps per block = chunks per batch; one more warp does the look-back
+constexpr uint32_t kEncMaxWorkers = 8;       // worker warps per block = chunks per batch; one more warp hands out
+                                             // the batches and places them
+constexpr uint32_t kRing = 8;                // batches of a block whose bookkeeping is alive at the same time
+constexpr uint32_t kTabSlots = 4;            // code tables (one per batch) alive at the same time
+constexpr uint32_t kNoTensor = 0xFFFFFFFFu;  // "no more batches"
+constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
 
 // What a worker warp keeps about a chunk between packing it and copying it out.
 struct PackedChunk {
-    uint32_t c;                 // chunk index; kNoChunk: this warp had no chunk in the batch
+    uint32_t c;                 // chunk index inside its tensor; kNoChunk: this warp had no chunk in the batch
+    uint32_t t;                 // tensor (index into the launch's items)
     uint32_t end[2];            // per stream: inclusive scan of the subchunks' bit counts over the lanes (= sub_end)
 };
-constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
 
-template <int FMT>
+// The kernel.  A block is up to kEncMaxWorkers worker warps plus one service warp.
+//
+// Batches: the chunks of every tensor are grouped into batches of n_workers consecutive chunks, the batches of
+// all tensors of the launch are numbered consecutively, and a global ticket counter hands them out in that
+// order.  Worker w of the block that owns a batch encodes chunk w of it:
+//   A  coalesced load, field split, raw stream stored as it is, coded stream staged per subchunk
+//   B  every lane packs the codes of its subchunk into a pack slot of its lane region
+//   C  subchunk end bits (sub_end table), the chunk's size in 16-byte units
+//   D  (up to n_slots batches later) copy-out: every lane moves its bits to their place in the payload area
+// The place of a chunk is the sum of the sizes of all earlier chunks of its tensor: the service warp adds up
+// its block's batch and finds the rest with a decoupled look-back over the words other blocks publish.
+//
+// Worker 0 takes the ticket of batch i + 1 after packing batch i (as late as possible: batches must start in
+// the order they were handed out, or the look-back of other blocks waits for a batch that is not even begun;
+// measured, an earlier ticket costs more in look-back waits than it saves).  Part of the ticket's latency
+// hides behind phase C; after it, if the ticket is another batch of the same tensor, worker 0 hands the batch
+// out itself; otherwise it leaves the ticket to the service warp.
+// The service warp never blocks on one thing: in a loop it (1) advances the look-back of the oldest unplaced
+// batch by one round; (2) turns a ticket left to it into a batch: finds the tensor, copies the tensor's code
+// table into a table slot and, for the first batch of a tensor, writes the fixed parts of the container.
+// The warps are coupled only through words in shared memory (no block barrier in the loop):
+//   s_ticket[i & 7], s_ticket_seq                  ticket of batch i; seq = tickets taken so far
+//   s_tensor/s_cbase/s_tabslot[i & 7], s_base_seq  batch i of this block; seq = batches handed out so far
+//   s_tot[i & 7][w], s_cnt[i & 7]                  size of worker w's chunk; cnt = workers that posted it
+//   s_off[i & 7][w], s_off_seq                     position of that chunk; seq = batches placed so far
+// A worker has copied out batch i - n_slots (n_slots <= 3) before it packs batch i; a batch is placed only
+// after every worker has posted its size, and a batch is handed out only while fewer than 4 handed-out
+// batches are unplaced.  So all warps of a block are within 4 batches of each other and rings of 8 are
+// enough.  A table slot is reused only when every worker has posted the last batch that used it.
+template <int FMT, int N_ITEMS>
 __global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, 3)
-encode_kernel(const __grid_constant__ EncParams P, const __grid_constant__ EncTables T)
+encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 {
     extern __shared__ __align__(16) uint8_t smem[];
+    const EncCommon& C = P.c;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_workers = (blockDim.x >> 5) - 1;
-    const bool scanner = warp == n_workers;                     // the last warp only does the look-back
-    const bool huff0 = P.mode[0] == ZC_MODE_HUFF, huff1 = P.mode[1] == ZC_MODE_HUFF;
+    const bool service = warp == n_workers;
+    const bool huff0 = C.mode[0] == ZC_MODE_HUFF, huff1 = C.mode[1] == ZC_MODE_HUFF;
     const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
-    const uint32_t n_slots = P.n_slots;
+    const uint32_t n_slots = C.n_slots;
 
-    // shared: enc[2][256] | per worker warp: regions[n_huff][stage_stride]
-    uint32_t* enc = reinterpret_cast<uint32_t*>(smem);
-    uint8_t* stage_all = smem + 2048;
-    for (uint32_t i = threadIdx.x; i < 512; i += blockDim.x) enc[i] = T.enc[i >> 8][i & 255];
-    uint8_t* stage = stage_all + (size_t)(scanner ? 0 : warp) * n_huff * P.stage_stride;
-    const uint32_t region = P.region_bytes;                     // (n_slots + 1) * sub + 4
-    const uint32_t sym_off = n_slots * P.sub;                   // symbols sit at this offset inside a region
+    // shared: tables[kTabSlots][n_huff][256] | per worker warp: regions[n_huff][stage_stride]
+    uint32_t* tabs = reinterpret_cast<uint32_t*>(smem);
+    const uint32_t tab_words = 256 * (n_huff ? n_huff : 1);     // words of one table slot
+    uint8_t* stage = smem + 4 * kTabSlots * tab_words + (size_t)(service ? 0 : warp) * n_huff * C.stage_stride;
+    const uint32_t region = C.region_bytes;                     // n_slots * slot_bytes + sub + 4
+    const uint32_t sym_off = n_slots * C.slot_bytes;            // symbols sit at this offset inside a region
 
-    // The warps of a block are coupled only through these words (no block barrier inside the loop):
-    //   s_base[it & 3], s_base_seq   first chunk of the block's batch `it`; seq = batches handed out so far
-    //   s_tot[it & 3][w], s_cnt[..]  payload size of worker w's chunk; cnt = workers that have posted it
-    //   s_off[it & 3][w], s_off_seq  position of that chunk in the payload area; seq = batches placed so far
-    // A worker has consumed the position of batch `it - n_slots` (n_slots <= 3) before it posts a size for
-    // batch `it`, and the look-back warp places a batch only after every worker has posted, so no warp is more
-    // than three batches away from any other and four copies of each word are enough.
-    __shared__ uint32_t s_base[4], s_base_seq, s_cnt[4], s_off_seq, s_fail;
-    __shared__ unsigned long long s_tot[4][kEncMaxWorkers], s_off[4][kEncMaxWorkers];
+    __shared__ uint32_t s_ticket[kRing], s_tensor[kRing], s_cbase[kRing], s_tabslot[kRing], s_cnt[kRing];
+    __shared__ uint32_t s_ticket_seq, s_base_seq, s_off_seq, s_fail;
+    __shared__ unsigned long long s_tot[kRing][kEncMaxWorkers], s_off[kRing][kEncMaxWorkers];
 
-    // block 0 writes the static parts of the table sections and the tail padding of raw bodies
-    if (blockIdx.x == 0) {
-        for (int s = 0; s < 2; ++s) {
-            if (P.mode[s] == ZC_MODE_HUFF) {
-                for (uint32_t v = threadIdx.x; v < 256; v += blockDim.x) P.out[P.lay.section_off[s] + v] = (uint8_t)(T.enc[s][v] & 15);
-                const uint32_t padded = (P.n_chunks + 3) & ~3u;
-                for (uint32_t i = P.n_chunks + threadIdx.x; i < padded; i += blockDim.x)
-                    reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[i] = 0;
-            } else {
-                const uint64_t lo = (P.n_syms + 7) & ~7ull, hi = (P.n_syms + 15) & ~15ull;
-                for (uint64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) P.out[P.lay.section_off[s] + i] = 0;
-            }
-        }
-    }
+    if (threadIdx.x < kRing) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) {
-        s_fail = 0; s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; s_cnt[3] = 0; s_off_seq = 0;
-        s_base[0] = atomicAdd(&P.ctl->ticket, n_workers);       // batches of n_workers consecutive chunks
-        s_base_seq = 1;
+        s_fail = 0; s_off_seq = 0; s_base_seq = 0;
+        s_ticket[0] = atomicAdd(&C.ctl->ticket, 1u);
+        s_ticket_seq = 1;
     }
     __syncthreads();
 
-    // Bounded wait of a whole warp until a sequence word reaches `target`; false on a failure flag or when
-    // the wait gives up (the caller then raises the failure flag itself).
-    auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
-        bool ok = false;
-        for (uint32_t n = 0; n < kSpinLimit; ++n) {
-            if (*reinterpret_cast<const volatile uint32_t*>(word) >= target) { ok = true; break; }
-            if (*reinterpret_cast<const volatile uint32_t*>(&s_fail)) break;
-            if (n > 64) __nanosleep(40);
-        }
-        __syncwarp();
-        __threadfence_block();
-        return ok;
-    };
+    auto vol32 = [](const uint32_t* p) { return *reinterpret_cast<const volatile uint32_t*>(p); };
+    auto item = [&](const uint32_t t) -> const EncItem& { return P.item[N_ITEMS == 1 ? 0u : t]; };
+    auto counters = [&](const uint32_t t) -> TensorCounters* { return C.counters + (N_ITEMS == 1 ? 0u : P.item[t].index); };
 
-    // ---- copy-out of a packed chunk: every lane moves its bits to their final position in the piece ----
-    auto copy_out = [&](const PackedChunk& pc, const uint32_t slot, const uint64_t off16) {
-        uint32_t hs = 0;
-        uint64_t piece_off16 = off16;
+    if (service) {
+        // =========================== the service warp ===========================
+        // block 0: tensors without chunks are all header
+        if (blockIdx.x == 0 && lane == 0)
+            for (uint32_t t = 0; t < C.n_tensors; ++t)
+                if (item(t).n_chunks == 0) write_header(C, item(t), counters(t));
+
+        uint32_t handed = 0, placed = 0;                         // batches of this block handed out / placed
+        uint32_t tcur = 0;                                       // tensor of the last ticket (tickets only grow)
+        uint32_t tab_tensor = kNoTensor, tab_slot = 0;           // the newest table slot and whose table it holds
+        uint32_t slot_last0 = 0, slot_last1 = 0, slot_last2 = 0, slot_last3 = 0;   // 1 + last batch that used slot k
+        bool ended = false, lb_on = false;
+        unsigned long long lb_sum = 0, lb_own = 0, lb_inc = 0, lb_v = 0;
+        long long lb_base = 0;
+        unsigned long long* lb_flags = nullptr;
+        uint32_t lb_b = 0, idle = 0;
+        for (;;) {
+            bool did = false;
+            // batches worker 0 handed out itself since the last look: they use the newest table slot
+            const uint32_t tickets = vol32(&s_ticket_seq);       // read before s_base_seq (worker 0 writes it after)
+            __threadfence_block();
+            const uint32_t published = vol32(&s_base_seq);
+            if (published > handed) {
+                handed = published;
+                if (tab_slot == 0) slot_last0 = handed; else if (tab_slot == 1) slot_last1 = handed;
+                else if (tab_slot == 2) slot_last2 = handed; else slot_last3 = handed;
+            }
+            // ---- (1) placement of the oldest unplaced batch ----
+            const uint32_t real = ended ? handed - 1 : handed;   // the last ticket was "no more batches"
+            if (placed < real) {
+                const uint32_t r = placed % kRing;
+                if (!lb_on && vol32(&s_cnt[r]) == n_workers) {   // every worker has posted a size (0 without a chunk)
+                    __threadfence_block();
+                    if (lane == 0) s_cnt[r] = 0;
+                    lb_v = lane < n_workers ? *reinterpret_cast<const volatile unsigned long long*>(&s_tot[r][lane]) : 0ull;
+                    lb_inc = lb_v;
 #pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            if (P.mode[s] != ZC_MODE_HUFF) continue;
-            const uint32_t end = pc.end[s];
-            uint32_t start = __shfl_up_sync(0xFFFFFFFFu, end, 1);
-            if (lane == 0) start = 0;
-            const uint32_t bits = end - start;
-            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
-            const uint32_t piece16 = (chunk_bits + 127) / 128;
-            if (lane == 0) reinterpret_cast<uint32_t*>(P.out + P.lay.chunk_off_tab[s])[pc.c] = (uint32_t)piece_off16;
-            uint32_t* piece = reinterpret_cast<uint32_t*>(P.out + P.lay.payload_off + 16 * piece_off16);
-            const uint32_t piece_words = 4 * piece16;
-            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region) + slot;
-            const uint32_t sh = start & 31, d0 = start >> 5;
-            const uint32_t n_dst = (sh + bits + 31) / 32;             // destination words I touch
-            const uint32_t n_src = (bits + 31) / 32;
-            if (__all_sync(0xFFFFFFFFu, bits >= 32)) {
-                // every lane spans a word boundary, so a destination word is shared by at most two neighbouring
-                // lanes: a lane hands its ragged last word to the next lane, which merges it into its first word
-                const bool ragged = ((sh + bits) & 31) != 0;
-                const uint32_t il = n_dst - 1;
-                const uint32_t lc = il < n_src ? lds32(reg_s + 4 * il) : 0u;
-                const uint32_t lp = il >= 1 ? lds32(reg_s + 4 * (il - 1)) : 0u;
-                const uint32_t tail = ragged ? __funnelshift_r(lc, lp, sh) : 0u;
-                uint32_t head = __shfl_up_sync(0xFFFFFFFFu, tail, 1);
-                if (lane == 0) head = 0;
-                const uint32_t n_mine = n_dst - ((ragged && lane != 31) ? 1u : 0u);
-                uint32_t prev = 0;
-                for (uint32_t i = 0; i < n_mine; ++i) {
-                    const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
-                    uint32_t v = __funnelshift_r(cur, prev, sh);      // (prev:cur) >> sh, low word
-                    prev = cur;
-                    if (i == 0) v |= head;
-                    piece[d0 + i] = v;
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned long long x = __shfl_up_sync(0xFFFFFFFFu, lb_inc, o);
+                        if (lane >= (uint32_t)o) lb_inc += x;
+                    }
+                    lb_own = __shfl_sync(0xFFFFFFFFu, lb_inc, 31);
+                    const EncItem& I = item(vol32(&s_tensor[r]));
+                    lb_flags = C.flags + I.first_batch;          // the look-back stays inside the tensor
+                    lb_b = vol32(&s_ticket[r]) - I.first_batch;
+                    lb_sum = 0;
+                    lb_base = (long long)lb_b - 1;               // lane i looks at batch lb_base - i
+                    if (n_huff && lb_b != 0 && lane == 0) st_flag(&lb_flags[lb_b], kFlagAggregate | lb_own);
+                    lb_on = true;
+                    did = true;
                 }
-                if (lane < 4 && piece_words) {                        // zero padding up to the 16-byte boundary
-                    const uint32_t w = piece_words - 4 + lane;
-                    if (32ull * w >= chunk_bits) piece[w] = 0;
-                }
-            } else {
-                // general case (short or empty subchunks): words shared between neighbours (and the padding)
-                // start from zero and are OR-ed into
-                if ((start >> 5) < piece_words) piece[start >> 5] = 0;
-                if (lane == 31 && (end >> 5) < piece_words) piece[end >> 5] = 0;
-                if (lane < 4 && piece_words) {
-                    const uint32_t w = piece_words - 4 + lane;
-                    if (32ull * w >= chunk_bits) piece[w] = 0;
-                }
-                __syncwarp();
-                if (bits) {
-                    uint32_t prev = 0;
-                    for (uint32_t i = 0; i < n_dst; ++i) {
-                        const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
-                        const uint32_t v = __funnelshift_r(cur, prev, sh);
-                        prev = cur;
-                        // the first word may hold the previous lane's bits, a ragged last word the next lane's
-                        const bool shared_word = i == 0 || (i == n_dst - 1 && ((sh + bits) & 31) != 0);
-                        if (shared_word) atomicOr(&piece[d0 + i], v);
-                        else piece[d0 + i] = v;
+                if (lb_on) {
+                    bool done = !n_huff || lb_b == 0;
+                    if (!done) {
+                        // one round of the look-back: 32 predecessors at a time, newest first, up to the first
+                        // one that already knows its prefix
+                        const long long idx = lb_base - lane;
+                        unsigned long long f = kFlagPrefix;      // before batch 0: prefix 0
+                        if (idx >= 0) f = ld_flag(&lb_flags[idx]);
+                        const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (f >> 62) != 0);
+                        const uint32_t prefix = __ballot_sync(0xFFFFFFFFu, (f >> 62) == 2);
+                        const uint32_t first_prefix = prefix ? (uint32_t)__ffs(prefix) - 1 : 32u;
+                        const uint32_t need = first_prefix == 32 ? 0xFFFFFFFFu : (0xFFFFFFFFu >> (31 - first_prefix));
+                        if ((ready & need) == need) {
+                            unsigned long long x = (lane <= first_prefix || first_prefix == 32) ? (f & kFlagValue) : 0;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+                            lb_sum += x;
+                            if (first_prefix != 32) done = true; else lb_base -= 32;
+                            did = true;
+                        }
+                    }
+                    if (done) {
+                        if (n_huff && lane == 0) st_flag(&lb_flags[lb_b], kFlagPrefix | (lb_sum + lb_own));
+                        if (lane < n_workers) s_off[r][lane] = lb_sum + lb_inc - lb_v;
+                        __threadfence_block();
+                        __syncwarp();
+                        if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = placed + 1;
+                        ++placed;
+                        lb_on = false;
+                        did = true;
                     }
                 }
             }
-            piece_off16 += piece16;
-            ++hs;
-        }
-        // the warp that owns the last chunk knows the size of the whole payload area
-        if (lane == 0 && pc.c == P.n_chunks - 1) P.ctl->total16 = piece_off16;
-        __syncwarp();
-    };
-
-    uint32_t bad = 0;
-
-    if (scanner) {
-        // ---- the look-back warp places batch after batch; the workers are a batch ahead of it ----
-        for (uint32_t it = 0; n_huff; ++it) {
-            if (!wait_seq(&s_base_seq, it + 1)) { s_fail = 1; break; }
-            const uint32_t base = *reinterpret_cast<const volatile uint32_t*>(&s_base[it & 3]);
-            if (base >= P.n_chunks) break;
-            bool ok = false;
-            for (uint32_t n = 0; n < kSpinLimit; ++n) {             // every worker posts a size (0 without a chunk)
-                if (*reinterpret_cast<const volatile uint32_t*>(&s_cnt[it & 3]) == n_workers) { ok = true; break; }
-                if (*reinterpret_cast<const volatile uint32_t*>(&s_fail)) break;
-                __nanosleep(40);
-            }
-            __syncwarp();
-            __threadfence_block();
-            if (!ok) { s_fail = 1; break; }
-            if (lane == 0) s_cnt[it & 3] = 0;
-            unsigned long long v = lane < n_workers ? *reinterpret_cast<const volatile unsigned long long*>(&s_tot[it & 3][lane]) : 0ull, inc = v;
+            // ---- (2) a new ticket becomes a batch ----
+            if (!ended && handed < tickets && handed < placed + 4) {
+                const uint32_t g = vol32(&s_ticket[handed % kRing]);
+                uint32_t t = kNoTensor, cbase = 0;
+                bool publish = true;
+                if (g < C.total_batches) {
+                    if (N_ITEMS > 1)                             // tensors without chunks share their start with the next one
+                        while (tcur + 1 < C.n_tensors && g >= P.item[tcur + 1].first_batch) ++tcur;
+                    t = tcur;
+                    const EncItem& I = item(t);
+                    cbase = (g - I.first_batch) * n_workers;
+                    if (n_huff && t != tab_tensor) {
+                        // another tensor: its table goes to the next slot, once every worker has posted the last
+                        // batch that was packed with the table that is there now
+                        const uint32_t nslot = (tab_slot + 1) % kTabSlots;
+                        const uint32_t last = nslot == 0 ? slot_last0 : nslot == 1 ? slot_last1 : nslot == 2 ? slot_last2 : slot_last3;
+                        if (placed + (lb_on ? 1u : 0u) < last) {
+                            publish = false;                     // not yet: look back some more first
+                        } else {
+                            uint32_t* tab = tabs + nslot * tab_words;
+                            uint32_t hs = 0;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                if (lane >= (uint32_t)o) inc += t;
+                            for (int s = 0; s < 2; ++s) {
+                                if (C.mode[s] != ZC_MODE_HUFF) continue;
+                                const uint32_t* src;
+                                if constexpr (N_ITEMS == 1) src = P.table.enc[s]; else src = C.tables[I.index].enc[s];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) tab[256 * hs + lane + 32 * i] = src[lane + 32 * i];
+                                ++hs;
+                            }
+                            tab_slot = nslot;
+                            tab_tensor = t;
+                            __syncwarp();
+                        }
+                    }
+                    if (publish && g == I.first_batch) {
+                        // the fixed parts of the tensor's container: code lengths, padding of the chunk offset
+                        // table, tail padding of raw bodies
+                        const uint32_t* tab = tabs + tab_slot * tab_words;
+                        uint32_t hs = 0;
+#pragma unroll
+                        for (int s = 0; s < 2; ++s) {
+                            if (C.mode[s] == ZC_MODE_HUFF) {
+                                for (uint32_t v = lane; v < 256; v += 32) I.out[I.lay.section_off[s] + v] = (uint8_t)(tab[256 * hs + v] & 15);
+                                const uint32_t padded = (I.n_chunks + 3) & ~3u;
+                                for (uint32_t i = I.n_chunks + lane; i < padded; i += 32)
+                                    reinterpret_cast<uint32_t*>(I.out + I.lay.chunk_off_tab[s])[i] = 0;
+                                ++hs;
+                            } else {
+                                const uint64_t lo = (I.n_syms + 7) & ~7ull, hi = (I.n_syms + 15) & ~15ull;
+                                for (uint64_t i = lo + lane; i < hi; i += 32) I.out[I.lay.section_off[s] + i] = 0;
+                            }
+                        }
+                    }
+                } else {
+                    ended = true;
+                }
+                if (publish) {
+                    if (t != kNoTensor) {
+                        if (tab_slot == 0) slot_last0 = handed + 1; else if (tab_slot == 1) slot_last1 = handed + 1;
+                        else if (tab_slot == 2) slot_last2 = handed + 1; else slot_last3 = handed + 1;
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        s_tensor[handed % kRing] = t; s_cbase[handed % kRing] = cbase; s_tabslot[handed % kRing] = tab_slot;
+                        __threadfence_block();
+                        *reinterpret_cast<volatile uint32_t*>(&s_base_seq) = handed + 1;
+                    }
+                    ++handed;
+                    did = true;
+                }
             }
-            const unsigned long long batch_total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            uint64_t batch_off = 0;
-            ok = lookback_exclusive(P.flags, base / n_workers, lane, batch_total, batch_off);
-            if (lane < n_workers) s_off[it & 3][lane] = batch_off + inc - v;
-            __threadfence_block();
-            __syncwarp();
-            if (!ok) { s_fail = 1; break; }
-            if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = it + 1;
+            if (ended && placed == handed - 1) break;
+            if (vol32(&s_fail)) break;
+            if (did) { idle = 0; continue; }
+            if (++idle > kSpinLimit) { s_fail = 1; break; }
+            if (lb_on) __nanosleep(50); else __nanosleep(300);      // a look-back in progress polls faster
         }
     } else {
-    // packed chunks that wait for their copy-out, newest first: q0 is batch it - 1, q1 batch it - 2, ...
-    PackedChunk q0{kNoChunk, {0, 0}}, q1 = q0, q2 = q0;
-    uint32_t n_pend = 0;
-    uint32_t slot_idx = 0;                                      // pack slot of batch `it`: it mod n_slots
-    // waits until the oldest pending batch is placed and copies this warp's chunk of it out
-    auto flush_oldest = [&](const uint32_t it) -> bool {
-        const uint32_t j = it - n_pend;                         // the batch in question
-        if (n_huff) {
-            if (!wait_seq(&s_off_seq, j + 1)) return false;
-            PackedChunk pc;
-            pc.c = n_pend == 1 ? q0.c : n_pend == 2 ? q1.c : q2.c;
-            pc.end[0] = n_pend == 1 ? q0.end[0] : n_pend == 2 ? q1.end[0] : q2.end[0];
-            pc.end[1] = n_pend == 1 ? q0.end[1] : n_pend == 2 ? q1.end[1] : q2.end[1];
-            // its slot: the slots are used round-robin, so it lies n_pend steps behind the current one
-            const uint32_t sl = (slot_idx + n_slots * 4 - n_pend) % n_slots;
-            if (pc.c != kNoChunk) copy_out(pc, sl * P.sub, *reinterpret_cast<const volatile unsigned long long*>(&s_off[j & 3][warp]));
-        }
-        --n_pend;
-        return true;
-    };
-    bool failed = false;
-    for (uint32_t it = 0;; ++it) {
-        if (!wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
-        const uint32_t base = *reinterpret_cast<const volatile uint32_t*>(&s_base[it & 3]);
-        const bool have = base < P.n_chunks;
-        if (!have) {
-            while (n_pend && !failed) failed = !flush_oldest(it);
-            break;
-        }
+        // =========================== a worker warp ===========================
+        // Bounded wait of the whole warp until a sequence word reaches `target`; false on a failure flag or
+        // when the wait gives up.
+        auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
+            bool ok = false;
+            for (uint32_t n = 0; n < kSpinLimit; ++n) {
+                if (vol32(word) >= target) { ok = true; break; }
+                if (vol32(&s_fail)) break;
+                if (n > 64) __nanosleep(40);
+            }
+            __syncwarp();
+            __threadfence_block();
+            return ok;
+        };
 
-        const bool active = base + warp < P.n_chunks;
-        PackedChunk cur{active ? base + warp : kNoChunk, {0, 0}};
-        const uint32_t slot = slot_idx * P.sub;
-        const uint64_t c_lo = (uint64_t)(active ? cur.c : 0) * P.cs;
-        const uint32_t c_syms = active ? (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo) : 0u;
-
-        // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
-        auto stage_group = [&](const uint4 x, const uint32_t k) {
-            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-            uint32_t sy[2][2];
-            split16<FMT>(w, sy[0], sy[1]);
-            uint32_t hs = 0;
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                if (P.mode[s] == ZC_MODE_RAW) {
-                    st_cs_v2(P.out + P.lay.section_off[s] + c_lo + k, make_uint2(sy[s][0], sy[s][1]));
-                } else {
-                    const uint32_t j = __umulhi(k, P.sub_magic);          // subchunk of these 8 symbols
-                    uint32_t* st = reinterpret_cast<uint32_t*>(stage + hs * P.stage_stride + j * region + sym_off + (k - j * P.sub));
-                    st[0] = sy[s][0];
-                    st[1] = sy[s][1];
-                    ++hs;
+        // Chunks this warp has completely written, per tensor; added to the tensor's counter (behind a fence)
+        // when the warp moves on to another tensor or leaves.  Whoever completes a tensor writes its header.
+        uint32_t acc_t = kNoTensor, acc_n = 0;
+        auto flush_acc = [&]() {
+            if (acc_n == 0) return;
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) {
+                TensorCounters* tc = counters(acc_t);
+                const uint32_t before = atomicAdd(&tc->done, acc_n);
+                if (before + acc_n == item(acc_t).n_chunks) {
+                    __threadfence();
+                    write_header(C, item(acc_t), tc);
                 }
             }
+            acc_n = 0;
         };
-        const uint32_t n_vec = (c_syms + 7) / 8;
-        const uint8_t* src_c = P.in + 2 * c_lo;
-        uint32_t g = lane;
-        if (2 * (c_lo + 8ull * n_vec) <= P.input_bytes) {           // every group of this chunk is complete
-            for (; g + 96 < n_vec; g += 128) {                          // four loads in flight per lane
-                const uint4 x0 = ld_nc_v4(src_c + 16 * g);
-                const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32));
-                const uint4 x2 = ld_nc_v4(src_c + 16 * (g + 64));
-                const uint4 x3 = ld_nc_v4(src_c + 16 * (g + 96));
-                stage_group(x0, 8 * g);
-                stage_group(x1, 8 * (g + 32));
-                stage_group(x2, 8 * (g + 64));
-                stage_group(x3, 8 * (g + 96));
-            }
-            for (; g < n_vec; g += 32) stage_group(ld_nc_v4(src_c + 16 * g), 8 * g);
-        } else {
-            for (; g < n_vec; g += 32) stage_group(load16_guarded(P.in, 2 * (c_lo + 8ull * g), P.input_bytes), 8 * g);
-        }
-        __syncwarp();
-
-        // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
-        if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
-
-        // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
-        const uint32_t lo_sym = lane * P.sub;
-        const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
-        // returns the bit count; stores stop at `room` bytes (the count goes on)
-        auto pack = [&](const int s, const uint32_t hs, const uint32_t slot, const uint32_t room) -> uint32_t {
-            const uint32_t reg_s = smem_u32(stage + hs * P.stage_stride + lane * region);
-            const uint32_t tab_s = smem_u32(enc + 256 * s);
-            const uint32_t w0 = reg_s + slot, limit = w0 + room;
-            uint32_t hi = 0, nb = 0, waddr = w0, seen = 0;
-            const uint32_t src = reg_s + sym_off;
-            const uint32_t full_words = n_my / 4;
-            for (uint32_t i = 0; i < full_words; ++i) {
-                const uint32_t four = lds32(src + 4 * i);
-                const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
-                const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
-                const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
-                const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
-                seen |= e0 | e1 | e2 | e3;
-                // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
-                // first entry = its length); the length fields end up below bit 8 and are masked off
-                const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
-                put_bits(ca, (e0 + e1) & 31, hi, nb, waddr, limit);
-                const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
-                put_bits(cb, (e2 + e3) & 31, hi, nb, waddr, limit);
-            }
-            for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
-                const uint32_t four = lds32(src + (i & ~3u));
-                const uint32_t e = lds32(tab_s + (((four >> (8 * (i & 3))) & 0xFF) << 2));
-                seen |= e;
-                put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr, limit);
-            }
-            if (active && waddr < limit) sts32(waddr, hi);          // pending bits (or zero)
-            bad |= seen & 16;                                       // an entry without a code carries bit 4
-            return 8 * (waddr - w0) + nb;
+        auto chunk_done = [&](const uint32_t t) {
+            if (t != acc_t) { flush_acc(); acc_t = t; }
+            ++acc_n;
         };
-        bool oversize = false;
-        uint32_t my_bits[2] = {0, 0};
-        const bool last_slot = slot_idx + 1 == n_slots;
-        {
+
+        // ---- copy-out of a packed chunk: every lane moves its bits to their final position in the piece ----
+        auto copy_out = [&](const PackedChunk& pc, const uint32_t slot, const uint64_t off16) {
+            const EncItem& I = item(pc.t);
             uint32_t hs = 0;
+            uint64_t piece_off16 = off16;
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
-                if (P.mode[s] != ZC_MODE_HUFF) continue;
-                // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
-                my_bits[s] = pack(s, hs, slot, last_slot ? 2 * P.sub : P.sub);
-                // more than 8 bits per symbol: the bits beyond the slot do not survive the next staging
-                oversize |= my_bits[s] > 8 * P.sub;
+                if (C.mode[s] != ZC_MODE_HUFF) continue;
+                const uint32_t end = pc.end[s];
+                uint32_t start = __shfl_up_sync(0xFFFFFFFFu, end, 1);
+                if (lane == 0) start = 0;
+                const uint32_t bits = end - start;
+                const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end, 31);
+                const uint32_t piece16 = (chunk_bits + 127) / 128;
+                if (lane == 0) reinterpret_cast<uint32_t*>(I.out + I.lay.chunk_off_tab[s])[pc.c] = (uint32_t)piece_off16;
+                uint32_t* piece = reinterpret_cast<uint32_t*>(I.out + I.lay.payload_off + 16 * piece_off16);
+                const uint32_t piece_words = 4 * piece16;
+                const uint32_t reg_s = smem_u32(stage + hs * C.stage_stride + lane * region) + slot;
+                const uint32_t sh = start & 31, d0 = start >> 5;
+                const uint32_t n_dst = (sh + bits + 31) / 32;             // destination words I touch
+                const uint32_t n_src = (bits + 31) / 32;
+                if (__all_sync(0xFFFFFFFFu, bits >= 32)) {
+                    // every lane spans a word boundary, so a destination word is shared by at most two neighbouring
+                    // lanes: a lane hands its ragged last word to the next lane, which merges it into its first word
+                    const bool ragged = ((sh + bits) & 31) != 0;
+                    const uint32_t il = n_dst - 1;
+                    const uint32_t lc = il < n_src ? lds32(reg_s + 4 * il) : 0u;
+                    const uint32_t lp = il >= 1 ? lds32(reg_s + 4 * (il - 1)) : 0u;
+                    const uint32_t tail = ragged ? __funnelshift_r(lc, lp, sh) : 0u;
+                    uint32_t head = __shfl_up_sync(0xFFFFFFFFu, tail, 1);
+                    if (lane == 0) head = 0;
+                    const uint32_t n_mine = n_dst - ((ragged && lane != 31) ? 1u : 0u);
+                    uint32_t prev = 0;
+                    for (uint32_t i = 0; i < n_mine; ++i) {
+                        const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
+                        uint32_t v = __funnelshift_r(cur, prev, sh);      // (prev:cur) >> sh, low word
+                        prev = cur;
+                        if (i == 0) v |= head;
+                        piece[d0 + i] = v;
+                    }
+                    if (lane < 4 && piece_words) {                        // zero padding up to the 16-byte boundary
+                        const uint32_t w = piece_words - 4 + lane;
+                        if (32ull * w >= chunk_bits) piece[w] = 0;
+                    }
+                } else {
+                    // general case (short or empty subchunks): words shared between neighbours (and the padding)
+                    // start from zero and are OR-ed into
+                    if ((start >> 5) < piece_words) piece[start >> 5] = 0;
+                    if (lane == 31 && (end >> 5) < piece_words) piece[end >> 5] = 0;
+                    if (lane < 4 && piece_words) {
+                        const uint32_t w = piece_words - 4 + lane;
+                        if (32ull * w >= chunk_bits) piece[w] = 0;
+                    }
+                    __syncwarp();
+                    if (bits) {
+                        uint32_t prev = 0;
+                        for (uint32_t i = 0; i < n_dst; ++i) {
+                            const uint32_t cur = i < n_src ? lds32(reg_s + 4 * i) : 0u;
+                            const uint32_t v = __funnelshift_r(cur, prev, sh);
+                            prev = cur;
+                            // the first word may hold the previous lane's bits, a ragged last word the next lane's
+                            const bool shared_word = i == 0 || (i == n_dst - 1 && ((sh + bits) & 31) != 0);
+                            if (shared_word) atomicOr(&piece[d0 + i], v);
+                            else piece[d0 + i] = v;
+                        }
+                    }
+                }
+                piece_off16 += piece16;
                 ++hs;
             }
-        }
+            // the warp that owns the last chunk knows the size of the whole payload area
+            if (lane == 0 && pc.c == I.n_chunks - 1) counters(pc.t)->total16 = piece_off16;
+            __syncwarp();
+            chunk_done(pc.t);
+        };
 
-        // the ticket of the next batch is taken as late as possible (batches must start in the order they
-        // were handed out, or the look-back of other blocks waits for a batch that is not even begun); its
-        // latency hides behind phase C
-        uint32_t next_base = 0;
-        if (threadIdx.x == 0) next_base = atomicAdd(&P.ctl->ticket, n_workers);
-
-        // ---- phase C: subchunk end bits and the chunk's size in the payload area ----
-        uint64_t tot16 = 0;
-        {
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                if (P.mode[s] != ZC_MODE_HUFF) continue;
-                uint32_t inc = my_bits[s];
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= (uint32_t)o) inc += t;
-                }
-                cur.end[s] = inc;
-                if (active) {
-                    if (P.sub_width == 2) reinterpret_cast<uint16_t*>(P.out + P.lay.sub_end_tab[s] + 64ull * cur.c)[lane] = (uint16_t)inc;
-                    else reinterpret_cast<uint32_t*>(P.out + P.lay.sub_end_tab[s] + 128ull * cur.c)[lane] = inc;
-                    const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                    tot16 += (chunk_bits + 127) / 128;
-                    if (lane == 0) atomicAdd(&P.ctl->payload_bits[s], (unsigned long long)chunk_bits);
-                }
+        uint32_t bad = 0;                                           // 1 + tensor in which a symbol had no code
+        // packed chunks that wait for their copy-out, newest first: q0 is batch it - 1, q1 batch it - 2, ...
+        PackedChunk q0{kNoChunk, 0, {0, 0}}, q1 = q0, q2 = q0;
+        uint32_t n_pend = 0;
+        uint32_t slot_idx = 0;                                      // pack slot of batch `it`: it mod n_slots
+        // waits until the oldest pending batch is placed and copies this warp's chunk of it out
+        auto flush_oldest = [&](const uint32_t it) -> bool {
+            const uint32_t j = it - n_pend;                         // the batch in question
+            if (!wait_seq(&s_off_seq, j + 1)) return false;
+            if (n_huff) {
+                PackedChunk pc;
+                pc.c = n_pend == 1 ? q0.c : n_pend == 2 ? q1.c : q2.c;
+                pc.t = n_pend == 1 ? q0.t : n_pend == 2 ? q1.t : q2.t;
+                pc.end[0] = n_pend == 1 ? q0.end[0] : n_pend == 2 ? q1.end[0] : q2.end[0];
+                pc.end[1] = n_pend == 1 ? q0.end[1] : n_pend == 2 ? q1.end[1] : q2.end[1];
+                // its slot: the slots are used round-robin, so it lies n_pend steps behind the current one
+                const uint32_t sl = (slot_idx + n_slots * 4 - n_pend) % n_slots;
+                if (pc.c != kNoChunk)
+                    copy_out(pc, sl * C.slot_bytes, *reinterpret_cast<const volatile unsigned long long*>(&s_off[j % kRing][warp]));
             }
-        }
-        if (lane == 0 && n_huff) {
-            s_tot[it & 3][warp] = tot16;
-            __threadfence_block();
-            atomicAdd(&s_cnt[it & 3], 1u);
-        }
-        if (threadIdx.x == 0) {
-            s_base[(it + 1) & 3] = next_base;
-            __threadfence_block();
-            *reinterpret_cast<volatile uint32_t*>(&s_base_seq) = it + 2;
-        }
+            --n_pend;
+            return true;
+        };
+        bool failed = false;
+        for (uint32_t it = 0;; ++it) {
+            if (!wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
+            const uint32_t t = vol32(&s_tensor[it % kRing]);
+            if (t == kNoTensor) {
+                while (n_pend && !failed) failed = !flush_oldest(it);
+                break;
+            }
+            const EncItem& I = item(t);
+            const uint32_t my_c = vol32(&s_cbase[it % kRing]) + warp;
+            const bool active = my_c < I.n_chunks;
+            PackedChunk cur{active ? my_c : kNoChunk, t, {0, 0}};
+            const uint32_t slot = slot_idx * C.slot_bytes;
+            const uint64_t c_lo = (uint64_t)(active ? my_c : 0) * C.cs;
+            const uint32_t c_syms = active ? (uint32_t)min((uint64_t)C.cs, I.n_syms - c_lo) : 0u;
 
-        q2 = q1; q1 = q0; q0 = cur;
-        ++n_pend;
-        slot_idx = last_slot ? 0 : slot_idx + 1;
-        if (__any_sync(0xFFFFFFFFu, oversize)) {
-            // some subchunk needs more than 8 bits per symbol: finish this chunk before anything else is staged.
-            // Once everything older has left, a packing that was clipped at the end of its slot is redone from
-            // slot 0 with the rest of the region as room.
-            while (n_pend > 1 && !failed) failed = !flush_oldest(it + 1);
-            if (failed) break;
-            if (!last_slot) {
+            // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
+            auto stage_group = [&](const uint4 x, const uint32_t k) {
+                const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                uint32_t sy[2][2];
+                split16<FMT>(w, sy[0], sy[1]);
                 uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
-                    if (P.mode[s] != ZC_MODE_HUFF) continue;
-                    pack(s, hs, 0, 2 * P.sub);
+                    if (C.mode[s] == ZC_MODE_RAW) {
+                        st_cs_v2(I.out + I.lay.section_off[s] + c_lo + k, make_uint2(sy[s][0], sy[s][1]));
+                    } else {
+                        const uint32_t j = __umulhi(k, C.sub_magic);          // subchunk of these 8 symbols
+                        uint32_t* st = reinterpret_cast<uint32_t*>(stage + hs * C.stage_stride + j * region + sym_off + (k - j * C.sub));
+                        st[0] = sy[s][0];
+                        st[1] = sy[s][1];
+                        ++hs;
+                    }
+                }
+            };
+            const uint32_t n_vec = (c_syms + 7) / 8;
+            const uint8_t* src_c = I.in + 2 * c_lo;
+            uint32_t g = lane;
+            if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {           // every group of this chunk is complete
+                for (; g + 96 < n_vec; g += 128) {                          // four loads in flight per lane
+                    const uint4 x0 = ld_nc_v4(src_c + 16 * g);
+                    const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32));
+                    const uint4 x2 = ld_nc_v4(src_c + 16 * (g + 64));
+                    const uint4 x3 = ld_nc_v4(src_c + 16 * (g + 96));
+                    stage_group(x0, 8 * g);
+                    stage_group(x1, 8 * (g + 32));
+                    stage_group(x2, 8 * (g + 64));
+                    stage_group(x3, 8 * (g + 96));
+                }
+                for (; g < n_vec; g += 32) stage_group(ld_nc_v4(src_c + 16 * g), 8 * g);
+            } else {
+                for (; g < n_vec; g += 32) stage_group(load16_guarded(I.in, 2 * (c_lo + 8ull * g), I.input_bytes), 8 * g);
+            }
+            __syncwarp();
+
+
+            // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
+            if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
+
+            // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
+            const uint32_t lo_sym = lane * C.sub;
+            const uint32_t n_my = lo_sym < c_syms ? min(C.sub, c_syms - lo_sym) : 0u;
+            const uint32_t tab_slot_idx = vol32(&s_tabslot[it % kRing]);
+            const uint32_t tab_slot_s = smem_u32(tabs + tab_slot_idx * tab_words);
+            // batches below this ticket belong to the same tensor
+            const uint32_t t_end = (N_ITEMS > 1 && t + 1 < C.n_tensors) ? P.item[N_ITEMS > 1 ? t + 1 : 0].first_batch : C.total_batches;
+            // returns the bit count; stores stop at `room` bytes (the count goes on)
+            auto pack = [&](const uint32_t hs, const uint32_t slot_off, const uint32_t room) -> uint32_t {
+                const uint32_t reg_s = smem_u32(stage + hs * C.stage_stride + lane * region);
+                const uint32_t tab_s = tab_slot_s + 1024 * hs;
+                const uint32_t w0 = reg_s + slot_off, limit = w0 + room;
+                uint32_t hi = 0, nb = 0, waddr = w0, seen = 0;
+                const uint32_t src = reg_s + sym_off;
+                const uint32_t full_words = n_my / 4;
+                for (uint32_t i = 0; i < full_words; ++i) {
+                    const uint32_t four = lds32(src + 4 * i);
+                    const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
+                    const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
+                    const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
+                    const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
+                    seen |= e0 | e1 | e2 | e3;
+                    // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
+                    // first entry = its length); the length fields end up below bit 8 and are masked off
+                    const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
+                    put_bits(ca, (e0 + e1) & 31, hi, nb, waddr, limit);
+                    const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
+                    put_bits(cb, (e2 + e3) & 31, hi, nb, waddr, limit);
+                }
+                for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
+                    const uint32_t four = lds32(src + (i & ~3u));
+                    const uint32_t e = lds32(tab_s + (((four >> (8 * (i & 3))) & 0xFF) << 2));
+                    seen |= e;
+                    put_bits(e & 0xFFFFFF00u, e & 31, hi, nb, waddr, limit);
+                }
+                if (active && waddr < limit) sts32(waddr, hi);          // pending bits (or zero)
+                if (seen & 16) bad = t + 1;                             // an entry without a code carries bit 4
+                return 8 * (waddr - w0) + nb;
+            };
+            bool oversize = false;
+            uint32_t my_bits[2] = {0, 0};
+            const bool last_slot = slot_idx + 1 == n_slots;
+            {
+                uint32_t hs = 0;
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    if (C.mode[s] != ZC_MODE_HUFF) continue;
+                    // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
+                    my_bits[s] = pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
+                    // more than the slot holds: the bits beyond it do not survive the next staging
+                    oversize |= my_bits[s] > 8 * C.slot_bytes;
                     ++hs;
                 }
-                __syncwarp();
-                slot_idx = 1;                                   // the chunk now sits in slot 0, one behind
             }
-            if (!flush_oldest(it + 1)) { failed = true; break; }
-            slot_idx = 0;                                       // nothing is pending: start over with slot 0
+
+            // the ticket of the next batch (see above)
+            uint32_t next_ticket = 0;
+            if (threadIdx.x == 0) next_ticket = atomicAdd(&C.ctl->ticket, 1u);
+
+            // ---- phase C: subchunk end bits and the chunk's size in the payload area ----
+            uint64_t tot16 = 0;
+            {
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    if (C.mode[s] != ZC_MODE_HUFF) continue;
+                    uint32_t inc = my_bits[s];
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t x = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                        if (lane >= (uint32_t)o) inc += x;
+                    }
+                    cur.end[s] = inc;
+                    if (active) {
+                        if (C.sub_width == 2) reinterpret_cast<uint16_t*>(I.out + I.lay.sub_end_tab[s] + 64ull * my_c)[lane] = (uint16_t)inc;
+                        else reinterpret_cast<uint32_t*>(I.out + I.lay.sub_end_tab[s] + 128ull * my_c)[lane] = inc;
+                        const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                        tot16 += (chunk_bits + 127) / 128;
+                        if (lane == 0) atomicAdd(&counters(t)->payload_bits[s], (unsigned long long)chunk_bits);
+                    }
+                }
+            }
+            if (lane == 0) {
+                s_tot[it % kRing][warp] = tot16;
+                __threadfence_block();
+                atomicAdd(&s_cnt[it % kRing], 1u);
+            }
+            if (threadIdx.x == 0) {
+                // another batch of this tensor is handed out right away; anything else is left to the service warp
+                const uint32_t r1 = (it + 1) % kRing;
+                const bool same = next_ticket < t_end;
+                s_ticket[r1] = next_ticket;
+                s_tensor[r1] = t;
+                s_cbase[r1] = (next_ticket - I.first_batch) * n_workers;
+                s_tabslot[r1] = tab_slot_idx;
+                __threadfence_block();
+                if (same) *reinterpret_cast<volatile uint32_t*>(&s_base_seq) = it + 2;
+                *reinterpret_cast<volatile uint32_t*>(&s_ticket_seq) = it + 2;   // after s_base_seq: the service warp reads it first
+            }
+            if (!n_huff && active) chunk_done(t);                   // nothing to copy out: the chunk is complete
+
+            q2 = q1; q1 = q0; q0 = cur;
+            ++n_pend;
+            slot_idx = last_slot ? 0 : slot_idx + 1;
+            if (__any_sync(0xFFFFFFFFu, oversize)) {
+                // some subchunk needs more than its slot holds: finish this chunk before anything else is staged.
+                // Once everything older has left, a packing that was clipped at the end of its slot is redone from
+                // slot 0 with the rest of the region as room.
+                while (n_pend > 1 && !failed) failed = !flush_oldest(it + 1);
+                if (failed) break;
+                if (!last_slot) {
+                    uint32_t hs = 0;
+#pragma unroll
+                    for (int s = 0; s < 2; ++s) {
+                        if (C.mode[s] != ZC_MODE_HUFF) continue;
+                        pack(hs, 0, 2 * C.sub);
+                        ++hs;
+                    }
+                    __syncwarp();
+                    slot_idx = 1;                                   // the chunk now sits in slot 0, one behind
+                }
+                if (!flush_oldest(it + 1)) { failed = true; break; }
+                slot_idx = 0;                                       // nothing is pending: start over with slot 0
+            }
         }
+        if (failed) s_fail = 1;
+        flush_acc();
+        if (bad && raise_status(C.ctl, 0, ZC_E_NO_CODE)) C.ctl->failed = item(bad - 1).index + 1;
     }
-    if (failed) s_fail = 1;
-    }
-    if (s_fail && threadIdx.x == 0) raise_status(P.ctl, 0, ZC_E_DEVICE_TIMEOUT);
-    if (bad) raise_status(P.ctl, 0, ZC_E_NO_CODE);
-    // the block that finishes last writes the header (every block's results are fenced before its count)
     __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(&P.ctl->done, 1u) == gridDim.x - 1) {
-            __threadfence();
-            write_header(P);
-        }
-    }
+    if (s_fail && threadIdx.x == 0) raise_status(C.ctl, 0, ZC_E_DEVICE_TIMEOUT);
 }
 
 }  // namespace zc
 
 using namespace zc;
+
+namespace {
+
+// Shared-memory shape of a launch for given chunk geometry, number of coded streams and slot size.
+struct EncShape { uint32_t n_slots, slot_bytes, region_bytes, stage_stride, workers, per_sm; size_t smem; };
+
+zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* out)
+{
+    EncShape s{};
+    const size_t fixed = (size_t)4 * kTabSlots * 256 * std::max<uint32_t>(n_huff, 1);
+    s.slot_bytes = wide ? p->syms_per_sub + p->syms_per_sub / 2 : p->syms_per_sub;
+    // as many pack slots per lane region (up to 3) as still leave three blocks of 8 worker warps per SM
+    s.n_slots = 1;
+    for (uint32_t ns = 3; ns > 1; --ns) {
+        const size_t block = fixed + (size_t)kEncMaxWorkers * std::max<uint32_t>(n_huff, 1) * kSubs * (ns * s.slot_bytes + p->syms_per_sub + 4);
+        if (3 * (block + 2048) <= kMaxSmem + 1024) { s.n_slots = ns; break; }
+    }
+    s.region_bytes = s.n_slots * s.slot_bytes + p->syms_per_sub + 4;
+    s.stage_stride = kSubs * s.region_bytes;
+    const size_t per_warp = std::max<size_t>((size_t)n_huff * s.stage_stride, 16);
+    // blocks of up to 8 worker warps (a batch of 8 consecutive chunks) plus the service warp; several
+    // blocks per SM so that loading, packing and copy-out phases of different blocks overlap
+    s.workers = (uint32_t)std::min<size_t>(kEncMaxWorkers, (kMaxSmem - fixed - 2048) / per_warp);
+    if (s.workers == 0) return ZC_E_UNSUPPORTED;
+    s.smem = fixed + s.workers * per_warp;
+    s.per_sm = std::max<uint32_t>((uint32_t)std::min<size_t>((kMaxSmem + 1024) / (s.smem + 2048 + 1024), 3), 1u);
+    *out = s;
+    return ZC_OK;
+}
+
+// Wide pack slots (12 bits per symbol) for code tables whose codes are long on average: with the symbol
+// probabilities the code lengths imply (2^-length), the expected length is above 6.5 bits.  Shorter codes get
+// slots of 8 bits per symbol and the slow path for the rare subchunk that needs more.
+bool wants_wide_slots(const zc_codebook_t* cb, const uint32_t mode[2])
+{
+    for (int s = 0; s < 2; ++s) {
+        if (mode[s] != ZC_MODE_HUFF) continue;
+        uint64_t acc = 0;                        // sum of length * 2^(12 - length)
+        for (int v = 0; v < 256; ++v)
+            if (cb->len[s][v]) acc += (uint64_t)cb->len[s][v] << (kLmax - cb->len[s][v]);
+        if (2 * acc > 13ull << kLmax) return true;
+    }
+    return false;
+}
+
+void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const EncShape& sh)
+{
+    c.cs = p->syms_per_chunk; c.sub = p->syms_per_sub; c.chunk_bytes = p->chunk_bytes;
+    c.format = p->format; c.group = p->group;
+    c.mode[0] = mode[0]; c.mode[1] = mode[1];
+    c.n_slots = sh.n_slots; c.slot_bytes = sh.slot_bytes; c.region_bytes = sh.region_bytes; c.stage_stride = sh.stage_stride;
+    c.sub_width = sub_end_width(p->chunk_bytes);
+    c.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
+}
+
+void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const void* d_in, void* d_out, uint32_t first_batch,
+               uint32_t index)
+{
+    it.in = (const uint8_t*)d_in;
+    it.out = (uint8_t*)d_out;
+    it.input_bytes = p->input_bytes; it.n_syms = p->n_syms; it.n_elems = p->n_elems;
+    it.n_chunks = p->n_chunks;
+    it.first_batch = first_batch;
+    it.index = index;
+    it.pad = 0;
+    it.lay = make_layout(*p, mode);
+}
+
+void fill_tables(EncTables& T, const zc_codebook_t* cb)
+{
+    for (int s = 0; s < 2; ++s)
+        for (int v = 0; v < 256; ++v)
+            T.enc[s][v] = cb->len[s][v] ? (cb->code[s][v] << (32 - cb->len[s][v])) | cb->len[s][v] : 16u;
+}
+
+template <int N_ITEMS>
+cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const EncShape& sh, cudaStream_t st)
+{
+    const uint32_t want = std::max<uint32_t>(P.c.total_batches, 1);
+    const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * sh.per_sm);
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kern) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
+        if (e != cudaSuccess) return;
+        kern<<<grid, (sh.workers + 1) * 32, sh.smem, st>>>(P);
+        e = cudaGetLastError();
+    };
+    switch (format) {
+    case ZC_FMT_BF16: launch(encode_kernel<ZC_FMT_BF16, N_ITEMS>); break;
+    case ZC_FMT_FP8_E4M3: launch(encode_kernel<ZC_FMT_FP8_E4M3, N_ITEMS>); break;
+    default: launch(encode_kernel<ZC_FMT_FP4_E2M1, N_ITEMS>); break;
+    }
+    return e;
+}
+
+// Workspace of a batched call: control block | counters[n] | tables[n] | look-back words[batches]
+struct BatchLayout { size_t counters, tables, flags, total; };
+
+BatchLayout batch_layout(uint32_t n_tensors, uint64_t total_batches)
+{
+    BatchLayout L{};
+    L.counters = kControlBytes;
+    L.tables = (size_t)round_up(L.counters + sizeof(TensorCounters) * (uint64_t)n_tensors, 256);
+    L.flags = (size_t)round_up(L.tables + sizeof(EncTables) * (uint64_t)n_tensors, 256);
+    L.total = (size_t)round_up(L.flags + 8ull * total_batches, 256);
+    return L;
+}
+
+// Upper bound of the batches a tensor is cut into, whatever the modes of its streams turn out to be.
+uint64_t max_batches_of(const zc_plan_t* p)
+{
+    EncShape sh;
+    if (enc_shape(p, 2, true, &sh) != ZC_OK) return p->n_chunks;
+    return (p->n_chunks + (uint64_t)sh.workers - 1) / sh.workers;
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -565,77 +852,142 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
     if (out_capacity < zc_max_compressed_bytes(p)) return ZC_E_BUFFER_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
-    EncParams P{};
-    P.in = (const uint8_t*)d_in;
-    P.out = (uint8_t*)d_out;
-    P.ctl = (Control*)d_workspace;
-    P.flags = (unsigned long long*)((uint8_t*)d_workspace + kControlBytes);
-    P.input_bytes = p->input_bytes; P.n_syms = p->n_syms; P.n_elems = p->n_elems;
-    P.n_chunks = p->n_chunks; P.cs = p->syms_per_chunk; P.sub = p->syms_per_sub; P.chunk_bytes = p->chunk_bytes;
-    P.format = p->format; P.group = p->group;
-    uint32_t n_huff = 0;
+    uint32_t mode[2], n_huff = 0;
     for (int s = 0; s < 2; ++s) {
         // an empty tensor has no symbols to code: both streams are stored raw
-        P.mode[s] = p->n_syms ? cb->mode[s] : (uint32_t)ZC_MODE_RAW;
-        n_huff += P.mode[s] == ZC_MODE_HUFF;
+        mode[s] = p->n_syms ? cb->mode[s] : (uint32_t)ZC_MODE_RAW;
+        n_huff += mode[s] == ZC_MODE_HUFF;
     }
-    P.lay = make_layout(*p, P.mode);
-    // as many pack slots per lane region (up to 3) as still leave three blocks of 8 worker warps per SM
-    P.n_slots = 1;
-    for (uint32_t ns = 3; ns > 1; --ns) {
-        const size_t block = 2048 + (size_t)kEncMaxWorkers * std::max<uint32_t>(n_huff, 1) * kSubs * ((ns + 1) * p->syms_per_sub + 4);
-        if (3 * (block + 1024) <= kMaxSmem + 1024) { P.n_slots = ns; break; }
-    }
-    P.region_bytes = (P.n_slots + 1) * p->syms_per_sub + 4;
-    P.sub_width = sub_end_width(p->chunk_bytes);
-    P.stage_stride = kSubs * P.region_bytes;
-    P.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
+    EncShape sh;
+    const zc_status ss = enc_shape(p, n_huff, wants_wide_slots(cb, mode), &sh);
+    if (ss != ZC_OK) return ss;
 
-    EncTables T;
-    for (int s = 0; s < 2; ++s)
-        for (int v = 0; v < 256; ++v)
-            T.enc[s][v] = cb->len[s][v] ? (cb->code[s][v] << (32 - cb->len[s][v])) | cb->len[s][v] : 16u;
+    static thread_local EncParamsT<1> P;
+    P.c = EncCommon{};
+    fill_common(P.c, p, mode, sh);
+    P.c.ctl = (Control*)d_workspace;
+    P.c.counters = &P.c.ctl->tc;
+    P.c.flags = (unsigned long long*)((uint8_t*)d_workspace + kControlBytes);
+    P.c.tables = nullptr;
+    P.c.n_tensors = 1;
+    P.c.total_batches = (uint32_t)((p->n_chunks + (uint64_t)sh.workers - 1) / sh.workers);
+    fill_item(P.item[0], p, mode, d_in, d_out, 0, 0);
+    fill_tables(P.table, cb);
 
-    if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * p->n_chunks, st) != cudaSuccess) return ZC_E_CUDA;
-
-    cudaError_t e = cudaSuccess;
-    if (p->n_chunks) {
-        const size_t fixed = 512 * sizeof(uint32_t);
-        const size_t per_warp = std::max<size_t>((size_t)n_huff * P.stage_stride, 16);
-        // blocks of up to 8 worker warps (a batch of 8 consecutive chunks) plus the look-back warp; several
-        // blocks per SM so that loading, packing and copy-out phases of different blocks overlap
-        const uint32_t workers = (uint32_t)std::min<size_t>(kEncMaxWorkers, (kMaxSmem - fixed - 1024) / per_warp);
-        if (workers == 0) return ZC_E_UNSUPPORTED;
-        const uint32_t warps = workers + 1;
-        const size_t smem = fixed + workers * per_warp;
-        uint32_t per_sm = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (smem + 1024 + 1024), 3);
-        per_sm = std::max(per_sm, 1u);
-        const uint32_t want = (p->n_chunks + workers - 1) / workers;
-        const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * per_sm);
-        auto launch = [&](auto kern) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return;
-            kern<<<grid, warps * 32, smem, st>>>(P, T);
-            e = cudaGetLastError();
-        };
-        switch (p->format) {
-        case ZC_FMT_BF16: launch(encode_kernel<ZC_FMT_BF16>); break;
-        case ZC_FMT_FP8_E4M3: launch(encode_kernel<ZC_FMT_FP8_E4M3>); break;
-        default: launch(encode_kernel<ZC_FMT_FP4_E2M1>); break;
-        }
-        if (e != cudaSuccess) return ZC_E_CUDA;
-    }
-    if (p->n_chunks == 0) {
-        finish_kernel<<<1, 32, 0, st>>>(P);
-        if (cudaGetLastError() != cudaSuccess) return ZC_E_CUDA;
-    }
+    if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * P.c.total_batches, st) != cudaSuccess) return ZC_E_CUDA;
+    if (launch_encode<1>(P, p->format, sh, st) != cudaSuccess) return ZC_E_CUDA;
 
     if (h_out_bytes) {
         Control h;
         if (cudaMemcpyAsync(&h, d_workspace, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
         if (h.status & 0xFF) return (zc_status)(h.status & 0xFF);
-        *h_out_bytes = h.total16;
+        *h_out_bytes = h.tc.total16;
+    }
+    return ZC_OK;
+}
+
+size_t zc_compress_batch_workspace_bytes(uint32_t n_tensors, const zc_plan_t* const* plans)
+{
+    if (!plans) return 0;
+    uint64_t batches = 0;
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        if (!plans[t]) return 0;
+        batches += max_batches_of(plans[t]);
+    }
+    return batch_layout(n_tensors, batches).total;
+}
+
+zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const zc_codebook_t* const* codebooks,
+                            const void* const* d_in, void* const* d_out, const size_t* out_capacity,
+                            void* d_workspace, size_t workspace_bytes, uint64_t* h_out_bytes, void* cuda_stream)
+{
+    if (!d_workspace || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
+    if (n_tensors == 0) return ZC_OK;
+    if (!plans || !codebooks || !d_in || !d_out || !out_capacity) return ZC_E_INVALID_ARG;
+    uint64_t max_batches = 0;
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        const zc_plan_t* p = plans[t];
+        if (!p || !codebooks[t] || !d_out[t] || (!d_in[t] && p->n_elems)) return ZC_E_INVALID_ARG;
+        if (!aligned16(d_in[t]) || !aligned16(d_out[t])) return ZC_E_INVALID_ARG;
+        if (p->format != plans[0]->format || p->chunk_bytes != plans[0]->chunk_bytes) return ZC_E_INVALID_ARG;
+        if (out_capacity[t] < zc_max_compressed_bytes(p)) return ZC_E_BUFFER_TOO_SMALL;
+        max_batches += max_batches_of(p);
+    }
+    const BatchLayout L = batch_layout(n_tensors, max_batches);
+    if (workspace_bytes < L.total) return ZC_E_BUFFER_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint8_t* ws = (uint8_t*)d_workspace;
+    const zc_plan_t* p0 = plans[0];
+
+    // control block, counters and look-back words start from zero; the tables are uploaded in one copy
+    if (cudaMemsetAsync(ws, 0, L.tables, st) != cudaSuccess) return ZC_E_CUDA;
+    if (cudaMemsetAsync(ws + L.flags, 0, L.total - L.flags, st) != cudaSuccess) return ZC_E_CUDA;
+    static thread_local std::vector<EncTables> h_tables;
+    h_tables.resize(n_tensors);
+    for (uint32_t t = 0; t < n_tensors; ++t) fill_tables(h_tables[t], codebooks[t]);
+    if (cudaMemcpyAsync(ws + L.tables, h_tables.data(), sizeof(EncTables) * (size_t)n_tensors, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return ZC_E_CUDA;
+
+    // one launch per combination of stream modes and slot size (the kernel's shared-memory layout depends on
+    // them) and per kEncBatchMax tensors of it
+    static thread_local EncParamsT<(int)kEncBatchMax> P;
+    uint64_t flag_base = 0;
+    static thread_local std::vector<uint8_t> group;              // per tensor: mode0 | mode1 << 1 | wide << 2
+    group.resize(n_tensors);
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        const bool any = plans[t]->n_syms != 0;                  // an empty tensor: both streams raw
+        const uint32_t m[2] = {any ? codebooks[t]->mode[0] : (uint32_t)ZC_MODE_RAW, any ? codebooks[t]->mode[1] : (uint32_t)ZC_MODE_RAW};
+        group[t] = (uint8_t)(m[0] | (m[1] << 1) | (wants_wide_slots(codebooks[t], m) ? 4u : 0u));
+    }
+    for (uint32_t combo = 0; combo < 8; ++combo) {
+        const uint32_t mode[2] = {combo & 1u, (combo >> 1) & 1u};
+        const uint32_t n_huff = (mode[0] == ZC_MODE_HUFF) + (mode[1] == ZC_MODE_HUFF);
+        auto in_combo = [&](uint32_t t) { return group[t] == combo; };
+        EncShape sh;
+        const zc_status ss = enc_shape(p0, n_huff, (combo & 4u) != 0, &sh);
+        if (ss != ZC_OK) return ss;
+        uint32_t t = 0;
+        while (t < n_tensors) {
+            P.c = EncCommon{};
+            fill_common(P.c, p0, mode, sh);
+            uint32_t n = 0;
+            uint64_t batches = 0;
+            for (; t < n_tensors && n < kEncBatchMax; ++t) {
+                if (!in_combo(t)) continue;
+                const uint64_t nb = (plans[t]->n_chunks + (uint64_t)sh.workers - 1) / sh.workers;
+                if (batches + nb >= (1ull << 32)) break;
+                fill_item(P.item[n], plans[t], mode, d_in[t], d_out[t], (uint32_t)batches, t);
+                batches += nb;
+                ++n;
+            }
+            if (n == 0) {
+                if (t < n_tensors) return ZC_E_UNSUPPORTED;      // a single tensor with 2^32 batches or more
+                break;
+            }
+            P.c.ctl = (Control*)ws;
+            P.c.counters = (TensorCounters*)(ws + L.counters);
+            P.c.tables = (const EncTables*)(ws + L.tables);
+            P.c.flags = (unsigned long long*)(ws + L.flags) + flag_base;
+            P.c.n_tensors = n;
+            P.c.total_batches = (uint32_t)batches;
+            flag_base += batches;
+            // the ticket counter restarts for every launch
+            if (cudaMemsetAsync(&((Control*)ws)->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
+            if (launch_encode<(int)kEncBatchMax>(P, p0->format, sh, st) != cudaSuccess) return ZC_E_CUDA;
+        }
+    }
+
+    if (h_out_bytes) {
+        static thread_local std::vector<TensorCounters> h_counters;
+        h_counters.resize(n_tensors);
+        Control h;
+        if (cudaMemcpyAsync(&h, ws, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
+        if (cudaMemcpyAsync(h_counters.data(), ws + L.counters, sizeof(TensorCounters) * (size_t)n_tensors, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return ZC_E_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
+        if (h.status & 0xFF) return (zc_status)(h.status & 0xFF);
+        for (uint32_t t = 0; t < n_tensors; ++t) h_out_bytes[t] = h_counters[t].total16;
     }
     return ZC_OK;
 }

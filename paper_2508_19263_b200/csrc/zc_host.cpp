@@ -1,10 +1,12 @@
 // Host logic of libzc: plans, codebooks, container checks, statistics.
 // Nothing in this file touches the GPU, so it also runs on machines without one.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "zc_bits.cuh"
@@ -182,6 +184,44 @@ zc_status zc_build_codebook(const zc_plan_t* plan, const uint64_t* h_hist, zc_po
         cb->mode[s] = mode;
     }
     *out = cb;
+    return ZC_OK;
+}
+
+zc_status zc_build_codebooks(uint32_t n_tensors, const zc_plan_t* const* plans, const uint64_t* h_hists, zc_policy policy,
+                             uint32_t n_threads, zc_codebook_t** out)
+{
+    if (n_tensors == 0) return ZC_OK;
+    if (!plans || !h_hists || !out) return ZC_E_INVALID_ARG;
+    if (policy != ZC_POLICY_AUTO && policy != ZC_POLICY_HUFF_ALL && policy != ZC_POLICY_RAW_ALL)
+        return ZC_E_UNSUPPORTED;
+    if (n_threads == 0) {
+        const uint32_t hw = std::max(1u, std::thread::hardware_concurrency());
+        n_threads = std::min<uint32_t>({hw, 16u, (n_tensors + 7) / 8});     // a codebook takes tens of microseconds
+    }
+    n_threads = std::max<uint32_t>(1, std::min<uint32_t>(n_threads, n_tensors));
+    std::vector<zc_codebook_t*> made(n_tensors, nullptr);
+    std::atomic<int> first_error{ZC_OK};
+    auto work = [&](uint32_t tid) {
+        for (uint32_t t = tid; t < n_tensors; t += n_threads) {
+            const zc_status st = zc_build_codebook(plans[t], h_hists + 512ull * t, policy, &made[t]);
+            if (st != ZC_OK) { int expected = ZC_OK; first_error.compare_exchange_strong(expected, (int)st); }
+        }
+    };
+    std::vector<std::thread> pool;
+    try {
+        for (uint32_t i = 1; i < n_threads; ++i) pool.emplace_back(work, i);
+    } catch (...) {
+        // fewer threads than asked for: the strides of the missing ones are done below
+        const uint32_t started = (uint32_t)pool.size() + 1;
+        for (uint32_t i = started; i < n_threads; ++i) work(i);
+    }
+    work(0);
+    for (auto& th : pool) th.join();
+    if (first_error.load() != ZC_OK) {
+        for (auto* cb : made) delete cb;
+        return (zc_status)first_error.load();
+    }
+    for (uint32_t t = 0; t < n_tensors; ++t) out[t] = made[t];
     return ZC_OK;
 }
 

@@ -73,15 +73,23 @@ inline Layout make_layout(const zc_plan_s& p, const uint32_t mode[2])
     return L;
 }
 
-// Device workspace: a control block followed by one look-back word per chunk.
+// What the encoder accumulates per tensor on the device.
+struct TensorCounters {
+    unsigned long long payload_bits[2];
+    unsigned long long total16;  // payload area size in 16-byte units
+    uint32_t done;               // chunks that are completely written
+    uint32_t pad;
+};
+
+// Device workspace: a control block, then whatever the call needs behind it (zc_compress: one look-back
+// word per chunk).
 struct Control {
     unsigned long long status;   // (call id << 8) | zc_status raised on the device; first error of a call wins
     unsigned long long call_id;  // id of the call that last used the block; a status with another id is stale.
-                                 // zc_compress clears the whole block and uses id 0.
-    uint32_t ticket;             // next batch of chunks to hand out
-    uint32_t done;               // encoder blocks finished
-    unsigned long long payload_bits[2];
-    unsigned long long total16;  // payload area size in 16-byte units; finally the container size in bytes
+                                 // The compress calls clear the whole block and use id 0.
+    uint32_t ticket;             // next batch of chunks (encoder) or range of chunks (batched decoder) to hand out
+    uint32_t failed;             // batched calls: 1 + index of the tensor the recorded error belongs to
+    TensorCounters tc;           // zc_compress: the counters of its one tensor
     uint32_t pad[4];
 };
 constexpr size_t kControlBytes = 256;

@@ -114,3 +114,96 @@ def test_batch_argument_checks():
         zc.decompress_batch(zc.DecompressBatch([pa, pa], d, [1 << 15, 64], o), ws)
     assert e.value.status == zc.E_CORRUPT
     zc.decompress_batch(zc.DecompressBatch([], [], [], []), ws)      # nothing to do
+
+
+# ---- the batched encoder ----
+
+def _batch_compress(fmt, sizes, chunk_bytes, seed, policies):
+    datas = [_weights(fmt, n, seed + i) for i, n in enumerate(sizes)]
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    hists = [zo.histogram(fmt, d, n) for d, n in zip(datas, sizes)]
+    cbs = [zc.build_codebook(p, h, policies[i % len(policies)]) for i, (p, h) in enumerate(zip(plans, hists))]
+    ocbs = [zo.build_codebook(h, policies[i % len(policies)]) for i, h in enumerate(hists)]
+    d_ins = [_to_dev(d) for d in datas]
+    d_outs = [torch.full((p.max_compressed_bytes + 64,), 0xA5, dtype=torch.uint8, device=DEV) for p in plans]
+    batch = zc.CompressBatch(plans, d_ins, [o[: p.max_compressed_bytes] for o, p in zip(d_outs, plans)])
+    batch.set_codebooks(cbs)
+    ws = torch.full((batch.workspace_bytes,), 0x5A, dtype=torch.uint8, device=DEV)
+    return datas, plans, ocbs, d_outs, batch, ws
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("chunk_bytes", [1024, 4096, 16384])
+def test_batched_encoder_writes_the_oracle_s_containers(fmt, chunk_bytes):
+    sizes = _sizes(fmt, chunk_bytes)
+    policies = [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL]
+    datas, plans, ocbs, d_outs, batch, ws = _batch_compress(fmt, sizes, chunk_bytes, 3000 * fmt + chunk_bytes, policies)
+    for _ in range(2):                                               # twice in a row on the same workspace
+        got_sizes = zc.compress_batch(batch, ws)
+        assert zc.batch_status(ws) == (zc.OK, None)
+        for n, data, p, ocb, out, nbytes in zip(sizes, datas, plans, ocbs, d_outs, got_sizes):
+            want = zo.compress(fmt, data, n, chunk_bytes, ocb)
+            cont = out.cpu().numpy()
+            assert nbytes == want.size
+            assert np.array_equal(cont[:nbytes], want)
+            assert (cont[p.max_compressed_bytes:] == 0xA5).all()     # canary after the buffer
+
+
+def test_batched_encoder_many_small_tensors_and_the_batched_decoder_after_it():
+    fmt, chunk_bytes = zc.FMT_BF16, 1024
+    rng = np.random.default_rng(11)
+    sizes = [int(v) for v in rng.integers(0, 6000, 700)]
+    datas, plans, ocbs, d_outs, batch, ws = _batch_compress(fmt, sizes, chunk_bytes, 9, [zc.POLICY_AUTO, zc.POLICY_HUFF_ALL])
+    got_sizes = zc.compress_batch(batch, ws)
+    for n, data, ocb, out, nbytes in zip(sizes, datas, ocbs, d_outs, got_sizes):
+        want = zo.compress(fmt, data, n, chunk_bytes, ocb)
+        assert nbytes == want.size and np.array_equal(out[:nbytes].cpu().numpy(), want)
+    backs = [torch.full((p.input_bytes + 16,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    zc.decompress_batch(zc.DecompressBatch(plans, d_outs, got_sizes, backs), ws)
+    assert zc.batch_status(ws) == (zc.OK, None)
+    for p, data, back in zip(plans, datas, backs):
+        assert np.array_equal(back[: p.input_bytes].cpu().numpy(), data[: p.input_bytes])
+
+
+def test_batched_encoder_reports_a_symbol_without_code_and_its_tensor():
+    fmt, chunk_bytes = zc.FMT_BF16, 4096
+    sizes = [30000, 50000, 20000]
+    datas = [_weights(fmt, n, 40 + i) for i, n in enumerate(sizes)]
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    hists = [zo.histogram(fmt, d, n) for d, n in zip(datas, sizes)]
+    missing = int(np.flatnonzero(hists[1][0] == 0)[0])
+    bad = datas[1].copy().view(np.uint16); bad[777] = missing << 7
+    datas[1] = bad.view(np.uint8)
+    cbs = [zc.build_codebook(p, h, zc.POLICY_HUFF_ALL) for p, h in zip(plans, hists)]
+    d_ins = [_to_dev(d) for d in datas]
+    d_outs = [torch.zeros(p.max_compressed_bytes, dtype=torch.uint8, device=DEV) for p in plans]
+    batch = zc.CompressBatch(plans, d_ins, d_outs)
+    batch.set_codebooks(cbs)
+    ws = torch.zeros(batch.workspace_bytes, dtype=torch.uint8, device=DEV)
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress_batch(batch, ws)
+    assert e.value.status == zc.E_NO_CODE
+    assert zc.batch_status(ws) == (zc.E_NO_CODE, 1)
+
+
+def test_compress_batch_argument_checks():
+    pa, pb = zc.plan(zc.FMT_BF16, 5000, 4096), zc.plan(zc.FMT_BF16, 5000, 8192)
+    d = [torch.zeros(1 << 15, dtype=torch.uint8, device=DEV) for _ in range(2)]
+    o = [torch.zeros(1 << 15, dtype=torch.uint8, device=DEV) for _ in range(2)]
+    cb = zc.build_codebook(pa, np.ones((2, 256)), zc.POLICY_AUTO)
+    batch = zc.CompressBatch([pa, pb], d, o)
+    batch.set_codebooks([cb, cb])
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress_batch(batch, ws)
+    assert e.value.status == zc.E_INVALID_ARG
+    batch = zc.CompressBatch([pa, pa], d, [o[0], o[1][:100]])
+    batch.set_codebooks([cb, cb])
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress_batch(batch, ws)
+    assert e.value.status == zc.E_BUFFER_TOO_SMALL
+    batch = zc.CompressBatch([pa, pa], d, o)
+    batch.set_codebooks([cb, cb])
+    with pytest.raises(zc.ZcError) as e:
+        zc.compress_batch(batch, ws[:256])
+    assert e.value.status == zc.E_BUFFER_TOO_SMALL

@@ -223,3 +223,25 @@ def test_stats_match_oracle():
             assert st.stream[0].payload_bits == hd["streams"][0]["payload_bits"]
         else:
             assert st.out_bytes == 0
+
+
+def test_threaded_codebook_builder_matches_the_single_one():
+    rng = np.random.default_rng(3)
+    n = 37
+    hists = np.zeros((n, 2, 256), np.uint64)
+    for t in range(n):
+        k = int(rng.integers(1, 256))
+        hists[t, 0, rng.choice(256, k, replace=False)] = rng.integers(1, 1 << 20, k)
+        hists[t, 1] = rng.integers(0, 1000, 256)
+    hists[5] = 0                                                       # an empty tensor
+    plans = [zc.plan(zc.FMT_BF16, int(hists[t, 0].sum()), 4096) for t in range(n)]
+    for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL):
+        for threads in (0, 1, 3, 64):
+            many = zc.build_codebooks(plans, hists, policy, threads)
+            assert len(many) == n
+            for t in range(n):
+                one = zc.build_codebook(plans[t], hists[t], policy)
+                for s in range(2):
+                    a, b = many[t].get(s), one.get(s)
+                    assert a[0] == b[0] and np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
+    assert zc.build_codebooks([], np.zeros((0, 2, 256), np.uint64)) == []
