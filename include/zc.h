@@ -153,6 +153,14 @@ size_t zc_workspace_bytes(const zc_plan_t* plan);
  * Asynchronous on cuda_stream.  Errors: INVALID_ARG, CUDA. */
 zc_status zc_histogram(const zc_plan_t* plan, const void* d_in, uint64_t* d_hist, void* cuda_stream);
 
+/* The histograms of many tensors with one call (one launch per 896 tensors).
+ * plans    host array of n_tensors plans; all must have the same format
+ * d_in     host array of DEVICE pointers (16-byte aligned), the tensors' element bytes
+ * d_hists  device, uint64_t[n_tensors][2][256]; overwritten, d_hists[t] as by zc_histogram
+ * Asynchronous on cuda_stream.  Errors: INVALID_ARG, CUDA. */
+zc_status zc_histogram_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_in,
+                             uint64_t* d_hists, void* cuda_stream);
+
 /* ---- codebook (Sec. 3.1 / 4.1: plain Huffman coding, one code per stream per tensor;
  *      Sec. 3.3 precomputed dictionaries: any histogram may be given) ------------------------
  * h_hist  host, uint64_t[2][256]

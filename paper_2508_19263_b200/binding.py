@@ -69,6 +69,8 @@ def _load():
     L.zc_workspace_bytes.argtypes = [vp]
     L.zc_histogram.restype = C.c_int
     L.zc_histogram.argtypes = [vp, vp, vp, vp]
+    L.zc_histogram_batch.restype = C.c_int
+    L.zc_histogram_batch.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), vp, vp]
     L.zc_build_codebook.restype = C.c_int
     L.zc_build_codebook.argtypes = [vp, u64p, C.c_int, C.POINTER(vp)]
     L.zc_build_codebooks.restype = C.c_int
@@ -183,6 +185,26 @@ def histogram(p: Plan, d_in: torch.Tensor, d_hist: Optional[torch.Tensor] = None
         d_hist = torch.empty((2, 256), dtype=torch.int64, device=d_in.device)
     _check(_lib.zc_histogram(p._h, d_in.data_ptr(), d_hist.data_ptr(), _stream_ptr(stream)), "zc_histogram")
     return d_hist
+
+
+class HistogramBatch:
+    """Argument arrays of zc_histogram_batch, marshalled once."""
+
+    def __init__(self, plans, d_ins):
+        n = len(plans)
+        assert len(d_ins) == n
+        self.n = n
+        self._keep = (list(plans), list(d_ins))
+        self.plans = (C.c_void_p * max(n, 1))(*[p._h.value for p in plans])
+        self.ins = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in d_ins])
+
+
+def histogram_batch(batch: HistogramBatch, d_hists: torch.Tensor, stream=None) -> torch.Tensor:
+    """zc_histogram_batch: d_hists is a device tensor int64 [n, 2, 256] (uint64 counts)."""
+    assert d_hists.is_cuda and d_hists.is_contiguous() and d_hists.numel() == 512 * batch.n and d_hists.element_size() == 8
+    _check(_lib.zc_histogram_batch(batch.n, batch.plans, batch.ins, d_hists.data_ptr(), _stream_ptr(stream)),
+           "zc_histogram_batch")
+    return d_hists
 
 
 def build_codebook(p: Plan, h_hist, policy: int = POLICY_AUTO) -> Codebook:

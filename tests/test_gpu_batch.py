@@ -207,3 +207,21 @@ def test_compress_batch_argument_checks():
     with pytest.raises(zc.ZcError) as e:
         zc.compress_batch(batch, ws[:256])
     assert e.value.status == zc.E_BUFFER_TOO_SMALL
+
+
+# ---- the batched histogram ----
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_batched_histogram_counts_every_tensor(fmt):
+    G = zo.group(fmt)
+    rng = np.random.default_rng(fmt)
+    sizes = [0, 2 * G, 8 * G - 2 * G, 8 * G, 8 * G + 2 * G, 100000 * G + 6 * G, 0, 16 * G, 3 * G * 2, 1 << 21, 12345 * 2 * G] + \
+            [int(v) * 2 * G for v in rng.integers(0, 5000, 40)]
+    datas = [_weights(fmt, n, 500 + i) for i, n in enumerate(sizes)]
+    plans = [zc.plan(fmt, n, 4096) for n in sizes]
+    d_ins = [_to_dev(d) for d in datas]
+    d_hists = torch.full((len(sizes), 2, 256), -1, dtype=torch.int64, device=DEV)
+    zc.histogram_batch(zc.HistogramBatch(plans, d_ins), d_hists)
+    got = d_hists.cpu().numpy().astype(np.uint64)
+    for i, (n, data) in enumerate(zip(sizes, datas)):
+        assert np.array_equal(got[i], zo.histogram(fmt, data, n)), f"tensor {i} ({n} elements)"
