@@ -195,7 +195,9 @@ struct PackedChunk {
 // after every worker has posted its size, and a batch is handed out only while fewer than 4 handed-out
 // batches are unplaced.  So all warps of a block are within 4 batches of each other and rings of 8 are
 // enough.  A table slot is reused only when every worker has posted the last batch that used it.
-template <int FMT, int N_ITEMS>
+// H0 / H1: stream 0 / 1 is Huffman-coded (the same for every tensor of a launch; a template parameter so that
+// the code of a raw stream's packing and copy-out does not exist and the kernel stays small).
+template <int FMT, int N_ITEMS, bool H0, bool H1>
 __global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, 3)
 encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 {
@@ -204,8 +206,8 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_workers = (blockDim.x >> 5) - 1;
     const bool service = warp == n_workers;
-    const bool huff0 = C.mode[0] == ZC_MODE_HUFF, huff1 = C.mode[1] == ZC_MODE_HUFF;
-    const uint32_t n_huff = (huff0 ? 1u : 0u) + (huff1 ? 1u : 0u);
+    constexpr uint32_t n_huff = (H0 ? 1u : 0u) + (H1 ? 1u : 0u);
+    auto is_huff = [](const int s) constexpr { return s == 0 ? H0 : H1; };
     const uint32_t n_slots = C.n_slots;
 
     // shared: tables[kTabSlots][n_huff][256] | per worker warp: regions[n_huff][stage_stride]
@@ -338,7 +340,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                             uint32_t hs = 0;
 #pragma unroll
                             for (int s = 0; s < 2; ++s) {
-                                if (C.mode[s] != ZC_MODE_HUFF) continue;
+                                if (!is_huff(s)) continue;
                                 const uint32_t* src;
                                 if constexpr (N_ITEMS == 1) src = P.table.enc[s]; else src = C.tables[I.index].enc[s];
 #pragma unroll
@@ -357,7 +359,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         uint32_t hs = 0;
 #pragma unroll
                         for (int s = 0; s < 2; ++s) {
-                            if (C.mode[s] == ZC_MODE_HUFF) {
+                            if (is_huff(s)) {
                                 for (uint32_t v = lane; v < 256; v += 32) I.out[I.lay.section_off[s] + v] = (uint8_t)(tab[256 * hs + v] & 15);
                                 const uint32_t padded = (I.n_chunks + 3) & ~3u;
                                 for (uint32_t i = I.n_chunks + lane; i < padded; i += 32)
@@ -438,7 +440,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             uint64_t piece_off16 = off16;
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
-                if (C.mode[s] != ZC_MODE_HUFF) continue;
+                if (!is_huff(s)) continue;
                 const uint32_t end = pc.end[s];
                 uint32_t start = __shfl_up_sync(0xFFFFFFFFu, end, 1);
                 if (lane == 0) start = 0;
@@ -554,7 +556,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
-                    if (C.mode[s] == ZC_MODE_RAW) {
+                    if (!is_huff(s)) {
                         st_cs_v2(I.out + I.lay.section_off[s] + c_lo + k, make_uint2(sy[s][0], sy[s][1]));
                     } else {
                         const uint32_t j = __umulhi(k, C.sub_magic);          // subchunk of these 8 symbols
@@ -635,7 +637,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
-                    if (C.mode[s] != ZC_MODE_HUFF) continue;
+                    if (!is_huff(s)) continue;
                     // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
                     my_bits[s] = pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
                     // more than the slot holds: the bits beyond it do not survive the next staging
@@ -653,7 +655,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             {
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
-                    if (C.mode[s] != ZC_MODE_HUFF) continue;
+                    if (!is_huff(s)) continue;
                     uint32_t inc = my_bits[s];
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
@@ -702,7 +704,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                     uint32_t hs = 0;
 #pragma unroll
                     for (int s = 0; s < 2; ++s) {
-                        if (C.mode[s] != ZC_MODE_HUFF) continue;
+                        if (!is_huff(s)) continue;
                         pack(hs, 0, 2 * C.sub);
                         ++hs;
                     }
@@ -811,11 +813,18 @@ cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const E
         kern<<<grid, (sh.workers + 1) * 32, sh.smem, st>>>(P);
         e = cudaGetLastError();
     };
+    const bool h0 = P.c.mode[0] == ZC_MODE_HUFF, h1 = P.c.mode[1] == ZC_MODE_HUFF;
+#define ZC_ENC_CASE(F)                                                                  \
+    if (h0 && h1) launch(encode_kernel<F, N_ITEMS, true, true>);                       \
+    else if (h0) launch(encode_kernel<F, N_ITEMS, true, false>);                       \
+    else if (h1) launch(encode_kernel<F, N_ITEMS, false, true>);                       \
+    else launch(encode_kernel<F, N_ITEMS, false, false>);
     switch (format) {
-    case ZC_FMT_BF16: launch(encode_kernel<ZC_FMT_BF16, N_ITEMS>); break;
-    case ZC_FMT_FP8_E4M3: launch(encode_kernel<ZC_FMT_FP8_E4M3, N_ITEMS>); break;
-    default: launch(encode_kernel<ZC_FMT_FP4_E2M1, N_ITEMS>); break;
+    case ZC_FMT_BF16: ZC_ENC_CASE(ZC_FMT_BF16) break;
+    case ZC_FMT_FP8_E4M3: ZC_ENC_CASE(ZC_FMT_FP8_E4M3) break;
+    default: ZC_ENC_CASE(ZC_FMT_FP4_E2M1) break;
     }
+#undef ZC_ENC_CASE
     return e;
 }
 
