@@ -37,11 +37,12 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 ORACLE_SAMPLE_BYTES = int(os.environ.get("ZC_ORACLE_SAMPLE_BYTES", 768 << 20))   # bytes the oracle is timed on (tests shrink it)
-# DRAM bytes (read + write) per uncompressed byte from the ncu captures summarised under profiles/ (one 14336x4096
-# BF16 tensor, 4 KiB chunks).  Only quoted for that workload class; the write part is undercounted there because
-# some of the output is still in L2 when the kernel ends.
-NCU_DRAM_BYTES_PER_INPUT_BYTE = {"decode_kernel": (80.008704e6 + 59.361280e6) / 117440512.0,
-                                 "encode_kernel": (117.541632e6 + 33.090048e6) / 117440512.0}
+# DRAM bytes (read + write) per uncompressed byte from the ncu captures summarised under profiles/ (two-layer BF16
+# stack of 872.4 MB, 4 KiB chunks, batched kernels); traffic grows in proportion to the input, so the figure for a
+# launch over the whole stack is this ratio times its input bytes.  The write part is undercounted in a capture
+# because some of the output is still in L2 when the kernel ends.
+NCU_DRAM_BYTES_PER_INPUT_BYTE = {"decode_kernel": (593.707008e6 + 813.984000e6) / 872415232.0,
+                                 "encode_kernel": (872.737024e6 + 537.671424e6) / 872415232.0}
 
 
 def measured_peaks():
@@ -471,9 +472,9 @@ def run_ours(args):
                 "launches_per_call": n_dec_launch if dom_name == "decode_kernel" else n_enc_launch,
                 "avg_launch_ms": (ms_dec / n_dec_launch if dom_name == "decode_kernel" else ms_enc / n_enc_launch),
                 "algorithmic_bytes_per_launch": (U + C) / (n_dec_launch if dom_name == "decode_kernel" else n_enc_launch),
-                "traffic": (NCU_DRAM_BYTES_PER_INPUT_BYTE[dom_name] * U / n_t
-                            if args.workload == "cfg2_bf16_llama8b" and args.chunk_kib == 4 else None),
-                "traffic_source": "ncu dram__bytes_read+write of one 117 MB tensor (profiles/), scaled by input bytes per launch"}
+                "traffic": (NCU_DRAM_BYTES_PER_INPUT_BYTE[dom_name] * U / (n_dec_launch if dom_name == "decode_kernel" else n_enc_launch)
+                            if args.workload == "cfg2_bf16_llama8b" and args.chunk_kib == 4 and args.batch else None),
+                "traffic_source": "ncu dram__bytes_read+write of the two-layer BF16 stack (profiles/), scaled by input bytes per launch"}
 
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only) ----
     cpu = None
@@ -495,7 +496,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.workload, "tensors": n_t, "uncompressed_bytes": U, "compressed_bytes": C,
-                   "chunk_kib": args.chunk_kib, "policy": "auto", "streams": args.streams,
+                   "chunk_kib": args.chunk_kib, "policy": "auto", "batched_calls": bool(args.batch), "streams": args.streams if not args.batch else 1,
                    "l2": "inputs larger than L2 (no flush)"},
         "decode": dec, "encode": enc, "histogram": hist, "codebook_host_ms": ms_codebook,
         "compression_ratio": {"total_container": C / U, "exponent_stream_payload": st_bits[0] / (8 * n_syms),
