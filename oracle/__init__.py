@@ -16,7 +16,7 @@ from dataclasses import dataclass
 
 import numpy as np
 
-BF16, FP8_E4M3, FP4_E2M1 = 1, 2, 3
+BF16, FP8_E4M3, FP4_E2M1, SCALE_U8 = 1, 2, 3, 4
 RAW, HUFF = 0, 1
 POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL = 0, 1, 2
 L_MAX = 12

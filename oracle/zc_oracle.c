@@ -22,6 +22,9 @@
  *     zo_canonical_codes.
  *   - The mantissa stream is Huffman-coded only when its entropy makes that
  *     worthwhile and is stored as is otherwise (Sec. 3.1, 4.3): zo_choose_mode.
+ *   - The scaling factors of FP4 blocks are Huffman-coded as a stream of bytes
+ *     (Sec. 3.4, last two paragraphs; Sec. 4.4): format ZO_SCALE_U8 of zo_split /
+ *     zo_merge (reading R11).
  *   - Chunks of one fixed size, each with a little metadata, so that chunks
  *     can be located and decoded independently (Sec. 3.1, Sec. 4): zo_compress,
  *     zo_decompress, zo_decompress_chunk.
@@ -54,6 +57,11 @@
  *       bit; each chunk payload starts on a 16-byte boundary.
  *   R6  AUTO policy: a stream is Huffman-coded iff
  *       64 * sum(count*len) <= 63 * 8 * n_syms, otherwise stored raw.
+ *   R11 A stream of scale bytes (E8M0 or E4M3 scales, one "element" per byte)
+ *       uses the same two-stream container: the bytes at odd offsets are the
+ *       symbols of stream 0, the bytes at even offsets those of stream 1, so
+ *       symbol k of both streams comes from bytes 2k and 2k+1 (a missing last
+ *       odd byte counts as zero).  Each half has its own code.
  *
  * Container layout (little-endian, every section 16-byte aligned):
  *   header 128 B:
@@ -81,7 +89,7 @@
 #include <string.h>
 #include <math.h>
 
-enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3 };
+enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3, ZO_SCALE_U8 = 4 };
 enum { ZO_RAW = 0, ZO_HUFF = 1 };
 enum { ZO_POLICY_AUTO = 0, ZO_POLICY_HUFF_ALL = 1, ZO_POLICY_RAW_ALL = 2 };
 enum { ZO_LMAX = 12, ZO_SUBS = 32, ZO_HEADER = 128 };
@@ -132,6 +140,7 @@ int zo_group(int fmt)
     case ZO_BF16: return 1;
     case ZO_FP8_E4M3: return 2;
     case ZO_FP4_E2M1: return 4;
+    case ZO_SCALE_U8: return 2;
     default: return 0;
     }
 }
@@ -148,6 +157,7 @@ uint64_t zo_input_bytes(int fmt, uint64_t n_elems)
     case ZO_BF16: return 2 * n_elems;
     case ZO_FP8_E4M3: return n_elems;
     case ZO_FP4_E2M1: return (n_elems + 1) / 2;
+    case ZO_SCALE_U8: return n_elems;
     default: return 0;
     }
 }
@@ -181,6 +191,13 @@ void zo_split(int fmt, const uint8_t *in, uint64_t n_elems, uint8_t *s0, uint8_t
     int g = zo_group(fmt);
     int w = 8 / g;
     uint64_t ns = zo_n_syms(fmt, n_elems);
+    if (fmt == ZO_SCALE_U8) {                    /* R11: whole bytes, odd offsets -> stream 0 */
+        for (uint64_t k = 0; k < ns; ++k) {
+            s1[k] = in[2 * k];
+            s0[k] = (2 * k + 1 < n_elems) ? in[2 * k + 1] : 0;
+        }
+        return;
+    }
     for (uint64_t k = 0; k < ns; ++k) {
         unsigned a = 0, b = 0;
         for (int i = 0; i < g; ++i) {
@@ -203,6 +220,10 @@ void zo_merge(int fmt, const uint8_t *s0, const uint8_t *s1, uint64_t n_elems, u
     int g = zo_group(fmt);
     int w = 8 / g;
     unsigned fmask = (1u << w) - 1u;
+    if (fmt == ZO_SCALE_U8) {
+        for (uint64_t el = 0; el < n_elems; ++el) out[el] = (el & 1) ? s0[el / 2] : s1[el / 2];
+        return;
+    }
     if (fmt == ZO_FP4_E2M1) memset(out, 0, (size_t)zo_input_bytes(fmt, n_elems));
     for (uint64_t el = 0; el < n_elems; ++el) {
         uint64_t k = el / (uint64_t)g;

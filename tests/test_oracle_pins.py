@@ -16,7 +16,7 @@ import torch
 import oracle as zo
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-FORMATS = [zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1]
+FORMATS = [zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8]
 
 
 # --------------------------------------------------------------------------------------------
@@ -134,6 +134,22 @@ def test_merge_inverts_split(fmt, n):
     s0, s1 = zo.split(fmt, data, n)
     assert s0.size == s1.size == -(-n // zo.group(fmt))
     assert np.array_equal(zo.merge(fmt, s0, s1, n), data)
+
+
+def test_scale_bytes_split_into_odd_and_even_offsets():
+    """Sec. 3.4 / 4.4: the scaling factors are coded as a stream of bytes.  Here: bytes at odd offsets are the
+    symbols of stream 0, bytes at even offsets those of stream 1; a missing last odd byte counts as zero."""
+    s0, s1 = zo.split(zo.SCALE_U8, np.array([0x7A, 0x7B, 0x7C, 0x7D, 0x7E], np.uint8), 5)
+    assert list(s0) == [0x7B, 0x7D, 0x00] and list(s1) == [0x7A, 0x7C, 0x7E]
+    assert zo.n_syms(zo.SCALE_U8, 5) == 3 and zo.input_bytes(zo.SCALE_U8, 5) == 5 and zo.group(zo.SCALE_U8) == 2
+    assert list(zo.merge(zo.SCALE_U8, s0, s1, 5)) == [0x7A, 0x7B, 0x7C, 0x7D, 0x7E]
+    # the two histograms are the plain byte counts of the two halves
+    rng = np.random.default_rng(8)
+    d = rng.integers(0, 256, 10001, dtype=np.uint8)
+    h = zo.histogram(zo.SCALE_U8, d, d.size)
+    assert np.array_equal(h[1], np.bincount(d[0::2], minlength=256))
+    odd = np.bincount(d[1::2], minlength=256); odd[0] += 1              # the zero that stands for the missing byte
+    assert np.array_equal(h[0], odd)
 
 
 def test_tail_fields_are_zero():
@@ -393,6 +409,8 @@ def _random_tensor(fmt, n, seed, skew=True):
     rng = np.random.default_rng(seed)
     if n == 0:
         return np.zeros(0, np.uint8)
+    if fmt == zo.SCALE_U8:                                # E8M0-like scale bytes: a narrow bell around 120
+        return np.clip(np.round(rng.normal(120, 1.5, n)), 0, 255).astype(np.uint8)
     if fmt == zo.BF16:
         x = (rng.standard_normal(n) * 0.02).astype(np.float32)
         return torch.from_numpy(x).to(torch.bfloat16).view(torch.uint8).numpy().reshape(-1).copy()
