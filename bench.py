@@ -65,6 +65,10 @@ def workload_specs(name: str):
         return wl.FP8_E4M3, wl.llama8b_stack(3)
     if name == "cfg4_fp4_llama8b":
         return wl.FP4_E2M1, wl.llama8b_stack(4)
+    if name == "cfg4_fp4_scales":
+        # the E8M0 block scales of the same stack as byte streams (config 4 stores them raw; coding them is
+        # what the paper's FP4 result rests on, Sec. 3.4 / 4.4): 225 streams, 234.5 MB
+        return wl.SCALE_U8, wl.llama8b_stack(4)
     if name in ("cfg5_kv_bf16", "cfg5_kv_fp8"):
         # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers)
         fmt = wl.BF16 if name.endswith("bf16") else wl.FP8_E4M3

@@ -52,6 +52,12 @@ ZC_HD uint32_t spread_hi(uint32_t p) { return byte_perm(p, 0, 0x4342); }
 
 template <int FMT> struct Fields;
 
+// Scale bytes have no fields: split16 / merge16 handle them whole (the word-level pair is never used).
+template <> struct Fields<ZC_FMT_SCALE_U8> {
+    static ZC_HD void split_word(uint32_t, uint32_t& e, uint32_t& sm) { e = 0; sm = 0; }
+    static ZC_HD uint32_t merge_word(uint32_t, uint32_t) { return 0; }
+};
+
 // BF16: two elements per word; exponent = bits 14..7, sign+mantissa = (bit 15 -> bit 7) | bits 6..0.
 template <> struct Fields<ZC_FMT_BF16> {
     static ZC_HD void split_word(uint32_t v, uint32_t& e, uint32_t& sm)
@@ -112,6 +118,15 @@ template <> struct Fields<ZC_FMT_FP4_E2M1> {
 template <int FMT>
 ZC_HD void split16(const uint32_t in[4], uint32_t e[2], uint32_t sm[2])
 {
+    if (FMT == ZC_FMT_SCALE_U8) {
+        // scale bytes: odd offsets are stream 0, even offsets stream 1
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            e[h] = byte_perm(in[2 * h], in[2 * h + 1], 0x7531);
+            sm[h] = byte_perm(in[2 * h], in[2 * h + 1], 0x6420);
+        }
+        return;
+    }
     if (FMT == ZC_FMT_BF16) {
         // gather the four high bytes (sign, exponent bits 7..1) and the four low bytes (exponent bit 0,
         // mantissa) of four elements, then recombine per byte lane
@@ -153,6 +168,14 @@ ZC_HD void split16(const uint32_t in[4], uint32_t e[2], uint32_t sm[2])
 template <int FMT>
 ZC_HD void merge16(const uint32_t e[2], const uint32_t sm[2], uint32_t out[4])
 {
+    if (FMT == ZC_FMT_SCALE_U8) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            out[2 * h] = byte_perm(sm[h], e[h], 0x5140);
+            out[2 * h + 1] = byte_perm(sm[h], e[h], 0x7362);
+        }
+        return;
+    }
     if (FMT == ZC_FMT_BF16) {
         // element = sign | exponent << 7 | mantissa.  The exponent byte goes to bits 14..7 (placed in byte 0
         // and multiplied by 128 on the multiply-add pipe); the sign+mantissa byte is duplicated into both bytes so that its bit 7

@@ -311,7 +311,7 @@ __device__ __forceinline__ void decode_words_plain(LaneStream& st, uint32_t lut_
 
 struct DecShared {                   // what the block's prologue leaves for the chunk loop
     uint32_t lut0_s, lut1_s;         // shared addresses of the decode tables
-    uint32_t pairs0;                 // stream 0's table yields two symbols per lookup
+    uint32_t pairs0, pairs1;         // the stream's table yields two symbols per lookup
     unsigned long long sec0, sec1;   // byte offsets of the streams' sections
     unsigned long long payload_off, payload_bytes;
 };
@@ -460,8 +460,9 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     }
                     if (H1) {
                         const uint32_t row_s = rows1_s + lane * kRowStride;
-                        if (staged1) decode_words_plain<true>(st1, S.lut1_s, row_s, n_words);
-                        else decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
+                        if (!staged1) decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
+                        else if (S.pairs1) decode_words<2>(st1, S.lut1_s, row_s, n_words);
+                        else decode_words<1>(st1, S.lut1_s, row_s, n_words);
                     }
                 }
                 __syncwarp();
@@ -624,6 +625,7 @@ __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem
     DecShared S;
     S.lut0_s = smem_u32(M.lut0); S.lut1_s = smem_u32(M.lut1);
     S.pairs0 = huff0 && s_per_lookup[0] == 2;
+    S.pairs1 = huff1 && s_per_lookup[1] == 2;
     S.sec0 = s_sec[0]; S.sec1 = s_sec[1];
     S.payload_off = s_payload_off; S.payload_bytes = s_payload_bytes;
     uint32_t first_end0 = spec_end, first_off0 = spec_off;
@@ -735,15 +737,17 @@ zc_status dec_shape(const zc_plan_t* p, DecShape* out)
     DecShape s{};
     // symbols per round and lane: the largest of 64 / 32 / 16 that divides the subchunk length
     s.ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;
+    // scale bytes have both halves coded as a rule, the element formats one stream (the other one is raw)
+    const uint32_t coded = p->format == ZC_FMT_SCALE_U8 ? 2 : 1;
     const uint32_t rows_bytes = 32 * (16 * s.ppl + 4);
-    // per warp: one stream's rows plus room to stage a piece as large as the raw chunk stream; pieces that
-    // do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
-    s.pool_bytes = std::max<uint32_t>(rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32, 2 * rows_bytes);
+    // per warp: the coded streams' rows plus room to stage, per coded stream, a piece as large as the raw chunk
+    // stream; pieces that do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
+    s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32), 2 * rows_bytes);
     const size_t fixed = kDecFixedSmem + 512 /* static shared */;
     size_t per_warp = 16 + s.pool_bytes;
     s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     if (s.warps < 8) {               // large chunks: stage less
-        s.pool_bytes = std::max<uint32_t>(rows_bytes + 4096 + 32, 2 * rows_bytes);
+        s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + 4096 + 32), 2 * rows_bytes);
         per_warp = 16 + s.pool_bytes;
         s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     }
@@ -803,6 +807,7 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
     switch (p->format) {
     case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
     case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
+    case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
     default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
     }
 #undef ZC_DEC_CASE
@@ -869,7 +874,8 @@ zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
         switch (p0->format) {
         case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
         case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
-        default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
+        case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
+    default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
         }
 #undef ZC_DEC_CASE
         if (e != cudaSuccess) return ZC_E_CUDA;

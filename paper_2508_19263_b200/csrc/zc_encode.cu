@@ -737,11 +737,14 @@ zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* ou
     EncShape s{};
     const size_t fixed = (size_t)4 * kTabSlots * 256 * std::max<uint32_t>(n_huff, 1);
     s.slot_bytes = wide ? p->syms_per_sub + p->syms_per_sub / 2 : p->syms_per_sub;
-    // as many pack slots per lane region (up to 3) as still leave three blocks of 8 worker warps per SM
+    // pack slots per lane region: first as many resident blocks of 8 worker warps per SM as possible (up to 3),
+    // then as many slots (up to 3) as that number of blocks leaves room for
     s.n_slots = 1;
-    for (uint32_t ns = 3; ns > 1; --ns) {
+    uint32_t best_blocks = 0;
+    for (uint32_t ns = 1; ns <= 3; ++ns) {
         const size_t block = fixed + (size_t)kEncMaxWorkers * std::max<uint32_t>(n_huff, 1) * kSubs * (ns * s.slot_bytes + p->syms_per_sub + 4);
-        if (3 * (block + 2048) <= kMaxSmem + 1024) { s.n_slots = ns; break; }
+        const uint32_t blocks = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (block + 2048 + 1024), 3);
+        if (blocks >= best_blocks && blocks > 0) { best_blocks = blocks; s.n_slots = ns; }
     }
     s.region_bytes = s.n_slots * s.slot_bytes + p->syms_per_sub + 4;
     s.stage_stride = kSubs * s.region_bytes;
@@ -822,6 +825,7 @@ cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const E
     switch (format) {
     case ZC_FMT_BF16: ZC_ENC_CASE(ZC_FMT_BF16) break;
     case ZC_FMT_FP8_E4M3: ZC_ENC_CASE(ZC_FMT_FP8_E4M3) break;
+    case ZC_FMT_SCALE_U8: ZC_ENC_CASE(ZC_FMT_SCALE_U8) break;
     default: ZC_ENC_CASE(ZC_FMT_FP4_E2M1) break;
     }
 #undef ZC_ENC_CASE

@@ -203,6 +203,7 @@ zc_status zc_histogram(const zc_plan_t* p, const void* d_in, uint64_t* d_hist, v
     switch (p->format) {
     case ZC_FMT_BF16: launch(hist_kernel<ZC_FMT_BF16>); break;
     case ZC_FMT_FP8_E4M3: launch(hist_kernel<ZC_FMT_FP8_E4M3>); break;
+    case ZC_FMT_SCALE_U8: launch(hist_kernel<ZC_FMT_SCALE_U8>); break;
     default: launch(hist_kernel<ZC_FMT_FP4_E2M1>); break;
     }
     return e == cudaSuccess ? ZC_OK : ZC_E_CUDA;
@@ -250,6 +251,7 @@ zc_status zc_histogram_batch(uint32_t n_tensors, const zc_plan_t* const* plans, 
         switch (plans[0]->format) {
         case ZC_FMT_BF16: launch(hist_batch_kernel<ZC_FMT_BF16>); break;
         case ZC_FMT_FP8_E4M3: launch(hist_batch_kernel<ZC_FMT_FP8_E4M3>); break;
+        case ZC_FMT_SCALE_U8: launch(hist_batch_kernel<ZC_FMT_SCALE_U8>); break;
         default: launch(hist_batch_kernel<ZC_FMT_FP4_E2M1>); break;
         }
         if (e != cudaSuccess) return ZC_E_CUDA;

@@ -23,6 +23,7 @@ uint32_t group_of(uint32_t fmt)
     case ZC_FMT_BF16: return 1;
     case ZC_FMT_FP8_E4M3: return 2;
     case ZC_FMT_FP4_E2M1: return 4;
+    case ZC_FMT_SCALE_U8: return 2;
     default: return 0;
     }
 }
@@ -134,7 +135,7 @@ zc_status zc_plan(zc_format fmt, uint64_t n_elems, uint32_t chunk_bytes, zc_plan
     const uint64_t nc = (p->n_syms + p->syms_per_chunk - 1) / p->syms_per_chunk;
     if (nc > 0xFFFFFFFFull) { delete p; return ZC_E_INVALID_ARG; }
     p->n_chunks = (uint32_t)nc;
-    p->input_bytes = fmt == ZC_FMT_BF16 ? 2 * n_elems : fmt == ZC_FMT_FP8_E4M3 ? n_elems : n_elems / 2;
+    p->input_bytes = fmt == ZC_FMT_BF16 ? 2 * n_elems : fmt == ZC_FMT_FP4_E2M1 ? n_elems / 2 : n_elems;
     *out = p;
     return ZC_OK;
 }
@@ -363,6 +364,7 @@ zc_status zc_test_split16(zc_format fmt, const uint8_t* h_in16, uint8_t* h_e8, u
     case ZC_FMT_BF16: split16<ZC_FMT_BF16>(in, e, sm); break;
     case ZC_FMT_FP8_E4M3: split16<ZC_FMT_FP8_E4M3>(in, e, sm); break;
     case ZC_FMT_FP4_E2M1: split16<ZC_FMT_FP4_E2M1>(in, e, sm); break;
+    case ZC_FMT_SCALE_U8: split16<ZC_FMT_SCALE_U8>(in, e, sm); break;
     default: return ZC_E_UNSUPPORTED;
     }
     std::memcpy(h_e8, e, 8);
@@ -380,6 +382,7 @@ zc_status zc_test_merge16(zc_format fmt, const uint8_t* h_e8, const uint8_t* h_s
     case ZC_FMT_BF16: merge16<ZC_FMT_BF16>(e, sm, out); break;
     case ZC_FMT_FP8_E4M3: merge16<ZC_FMT_FP8_E4M3>(e, sm, out); break;
     case ZC_FMT_FP4_E2M1: merge16<ZC_FMT_FP4_E2M1>(e, sm, out); break;
+    case ZC_FMT_SCALE_U8: merge16<ZC_FMT_SCALE_U8>(e, sm, out); break;
     default: return ZC_E_UNSUPPORTED;
     }
     std::memcpy(h_out16, out, 16);

@@ -22,7 +22,7 @@ from typing import Iterator, List, Optional, Tuple
 
 import torch
 
-BF16, FP8_E4M3, FP4_E2M1 = 1, 2, 3
+BF16, FP8_E4M3, FP4_E2M1, SCALE_U8 = 1, 2, 3, 4
 FORMAT_NAMES = {BF16: "bf16", FP8_E4M3: "fp8_e4m3", FP4_E2M1: "fp4_e2m1"}
 
 
@@ -119,6 +119,9 @@ def make_weight(spec: TensorSpec, fmt: int, device) -> Tuple[torch.Tensor, int, 
     if fmt == FP4_E2M1:
         packed, scales = to_mxfp4_bytes(x)
         return packed, spec.n_elems, scales
+    if fmt == SCALE_U8:                          # the E8M0 block scales of the tensor's MXFP4 form, as a byte stream
+        _, scales = to_mxfp4_bytes(x)
+        return scales, scales.numel(), None
     raise ValueError(fmt)
 
 

@@ -11,7 +11,7 @@ from paper_2508_19263_b200 import binding as zc
 from paper_2508_19263_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
-FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1]
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8]
 DEV = "cuda"
 
 
@@ -57,6 +57,8 @@ def _weights(fmt, n, seed):
     rng = np.random.default_rng(seed)
     if n == 0:
         return np.zeros(0, np.uint8)
+    if fmt == zc.FMT_SCALE_U8:                                       # E8M0-like scale bytes: a narrow bell around 120
+        return np.clip(np.round(rng.normal(120, 1.5, n)), 0, 255).astype(np.uint8)
     if fmt == zc.FMT_BF16:
         x = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
         return x.to(torch.bfloat16).view(torch.uint8).numpy().reshape(-1).copy()
