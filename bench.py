@@ -73,6 +73,10 @@ def workload_specs(name: str):
         # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers)
         fmt = wl.BF16 if name.endswith("bf16") else wl.FP8_E4M3
         return fmt, [wl.TensorSpec(f"kv.{l}.{'kv'[w]}", (8, 8, 32768, 128), 0.0, 10 * l + w) for l in range(4) for w in range(2)]
+    if name in ("next2_bf16_delta", "small_bf16_delta"):
+        # delta checkpoints (Sec. 3.1 / 4.1): the XOR of two consecutive BF16 checkpoints of the config-2 stack is
+        # coded; the earlier checkpoint is a second resident input of every call
+        return wl.BF16, wl.llama8b_stack(2) if name.startswith("next2") else wl.llama8b_stack(2, n_layers=2, include_embedding=False)
     if name == "small_bf16":
         return wl.BF16, wl.llama8b_stack(2, n_layers=2, include_embedding=False)
     if name == "small_fp8":
@@ -131,11 +135,15 @@ class ClockSampler:
 # the CPU oracle as baseline / reference arm
 # --------------------------------------------------------------------------------------------
 
-def oracle_sample(fmt, specs, device):
-    """The first tensors of the workload up to ORACLE_SAMPLE_BYTES, as host arrays."""
+def oracle_sample(fmt, specs, device, delta=False):
+    """The first tensors of the workload up to ORACLE_SAMPLE_BYTES, as host arrays (delta workloads: the XOR of
+    the two checkpoints, which is what the oracle codes)."""
     out, total = [], 0
     for spec in specs:
-        if spec.name.startswith("kv."):
+        if delta:
+            cur, base, n = wl.checkpoint_pair(spec, device)
+            t = cur ^ base
+        elif spec.name.startswith("kv."):
             t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, device)
         else:
             t, n, _ = wl.make_weight(spec, fmt, device)
@@ -174,7 +182,7 @@ def run_reference(args):
     if rank != 0:
         return
     fmt, specs = workload_specs(args.workload)
-    sample, total = oracle_sample(fmt, specs, "cpu")
+    sample, total = oracle_sample(fmt, specs, "cpu", args.workload.endswith("_delta"))
     chunk_bytes = args.chunk_kib * 1024
     for _ in range(min(args.warmup, 1)):
         oracle_step(fmt, sample[:1], chunk_bytes)
@@ -256,13 +264,17 @@ def run_ours(args):
 
     # ---- resident inputs, plans, output buffers ----
     tensors = []
+    delta = args.workload.endswith("_delta")
     for spec in specs:
-        if spec.name.startswith("kv."):
+        base_t = None
+        if delta:
+            t, base_t, n = wl.checkpoint_pair(spec, dev)
+        elif spec.name.startswith("kv."):
             t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, dev)
         else:
             t, n, _ = wl.make_weight(spec, fmt, dev)
         p = zc.plan(fmt, n, chunk_bytes)
-        tensors.append({"name": spec.name, "in": t, "n": n, "plan": p,
+        tensors.append({"name": spec.name, "in": t, "base": base_t, "n": n, "plan": p,
                         "comp": torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=dev),
                         "out": torch.empty(p.input_bytes, dtype=torch.uint8, device=dev),
                         "ws": torch.empty(p.workspace_bytes, dtype=torch.uint8, device=dev)})
@@ -282,7 +294,8 @@ def run_ours(args):
         for s in side:
             stream.wait_stream(s)
 
-    hist_batch = zc.HistogramBatch([t["plan"] for t in tensors], [t["in"] for t in tensors])
+    bases = [t["base"] for t in tensors] if delta else None
+    hist_batch = zc.HistogramBatch([t["plan"] for t in tensors], [t["in"] for t in tensors], bases)
 
     def phase_hist():
         if args.batch:
@@ -292,7 +305,7 @@ def run_ours(args):
             return
         fork()
         for i, t in enumerate(tensors):
-            zc.histogram(t["plan"], t["in"], d_hist[i], stream=lanes[i % len(lanes)])
+            zc.histogram(t["plan"], t["in"], d_hist[i], stream=lanes[i % len(lanes)], d_base=t["base"])
         join()
         h_hist.copy_(d_hist, non_blocking=True)
         stream.synchronize()
@@ -308,7 +321,7 @@ def run_ours(args):
         for i, t in enumerate(tensors):
             t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
 
-    enc_batch = zc.CompressBatch([t["plan"] for t in tensors], [t["in"] for t in tensors], [t["comp"] for t in tensors])
+    enc_batch = zc.CompressBatch([t["plan"] for t in tensors], [t["in"] for t in tensors], [t["comp"] for t in tensors], bases)
     enc_ws = torch.empty(enc_batch.workspace_bytes, dtype=torch.uint8, device=dev)
 
     def phase_compress():
@@ -317,13 +330,13 @@ def run_ours(args):
             return
         fork()
         for i, t in enumerate(tensors):
-            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=lanes[i % len(lanes)])
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=lanes[i % len(lanes)], d_base=t["base"])
         join()
 
     # every tensor of the stack in one call; the decoder only needs an upper bound of each container's size
     # (the header carries the exact one)
     dec_batch = zc.DecompressBatch([t["plan"] for t in tensors], [t["comp"] for t in tensors],
-                                   [t["plan"].max_compressed_bytes for t in tensors], [t["out"] for t in tensors])
+                                   [t["plan"].max_compressed_bytes for t in tensors], [t["out"] for t in tensors], bases)
     batch_ws = torch.zeros(256, dtype=torch.uint8, device=dev)
 
     def phase_decompress():
@@ -332,7 +345,7 @@ def run_ours(args):
             return
         fork()
         for i, t in enumerate(tensors):
-            zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"], stream=lanes[i % len(lanes)])
+            zc.decompress(t["plan"], t["comp"], t["cbytes"], t["out"], t["ws"], stream=lanes[i % len(lanes)], d_base=t["base"])
         join()
 
     def read_sizes():
@@ -357,8 +370,8 @@ def run_ours(args):
         for i, t in enumerate(tensors):
             ln = lanes[i % len(lanes)]
             t["cb"] = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
-            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=ln)
-            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], stream=ln)
+            zc.compress(t["plan"], t["cb"], t["in"], t["comp"], t["ws"], sync=False, stream=ln, d_base=t["base"])
+            zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], stream=ln, d_base=t["base"])
         join()
 
     def timed(fn, reps):
@@ -426,15 +439,15 @@ def run_ours(args):
                 return
             for i, t in enumerate(tensors):
                 t["in"].copy_(h_in[i], non_blocking=True)
-                zc.histogram(t["plan"], t["in"], d_hist[i])
+                zc.histogram(t["plan"], t["in"], d_hist[i], d_base=t["base"])
             h_hist.copy_(d_hist, non_blocking=True)
             stream.synchronize()
             hh = h_hist.numpy()
             for i, t in enumerate(tensors):
                 cb = zc.build_codebook(t["plan"], hh[i], zc.POLICY_AUTO)
-                zc.compress(t["plan"], cb, t["in"], t["comp"], t["ws"], sync=False)
+                zc.compress(t["plan"], cb, t["in"], t["comp"], t["ws"], sync=False, d_base=t["base"])
                 h_out[i].copy_(t["comp"][: t["cbytes"]], non_blocking=True)
-                zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"])
+                zc.decompress(t["plan"], t["comp"], t["plan"].max_compressed_bytes, t["out"], t["ws"], d_base=t["base"])
 
         e2e_step()
         ms_e2e = timed(e2e_step, max(1, min(args.steps, 3)))
@@ -465,11 +478,13 @@ def run_ours(args):
             key = tuple(t["cb"].modes) if t["n"] else (0, 0)
             combos[key] = combos.get(key, 0) + 1
         n_enc_launch = sum((c + 255) // 256 for c in combos.values())
-        n_dec_launch = (n_t + 511) // 512
-        n_hist_launch = (n_t + 895) // 896
+        n_dec_launch = (n_t + 447) // 448
+        n_hist_launch = (n_t + 767) // 768
     else:
         n_enc_launch = n_dec_launch = n_hist_launch = n_t
-    dec, enc, hist = leg(ms_dec, U + C), leg(ms_enc, U + C), leg(ms_hist, U)
+    # delta form: the earlier checkpoint is read once more by every kernel
+    B_extra = U if delta else 0
+    dec, enc, hist = leg(ms_dec, U + C + B_extra), leg(ms_enc, U + C + B_extra), leg(ms_hist, U + B_extra)
     dom_name, dom = ("decode_kernel", dec) if ms_dec >= ms_enc else ("encode_kernel", enc)
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": dom["hbm_gbs"], "peak": peak, "unit": "GB/s",
                 "frac": dom["hbm_gbs"] / peak, "peak_source": peak_src,
@@ -483,7 +498,7 @@ def run_ours(args):
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only) ----
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        sample, total = oracle_sample(fmt, specs, dev)
+        sample, total = oracle_sample(fmt, specs, dev, delta)
         t_h, t_e, t_d, cb_sample = oracle_step(fmt, sample, chunk_bytes)
         cpu = {"value": total / (t_h + t_e + t_d) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {len(sample)} tensors of {args.workload}, {total} bytes",

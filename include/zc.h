@@ -156,7 +156,7 @@ size_t zc_workspace_bytes(const zc_plan_t* plan);
  * Asynchronous on cuda_stream.  Errors: INVALID_ARG, CUDA. */
 zc_status zc_histogram(const zc_plan_t* plan, const void* d_in, uint64_t* d_hist, void* cuda_stream);
 
-/* The histograms of many tensors with one call (one launch per 896 tensors).
+/* The histograms of many tensors with one call (one launch per 768 tensors).
  * plans    host array of n_tensors plans; all must have the same format
  * d_in     host array of DEVICE pointers (16-byte aligned), the tensors' element bytes
  * d_hists  device, uint64_t[n_tensors][2][256]; overwritten, d_hists[t] as by zc_histogram
@@ -277,7 +277,7 @@ zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
 /* ---- decompress many tensors with one call (Sec. 4 and 4.1: a model or a checkpoint is a set of
  *      tensors, each compressed on its own; Sec. 3.3: the K and V tensors of all layers) --------
  * The result is the same as n_tensors calls of zc_decompress; the work of all tensors is spread
- * over the GPU in one launch (per 512 tensors), so that small tensors do not pay a launch and a
+ * over the GPU in one launch (per 448 tensors), so that small tensors do not pay a launch and a
  * table build per block each.
  * n_tensors     number of tensors (0 returns ZC_OK and launches nothing)
  * plans         host array of n_tensors plans; all must have the same format and chunk_bytes
@@ -300,6 +300,35 @@ zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
  * the device (ZC_OK if none).  h_failed_tensor (optional, host) receives the index of the tensor
  * the first recorded error belongs to, or 0xFFFFFFFF. */
 zc_status zc_batch_status(const void* d_workspace, uint32_t* h_failed_tensor, void* cuda_stream);
+
+/* ---- XOR-delta forms (Sec. 3.1 and 4.1, delta checkpoints: the bitwise XOR of two consecutive
+ *      checkpoints is what gets split and coded) ----------------------------------------------
+ * Every call below is its namesake with one more argument, d_base: a DEVICE tensor of the same
+ * size as the input (16-byte aligned; the batched calls take a host array of such pointers).
+ * The XOR is fused into the kernels, nothing is materialised:
+ *   zc_histogram_xor   counts the symbols of (d_in XOR d_base)
+ *   zc_compress_xor    writes the container of (d_in XOR d_base)
+ *   zc_decompress_xor  writes (decoded tensor XOR d_base), i.e. the tensor d_in was
+ * A null d_base (for the batched calls: a null array, or a null entry) means "no base": the call
+ * then is exactly its namesake.  The container does not record that it holds a delta: the
+ * caller pairs it with the right base.  Errors: as the namesakes. */
+zc_status zc_histogram_xor(const zc_plan_t* plan, const void* d_in, const void* d_base, uint64_t* d_hist,
+                           void* cuda_stream);
+zc_status zc_histogram_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_in,
+                                 const void* const* d_base, uint64_t* d_hists, void* cuda_stream);
+zc_status zc_compress_xor(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, const void* d_base,
+                          void* d_out, size_t out_capacity, void* d_workspace, uint64_t* h_out_bytes,
+                          void* cuda_stream);
+zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans,
+                                const zc_codebook_t* const* codebooks, const void* const* d_in,
+                                const void* const* d_base, void* const* d_out, const size_t* out_capacity,
+                                void* d_workspace, size_t workspace_bytes, uint64_t* h_out_bytes,
+                                void* cuda_stream);
+zc_status zc_decompress_xor(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes, const void* d_base,
+                            void* d_out, void* d_workspace, void* cuda_stream);
+zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_comp,
+                                  const size_t* comp_bytes, const void* const* d_base, void* const* d_out,
+                                  void* d_workspace, void* cuda_stream);
 
 /* Synchronise cuda_stream and return the status word the last zc_compress / zc_decompress
  * call on this workspace left on the device (ZC_OK if none was raised). */

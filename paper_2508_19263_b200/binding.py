@@ -94,6 +94,20 @@ def _load():
     L.zc_decompress_batch.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), vp, vp]
     L.zc_batch_status.restype = C.c_int
     L.zc_batch_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    L.zc_histogram_xor.restype = C.c_int
+    L.zc_histogram_xor.argtypes = [vp, vp, vp, vp, vp]
+    L.zc_histogram_batch_xor.restype = C.c_int
+    L.zc_histogram_batch_xor.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp]
+    L.zc_compress_xor.restype = C.c_int
+    L.zc_compress_xor.argtypes = [vp, vp, vp, vp, vp, C.c_size_t, vp, u64p, vp]
+    L.zc_compress_batch_xor.restype = C.c_int
+    L.zc_compress_batch_xor.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                        C.POINTER(C.c_size_t), vp, C.c_size_t, u64p, vp]
+    L.zc_decompress_xor.restype = C.c_int
+    L.zc_decompress_xor.argtypes = [vp, vp, C.c_size_t, vp, vp, vp, vp]
+    L.zc_decompress_batch_xor.restype = C.c_int
+    L.zc_decompress_batch_xor.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), C.POINTER(vp),
+                                          vp, vp]
     L.zc_device_status.restype = C.c_int
     L.zc_device_status.argtypes = [vp, vp, vp]
     L.zc_validate_container.restype = C.c_int
@@ -178,31 +192,44 @@ class Codebook:
             self._h = None
 
 
-def histogram(p: Plan, d_in: torch.Tensor, d_hist: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """zc_histogram: returns a device tensor uint64-as-int64 [2, 256]."""
+def histogram(p: Plan, d_in: torch.Tensor, d_hist: Optional[torch.Tensor] = None, stream=None,
+              d_base: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """zc_histogram (zc_histogram_xor when d_base is given): returns a device tensor uint64-as-int64 [2, 256]."""
     assert d_in.is_cuda and d_in.is_contiguous()
     if d_hist is None:
         d_hist = torch.empty((2, 256), dtype=torch.int64, device=d_in.device)
-    _check(_lib.zc_histogram(p._h, d_in.data_ptr(), d_hist.data_ptr(), _stream_ptr(stream)), "zc_histogram")
+    if d_base is None:
+        _check(_lib.zc_histogram(p._h, d_in.data_ptr(), d_hist.data_ptr(), _stream_ptr(stream)), "zc_histogram")
+    else:
+        _check(_lib.zc_histogram_xor(p._h, d_in.data_ptr(), d_base.data_ptr(), d_hist.data_ptr(), _stream_ptr(stream)),
+               "zc_histogram_xor")
     return d_hist
+
+
+def _base_array(d_bases, n):
+    """Host array of base-tensor pointers for the XOR-delta forms (None: no base at all, a None entry: none for that tensor)."""
+    if d_bases is None:
+        return None
+    return (C.c_void_p * max(n, 1))(*[(t.data_ptr() if t is not None else None) for t in d_bases])
 
 
 class HistogramBatch:
     """Argument arrays of zc_histogram_batch, marshalled once."""
 
-    def __init__(self, plans, d_ins):
+    def __init__(self, plans, d_ins, d_bases=None):
         n = len(plans)
-        assert len(d_ins) == n
+        assert len(d_ins) == n and (d_bases is None or len(d_bases) == n)
         self.n = n
-        self._keep = (list(plans), list(d_ins))
+        self._keep = (list(plans), list(d_ins), list(d_bases) if d_bases is not None else None)
         self.plans = (C.c_void_p * max(n, 1))(*[p._h.value for p in plans])
         self.ins = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in d_ins])
+        self.bases = _base_array(d_bases, n)     # XOR-delta form when given
 
 
 def histogram_batch(batch: HistogramBatch, d_hists: torch.Tensor, stream=None) -> torch.Tensor:
     """zc_histogram_batch: d_hists is a device tensor int64 [n, 2, 256] (uint64 counts)."""
     assert d_hists.is_cuda and d_hists.is_contiguous() and d_hists.numel() == 512 * batch.n and d_hists.element_size() == 8
-    _check(_lib.zc_histogram_batch(batch.n, batch.plans, batch.ins, d_hists.data_ptr(), _stream_ptr(stream)),
+    _check(_lib.zc_histogram_batch_xor(batch.n, batch.plans, batch.ins, batch.bases, d_hists.data_ptr(), _stream_ptr(stream)),
            "zc_histogram_batch")
     return d_hists
 
@@ -239,14 +266,19 @@ def build_codebooks(plans, h_hists, policy: int = POLICY_AUTO, n_threads: int = 
 
 
 def compress(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Tensor, d_workspace: torch.Tensor,
-             sync: bool = True, stream=None) -> Optional[int]:
-    """zc_compress.  With sync=True returns the container size in bytes (and raises on a device-side
-    error); with sync=False the call is asynchronous and returns None."""
+             sync: bool = True, stream=None, d_base: Optional[torch.Tensor] = None) -> Optional[int]:
+    """zc_compress (zc_compress_xor when d_base is given).  With sync=True returns the container size in bytes
+    (and raises on a device-side error); with sync=False the call is asynchronous and returns None."""
     assert d_in.is_cuda and d_out.is_cuda and d_workspace.is_cuda
     assert d_workspace.numel() * d_workspace.element_size() >= p.workspace_bytes
     n = C.c_uint64(0)
-    st = _lib.zc_compress(p._h, cb._h, d_in.data_ptr(), d_out.data_ptr(), d_out.numel() * d_out.element_size(),
-                          d_workspace.data_ptr(), C.byref(n) if sync else None, _stream_ptr(stream))
+    if d_base is None:
+        st = _lib.zc_compress(p._h, cb._h, d_in.data_ptr(), d_out.data_ptr(), d_out.numel() * d_out.element_size(),
+                              d_workspace.data_ptr(), C.byref(n) if sync else None, _stream_ptr(stream))
+    else:
+        st = _lib.zc_compress_xor(p._h, cb._h, d_in.data_ptr(), d_base.data_ptr(), d_out.data_ptr(),
+                                  d_out.numel() * d_out.element_size(), d_workspace.data_ptr(), C.byref(n) if sync else None,
+                                  _stream_ptr(stream))
     _check(st, "zc_compress")
     return n.value if sync else None
 
@@ -265,12 +297,17 @@ def compress_noalloc(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Ten
 
 
 def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tensor, d_workspace: torch.Tensor,
-               stream=None) -> None:
-    """zc_decompress (asynchronous; call device_status() to learn the outcome)."""
+               stream=None, d_base: Optional[torch.Tensor] = None) -> None:
+    """zc_decompress, or zc_decompress_xor when d_base is given (asynchronous; call device_status() to learn the
+    outcome)."""
     assert d_comp.is_cuda and d_out.is_cuda and d_workspace.is_cuda
     assert d_out.numel() * d_out.element_size() >= p.input_bytes
-    _check(_lib.zc_decompress(p._h, d_comp.data_ptr(), comp_bytes, d_out.data_ptr(), d_workspace.data_ptr(),
-                              _stream_ptr(stream)), "zc_decompress")
+    if d_base is None:
+        _check(_lib.zc_decompress(p._h, d_comp.data_ptr(), comp_bytes, d_out.data_ptr(), d_workspace.data_ptr(),
+                                  _stream_ptr(stream)), "zc_decompress")
+    else:
+        _check(_lib.zc_decompress_xor(p._h, d_comp.data_ptr(), comp_bytes, d_base.data_ptr(), d_out.data_ptr(),
+                                      d_workspace.data_ptr(), _stream_ptr(stream)), "zc_decompress_xor")
 
 
 def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:
@@ -280,11 +317,12 @@ def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:
 class CompressBatch:
     """Argument arrays of zc_compress_batch, marshalled once; set_codebooks() swaps in new codebooks."""
 
-    def __init__(self, plans, d_ins, d_outs):
+    def __init__(self, plans, d_ins, d_outs, d_bases=None):
         n = len(plans)
-        assert len(d_ins) == n and len(d_outs) == n
+        assert len(d_ins) == n and len(d_outs) == n and (d_bases is None or len(d_bases) == n)
         self.n = n
-        self._keep = (list(plans), list(d_ins), list(d_outs))          # the arrays hold raw pointers
+        self._keep = (list(plans), list(d_ins), list(d_outs), list(d_bases) if d_bases is not None else None)
+        self.bases = _base_array(d_bases, n)     # XOR-delta form when given
         self.plans = (C.c_void_p * n)(*[p._h.value for p in plans])
         self.ins = (C.c_void_p * n)(*[t.data_ptr() for t in d_ins])
         self.outs = (C.c_void_p * n)(*[t.data_ptr() for t in d_outs])
@@ -303,19 +341,21 @@ class CompressBatch:
 def compress_batch(batch: CompressBatch, d_workspace: torch.Tensor, sync: bool = True, stream=None):
     """zc_compress_batch.  Returns the list of container sizes (sync=True) or None (asynchronous)."""
     sizes = (C.c_uint64 * max(batch.n, 1))()
-    _check(_lib.zc_compress_batch(batch.n, batch.plans, batch.cbs, batch.ins, batch.outs, batch.caps, d_workspace.data_ptr(),
-                                  d_workspace.numel(), sizes if sync else None, _stream_ptr(stream)), "zc_compress_batch")
+    _check(_lib.zc_compress_batch_xor(batch.n, batch.plans, batch.cbs, batch.ins, batch.bases, batch.outs, batch.caps,
+                                      d_workspace.data_ptr(), d_workspace.numel(), sizes if sync else None, _stream_ptr(stream)),
+           "zc_compress_batch")
     return [int(v) for v in sizes[: batch.n]] if sync else None
 
 
 class DecompressBatch:
     """Argument arrays of zc_decompress_batch, marshalled once and reusable for repeated calls."""
 
-    def __init__(self, plans, d_comps, comp_bytes, d_outs):
+    def __init__(self, plans, d_comps, comp_bytes, d_outs, d_bases=None):
         n = len(plans)
-        assert len(d_comps) == n and len(comp_bytes) == n and len(d_outs) == n
+        assert len(d_comps) == n and len(comp_bytes) == n and len(d_outs) == n and (d_bases is None or len(d_bases) == n)
         self.n = n
-        self._keep = (list(plans), list(d_comps), list(d_outs))        # the arrays hold raw pointers
+        self._keep = (list(plans), list(d_comps), list(d_outs), list(d_bases) if d_bases is not None else None)
+        self.bases = _base_array(d_bases, n)     # XOR-delta form when given
         self.plans = (C.c_void_p * n)(*[p._h.value for p in plans])
         self.comps = (C.c_void_p * n)(*[t.data_ptr() for t in d_comps])
         self.sizes = (C.c_size_t * n)(*[int(b) for b in comp_bytes])
@@ -324,8 +364,8 @@ class DecompressBatch:
 
 def decompress_batch(batch: DecompressBatch, d_workspace: torch.Tensor, stream=None) -> None:
     """zc_decompress_batch (asynchronous; read the outcome with batch_status)."""
-    _check(_lib.zc_decompress_batch(batch.n, batch.plans, batch.comps, batch.sizes, batch.outs, d_workspace.data_ptr(),
-                                    _stream_ptr(stream)), "zc_decompress_batch")
+    _check(_lib.zc_decompress_batch_xor(batch.n, batch.plans, batch.comps, batch.sizes, batch.bases, batch.outs,
+                                        d_workspace.data_ptr(), _stream_ptr(stream)), "zc_decompress_batch")
 
 
 def batch_status(d_workspace: torch.Tensor, stream=None):

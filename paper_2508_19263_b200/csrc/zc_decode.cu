@@ -15,6 +15,7 @@ namespace zc {
 
 struct DecParams {
     const uint8_t* comp;
+    const uint8_t* base;     // XOR-delta form: the decoded tensor is XOR-ed with this one before it is written; or null
     uint8_t* out;
     Control* ctl;
     uint64_t comp_bytes, input_bytes, n_syms, n_elems;
@@ -28,11 +29,12 @@ struct DecParams {
 // the chunks of all of them form one index space that is cut into equal contiguous ranges, one per block.
 struct DecItem {
     const uint8_t* comp;
+    const uint8_t* base;
     uint8_t* out;
     uint64_t comp_bytes, input_bytes, n_syms, n_elems;
     uint32_t n_chunks, first_chunk;          // first_chunk = chunks of all earlier tensors of the launch
 };
-constexpr uint32_t kDecBatchMax = 512;       // tensors per launch: the parameter block stays below 32 KiB
+constexpr uint32_t kDecBatchMax = 448;       // tensors per launch: the parameter block stays below 32 KiB
 struct DecBatchParams {
     Control* ctl;
     unsigned long long call_id;
@@ -317,7 +319,7 @@ struct DecShared {                   // what the block's prologue leaves for the
 };
 
 // PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
-template <int FMT, int PPL, bool H0, bool H1>
+template <int FMT, int PPL, bool H0, bool H1, bool XOR>
 __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShared& S, uint8_t* pool, uint64_t* bar,
                                                uint32_t first_end0, uint32_t first_off0,
                                                uint32_t c, const uint32_t c_end, const uint32_t step,
@@ -488,6 +490,12 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                 merge16<FMT>(e, m, o);
                 merge16<FMT>(e + 2, m + 2, o + 4);
                 uint8_t* dst = dst_lane + 2 * (i * k_step + r * R);
+                if (XOR && P.base) {                              // delta form: XOR the base tensor back in
+                    const uint64_t off = (uint64_t)(dst - P.out);
+                    const uint4 b0 = load16_guarded(P.base, off, P.input_bytes), b1 = load16_guarded(P.base, off + 16, P.input_bytes);
+                    o[0] ^= b0.x; o[1] ^= b0.y; o[2] ^= b0.z; o[3] ^= b0.w;
+                    o[4] ^= b1.x; o[5] ^= b1.y; o[6] ^= b1.z; o[7] ^= b1.w;
+                }
                 if (2 * k + 32 <= out_bytes) {
                     st_cs_v8(dst, o);
                 } else {
@@ -542,7 +550,7 @@ __device__ __forceinline__ DecSmem carve_smem(uint8_t* smem, uint32_t pool_bytes
 // Decodes the chunks c0, c0 + step, ... (< c_end) of one tensor with this warp; the whole block calls it
 // together (the header check and the table build are block-wide).  Returns a zc_status, the same in every
 // thread for the block-wide checks.
-template <int FMT, int PPL>
+template <int FMT, int PPL, bool XOR>
 __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem& M, const uint32_t c0, const uint32_t c_end,
                                                const uint32_t step, uint32_t& parity0, uint32_t& parity1)
 {
@@ -633,10 +641,10 @@ __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem
         first_end0 = load_sub_end(P.comp + S.sec0 + tab_sub, sub_w, c0, lane);
         first_off0 = reinterpret_cast<const uint32_t*>(P.comp + S.sec0 + tab_chunk)[c0];
     }
-    if (huff0 && !huff1) return run_chunks<FMT, PPL, true, false>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
-    if (!huff0 && !huff1) return run_chunks<FMT, PPL, false, false>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
-    if (huff0) return run_chunks<FMT, PPL, true, true>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
-    return run_chunks<FMT, PPL, false, true>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+    if (huff0 && !huff1) return run_chunks<FMT, PPL, true, false, XOR>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    if (!huff0 && !huff1) return run_chunks<FMT, PPL, false, false, XOR>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+    if (huff0) return run_chunks<FMT, PPL, true, true, XOR>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    return run_chunks<FMT, PPL, false, true, XOR>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
 }
 
 // One tensor per launch: the warps of all blocks take the chunks in turn.
@@ -649,13 +657,14 @@ decode_kernel(const __grid_constant__ DecParams P)
     const DecSmem M = carve_smem(smem, P.pool_bytes);
     if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
     uint32_t parity0 = 0, parity1 = 0;
-    const uint32_t err = decode_one<FMT, PPL>(P, M, blockIdx.x * n_warps + warp, P.n_chunks, gridDim.x * n_warps, parity0, parity1);
+    const uint32_t err = decode_one<FMT, PPL, false>(P, M, blockIdx.x * n_warps + warp, P.n_chunks, gridDim.x * n_warps, parity0, parity1);
     if (err) raise_status(P.ctl, P.call_id, err);
 }
 
 // Many tensors per launch: block b takes the chunks [b * total / grid, (b + 1) * total / grid) of the
 // concatenated chunk index space, tensor by tensor; it builds the tables of a tensor once for its whole share.
-template <int FMT, int PPL>
+// XOR: the launch has base tensors (delta form); a kernel of its own so that the plain form pays nothing for it.
+template <int FMT, int PPL, bool XOR>
 __global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
 decode_batch_kernel(const __grid_constant__ DecBatchParams B)
 {
@@ -667,7 +676,7 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
 
     auto run = [&](const uint32_t t, const uint32_t seg_lo, const uint32_t seg_hi) {
         DecParams P;
-        P.comp = B.item[t].comp; P.out = B.item[t].out; P.ctl = B.ctl;
+        P.comp = B.item[t].comp; P.base = XOR ? B.item[t].base : nullptr; P.out = B.item[t].out; P.ctl = B.ctl;
         P.comp_bytes = B.item[t].comp_bytes; P.input_bytes = B.item[t].input_bytes;
         P.n_syms = B.item[t].n_syms; P.n_elems = B.item[t].n_elems; P.n_chunks = B.item[t].n_chunks;
         P.cs = B.cs; P.sub = B.sub; P.chunk_bytes = B.chunk_bytes; P.format = B.format; P.group = B.group;
@@ -675,7 +684,7 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
         const uint64_t tables = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * (P.chunk_bytes <= 8192 ? 2u : 4u) * P.n_chunks;
         P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
         __syncthreads();                                         // everybody is done with the previous tensor's tables
-        const uint32_t err = decode_one<FMT, PPL>(P, M, seg_lo + warp, seg_hi, n_warps, parity0, parity1);
+        const uint32_t err = decode_one<FMT, PPL, XOR>(P, M, seg_lo + warp, seg_hi, n_warps, parity0, parity1);
         if (err && raise_status(B.ctl, B.call_id, err)) B.ctl->failed = B.tensor_base + t + 1;
     };
 
@@ -732,13 +741,14 @@ namespace {
 // Launch shape for a plan: symbols per round and lane, per-warp pool, warps per block, shared memory.
 struct DecShape { uint32_t ppl, pool_bytes, warps; size_t smem; };
 
-zc_status dec_shape(const zc_plan_t* p, DecShape* out)
+// both_coded: expect both streams to be Huffman-coded (scale bytes, deltas) instead of one
+zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
 {
     DecShape s{};
     // symbols per round and lane: the largest of 64 / 32 / 16 that divides the subchunk length
     s.ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;
-    // scale bytes have both halves coded as a rule, the element formats one stream (the other one is raw)
-    const uint32_t coded = p->format == ZC_FMT_SCALE_U8 ? 2 : 1;
+    // scale bytes and deltas have both streams coded as a rule, plain tensors one (the other one is raw)
+    const uint32_t coded = (both_coded || p->format == ZC_FMT_SCALE_U8) ? 2 : 1;
     const uint32_t rows_bytes = 32 * (16 * s.ppl + 4);
     // per warp: the coded streams' rows plus room to stage, per coded stream, a piece as large as the raw chunk
     // stream; pieces that do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
@@ -771,15 +781,27 @@ unsigned long long new_call_id()
 zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_bytes, void* d_out, void* d_workspace,
                         void* cuda_stream)
 {
+    return zc_decompress_xor(p, d_comp, comp_bytes, nullptr, d_out, d_workspace, cuda_stream);
+}
+
+zc_status zc_decompress_xor(const zc_plan_t* p, const void* d_comp, size_t comp_bytes, const void* d_base, void* d_out,
+                            void* d_workspace, void* cuda_stream)
+{
+    if (d_base) {                                            // the delta form lives in the batched kernel
+        if (!p) return ZC_E_INVALID_ARG;
+        void* out1 = d_out;
+        return zc_decompress_batch_xor(1, &p, &d_comp, &comp_bytes, &d_base, &out1, d_workspace, cuda_stream);
+    }
     if (!p || !d_comp || !d_workspace || (!d_out && p->n_elems)) return ZC_E_INVALID_ARG;
-    if (!aligned16(d_comp) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
+    if (!aligned16(d_comp) || !aligned16(d_base) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (comp_bytes < kHeaderBytes) return ZC_E_CORRUPT;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     DecShape shape;
-    const zc_status ss = dec_shape(p, &shape);
+    const zc_status ss = dec_shape(p, false, &shape);
     if (ss != ZC_OK) return ss;
     DecParams P{};
     P.comp = (const uint8_t*)d_comp;
+    P.base = nullptr;
     P.out = (uint8_t*)d_out;
     P.ctl = (Control*)d_workspace;
     P.comp_bytes = comp_bytes; P.input_bytes = p->input_bytes; P.n_syms = p->n_syms; P.n_elems = p->n_elems;
@@ -817,20 +839,29 @@ zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_byte
 zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_comp,
                               const size_t* comp_bytes, void* const* d_out, void* d_workspace, void* cuda_stream)
 {
+    return zc_decompress_batch_xor(n_tensors, plans, d_comp, comp_bytes, nullptr, d_out, d_workspace, cuda_stream);
+}
+
+zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_comp,
+                                  const size_t* comp_bytes, const void* const* d_base, void* const* d_out,
+                                  void* d_workspace, void* cuda_stream)
+{
     if (!d_workspace || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (n_tensors == 0) return ZC_OK;
     if (!plans || !d_comp || !comp_bytes || !d_out) return ZC_E_INVALID_ARG;
     for (uint32_t t = 0; t < n_tensors; ++t) {
         const zc_plan_t* p = plans[t];
         if (!p || !d_comp[t] || (!d_out[t] && p->n_elems)) return ZC_E_INVALID_ARG;
-        if (!aligned16(d_comp[t]) || !aligned16(d_out[t])) return ZC_E_INVALID_ARG;
+        if (!aligned16(d_comp[t]) || !aligned16(d_out[t]) || (d_base && !aligned16(d_base[t]))) return ZC_E_INVALID_ARG;
         if (p->format != plans[0]->format || p->chunk_bytes != plans[0]->chunk_bytes) return ZC_E_INVALID_ARG;
         if (comp_bytes[t] < kHeaderBytes) return ZC_E_CORRUPT;
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const zc_plan_t* p0 = plans[0];
     DecShape shape;
-    const zc_status ss = dec_shape(p0, &shape);
+    bool delta = false;
+    if (d_base) for (uint32_t t = 0; t < n_tensors; ++t) delta = delta || d_base[t] != nullptr;
+    const zc_status ss = dec_shape(p0, delta, &shape);
     if (ss != ZC_OK) return ss;
     const unsigned long long call_id = new_call_id();
     static thread_local DecBatchParams B;                    // 28 KiB: kept off the stack
@@ -847,6 +878,7 @@ zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
             const zc_plan_t* p = plans[base + n];
             DecItem& it = B.item[n];
             it.comp = (const uint8_t*)d_comp[base + n];
+            it.base = d_base ? (const uint8_t*)d_base[base + n] : nullptr;
             it.out = (uint8_t*)d_out[base + n];
             it.comp_bytes = comp_bytes[base + n]; it.input_bytes = p->input_bytes; it.n_syms = p->n_syms; it.n_elems = p->n_elems;
             it.n_chunks = p->n_chunks; it.first_chunk = (uint32_t)total;
@@ -867,10 +899,18 @@ zc_status zc_decompress_batch(uint32_t n_tensors, const zc_plan_t* const* plans,
             kern<<<grid, shape.warps * 32, shape.smem, st>>>(B);
             e = cudaGetLastError();
         };
-#define ZC_DEC_CASE(F)                                                     \
-    if (shape.ppl == 4) launch(decode_batch_kernel<F, 4>);                 \
-    else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2>);            \
-    else launch(decode_batch_kernel<F, 1>);
+        bool any_base = false;
+        for (uint32_t i = 0; i < n; ++i) any_base = any_base || B.item[i].base != nullptr;
+#define ZC_DEC_CASE(F)                                                                               \
+    if (any_base) {                                                                                  \
+        if (shape.ppl == 4) launch(decode_batch_kernel<F, 4, true>);                                 \
+        else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2, true>);                            \
+        else launch(decode_batch_kernel<F, 1, true>);                                                \
+    } else {                                                                                         \
+        if (shape.ppl == 4) launch(decode_batch_kernel<F, 4, false>);                                \
+        else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2, false>);                           \
+        else launch(decode_batch_kernel<F, 1, false>);                                               \
+    }
         switch (p0->format) {
         case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
         case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;

@@ -16,6 +16,7 @@ struct EncTables { uint32_t enc[2][256]; };
 // One tensor of a launch.
 struct EncItem {
     const uint8_t* in;
+    const uint8_t* base;                         // XOR-delta form: what is coded is in XOR base; or null
     uint8_t* out;
     uint64_t input_bytes, n_syms, n_elems;
     uint32_t n_chunks;
@@ -570,7 +571,24 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             const uint32_t n_vec = (c_syms + 7) / 8;
             const uint8_t* src_c = I.in + 2 * c_lo;
             uint32_t g = lane;
-            if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {           // every group of this chunk is complete
+            if (I.base) {
+                // delta form: the chunk of the base tensor is read alongside and XOR-ed in (two pairs of loads in flight)
+                const uint8_t* base_c = I.base + 2 * c_lo;
+                auto x4 = [](const uint4 a, const uint4 b) { return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w); };
+                if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {
+                    for (; g + 32 < n_vec; g += 64) {
+                        const uint4 x0 = ld_nc_v4(src_c + 16 * g), y0 = ld_nc_v4(base_c + 16 * g);
+                        const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32)), y1 = ld_nc_v4(base_c + 16 * (g + 32));
+                        stage_group(x4(x0, y0), 8 * g);
+                        stage_group(x4(x1, y1), 8 * (g + 32));
+                    }
+                    for (; g < n_vec; g += 32) stage_group(x4(ld_nc_v4(src_c + 16 * g), ld_nc_v4(base_c + 16 * g)), 8 * g);
+                } else {
+                    for (; g < n_vec; g += 32)
+                        stage_group(x4(load16_guarded(I.in, 2 * (c_lo + 8ull * g), I.input_bytes),
+                                       load16_guarded(I.base, 2 * (c_lo + 8ull * g), I.input_bytes)), 8 * g);
+                }
+            } else if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {    // every group of this chunk is complete
                 for (; g + 96 < n_vec; g += 128) {                          // four loads in flight per lane
                     const uint4 x0 = ld_nc_v4(src_c + 16 * g);
                     const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32));
@@ -784,10 +802,11 @@ void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const
     c.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
 }
 
-void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const void* d_in, void* d_out, uint32_t first_batch,
-               uint32_t index)
+void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const void* d_in, const void* d_base, void* d_out,
+               uint32_t first_batch, uint32_t index)
 {
     it.in = (const uint8_t*)d_in;
+    it.base = (const uint8_t*)d_base;
     it.out = (uint8_t*)d_out;
     it.input_bytes = p->input_bytes; it.n_syms = p->n_syms; it.n_elems = p->n_elems;
     it.n_chunks = p->n_chunks;
@@ -860,8 +879,14 @@ extern "C" {
 zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d_in, void* d_out, size_t out_capacity,
                       void* d_workspace, uint64_t* h_out_bytes, void* cuda_stream)
 {
+    return zc_compress_xor(p, cb, d_in, nullptr, d_out, out_capacity, d_workspace, h_out_bytes, cuda_stream);
+}
+
+zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const void* d_in, const void* d_base, void* d_out,
+                          size_t out_capacity, void* d_workspace, uint64_t* h_out_bytes, void* cuda_stream)
+{
     if (!p || !cb || !d_out || !d_workspace || (!d_in && p->n_elems)) return ZC_E_INVALID_ARG;
-    if (!aligned16(d_in) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
+    if (!aligned16(d_in) || !aligned16(d_base) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (out_capacity < zc_max_compressed_bytes(p)) return ZC_E_BUFFER_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
@@ -884,7 +909,7 @@ zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d
     P.c.tables = nullptr;
     P.c.n_tensors = 1;
     P.c.total_batches = (uint32_t)((p->n_chunks + (uint64_t)sh.workers - 1) / sh.workers);
-    fill_item(P.item[0], p, mode, d_in, d_out, 0, 0);
+    fill_item(P.item[0], p, mode, d_in, d_base, d_out, 0, 0);
     fill_tables(P.table, cb);
 
     if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * P.c.total_batches, st) != cudaSuccess) return ZC_E_CUDA;
@@ -915,6 +940,15 @@ zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, c
                             const void* const* d_in, void* const* d_out, const size_t* out_capacity,
                             void* d_workspace, size_t workspace_bytes, uint64_t* h_out_bytes, void* cuda_stream)
 {
+    return zc_compress_batch_xor(n_tensors, plans, codebooks, d_in, nullptr, d_out, out_capacity, d_workspace, workspace_bytes,
+                                 h_out_bytes, cuda_stream);
+}
+
+zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans, const zc_codebook_t* const* codebooks,
+                                const void* const* d_in, const void* const* d_base, void* const* d_out,
+                                const size_t* out_capacity, void* d_workspace, size_t workspace_bytes,
+                                uint64_t* h_out_bytes, void* cuda_stream)
+{
     if (!d_workspace || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (n_tensors == 0) return ZC_OK;
     if (!plans || !codebooks || !d_in || !d_out || !out_capacity) return ZC_E_INVALID_ARG;
@@ -922,7 +956,7 @@ zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, c
     for (uint32_t t = 0; t < n_tensors; ++t) {
         const zc_plan_t* p = plans[t];
         if (!p || !codebooks[t] || !d_out[t] || (!d_in[t] && p->n_elems)) return ZC_E_INVALID_ARG;
-        if (!aligned16(d_in[t]) || !aligned16(d_out[t])) return ZC_E_INVALID_ARG;
+        if (!aligned16(d_in[t]) || !aligned16(d_out[t]) || (d_base && !aligned16(d_base[t]))) return ZC_E_INVALID_ARG;
         if (p->format != plans[0]->format || p->chunk_bytes != plans[0]->chunk_bytes) return ZC_E_INVALID_ARG;
         if (out_capacity[t] < zc_max_compressed_bytes(p)) return ZC_E_BUFFER_TOO_SMALL;
         max_batches += max_batches_of(p);
@@ -970,7 +1004,7 @@ zc_status zc_compress_batch(uint32_t n_tensors, const zc_plan_t* const* plans, c
                 if (!in_combo(t)) continue;
                 const uint64_t nb = (plans[t]->n_chunks + (uint64_t)sh.workers - 1) / sh.workers;
                 if (batches + nb >= (1ull << 32)) break;
-                fill_item(P.item[n], plans[t], mode, d_in[t], d_out[t], (uint32_t)batches, t);
+                fill_item(P.item[n], plans[t], mode, d_in[t], d_base ? d_base[t] : nullptr, d_out[t], (uint32_t)batches, t);
                 batches += nb;
                 ++n;
             }

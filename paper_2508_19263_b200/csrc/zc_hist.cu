@@ -1,4 +1,7 @@
-// Split + histogram kernel and zc_histogram.
+// Split + histogram kernels and zc_histogram, zc_histogram_batch (and their XOR-delta forms).
+//
+// Delta form (Sec. 3.1 / 4.1, delta checkpoints): when a base tensor is given, what is counted is the
+// bitwise XOR of the input with the base, computed on the fly in registers.
 #include "zc_device.cuh"
 
 namespace zc {
@@ -37,9 +40,12 @@ __device__ __forceinline__ void count16(const uint4 x, uint32_t lane_bins)
     }
 }
 
+__device__ __forceinline__ uint4 xor4(const uint4 a, const uint4 b) { return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w); }
+
 template <int FMT>
 __global__ void __launch_bounds__(kHistThreads)
-hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_syms, unsigned long long* __restrict__ hist)
+hist_kernel(const uint8_t* __restrict__ in, const uint8_t* __restrict__ base, uint64_t input_bytes, uint64_t n_syms,
+            unsigned long long* __restrict__ hist)
 {
     extern __shared__ uint32_t bins[];           // [2][256][32]
     const uint32_t lane = threadIdx.x & 31;
@@ -51,6 +57,15 @@ hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_sym
     const uint64_t n_full = n_syms / 8 < input_bytes / 16 ? n_syms / 8 : input_bytes / 16;
     const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
     uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x;
+    if (base) {
+        for (; v + stride < n_full; v += 2 * stride) {          // two pairs of loads in flight
+            const uint4 x0 = ld_nc_v4(in + 16 * v), y0 = ld_nc_v4(base + 16 * v);
+            const uint4 x1 = ld_nc_v4(in + 16 * (v + stride)), y1 = ld_nc_v4(base + 16 * (v + stride));
+            count16<FMT>(xor4(x0, y0), lane_bins);
+            count16<FMT>(xor4(x1, y1), lane_bins);
+        }
+        for (; v < n_full; v += stride) count16<FMT>(xor4(ld_nc_v4(in + 16 * v), ld_nc_v4(base + 16 * v)), lane_bins);
+    }
     for (; v + 3 * stride < n_full; v += 4 * stride) {
         const uint4 x0 = ld_nc_v4(in + 16 * v);
         const uint4 x1 = ld_nc_v4(in + 16 * (v + stride));
@@ -64,7 +79,8 @@ hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_sym
     for (; v < n_full; v += stride) count16<FMT>(ld_nc_v4(in + 16 * v), lane_bins);
     // the ragged last group (fewer than 8 symbols, or input bytes that end inside the group)
     if (blockIdx.x == 0 && threadIdx.x == 0 && 8 * n_full < n_syms) {
-        const uint4 x = load16_guarded(in, 16 * n_full, input_bytes);
+        uint4 x = load16_guarded(in, 16 * n_full, input_bytes);
+        if (base) x = xor4(x, load16_guarded(base, 16 * n_full, input_bytes));
         const uint32_t w[4] = {x.x, x.y, x.z, x.w};
         uint32_t e[2], sm[2];
         split16<FMT>(w, e, sm);
@@ -90,10 +106,11 @@ hist_kernel(const uint8_t* __restrict__ in, uint64_t input_bytes, uint64_t n_sym
 // moves on to the next tensor.  Ragged last groups are counted straight into global memory.
 struct HistItem {
     const uint8_t* in;
+    const uint8_t* base;                         // XOR-delta form: the tensor the input is XOR-ed with, or null
     uint64_t input_bytes, n_syms;
     uint64_t first_vec;                          // complete groups of all earlier tensors of the launch
 };
-constexpr uint32_t kHistBatchMax = 896;          // keeps the parameter block below 32 KiB
+constexpr uint32_t kHistBatchMax = 768;          // keeps the parameter block below 32 KiB
 struct HistBatchParams {
     unsigned long long* hist;                    // [n_tensors][2][256]
     uint64_t total_vec;
@@ -117,7 +134,8 @@ hist_batch_kernel(const __grid_constant__ HistBatchParams B)
             const HistItem& I = B.item[t];
             const uint64_t n_full = I.n_syms / 8 < I.input_bytes / 16 ? I.n_syms / 8 : I.input_bytes / 16;
             if (8 * n_full >= I.n_syms) continue;
-            const uint4 x = load16_guarded(I.in, 16 * n_full, I.input_bytes);
+            uint4 x = load16_guarded(I.in, 16 * n_full, I.input_bytes);
+            if (I.base) x = xor4(x, load16_guarded(I.base, 16 * n_full, I.input_bytes));
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
             uint32_t e[2], sm[2];
             split16<FMT>(w, e, sm);
@@ -146,9 +164,19 @@ hist_batch_kernel(const __grid_constant__ HistBatchParams B)
         const uint64_t end = t + 1 < B.n_tensors ? B.item[t + 1].first_vec : B.total_vec;
         if (v_lo >= end) continue;
         const uint8_t* in = B.item[t].in;
+        const uint8_t* base = B.item[t].base;
         const uint64_t seg_hi = (v_hi < end ? v_hi : end) - first;
         uint64_t v = v_lo - first + threadIdx.x;
         constexpr uint64_t stride = kHistThreads;
+        if (base) {
+            for (; v + stride < seg_hi; v += 2 * stride) {       // two pairs of loads in flight
+                const uint4 x0 = ld_nc_v4(in + 16 * v), y0 = ld_nc_v4(base + 16 * v);
+                const uint4 x1 = ld_nc_v4(in + 16 * (v + stride)), y1 = ld_nc_v4(base + 16 * (v + stride));
+                count16<FMT>(xor4(x0, y0), lane_bins);
+                count16<FMT>(xor4(x1, y1), lane_bins);
+            }
+            for (; v < seg_hi; v += stride) count16<FMT>(xor4(ld_nc_v4(in + 16 * v), ld_nc_v4(base + 16 * v)), lane_bins);
+        }
         for (; v + 3 * stride < seg_hi; v += 4 * stride) {       // four loads in flight
             const uint4 x0 = ld_nc_v4(in + 16 * v);
             const uint4 x1 = ld_nc_v4(in + 16 * (v + stride));
@@ -185,7 +213,12 @@ extern "C" {
 
 zc_status zc_histogram(const zc_plan_t* p, const void* d_in, uint64_t* d_hist, void* cuda_stream)
 {
-    if (!p || !d_hist || (!d_in && p->n_elems) || !aligned16(d_in)) return ZC_E_INVALID_ARG;
+    return zc_histogram_xor(p, d_in, nullptr, d_hist, cuda_stream);
+}
+
+zc_status zc_histogram_xor(const zc_plan_t* p, const void* d_in, const void* d_base, uint64_t* d_hist, void* cuda_stream)
+{
+    if (!p || !d_hist || (!d_in && p->n_elems) || !aligned16(d_in) || !aligned16(d_base)) return ZC_E_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (cudaMemsetAsync(d_hist, 0, 2 * 256 * sizeof(uint64_t), st) != cudaSuccess) return ZC_E_CUDA;
     if (p->n_syms == 0) return ZC_OK;
@@ -197,7 +230,8 @@ zc_status zc_histogram(const zc_plan_t* p, const void* d_in, uint64_t* d_hist, v
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return;
-        kern<<<grid, kHistThreads, smem, st>>>((const uint8_t*)d_in, p->input_bytes, p->n_syms, (unsigned long long*)d_hist);
+        kern<<<grid, kHistThreads, smem, st>>>((const uint8_t*)d_in, (const uint8_t*)d_base, p->input_bytes, p->n_syms,
+                                                (unsigned long long*)d_hist);
         e = cudaGetLastError();
     };
     switch (p->format) {
@@ -212,10 +246,17 @@ zc_status zc_histogram(const zc_plan_t* p, const void* d_in, uint64_t* d_hist, v
 zc_status zc_histogram_batch(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_in, uint64_t* d_hists,
                              void* cuda_stream)
 {
+    return zc_histogram_batch_xor(n_tensors, plans, d_in, nullptr, d_hists, cuda_stream);
+}
+
+zc_status zc_histogram_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plans, const void* const* d_in,
+                                 const void* const* d_base, uint64_t* d_hists, void* cuda_stream)
+{
     if (n_tensors == 0) return ZC_OK;
     if (!plans || !d_in || !d_hists) return ZC_E_INVALID_ARG;
     for (uint32_t t = 0; t < n_tensors; ++t) {
         if (!plans[t] || (!d_in[t] && plans[t]->n_elems) || !aligned16(d_in[t])) return ZC_E_INVALID_ARG;
+        if (d_base && !aligned16(d_base[t])) return ZC_E_INVALID_ARG;
         if (plans[t]->format != plans[0]->format) return ZC_E_INVALID_ARG;
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -228,6 +269,7 @@ zc_status zc_histogram_batch(uint32_t n_tensors, const zc_plan_t* const* plans, 
         for (uint32_t i = 0; i < n; ++i) {
             const zc_plan_t* p = plans[base + i];
             B.item[i].in = (const uint8_t*)d_in[base + i];
+            B.item[i].base = d_base ? (const uint8_t*)d_base[base + i] : nullptr;
             B.item[i].input_bytes = p->input_bytes;
             B.item[i].n_syms = p->n_syms;
             B.item[i].first_vec = total;

@@ -125,6 +125,16 @@ def make_weight(spec: TensorSpec, fmt: int, device) -> Tuple[torch.Tensor, int, 
     raise ValueError(fmt)
 
 
+def checkpoint_pair(spec: TensorSpec, device, rel_step: float = 0.03) -> Tuple[torch.Tensor, torch.Tensor, int]:
+    """Two consecutive BF16 checkpoints of one weight tensor: the earlier one is the tensor of `make_weight`, the
+    later one is every weight moved by a relative step N(0, rel_step^2) (seed + 7) before the BF16 cast, so that
+    most exponents and the upper mantissa bits stay the same.  Returns (later bytes, earlier bytes, n_elems)."""
+    x = _randn(spec.shape, spec.std, spec.seed, device)
+    base = to_bf16_bytes(x)
+    x.mul_(1.0 + rel_step * torch.randn(spec.shape, generator=_gen(spec.seed + 7, device), device=device, dtype=torch.float32))
+    return to_bf16_bytes(x), base, spec.n_elems
+
+
 def config1_tensor(device) -> Tuple[torch.Tensor, int]:
     """One 1024x1024 FP8 E4M3 weight tensor, N(0, 0.02^2), per-tensor scale amax/448, seed 0."""
     x = _randn((1024, 1024), 0.02, 0, device)

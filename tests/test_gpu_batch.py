@@ -225,3 +225,75 @@ def test_batched_histogram_counts_every_tensor(fmt):
     got = d_hists.cpu().numpy().astype(np.uint64)
     for i, (n, data) in enumerate(zip(sizes, datas)):
         assert np.array_equal(got[i], zo.histogram(fmt, data, n)), f"tensor {i} ({n} elements)"
+
+
+# ---- XOR-delta forms (delta checkpoints, Sec. 3.1 / 4.1) ----
+
+def _checkpoint_pair(fmt, n, seed):
+    """Two tensors that differ little: the second one is the first with a few low mantissa bits flipped here and
+    there and a sprinkling of completely different elements."""
+    rng = np.random.default_rng(seed)
+    a = _weights(fmt, n, seed)
+    b = a.copy()
+    if b.size:
+        flip = rng.random(b.size) < 0.3
+        b[flip] ^= rng.integers(0, 4, int(flip.sum()), dtype=np.uint8)
+        wild = rng.random(b.size) < 0.002
+        b[wild] = rng.integers(0, 256, int(wild.sum()), dtype=np.uint8)
+    return a, b
+
+
+@pytest.mark.parametrize("fmt", [zc.FMT_BF16, zc.FMT_FP8_E4M3])
+@pytest.mark.parametrize("chunk_bytes", [1024, 4096, 16384])
+def test_xor_delta_single_calls_match_the_oracle_on_the_xor(fmt, chunk_bytes):
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    for n in [0, 2 * G, 5 * cs * G + cs * G // 3 + 2 * G, 23 * cs * G + 6 * G]:
+        base, cur = _checkpoint_pair(fmt, n, chunk_bytes + n)
+        delta = base ^ cur                                            # the plain definition of what is coded
+        p = zc.plan(fmt, n, chunk_bytes)
+        d_cur, d_base = _to_dev(cur), _to_dev(base)
+        hist = zc.histogram(p, d_cur, d_base=d_base).cpu().numpy().astype(np.uint64)
+        assert np.array_equal(hist, zo.histogram(fmt, delta, n))
+        cb, ocb = zc.build_codebook(p, hist, zc.POLICY_AUTO), zo.build_codebook(hist, zc.POLICY_AUTO)
+        d_out = torch.full((p.max_compressed_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+        ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+        nbytes = zc.compress(p, cb, d_cur, d_out, ws, d_base=d_base)
+        want = zo.compress(fmt, delta, n, chunk_bytes, ocb)
+        assert nbytes == want.size and np.array_equal(d_out[:nbytes].cpu().numpy(), want)
+        d_back = torch.full((p.input_bytes + 32,), 0xEE, dtype=torch.uint8, device=DEV)
+        zc.decompress(p, d_out, nbytes, d_back, ws, d_base=d_base)
+        assert zc.device_status(p, ws) == zc.OK
+        back = d_back.cpu().numpy()
+        assert np.array_equal(back[: p.input_bytes], cur[: p.input_bytes]) and (back[p.input_bytes:] == 0xEE).all()
+
+
+def test_xor_delta_batched_calls():
+    fmt, chunk_bytes = zc.FMT_BF16, 4096
+    sizes = _sizes(fmt, chunk_bytes)
+    pairs = [_checkpoint_pair(fmt, n, 900 + i) for i, n in enumerate(sizes)]
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    d_bases = [_to_dev(a) for a, _ in pairs]
+    d_curs = [_to_dev(b) for _, b in pairs]
+    d_bases[3] = None                                                 # one tensor of the batch without a base
+    deltas = [(b if i == 3 else a ^ b) for i, (a, b) in enumerate(pairs)]
+    d_hists = torch.zeros((len(sizes), 2, 256), dtype=torch.int64, device=DEV)
+    zc.histogram_batch(zc.HistogramBatch(plans, d_curs, d_bases), d_hists)
+    hists = d_hists.cpu().numpy().astype(np.uint64)
+    for i, (n, d) in enumerate(zip(sizes, deltas)):
+        assert np.array_equal(hists[i], zo.histogram(fmt, d, n))
+    cbs = zc.build_codebooks(plans, hists, zc.POLICY_AUTO)
+    d_outs = [torch.zeros(p.max_compressed_bytes, dtype=torch.uint8, device=DEV) for p in plans]
+    batch = zc.CompressBatch(plans, d_curs, d_outs, d_bases)
+    batch.set_codebooks(cbs)
+    ws = torch.empty(batch.workspace_bytes, dtype=torch.uint8, device=DEV)
+    got = zc.compress_batch(batch, ws)
+    for i, (n, d) in enumerate(zip(sizes, deltas)):
+        want = zo.compress(fmt, d, n, chunk_bytes, zo.build_codebook(hists[i], zc.POLICY_AUTO))
+        assert got[i] == want.size and np.array_equal(d_outs[i][: got[i]].cpu().numpy(), want)
+    backs = [torch.full((p.input_bytes + 16,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    zc.decompress_batch(zc.DecompressBatch(plans, d_outs, got, backs, d_bases), ws)
+    assert zc.batch_status(ws) == (zc.OK, None)
+    for p, (a, b), back in zip(plans, pairs, backs):
+        out = back.cpu().numpy()
+        assert np.array_equal(out[: p.input_bytes], b[: p.input_bytes]) and (out[p.input_bytes:] == 0xEE).all()
