@@ -247,6 +247,16 @@ zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, co
 zc_status zc_decompress(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes, void* d_out,
                         void* d_workspace, void* cuda_stream);
 
+/* ---- random access (Sec. 3.1: any chunk can be located and decoded on its own) ---------------
+ * Decodes chunks first_chunk .. first_chunk + n_chunks - 1 of a container and nothing else.
+ * d_out receives their element bytes, starting with the first byte of chunk first_chunk (so it
+ * needs n_chunks * chunk_bytes bytes, fewer if the range includes the tensor's last chunk).
+ * Everything else as zc_decompress (header and tables are checked the same way).
+ * Errors: INVALID_ARG (also for a range that does not lie inside the plan's chunks), CUDA. */
+zc_status zc_decompress_chunks(const zc_plan_t* plan, const void* d_comp, size_t comp_bytes,
+                               uint32_t first_chunk, uint32_t n_chunks, void* d_out, void* d_workspace,
+                               void* cuda_stream);
+
 /* ---- compress many tensors with one call (Sec. 4 and 4.1: a model or a checkpoint is a set of
  *      tensors, each compressed on its own with its own codes; Sec. 3.3: K and V of all layers) -
  * The containers are byte for byte those of n_tensors calls of zc_compress; the chunks of all

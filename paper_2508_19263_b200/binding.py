@@ -108,6 +108,8 @@ def _load():
     L.zc_decompress_batch_xor.restype = C.c_int
     L.zc_decompress_batch_xor.argtypes = [C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), C.POINTER(vp),
                                           vp, vp]
+    L.zc_decompress_chunks.restype = C.c_int
+    L.zc_decompress_chunks.argtypes = [vp, vp, C.c_size_t, C.c_uint32, C.c_uint32, vp, vp, vp]
     L.zc_device_status.restype = C.c_int
     L.zc_device_status.argtypes = [vp, vp, vp]
     L.zc_validate_container.restype = C.c_int
@@ -308,6 +310,14 @@ def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tens
     else:
         _check(_lib.zc_decompress_xor(p._h, d_comp.data_ptr(), comp_bytes, d_base.data_ptr(), d_out.data_ptr(),
                                       d_workspace.data_ptr(), _stream_ptr(stream)), "zc_decompress_xor")
+
+
+def decompress_chunks(p: Plan, d_comp: torch.Tensor, comp_bytes: int, first_chunk: int, n_chunks: int, d_out: torch.Tensor,
+                      d_workspace: torch.Tensor, stream=None) -> None:
+    """zc_decompress_chunks: d_out receives the element bytes of chunks first_chunk .. first_chunk + n_chunks - 1."""
+    assert d_comp.is_cuda and d_out.is_cuda and d_workspace.is_cuda
+    _check(_lib.zc_decompress_chunks(p._h, d_comp.data_ptr(), comp_bytes, first_chunk, n_chunks, d_out.data_ptr(),
+                                     d_workspace.data_ptr(), _stream_ptr(stream)), "zc_decompress_chunks")
 
 
 def device_status(p: Plan, d_workspace: torch.Tensor, stream=None) -> int:

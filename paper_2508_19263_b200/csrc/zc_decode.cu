@@ -21,6 +21,7 @@ struct DecParams {
     uint64_t comp_bytes, input_bytes, n_syms, n_elems;
     uint32_t n_chunks, cs, sub, chunk_bytes, format, group;
     uint32_t pool_bytes;     // per-warp shared memory: symbol rows first, the rest stages compressed pieces
+    uint32_t c_begin, c_end; // chunks the launch decodes (zc_decompress: all of them)
     uint32_t spec;           // the container is long enough to read stream 0's tables before the header is checked
     unsigned long long call_id;
 };
@@ -657,7 +658,7 @@ decode_kernel(const __grid_constant__ DecParams P)
     const DecSmem M = carve_smem(smem, P.pool_bytes);
     if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
     uint32_t parity0 = 0, parity1 = 0;
-    const uint32_t err = decode_one<FMT, PPL, false>(P, M, blockIdx.x * n_warps + warp, P.n_chunks, gridDim.x * n_warps, parity0, parity1);
+    const uint32_t err = decode_one<FMT, PPL, false>(P, M, P.c_begin + blockIdx.x * n_warps + warp, P.c_end, gridDim.x * n_warps, parity0, parity1);
     if (err) raise_status(P.ctl, P.call_id, err);
 }
 
@@ -680,7 +681,7 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
         P.comp_bytes = B.item[t].comp_bytes; P.input_bytes = B.item[t].input_bytes;
         P.n_syms = B.item[t].n_syms; P.n_elems = B.item[t].n_elems; P.n_chunks = B.item[t].n_chunks;
         P.cs = B.cs; P.sub = B.sub; P.chunk_bytes = B.chunk_bytes; P.format = B.format; P.group = B.group;
-        P.pool_bytes = B.pool_bytes; P.call_id = B.call_id;
+        P.pool_bytes = B.pool_bytes; P.call_id = B.call_id; P.c_begin = 0; P.c_end = P.n_chunks;
         const uint64_t tables = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * (P.chunk_bytes <= 8192 ? 2u : 4u) * P.n_chunks;
         P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
         __syncthreads();                                         // everybody is done with the previous tensor's tables
@@ -792,8 +793,16 @@ zc_status zc_decompress_xor(const zc_plan_t* p, const void* d_comp, size_t comp_
         void* out1 = d_out;
         return zc_decompress_batch_xor(1, &p, &d_comp, &comp_bytes, &d_base, &out1, d_workspace, cuda_stream);
     }
+    if (!p) return ZC_E_INVALID_ARG;
+    return zc_decompress_chunks(p, d_comp, comp_bytes, 0, p->n_chunks, d_out, d_workspace, cuda_stream);
+}
+
+zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t comp_bytes, uint32_t first_chunk, uint32_t n_chunks,
+                               void* d_out, void* d_workspace, void* cuda_stream)
+{
     if (!p || !d_comp || !d_workspace || (!d_out && p->n_elems)) return ZC_E_INVALID_ARG;
-    if (!aligned16(d_comp) || !aligned16(d_base) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
+    if ((uint64_t)first_chunk + n_chunks > p->n_chunks) return ZC_E_INVALID_ARG;
+    if (!aligned16(d_comp) || !aligned16(d_out) || !aligned16(d_workspace)) return ZC_E_INVALID_ARG;
     if (comp_bytes < kHeaderBytes) return ZC_E_CORRUPT;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     DecShape shape;
@@ -802,7 +811,9 @@ zc_status zc_decompress_xor(const zc_plan_t* p, const void* d_comp, size_t comp_
     DecParams P{};
     P.comp = (const uint8_t*)d_comp;
     P.base = nullptr;
-    P.out = (uint8_t*)d_out;
+    // the kernel addresses the output by position in the tensor: d_out is where chunk first_chunk goes
+    P.out = (uint8_t*)d_out - (size_t)first_chunk * p->chunk_bytes;
+    P.c_begin = first_chunk; P.c_end = first_chunk + n_chunks;
     P.ctl = (Control*)d_workspace;
     P.comp_bytes = comp_bytes; P.input_bytes = p->input_bytes; P.n_syms = p->n_syms; P.n_elems = p->n_elems;
     P.n_chunks = p->n_chunks; P.cs = p->syms_per_chunk; P.sub = p->syms_per_sub; P.chunk_bytes = p->chunk_bytes;
@@ -812,8 +823,8 @@ zc_status zc_decompress_xor(const zc_plan_t* p, const void* d_comp, size_t comp_
     P.pool_bytes = shape.pool_bytes;
     const uint32_t warps = shape.warps, ppl = shape.ppl;
     const size_t smem = shape.smem;
-    // at least one block even for an empty tensor: the header is still checked
-    const uint32_t want = std::max<uint32_t>((p->n_chunks + warps - 1) / warps, 1);
+    // at least one block even for an empty range: the header is still checked
+    const uint32_t want = std::max<uint32_t>((n_chunks + warps - 1) / warps, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
     cudaError_t e = cudaSuccess;
     auto launch = [&](auto kern) {

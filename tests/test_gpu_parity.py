@@ -200,6 +200,34 @@ def test_decoder_accepts_oracle_containers_and_flags_damage():
         assert zc.device_status(p2, d_ws2) == zc.E_CORRUPT
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_random_access_decodes_chunk_ranges_like_the_oracle(fmt):
+    """Sec. 3.1: chunks decode independently.  Ranges of chunks (first, last, single, all, empty) against the
+    oracle's chunk-by-chunk decoder; bytes outside the range stay untouched."""
+    chunk_bytes = 2048
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    n = (37 * cs + cs // 2 + 5) * G
+    if fmt == zc.FMT_FP4_E2M1:
+        n -= n % 2
+    data = _weights(fmt, n, 321 + fmt)
+    for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL):
+        p, cb, hist, cont = _gpu_round_trip(fmt, data, n, chunk_bytes, policy)
+        d_c = torch.from_numpy(cont).to(DEV)
+        ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+        for first, count in [(0, 1), (0, p.n_chunks), (p.n_chunks - 1, 1), (5, 1), (7, 13), (30, p.n_chunks - 30), (9, 0)]:
+            want = np.concatenate([zo.decompress_chunk(cont, c, chunk_bytes) for c in range(first, first + count)] + [np.zeros(0, np.uint8)])
+            d_out = torch.full((want.size + 64,), 0xEE, dtype=torch.uint8, device=DEV)
+            zc.decompress_chunks(p, d_c, cont.size, first, count, d_out[32:], ws)
+            assert zc.device_status(p, ws) == zc.OK
+            got = d_out.cpu().numpy()
+            assert np.array_equal(got[32: 32 + want.size], want), (first, count)
+            assert (got[:32] == 0xEE).all() and (got[32 + want.size:] == 0xEE).all()
+        with pytest.raises(zc.ZcError) as e:
+            zc.decompress_chunks(p, d_c, cont.size, p.n_chunks - 1, 2, d_out, ws)
+        assert e.value.status == zc.E_INVALID_ARG
+
+
 def test_argument_checks():
     p = zc.plan(zc.FMT_BF16, 1000, 1024)
     d = torch.zeros(4096, dtype=torch.uint8, device=DEV)
