@@ -297,3 +297,49 @@ def test_xor_delta_batched_calls():
     for p, (a, b), back in zip(plans, pairs, backs):
         out = back.cpu().numpy()
         assert np.array_equal(out[: p.input_bytes], b[: p.input_bytes]) and (out[p.input_bytes:] == 0xEE).all()
+
+
+def test_batched_calls_at_bench_size_on_sampled_chunks():
+    """Tensors of the size class the benchmark times (a 14336 x 4096 and a 4096 x 4096 BF16 matrix and a 1024 x 4096
+    one, 4 KiB chunks, the batched calls): the oracle decodes sampled chunks one by one, properties that hold at
+    any size cover the rest."""
+    fmt, chunk_bytes = zc.FMT_BF16, 4096
+    shapes = [(14336, 4096), (4096, 4096), (1024, 4096)]
+    g = torch.Generator(device=DEV); g.manual_seed(99)
+    d_ins, plans = [], []
+    for r, c in shapes:
+        x = (torch.randn(r * c, generator=g, device=DEV) * 0.02).to(torch.bfloat16)
+        d_ins.append(x.view(torch.uint8))
+        plans.append(zc.plan(fmt, r * c, chunk_bytes))
+    n_t = len(plans)
+    d_hists = torch.zeros((n_t, 2, 256), dtype=torch.int64, device=DEV)
+    zc.histogram_batch(zc.HistogramBatch(plans, d_ins), d_hists)
+    hists = d_hists.cpu().numpy().astype(np.uint64)
+    for t in range(n_t):
+        assert int(hists[t, 0].sum()) == plans[t].n_syms and int(hists[t, 1].sum()) == plans[t].n_syms
+    cbs = zc.build_codebooks(plans, hists, zc.POLICY_AUTO)
+    d_outs = [torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=DEV) for p in plans]
+    enc = zc.CompressBatch(plans, d_ins, d_outs)
+    enc.set_codebooks(cbs)
+    ws = torch.empty(enc.workspace_bytes, dtype=torch.uint8, device=DEV)
+    sizes = zc.compress_batch(enc, ws)
+    rng = np.random.default_rng(0)
+    for t in range(n_t):
+        p = plans[t]
+        cont = d_outs[t][: sizes[t]].cpu().numpy()
+        assert zc.validate_container(p, cont) == zc.OK
+        hd = zo.parse_header(cont)
+        assert hd["total_bytes"] == sizes[t] and hd["n_chunks"] == p.n_chunks
+        for s in range(2):
+            mode, lens, _ = cbs[t].get(s)
+            want_bits = int((hists[t, s].astype(np.int64) * lens).sum()) if mode == zc.MODE_HUFF else 8 * p.n_syms
+            assert hd["streams"][s]["payload_bits"] == want_bits
+        data = d_ins[t].cpu().numpy()
+        for c in [0, 1, p.n_chunks - 1] + [int(v) for v in rng.integers(0, p.n_chunks, 10)]:
+            got = zo.decompress_chunk(cont, c, chunk_bytes)
+            assert np.array_equal(got, data[c * chunk_bytes: c * chunk_bytes + got.size]), (t, c)
+    d_backs = [torch.empty(p.input_bytes, dtype=torch.uint8, device=DEV) for p in plans]
+    zc.decompress_batch(zc.DecompressBatch(plans, d_outs, sizes, d_backs), ws)
+    assert zc.batch_status(ws) == (zc.OK, None)
+    for b, x in zip(d_backs, d_ins):
+        assert torch.equal(b, x)
