@@ -156,7 +156,7 @@ __device__ void write_header(const EncCommon& C, const EncItem& I, TensorCounter
 constexpr uint32_t kEncMaxWorkers = 8;       // worker warps per block = chunks per batch; one more warp hands out
                                              // the batches and places them
 constexpr uint32_t kRing = 8;                // batches of a block whose bookkeeping is alive at the same time
-constexpr uint32_t kTabSlots = 4;            // code tables (one per batch) alive at the same time
+constexpr uint32_t kTabSlots = 4;            // code tables (of the tensors the last batches belong to) alive at the same time
 constexpr uint32_t kNoTensor = 0xFFFFFFFFu;  // "no more batches"
 constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
 
@@ -193,9 +193,9 @@ struct PackedChunk {
 //   s_tot[i & 7][w], s_cnt[i & 7]                  size of worker w's chunk; cnt = workers that posted it
 //   s_off[i & 7][w], s_off_seq                     position of that chunk; seq = batches placed so far
 // A worker has copied out batch i - n_slots (n_slots <= 3) before it packs batch i; a batch is placed only
-// after every worker has posted its size, and a batch is handed out only while fewer than 4 handed-out
-// batches are unplaced.  So all warps of a block are within 4 batches of each other and rings of 8 are
-// enough.  A table slot is reused only when every worker has posted the last batch that used it.
+// after every worker has posted its size, so worker 0 never hands out a batch more than 3 ahead of the last
+// placed one, and the service warp hands one out only while fewer than 4 are unplaced.  So all warps of a
+// block are within 4 batches of each other and rings of 8 are enough.  A table slot is reused only when every worker has posted the last batch that used it.
 // H0 / H1: stream 0 / 1 is Huffman-coded (the same for every tensor of a launch; a template parameter so that
 // the code of a raw stream's packing and copy-out does not exist and the kernel stays small).
 template <int FMT, int N_ITEMS, bool H0, bool H1>
