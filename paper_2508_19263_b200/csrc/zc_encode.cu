@@ -107,7 +107,10 @@ __device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& 
     const uint32_t lo = __funnelshift_r(0, code, nb);           // the bits that do not fit: code << (32 - nb), 0 if nb == 0
     const uint32_t n = nb + len;
     const bool full = n >= 32;
-    sts32_if(full && waddr < limit, waddr, hi);
+    // store if (n > 31 && waddr < limit): both compares and the store in one piece, so that the predicate never
+    // travels through a register
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.gt.u32 p, %2, 31;\n\tsetp.lt.and.u32 q, %0, %3, p;\n\t@q st.shared.u32 [%0], %1;\n\t}"
+                 :: "r"(waddr), "r"(hi), "r"(n), "r"(limit) : "memory");
     waddr += full ? 4 : 0;
     hi = full ? lo : hi;
     nb = n & 31;
@@ -394,7 +397,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             if (vol32(&s_fail)) break;
             if (did) { idle = 0; continue; }
             if (++idle > kSpinLimit) { s_fail = 1; break; }
-            if (lb_on) __nanosleep(50); else __nanosleep(300);      // a look-back in progress polls faster
+            __nanosleep(1000);                                   // nothing to do right now: leave the issue slots to the workers
         }
     } else {
         // =========================== a worker warp ===========================
@@ -626,16 +629,18 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 const uint32_t full_words = n_my / 4;
                 for (uint32_t i = 0; i < full_words; ++i) {
                     const uint32_t four = lds32(src + 4 * i);
-                    const uint32_t e0 = lds32(tab_s + ((four << 2) & 0x3FC));
-                    const uint32_t e1 = lds32(tab_s + ((four >> 6) & 0x3FC));
-                    const uint32_t e2 = lds32(tab_s + ((four >> 14) & 0x3FC));
-                    const uint32_t e3 = lds32(tab_s + ((four >> 22) & 0x3FC));
+                    // table index = one byte of the word (byte permute), scaled by 4 in the address add
+                    const uint32_t e0 = lds32(tab_s + 4u * __byte_perm(four, 0, 0x4440));
+                    const uint32_t e1 = lds32(tab_s + 4u * __byte_perm(four, 0, 0x4441));
+                    const uint32_t e2 = lds32(tab_s + 4u * __byte_perm(four, 0, 0x4442));
+                    const uint32_t e3 = lds32(tab_s + 4u * __byte_perm(four, 0, 0x4443));
                     seen |= e0 | e1 | e2 | e3;
-                    // two codes at a time: the second one shifted behind the first (shift count = low 5 bits of the
-                    // first entry = its length); the length fields end up below bit 8 and are masked off
-                    const uint32_t ca = (e0 | (e1 >> (e0 & 31))) & 0xFFFFFF00u;
+                    // two codes at a time: the second one shifted behind the first (the funnel shift takes its
+                    // count from the low 5 bits of the first entry = its length); the length fields end up below
+                    // bit 8 and are masked off
+                    const uint32_t ca = (e0 | __funnelshift_r(e1, 0, e0)) & 0xFFFFFF00u;
                     put_bits(ca, (e0 + e1) & 31, hi, nb, waddr, limit);
-                    const uint32_t cb = (e2 | (e3 >> (e2 & 31))) & 0xFFFFFF00u;
+                    const uint32_t cb = (e2 | __funnelshift_r(e3, 0, e2)) & 0xFFFFFF00u;
                     put_bits(cb, (e2 + e3) & 31, hi, nb, waddr, limit);
                 }
                 for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
