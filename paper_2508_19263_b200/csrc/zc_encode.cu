@@ -45,6 +45,8 @@ struct EncCommon {
     uint32_t sub_width;                          // bytes per sub_end entry (2 or 4)
     uint32_t n_slots;                            // pack slots per lane region (1..3, see encode_kernel)
     uint32_t sub_magic;                          // ceil(2^32 / sub): k / sub == umulhi(k, sub_magic) for k < 2^17
+    uint32_t stage_step;                         // staging offset between a lane's consecutive groups (256 symbols apart)
+                                                 // when that is a constant, i.e. sub divides 256; else 0
     uint32_t n_tensors, total_batches;
 };
 
@@ -553,7 +555,17 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             const uint32_t c_syms = active ? (uint32_t)min((uint64_t)C.cs, I.n_syms - c_lo) : 0u;
 
             // ---- phase A: coalesced load, split, raw stream stored as is, coded stream staged per subchunk ----
-            auto stage_group = [&](const uint4 x, const uint32_t k) {
+            // Group g (16 input bytes = symbols 8 g .. 8 g + 7) is staged at byte (8 g / sub) * region + 8 g % sub of
+            // the symbol area.  A lane's groups are 32 apart: when sub divides 256 that is a constant step.
+            uint8_t* const raw0 = I.out + I.lay.section_off[0] + c_lo;      // this chunk in the raw bodies
+            uint8_t* const raw1 = I.out + I.lay.section_off[1] + c_lo;
+            const uint32_t sym_s = smem_u32(stage) + sym_off;
+            const uint32_t step = C.stage_step;
+            auto stage_off = [&](const uint32_t g_) {
+                const uint32_t k = 8 * g_, j = __umulhi(k, C.sub_magic);
+                return j * region + (k - j * C.sub);
+            };
+            auto stage_group = [&](const uint4 x, const uint32_t g_, const uint32_t off) {
                 const uint32_t w[4] = {x.x, x.y, x.z, x.w};
                 uint32_t sy[2][2];
                 split16<FMT>(w, sy[0], sy[1]);
@@ -561,12 +573,10 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     if (!is_huff(s)) {
-                        st_cs_v2(I.out + I.lay.section_off[s] + c_lo + k, make_uint2(sy[s][0], sy[s][1]));
+                        st_cs_v2((s == 0 ? raw0 : raw1) + 8 * g_, make_uint2(sy[s][0], sy[s][1]));
                     } else {
-                        const uint32_t j = __umulhi(k, C.sub_magic);          // subchunk of these 8 symbols
-                        uint32_t* st = reinterpret_cast<uint32_t*>(stage + hs * C.stage_stride + j * region + sym_off + (k - j * C.sub));
-                        st[0] = sy[s][0];
-                        st[1] = sy[s][1];
+                        sts32(sym_s + hs * C.stage_stride + off, sy[s][0]);
+                        sts32(sym_s + hs * C.stage_stride + off + 4, sy[s][1]);
                         ++hs;
                     }
                 }
@@ -574,37 +584,40 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             const uint32_t n_vec = (c_syms + 7) / 8;
             const uint8_t* src_c = I.in + 2 * c_lo;
             uint32_t g = lane;
+            uint32_t off = stage_off(lane);                             // running offset (constant-step case)
+            auto off_at = [&](const uint32_t g_, const uint32_t i) { return step ? off + i * step : stage_off(g_); };
             if (I.base) {
                 // delta form: the chunk of the base tensor is read alongside and XOR-ed in (two pairs of loads in flight)
                 const uint8_t* base_c = I.base + 2 * c_lo;
                 auto x4 = [](const uint4 a, const uint4 b) { return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w); };
                 if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {
-                    for (; g + 32 < n_vec; g += 64) {
+                    for (; g + 32 < n_vec; g += 64, off += 2 * step) {
                         const uint4 x0 = ld_nc_v4(src_c + 16 * g), y0 = ld_nc_v4(base_c + 16 * g);
                         const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32)), y1 = ld_nc_v4(base_c + 16 * (g + 32));
-                        stage_group(x4(x0, y0), 8 * g);
-                        stage_group(x4(x1, y1), 8 * (g + 32));
+                        stage_group(x4(x0, y0), g, off_at(g, 0));
+                        stage_group(x4(x1, y1), g + 32, off_at(g + 32, 1));
                     }
-                    for (; g < n_vec; g += 32) stage_group(x4(ld_nc_v4(src_c + 16 * g), ld_nc_v4(base_c + 16 * g)), 8 * g);
+                    for (; g < n_vec; g += 32, off += step)
+                        stage_group(x4(ld_nc_v4(src_c + 16 * g), ld_nc_v4(base_c + 16 * g)), g, off_at(g, 0));
                 } else {
                     for (; g < n_vec; g += 32)
                         stage_group(x4(load16_guarded(I.in, 2 * (c_lo + 8ull * g), I.input_bytes),
-                                       load16_guarded(I.base, 2 * (c_lo + 8ull * g), I.input_bytes)), 8 * g);
+                                       load16_guarded(I.base, 2 * (c_lo + 8ull * g), I.input_bytes)), g, stage_off(g));
                 }
             } else if (2 * (c_lo + 8ull * n_vec) <= I.input_bytes) {    // every group of this chunk is complete
-                for (; g + 96 < n_vec; g += 128) {                          // four loads in flight per lane
+                for (; g + 96 < n_vec; g += 128, off += 4 * step) {         // four loads in flight per lane
                     const uint4 x0 = ld_nc_v4(src_c + 16 * g);
                     const uint4 x1 = ld_nc_v4(src_c + 16 * (g + 32));
                     const uint4 x2 = ld_nc_v4(src_c + 16 * (g + 64));
                     const uint4 x3 = ld_nc_v4(src_c + 16 * (g + 96));
-                    stage_group(x0, 8 * g);
-                    stage_group(x1, 8 * (g + 32));
-                    stage_group(x2, 8 * (g + 64));
-                    stage_group(x3, 8 * (g + 96));
+                    stage_group(x0, g, off_at(g, 0));
+                    stage_group(x1, g + 32, off_at(g + 32, 1));
+                    stage_group(x2, g + 64, off_at(g + 64, 2));
+                    stage_group(x3, g + 96, off_at(g + 96, 3));
                 }
-                for (; g < n_vec; g += 32) stage_group(ld_nc_v4(src_c + 16 * g), 8 * g);
+                for (; g < n_vec; g += 32, off += step) stage_group(ld_nc_v4(src_c + 16 * g), g, off_at(g, 0));
             } else {
-                for (; g < n_vec; g += 32) stage_group(load16_guarded(I.in, 2 * (c_lo + 8ull * g), I.input_bytes), 8 * g);
+                for (; g < n_vec; g += 32) stage_group(load16_guarded(I.in, 2 * (c_lo + 8ull * g), I.input_bytes), g, stage_off(g));
             }
             __syncwarp();
 
@@ -805,6 +818,7 @@ void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const
     c.n_slots = sh.n_slots; c.slot_bytes = sh.slot_bytes; c.region_bytes = sh.region_bytes; c.stage_stride = sh.stage_stride;
     c.sub_width = sub_end_width(p->chunk_bytes);
     c.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
+    c.stage_step = 256 % p->syms_per_sub == 0 ? (256 / p->syms_per_sub) * sh.region_bytes : 0;
 }
 
 void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const void* d_in, const void* d_base, void* d_out,
