@@ -227,7 +227,7 @@ __device__ __forceinline__ void lane_refill(LaneStream& st)
 
 __device__ __forceinline__ uint32_t lane_peek(const LaneStream& st, uint32_t lut_s)
 {
-    return lds32(lut_s + ((st.hi >> (30 - kLmax)) & (4 * kLutEntries - 4)));
+    return lds32(lut_s + 4u * (st.hi >> (32 - kLmax)));         // window = top 12 bits; scaled by the address add
 }
 __device__ __forceinline__ void lane_consume(LaneStream& st, uint32_t n)    // n < 32 in its low 5 bits
 {
