@@ -69,9 +69,11 @@ def workload_specs(name: str):
         # the E8M0 block scales of the same stack as byte streams (config 4 stores them raw; coding them is
         # what the paper's FP4 result rests on, Sec. 3.4 / 4.4): 225 streams, 234.5 MB
         return wl.SCALE_U8, wl.llama8b_stack(4)
-    if name in ("cfg5_kv_bf16", "cfg5_kv_fp8"):
-        # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers)
-        fmt = wl.BF16 if name.endswith("bf16") else wl.FP8_E4M3
+    if name in ("cfg5_kv_bf16", "cfg5_kv_fp8", "next3_kv_bf16_static", "next3_kv_fp8_static"):
+        # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers).
+        # The *_static workloads code them the way Sec. 3.3 describes the run-time use: with dictionaries computed
+        # ahead of time (from layer 0's K and V), no histogram pass and no codebook build in the step
+        fmt = wl.BF16 if "bf16" in name else wl.FP8_E4M3
         return fmt, [wl.TensorSpec(f"kv.{l}.{'kv'[w]}", (8, 8, 32768, 128), 0.0, 10 * l + w) for l in range(4) for w in range(2)]
     if name in ("next2_bf16_delta", "small_bf16_delta"):
         # delta checkpoints (Sec. 3.1 / 4.1): the XOR of two consecutive BF16 checkpoints of the config-2 stack is
@@ -135,6 +137,13 @@ class ClockSampler:
 # the CPU oracle as baseline / reference arm
 # --------------------------------------------------------------------------------------------
 
+def oracle_static_codebook(fmt, sample):
+    """The dictionary of the *_static workloads for the oracle legs: from the first tensor of the sample."""
+    import oracle as zo
+    name, data, n = sample[0]
+    return zo.build_codebook(zo.histogram(fmt, data, n), zo.POLICY_STATIC)
+
+
 def oracle_sample(fmt, specs, device, delta=False):
     """The first tensors of the workload up to ORACLE_SAMPLE_BYTES, as host arrays (delta workloads: the XOR of
     the two checkpoints, which is what the oracle codes)."""
@@ -156,15 +165,19 @@ def oracle_sample(fmt, specs, device, delta=False):
     return out, total
 
 
-def oracle_step(fmt, sample, chunk_bytes):
-    """Whole path on the CPU oracle (single thread): histogram, codebook, compress, decompress."""
+def oracle_step(fmt, sample, chunk_bytes, static_cb=None):
+    """Whole path on the CPU oracle (single thread): histogram, codebook, compress, decompress; with a static
+    dictionary (Sec. 3.3) the first two fall away."""
     import oracle as zo
     t_h = t_e = t_d = 0.0
     cbytes = 0
     for name, data, n in sample:
         t0 = time.perf_counter()
-        h = zo.histogram(fmt, data, n)
-        cb = zo.build_codebook(h, zo.POLICY_AUTO)
+        if static_cb is None:
+            h = zo.histogram(fmt, data, n)
+            cb = zo.build_codebook(h, zo.POLICY_AUTO)
+        else:
+            cb = static_cb
         t1 = time.perf_counter()
         c = zo.compress(fmt, data, n, chunk_bytes, cb)
         t2 = time.perf_counter()
@@ -184,12 +197,13 @@ def run_reference(args):
     fmt, specs = workload_specs(args.workload)
     sample, total = oracle_sample(fmt, specs, "cpu", args.workload.endswith("_delta"))
     chunk_bytes = args.chunk_kib * 1024
+    static_cb = oracle_static_codebook(fmt, sample) if args.workload.endswith("_static") else None
     for _ in range(min(args.warmup, 1)):
-        oracle_step(fmt, sample[:1], chunk_bytes)
+        oracle_step(fmt, sample[:1], chunk_bytes, static_cb)
     times = []
     for _ in range(args.steps):
         t0 = time.perf_counter()
-        t_h, t_e, t_d, cbytes = oracle_step(fmt, sample, chunk_bytes)
+        t_h, t_e, t_d, cbytes = oracle_step(fmt, sample, chunk_bytes, static_cb)
         times.append(time.perf_counter() - t0)
     dt = float(np.mean(times))
     value = total / dt / 1e9
@@ -197,7 +211,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": args.workload, "chunk_kib": args.chunk_kib, "policy": "auto",
+        "config": {"workload": args.workload, "chunk_kib": args.chunk_kib, "policy": "static" if static_cb else "auto",
                    "sample": f"first {len(sample)} tensors, {total} bytes"},
         "decode": {"value": total / t_d / 1e9, "unit": UNIT}, "encode": {"value": total / t_e / 1e9, "unit": UNIT},
         "compression_ratio": cbytes / total,
@@ -265,6 +279,9 @@ def run_ours(args):
     # ---- resident inputs, plans, output buffers ----
     tensors = []
     delta = args.workload.endswith("_delta")
+    static = args.workload.endswith("_static")
+    if static and not args.batch:
+        raise SystemExit("the *_static workloads use the batched calls")
     for spec in specs:
         base_t = None
         if delta:
@@ -310,8 +327,16 @@ def run_ours(args):
         h_hist.copy_(d_hist, non_blocking=True)
         stream.synchronize()
 
+    STATIC_TOLERANCE = 0.05
+    dicts = []                                   # *_static: [dictionary of the K tensors, dictionary of the V tensors]
+
     def phase_codebooks():
         hh = h_hist.numpy()
+        if static and dicts:
+            for i, t in enumerate(tensors):
+                t["cb"] = dicts[i % 2].codebook
+            enc_batch.set_codebooks([t["cb"] for t in tensors])
+            return
         if args.batch:
             cbs = zc.build_codebooks([t["plan"] for t in tensors], hh, zc.POLICY_AUTO)
             for t, cb in zip(tensors, cbs):
@@ -367,7 +392,7 @@ def run_ours(args):
 
     # the step compresses in a few groups: the host builds the codebooks of the next group while the GPU encodes
     step_groups = []
-    if args.batch:
+    if args.batch and not static:
         for idx in split_groups(max(1, min(4, n_t // 8))):
             sel = [tensors[i] for i in idx]
             eb = zc.CompressBatch([t["plan"] for t in sel], [t["in"] for t in sel], [t["comp"] for t in sel],
@@ -377,6 +402,15 @@ def run_ours(args):
     def step():
         # histogram of every tensor, then codebook / compress / decompress per tensor: the host builds the
         # next codebook while the GPU is busy with the previous tensors
+        if static:
+            # run-time use (Sec. 3.3): no histogram, no codebook build; the sizes come back with the call and tell
+            # the dictionaries whether they still fit
+            sizes = zc.compress_batch(enc_batch, enc_ws, sync=True, stream=stream)
+            for i, t in enumerate(tensors):
+                if dicts[i % 2].observe(t["plan"].input_bytes, sizes[i]):
+                    raise SystemExit(f"dictionary {i % 2} no longer fits tensor {t['name']}")
+            zc.decompress_batch(dec_batch, batch_ws, stream=stream)
+            return
         phase_hist()
         if args.batch:
             hh = h_hist.numpy()
@@ -407,6 +441,18 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         return max_over_ranks(e0.elapsed_time(e1), dist, dev) / reps
+
+    C_own = None
+    if static:
+        # for comparison: the container sizes with every tensor's own codebook
+        phase_hist()
+        phase_codebooks()
+        phase_compress()
+        read_sizes()
+        C_own = sum(t["cbytes"] for t in tensors)
+        hh = h_hist.numpy()
+        dicts.extend(zc.Dictionary(tensors[w]["plan"], hh[w], STATIC_TOLERANCE) for w in range(2))
+        phase_codebooks()
 
     # ---- correctness of what is timed (untimed): statuses, byte-identical round trip ----
     step()
@@ -483,11 +529,14 @@ def run_ours(args):
                 for g in gb:
                     lo, hi = g["idx"][0], g["idx"][-1] + 1
                     stream.wait_event(g["ev_in"])
-                    zc.histogram_batch(g["hist"], d_hist[lo:hi], stream=stream)
-                    h_hist[lo:hi].copy_(d_hist[lo:hi], non_blocking=True)
-                    stream.synchronize()                       # the host needs the counts for the codebooks
-                    cbs = zc.build_codebooks([tensors[i]["plan"] for i in g["idx"]], h_hist[lo:hi].numpy(), zc.POLICY_AUTO)
-                    g["enc"].set_codebooks(cbs)
+                    if static:
+                        g["enc"].set_codebooks([tensors[i]["cb"] for i in g["idx"]])
+                    else:
+                        zc.histogram_batch(g["hist"], d_hist[lo:hi], stream=stream)
+                        h_hist[lo:hi].copy_(d_hist[lo:hi], non_blocking=True)
+                        stream.synchronize()                   # the host needs the counts for the codebooks
+                        cbs = zc.build_codebooks([tensors[i]["plan"] for i in g["idx"]], h_hist[lo:hi].numpy(), zc.POLICY_AUTO)
+                        g["enc"].set_codebooks(cbs)
                     zc.compress_batch(g["enc"], g["enc_ws"], sync=False, stream=stream)
                     g["ev_enc"].record(stream)
                     with torch.cuda.stream(s_out):
@@ -570,10 +619,10 @@ def run_ours(args):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         sample, total = oracle_sample(fmt, specs, dev, delta)
-        t_h, t_e, t_d, cb_sample = oracle_step(fmt, sample, chunk_bytes)
+        t_h, t_e, t_d, cb_sample = oracle_step(fmt, sample, chunk_bytes, oracle_static_codebook(fmt, sample) if static else None)
         cpu = {"value": total / (t_h + t_e + t_d) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {len(sample)} tensors of {args.workload}, {total} bytes",
-               "decode_gbs": total / t_d / 1e9, "encode_gbs": total / t_e / 1e9, "histogram_codebook_gbs": total / t_h / 1e9}
+               "decode_gbs": total / t_d / 1e9, "encode_gbs": total / t_e / 1e9, "histogram_codebook_gbs": (total / t_h / 1e9 if not static else None)}
 
     # compression ratios next to the paper's (context): exponent stream, sign+mantissa stream, total
     st_bits = [0, 0]
@@ -586,14 +635,16 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.workload, "tensors": n_t, "uncompressed_bytes": U, "compressed_bytes": C,
-                   "chunk_kib": args.chunk_kib, "policy": "auto", "batched_calls": bool(args.batch), "streams": args.streams if not args.batch else 1,
+                   "chunk_kib": args.chunk_kib,
+                   "policy": f"static dictionaries from layer 0's K and V, tolerance {STATIC_TOLERANCE}" if static else "auto",
+                   "batched_calls": bool(args.batch), "streams": args.streams if not args.batch else 1,
                    "l2": "inputs larger than L2 (no flush)"},
         "decode": dec, "encode": enc, "histogram": hist, "codebook_host_ms": ms_codebook,
-        "compression_ratio": {"total_container": C / U, "exponent_stream_payload": st_bits[0] / (8 * n_syms),
+        "compression_ratio": {"total_container": C / U, "total_container_own_codebooks": (C_own / U if C_own else None), "exponent_stream_payload": st_bits[0] / (8 * n_syms),
                               "sign_mantissa_stream_payload": st_bits[1] / (8 * n_syms),
                               "paper_context": "abstract: up to 62% (BF16) / 83% (FP8) total"},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": (n_hist_launch + n_enc_launch_step + n_dec_launch) * args.steps,
+        "gpu_launches": ((n_enc_launch if static else n_hist_launch + n_enc_launch_step) + n_dec_launch) * args.steps,
     }
     print(json.dumps(line))
     if dist is not None:

@@ -93,13 +93,29 @@ typedef enum zc_format {
 typedef enum zc_policy {
     ZC_POLICY_AUTO = 0,         /* Huffman only for a stream that saves at least 1/64 (Sec. 3.1 rule) */
     ZC_POLICY_HUFF_ALL = 1,     /* Huffman for every non-empty stream */
-    ZC_POLICY_RAW_ALL = 2       /* both streams stored raw (split / merge only) */
+    ZC_POLICY_RAW_ALL = 2,      /* both streams stored raw (split / merge only) */
+    ZC_POLICY_STATIC = 3        /* a dictionary meant for OTHER tensors than the one it was counted on
+                                   (Sec. 3.3, precomputed dictionaries): every one of the 256 symbols gets
+                                   a code, so no later tensor can hit a missing code; the RAW / HUFF
+                                   decision is the AUTO rule on the histogram given */
 } zc_policy;
 
 typedef enum zc_mode { ZC_MODE_RAW = 0, ZC_MODE_HUFF = 1 } zc_mode;
 
 typedef struct zc_plan_s zc_plan_t;
 typedef struct zc_codebook_s zc_codebook_t;
+typedef struct zc_dict_s zc_dict_t;
+
+typedef struct zc_dict_info {
+    double tolerance;           /* as given to zc_dict_create */
+    double baseline_ratio;      /* container bytes / input bytes of the first tensor coded since the last
+                                   (re)build; 0 while there is none */
+    double last_ratio;          /* of the latest observation; 0 before the first */
+    uint64_t n_observed;        /* calls of zc_dict_observe */
+    uint64_t n_rebuilds;        /* calls of zc_dict_rebuild */
+    uint32_t has_baseline;
+    uint32_t reserved;
+} zc_dict_info;
 
 typedef struct zc_plan_info {
     uint32_t format, group, chunk_bytes, n_chunks;
@@ -355,6 +371,35 @@ zc_status zc_validate_container(const zc_plan_t* plan, const void* h_container, 
  * 128 container bytes) is optional and adds the container-inclusive figures. */
 zc_status zc_stats(const zc_plan_t* plan, const zc_codebook_t* cb, const uint64_t* h_hist,
                    const void* h_header, zc_stats_t* out);
+
+/* ---- runtime dictionaries for K/V cache tensors (Sec. 3.3: dictionaries are computed ahead of
+ *      time while the exponent distribution stays stable, and replaced only when the achieved
+ *      ratio gets worse; Sec. 5.2 reports the savings of such static dictionaries) -------------
+ * A zc_dict_t owns one ZC_POLICY_STATIC codebook and the bookkeeping that decides when to replace
+ * it.  The paper gives no threshold; here the caller does: `tolerance` is the relative growth of
+ * the container ratio (container bytes / input bytes) over the baseline that is still accepted.
+ * The baseline is the ratio of the first tensor observed after the dictionary was (re)built.
+ * Host-only objects; one dictionary per kind of tensor (say, per layer and K or V), used from
+ * one thread at a time.
+ *
+ * zc_dict_create   codebook from the histogram of a representative tensor (h_hist as for
+ *                  zc_build_codebook); tolerance >= 0.  Errors: INVALID_ARG, NOMEM.
+ * zc_dict_codebook the current codebook, for zc_compress / zc_compress_batch on tensors of the
+ *                  same format; owned by the dictionary, valid until zc_dict_rebuild / destroy.
+ * zc_dict_observe  report one coded tensor: input_bytes > 0 and the container size the compress
+ *                  call returned.  *rebuild is set to 1 when container_bytes / input_bytes exceeds
+ *                  baseline * (1 + tolerance), else 0; the first observation after a (re)build
+ *                  becomes the baseline and never asks for a rebuild.  Errors: INVALID_ARG.
+ * zc_dict_rebuild  replace the codebook by one built from h_hist (the histogram of the tensor
+ *                  that was coded badly); the baseline is taken anew from the next observation.
+ *                  The caller compresses that tensor again if it wants the better ratio now.
+ * zc_dict_get_info the bookkeeping above. */
+zc_status zc_dict_create(const zc_plan_t* plan, const uint64_t* h_hist, double tolerance, zc_dict_t** out);
+void zc_dict_destroy(zc_dict_t* dict);
+const zc_codebook_t* zc_dict_codebook(const zc_dict_t* dict);
+zc_status zc_dict_observe(zc_dict_t* dict, uint64_t input_bytes, uint64_t container_bytes, int* rebuild);
+zc_status zc_dict_rebuild(zc_dict_t* dict, const zc_plan_t* plan, const uint64_t* h_hist);
+zc_status zc_dict_get_info(const zc_dict_t* dict, zc_dict_info* out);
 
 const char* zc_strerror(zc_status s);
 

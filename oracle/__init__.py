@@ -18,7 +18,7 @@ import numpy as np
 
 BF16, FP8_E4M3, FP4_E2M1, SCALE_U8 = 1, 2, 3, 4
 RAW, HUFF = 0, 1
-POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL = 0, 1, 2
+POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL, POLICY_STATIC = 0, 1, 2, 3
 L_MAX = 12
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -64,6 +64,10 @@ def lib():
         L.zo_histogram.argtypes = [u8p, C.c_uint64, u64p]
         L.zo_code_lengths.restype = C.c_int
         L.zo_code_lengths.argtypes = [u64p, C.c_int, u8p]
+        L.zo_static_lengths.restype = C.c_int
+        L.zo_static_lengths.argtypes = [u64p, C.c_int, u8p]
+        L.zo_dict_wants_rebuild.restype = C.c_int
+        L.zo_dict_wants_rebuild.argtypes = [C.c_double, C.c_double, C.c_double]
         L.zo_canonical_codes.restype = None
         L.zo_canonical_codes.argtypes = [u8p, u32p]
         L.zo_payload_bits.restype = C.c_uint64
@@ -167,6 +171,17 @@ def code_lengths(hist, L: int = L_MAX) -> np.ndarray:
     return out
 
 
+def static_lengths(hist, L: int = L_MAX) -> np.ndarray:
+    """Code lengths of a static dictionary (Sec. 3.3): every symbol gets a code."""
+    h = np.ascontiguousarray(hist, np.uint64)
+    assert h.shape == (256,)
+    out = np.zeros(256, np.uint8)
+    rc = lib().zo_static_lengths(_p(h, C.c_uint64), L, _p(out, C.c_uint8))
+    if rc:
+        raise ValueError(f"zo_static_lengths failed: {rc}")
+    return out
+
+
 def canonical_codes(lengths) -> np.ndarray:
     l = np.ascontiguousarray(lengths, np.uint8)
     out = np.zeros(256, np.uint32)
@@ -195,10 +210,34 @@ class Codebook:
 
 def build_codebook(hist2, policy: int = POLICY_AUTO) -> Codebook:
     hist2 = np.ascontiguousarray(hist2, np.uint64).reshape(2, 256)
-    lens = np.stack([code_lengths(hist2[s]) for s in range(2)])
+    lens = np.stack([(static_lengths if policy == POLICY_STATIC else code_lengths)(hist2[s]) for s in range(2)])
     codes = np.stack([canonical_codes(lens[s]) for s in range(2)])
     modes = [choose_mode(hist2[s], lens[s], policy) for s in range(2)]
     return Codebook(modes, lens, codes)
+
+
+class StaticDictionary:
+    """A precomputed dictionary for K/V cache tensors and the rule that replaces it (Sec. 3.3): built from the
+    histogram of a representative tensor, reused for the tensors that follow, replaced when a tensor's ratio
+    (container bytes / input bytes) exceeds the baseline by more than `tolerance` (relative)."""
+
+    def __init__(self, hist2, tolerance: float):
+        self.tolerance = float(tolerance)
+        self.codebook = build_codebook(hist2, POLICY_STATIC)
+        self.baseline = None
+        self.n_rebuilds = 0
+
+    def observe(self, input_bytes: int, container_bytes: int) -> bool:
+        ratio = container_bytes / input_bytes
+        if self.baseline is None:
+            self.baseline = ratio
+            return False
+        return bool(lib().zo_dict_wants_rebuild(self.baseline, ratio, self.tolerance))
+
+    def rebuild(self, hist2) -> None:
+        self.codebook = build_codebook(hist2, POLICY_STATIC)
+        self.baseline = None
+        self.n_rebuilds += 1
 
 
 # ---- container -------------------------------------------------------------------------------

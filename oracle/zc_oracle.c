@@ -25,6 +25,9 @@
  *   - The scaling factors of FP4 blocks are Huffman-coded as a stream of bytes
  *     (Sec. 3.4, last two paragraphs; Sec. 4.4): format ZO_SCALE_U8 of zo_split /
  *     zo_merge (reading R11).
+ *   - Dictionaries for K/V cache tensors are computed ahead of time and replaced
+ *     only when the achieved ratio gets worse (Sec. 3.3, last paragraph but one;
+ *     Sec. 5.2): zo_static_lengths, zo_dict_wants_rebuild (reading R12).
  *   - Chunks of one fixed size, each with a little metadata, so that chunks
  *     can be located and decoded independently (Sec. 3.1, Sec. 4): zo_compress,
  *     zo_decompress, zo_decompress_chunk.
@@ -62,6 +65,14 @@
  *       symbols of stream 0, the bytes at even offsets those of stream 1, so
  *       symbol k of both streams comes from bytes 2k and 2k+1 (a missing last
  *       odd byte counts as zero).  Each half has its own code.
+ *   R12 A static dictionary has to code tensors it was not counted on, so its
+ *       lengths come from the counts 256*count + 1 (every symbol counts as
+ *       1/256 of an occurrence more and therefore gets a code); RAW/HUFF is
+ *       decided by R6 on the counts themselves.  "The ratio drops" is read as:
+ *       container bytes / input bytes of a tensor exceeds baseline*(1+tolerance),
+ *       where the baseline is that quotient for the first tensor coded after the
+ *       dictionary was built and the tolerance is the caller's (the paper gives
+ *       no number).
  *
  * Container layout (little-endian, every section 16-byte aligned):
  *   header 128 B:
@@ -91,7 +102,7 @@
 
 enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3, ZO_SCALE_U8 = 4 };
 enum { ZO_RAW = 0, ZO_HUFF = 1 };
-enum { ZO_POLICY_AUTO = 0, ZO_POLICY_HUFF_ALL = 1, ZO_POLICY_RAW_ALL = 2 };
+enum { ZO_POLICY_AUTO = 0, ZO_POLICY_HUFF_ALL = 1, ZO_POLICY_RAW_ALL = 2, ZO_POLICY_STATIC = 3 };
 enum { ZO_LMAX = 12, ZO_SUBS = 32, ZO_HEADER = 128 };
 
 /* ------------------------------------------------------------------ */
@@ -353,6 +364,22 @@ uint64_t zo_payload_bits(const uint64_t hist[256], const uint8_t len[256])
     return t;
 }
 
+/* Code lengths of a static dictionary (reading R12; Sec. 3.3): the plain
+ * construction on counts raised so that no symbol is left without a code. */
+int zo_static_lengths(const uint64_t hist[256], int L, uint8_t len[256])
+{
+    uint64_t raised[256];
+    for (int v = 0; v < 256; ++v) raised[v] = 256 * hist[v] + 1;
+    return zo_code_lengths(raised, L, len);
+}
+
+/* Whether a dictionary is to be replaced after a tensor was coded at `ratio`
+ * (container bytes / input bytes) (reading R12; Sec. 3.3). */
+int zo_dict_wants_rebuild(double baseline, double ratio, double tolerance)
+{
+    return ratio > baseline * (1.0 + tolerance);
+}
+
 /* RAW/HUFF decision of one stream (reading R6; Sec. 3.1: a stream is coded
  * only when that pays, and stored uncompressed otherwise). */
 int zo_choose_mode(const uint64_t hist[256], const uint8_t len[256], int policy)
@@ -362,6 +389,7 @@ int zo_choose_mode(const uint64_t hist[256], const uint8_t len[256], int policy)
     if (n == 0) return ZO_RAW;
     if (policy == ZO_POLICY_RAW_ALL) return ZO_RAW;
     if (policy == ZO_POLICY_HUFF_ALL) return ZO_HUFF;
+    /* ZO_POLICY_AUTO and ZO_POLICY_STATIC */
     return (64 * zo_payload_bits(hist, len) <= 63 * 8 * n) ? ZO_HUFF : ZO_RAW;
 }
 

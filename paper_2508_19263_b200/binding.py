@@ -19,7 +19,7 @@ import torch
 from . import build as _build
 
 FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1, FMT_SCALE_U8 = 1, 2, 3, 4
-POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL = 0, 1, 2
+POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL, POLICY_STATIC = 0, 1, 2, 3
 MODE_RAW, MODE_HUFF = 0, 1
 (OK, E_INVALID_ARG, E_UNSUPPORTED, E_BUFFER_TOO_SMALL, E_CORRUPT, E_CUDA, E_NOMEM, E_DEVICE_TIMEOUT, E_NO_CODE,
  E_TOO_LARGE) = range(10)
@@ -48,6 +48,11 @@ class StreamStats(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("stream", StreamStats * 2), ("in_bytes", C.c_uint64), ("out_bytes", C.c_uint64),
                 ("ratio_payload", C.c_double), ("ratio_container", C.c_double)]
+
+
+class DictInfo(C.Structure):
+    _fields_ = [("tolerance", C.c_double), ("baseline_ratio", C.c_double), ("last_ratio", C.c_double),
+                ("n_observed", C.c_uint64), ("n_rebuilds", C.c_uint64), ("has_baseline", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 def _load():
@@ -116,6 +121,18 @@ def _load():
     L.zc_validate_container.argtypes = [vp, vp, C.c_size_t]
     L.zc_stats.restype = C.c_int
     L.zc_stats.argtypes = [vp, vp, u64p, vp, C.POINTER(Stats)]
+    L.zc_dict_create.restype = C.c_int
+    L.zc_dict_create.argtypes = [vp, u64p, C.c_double, C.POINTER(vp)]
+    L.zc_dict_destroy.restype = None
+    L.zc_dict_destroy.argtypes = [vp]
+    L.zc_dict_codebook.restype = vp
+    L.zc_dict_codebook.argtypes = [vp]
+    L.zc_dict_observe.restype = C.c_int
+    L.zc_dict_observe.argtypes = [vp, C.c_uint64, C.c_uint64, C.POINTER(C.c_int)]
+    L.zc_dict_rebuild.restype = C.c_int
+    L.zc_dict_rebuild.argtypes = [vp, vp, u64p]
+    L.zc_dict_get_info.restype = C.c_int
+    L.zc_dict_get_info.argtypes = [vp, C.POINTER(DictInfo)]
     L.zc_strerror.restype = C.c_char_p
     L.zc_strerror.argtypes = [C.c_int]
     L.zc_test_split16.restype = C.c_int
@@ -172,8 +189,9 @@ def plan(fmt: int, n_elems: int, chunk_bytes: int) -> Plan:
 class Codebook:
     """zc_build_codebook result: per stream a mode, 256 code lengths and 256 canonical code values."""
 
-    def __init__(self, handle):
+    def __init__(self, handle, owned: bool = True):
         self._h = handle
+        self._owned = owned                      # a dictionary's codebook belongs to the dictionary
 
     def get(self, stream_idx: int):
         mode = C.c_uint32()
@@ -189,7 +207,7 @@ class Codebook:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h and _lib is not None:
+        if h and _lib is not None and getattr(self, "_owned", True):
             _lib.zc_codebook_destroy(h)
             self._h = None
 
@@ -248,6 +266,51 @@ def build_codebook(p: Plan, h_hist, policy: int = POLICY_AUTO) -> Codebook:
     _check(_lib.zc_build_codebook(p._h, C.cast(h.ctypes.data, C.POINTER(C.c_uint64)), policy, C.byref(out)),
            "zc_build_codebook")
     return Codebook(out)
+
+
+def _hist_ptr(h_hist):
+    h = np.asarray(h_hist)
+    if h.dtype == np.int64 and h.flags.c_contiguous:
+        h = h.view(np.uint64)
+    elif h.dtype != np.uint64 or not h.flags.c_contiguous:
+        h = np.ascontiguousarray(h.astype(np.uint64))
+    assert h.size == 512
+    return h, C.cast(h.ctypes.data, C.POINTER(C.c_uint64))
+
+
+class Dictionary:
+    """zc_dict_*: a static codebook for K/V cache tensors plus the rule that says when to replace it."""
+
+    def __init__(self, p: Plan, h_hist, tolerance: float):
+        _keep, ptr = _hist_ptr(h_hist)
+        self._h = C.c_void_p()
+        _check(_lib.zc_dict_create(p._h, ptr, tolerance, C.byref(self._h)), "zc_dict_create")
+
+    @property
+    def codebook(self) -> Codebook:
+        """The current codebook (not owned: valid until rebuild())."""
+        return Codebook(C.c_void_p(_lib.zc_dict_codebook(self._h)), owned=False)
+
+    def observe(self, input_bytes: int, container_bytes: int) -> bool:
+        flag = C.c_int(0)
+        _check(_lib.zc_dict_observe(self._h, input_bytes, container_bytes, C.byref(flag)), "zc_dict_observe")
+        return bool(flag.value)
+
+    def rebuild(self, p: Plan, h_hist) -> None:
+        _keep, ptr = _hist_ptr(h_hist)
+        _check(_lib.zc_dict_rebuild(self._h, p._h, ptr), "zc_dict_rebuild")
+
+    @property
+    def info(self) -> DictInfo:
+        out = DictInfo()
+        _check(_lib.zc_dict_get_info(self._h, C.byref(out)), "zc_dict_get_info")
+        return out
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h and _lib is not None:
+            _lib.zc_dict_destroy(h)
+            self._h = None
 
 
 def build_codebooks(plans, h_hists, policy: int = POLICY_AUTO, n_threads: int = 0):

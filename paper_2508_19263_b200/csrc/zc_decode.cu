@@ -94,7 +94,8 @@ __device__ __forceinline__ CodeBook codebook_views(uint32_t* scratch)
 // Two-symbol mode: a lookup normally yields the two symbols whose codes start the 12-bit window; when the two
 // codes together are longer than 12 bits the entry carries the first one and bit 31, and the decoder fetches
 // the second with one more lookup.  That mode is chosen when such pairs are rare (estimated from the code
-// lengths with p(symbol) = 2^-length); otherwise every lookup yields exactly one symbol.  A fixed number of
+// lengths with p(symbol) = 2^-length, an eighth of that for the two longest lengths); otherwise every lookup
+// yields exactly one symbol.  A fixed number of
 // symbols per lookup lets a lane assemble words of 4 symbols in registers without any bookkeeping.
 // `single` is a 4096 x u16 scratch table (length << 8 | symbol of the first code of every window).
 // Returns false to all threads if the lengths are not a complete prefix code (or the one-symbol code).
@@ -133,6 +134,9 @@ __device__ bool build_lut(uint32_t my_len, uint32_t* lut, uint16_t* single, uint
             off += cnt;
             active += cnt;
             p[l] = cnt << (kLmax - l);
+            // codes at or next to the length limit belong to symbols that are rarer than 2^-length says: the limit
+            // clipped them, or they are the never-seen symbols of a static dictionary
+            if (l + 1 >= kLmax) p[l] >>= 3;
         }
         const bool complete = b.limit[kLmax] == kLutEntries;      // Kraft sum is exactly one
         const bool one = active == 1 && b.count[1] == 1;

@@ -166,22 +166,33 @@ size_t zc_workspace_bytes(const zc_plan_t* p)
     return (size_t)round_up(kControlBytes + 8ull * p->n_chunks, 256);
 }
 
+static bool known_policy(zc_policy policy)
+{
+    return policy == ZC_POLICY_AUTO || policy == ZC_POLICY_HUFF_ALL || policy == ZC_POLICY_RAW_ALL || policy == ZC_POLICY_STATIC;
+}
+
 zc_status zc_build_codebook(const zc_plan_t* plan, const uint64_t* h_hist, zc_policy policy, zc_codebook_t** out)
 {
     if (!plan || !h_hist || !out) return ZC_E_INVALID_ARG;
-    if (policy != ZC_POLICY_AUTO && policy != ZC_POLICY_HUFF_ALL && policy != ZC_POLICY_RAW_ALL)
-        return ZC_E_UNSUPPORTED;
+    if (!known_policy(policy)) return ZC_E_UNSUPPORTED;
     zc_codebook_s* cb = new (std::nothrow) zc_codebook_s;
     if (!cb) return ZC_E_NOMEM;
     for (int s = 0; s < 2; ++s) {
         const uint64_t* h = h_hist + 256 * s;
-        if (!limited_lengths(h, kLmax, cb->len[s])) { delete cb; return ZC_E_INVALID_ARG; }
-        canonical(cb->len[s], cb->code[s]);
         uint64_t n = 0;
         for (int v = 0; v < 256; ++v) n += h[v];
+        // a static dictionary codes tensors it has not seen: every symbol counts as 1/256 of an occurrence more
+        uint64_t smoothed[256];
+        if (policy == ZC_POLICY_STATIC) {
+            if (n >> 54) { delete cb; return ZC_E_INVALID_ARG; }
+            for (int v = 0; v < 256; ++v) smoothed[v] = 256 * h[v] + 1;
+        }
+        if (!limited_lengths(policy == ZC_POLICY_STATIC ? smoothed : h, kLmax, cb->len[s])) { delete cb; return ZC_E_INVALID_ARG; }
+        canonical(cb->len[s], cb->code[s]);
         uint32_t mode = ZC_MODE_RAW;
         if (n != 0 && policy == ZC_POLICY_HUFF_ALL) mode = ZC_MODE_HUFF;
-        if (n != 0 && policy == ZC_POLICY_AUTO && 64 * cost_bits(h, cb->len[s]) <= 63 * 8 * n) mode = ZC_MODE_HUFF;
+        if (n != 0 && (policy == ZC_POLICY_AUTO || policy == ZC_POLICY_STATIC) && 64 * cost_bits(h, cb->len[s]) <= 63 * 8 * n)
+            mode = ZC_MODE_HUFF;
         cb->mode[s] = mode;
     }
     *out = cb;
@@ -193,8 +204,7 @@ zc_status zc_build_codebooks(uint32_t n_tensors, const zc_plan_t* const* plans, 
 {
     if (n_tensors == 0) return ZC_OK;
     if (!plans || !h_hists || !out) return ZC_E_INVALID_ARG;
-    if (policy != ZC_POLICY_AUTO && policy != ZC_POLICY_HUFF_ALL && policy != ZC_POLICY_RAW_ALL)
-        return ZC_E_UNSUPPORTED;
+    if (!known_policy(policy)) return ZC_E_UNSUPPORTED;
     if (n_threads == 0) {
         const uint32_t hw = std::max(1u, std::thread::hardware_concurrency());
         n_threads = std::min<uint32_t>({hw, 16u, (n_tensors + 7) / 8});     // a codebook takes tens of microseconds
@@ -227,6 +237,74 @@ zc_status zc_build_codebooks(uint32_t n_tensors, const zc_plan_t* const* plans, 
 }
 
 void zc_codebook_destroy(zc_codebook_t* cb) { delete cb; }
+
+// ---- runtime dictionaries (Sec. 3.3): one static codebook and the rule that says when to replace it ----
+struct zc_dict_s {
+    zc_codebook_t* cb = nullptr;
+    double tolerance = 0, baseline = 0, last = 0;
+    uint64_t n_observed = 0, n_rebuilds = 0;
+    bool has_baseline = false;
+};
+
+zc_status zc_dict_create(const zc_plan_t* plan, const uint64_t* h_hist, double tolerance, zc_dict_t** out)
+{
+    if (!plan || !h_hist || !out || !(tolerance >= 0) || !std::isfinite(tolerance)) return ZC_E_INVALID_ARG;
+    zc_dict_s* d = new (std::nothrow) zc_dict_s;
+    if (!d) return ZC_E_NOMEM;
+    const zc_status st = zc_build_codebook(plan, h_hist, ZC_POLICY_STATIC, &d->cb);
+    if (st != ZC_OK) { delete d; return st; }
+    d->tolerance = tolerance;
+    *out = d;
+    return ZC_OK;
+}
+
+void zc_dict_destroy(zc_dict_t* d)
+{
+    if (!d) return;
+    zc_codebook_destroy(d->cb);
+    delete d;
+}
+
+const zc_codebook_t* zc_dict_codebook(const zc_dict_t* d) { return d ? d->cb : nullptr; }
+
+zc_status zc_dict_observe(zc_dict_t* d, uint64_t input_bytes, uint64_t container_bytes, int* rebuild)
+{
+    if (!d || !rebuild || input_bytes == 0) return ZC_E_INVALID_ARG;
+    const double ratio = (double)container_bytes / (double)input_bytes;
+    d->last = ratio;
+    ++d->n_observed;
+    if (!d->has_baseline) {
+        d->baseline = ratio;
+        d->has_baseline = true;
+        *rebuild = 0;
+    } else {
+        *rebuild = ratio > d->baseline * (1.0 + d->tolerance) ? 1 : 0;
+    }
+    return ZC_OK;
+}
+
+zc_status zc_dict_rebuild(zc_dict_t* d, const zc_plan_t* plan, const uint64_t* h_hist)
+{
+    if (!d || !plan || !h_hist) return ZC_E_INVALID_ARG;
+    zc_codebook_t* fresh = nullptr;
+    const zc_status st = zc_build_codebook(plan, h_hist, ZC_POLICY_STATIC, &fresh);
+    if (st != ZC_OK) return st;
+    zc_codebook_destroy(d->cb);
+    d->cb = fresh;
+    d->has_baseline = false;
+    d->baseline = 0;
+    ++d->n_rebuilds;
+    return ZC_OK;
+}
+
+zc_status zc_dict_get_info(const zc_dict_t* d, zc_dict_info* out)
+{
+    if (!d || !out) return ZC_E_INVALID_ARG;
+    out->tolerance = d->tolerance; out->baseline_ratio = d->baseline; out->last_ratio = d->last;
+    out->n_observed = d->n_observed; out->n_rebuilds = d->n_rebuilds;
+    out->has_baseline = d->has_baseline ? 1u : 0u; out->reserved = 0;
+    return ZC_OK;
+}
 
 zc_status zc_codebook_get(const zc_codebook_t* cb, uint32_t s, uint32_t* mode, uint8_t* len256, uint32_t* code256)
 {

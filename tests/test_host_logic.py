@@ -28,7 +28,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_enums_match_the_oracle_s_numbering():
     assert (zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8) == (zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8)
-    assert (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL) == (zo.POLICY_AUTO, zo.POLICY_HUFF_ALL, zo.POLICY_RAW_ALL)
+    assert (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL, zc.POLICY_STATIC) == \
+        (zo.POLICY_AUTO, zo.POLICY_HUFF_ALL, zo.POLICY_RAW_ALL, zo.POLICY_STATIC)
     assert (zc.MODE_RAW, zc.MODE_HUFF) == (zo.RAW, zo.HUFF)
 
 
@@ -100,7 +101,7 @@ def test_codebook_matches_oracle_on_adversarial_histograms():
     H = _adversarial_histograms(rng)
     for i in range(0, len(H) - 1, 2):
         h2 = np.stack([H[i][1], H[i + 1][1]])
-        for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL):
+        for policy in (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL, zc.POLICY_STATIC):
             _compare_codebook(h2, policy)
 
 
@@ -124,6 +125,47 @@ def test_codebook_matches_oracle_on_random_histograms():
             idx = rng.permutation(256)[:n]
             h2[s, idx] = np.asarray(c, dtype=np.uint64)
         _compare_codebook(h2, zc.POLICY_AUTO)
+        if trial % 4 == 0:
+            _compare_codebook(h2, zc.POLICY_STATIC)
+
+
+def test_dictionary_object_follows_the_replacement_rule():
+    """zc_dict_*: the same decisions as the oracle's statement of the rule on seeded sequences of sizes, the same
+    codebooks after every rebuild, and the argument checks."""
+    rng = np.random.default_rng(5)
+    p = zc.plan(zc.FMT_BF16, 1 << 16, 4096)
+    for trial in range(20):
+        tol = float(rng.choice([0.0, 0.01, 0.05, 0.25]))
+        h = rng.integers(0, 1 << 20, (2, 256)).astype(np.uint64) * (rng.random((2, 256)) < 0.4)
+        d, o = zc.Dictionary(p, h, tol), zo.StaticDictionary(h, tol)
+        ratio = 0.7
+        for step in range(60):
+            ratio = min(max(ratio * float(rng.uniform(0.97, 1.04)), 0.05), 1.2)
+            nin = int(rng.integers(1, 1 << 30))
+            nout = int(round(nin * ratio))
+            got, want = d.observe(nin, nout), o.observe(nin, nout)
+            assert got == want, (trial, step)
+            if got:
+                h = rng.integers(0, 1 << 16, (2, 256)).astype(np.uint64)
+                d.rebuild(p, h)
+                o.rebuild(h)
+            cb = d.codebook
+            for s in range(2):
+                mode, lens, codes = cb.get(s)
+                assert mode == o.codebook.modes[s] and np.array_equal(lens, o.codebook.lengths[s])
+                assert np.array_equal(codes, o.codebook.codes[s]) and lens.min() >= 1
+        info = d.info
+        assert info.n_observed == 60 and info.n_rebuilds == o.n_rebuilds and info.tolerance == tol
+        assert bool(info.has_baseline) == (o.baseline is not None)
+        if o.baseline is not None:
+            assert info.baseline_ratio == o.baseline
+    h = np.ones((2, 256), np.uint64)
+    for bad in (-0.1, float("nan"), float("inf")):
+        with pytest.raises(zc.ZcError):
+            zc.Dictionary(p, h, bad)
+    d = zc.Dictionary(p, h, 0.1)
+    with pytest.raises(zc.ZcError):
+        d.observe(0, 10)
 
 
 def test_codebook_on_workload_like_histograms():

@@ -545,6 +545,68 @@ def test_static_dictionary_from_another_tensor():
         zo.compress(zo.BF16, bad, 20000, 4096, cb2)
 
 
+def test_static_dictionary_lengths_cover_every_symbol():
+    """A precomputed dictionary (Sec. 3.3) must be able to code a tensor it was not counted on: all 256 symbols
+    get a code, the code is complete (Kraft sum exactly 1), and wherever the length limit does not bind its cost
+    on the raised counts is that of a textbook Huffman tree."""
+    rng = np.random.default_rng(21)
+    for trial in range(40):
+        n = int(rng.integers(0, 257))
+        h = np.zeros(256, np.uint64)
+        h[rng.permutation(256)[:n]] = rng.integers(1, 1 << int(rng.integers(1, 34)), n).astype(np.uint64)
+        lens = zo.static_lengths(h)
+        assert lens.min() >= 1 and lens.max() <= 12
+        assert sum(1 << (12 - int(l)) for l in lens) == 1 << 12
+        # frequent symbols never get longer codes than rarer ones
+        order = np.argsort(h, kind="stable")
+        assert all(lens[order[i]] >= lens[order[i + 1]] or h[order[i]] == h[order[i + 1]] for i in range(255))
+    assert np.array_equal(zo.static_lengths(np.zeros(256, np.uint64)), np.full(256, 8))
+    assert np.array_equal(zo.static_lengths(np.full(256, 12345, np.uint64)), np.full(256, 8))
+    for trial in range(20):                      # Huffman depth stays below 12: the limit is loose
+        counts = rng.integers(1000, 2000, 256).astype(np.uint64)
+        lens = zo.static_lengths(counts)
+        raised = [256 * int(c) + 1 for c in counts]
+        assert sum(r * int(l) for r, l in zip(raised, lens)) == _huffman_cost(raised)
+    # a symbol that never occurred costs a long code; the frequent ones make room for them with one more bit at the end
+    h = _hist_of([1 << 20, 1 << 19, 1 << 18, 1 << 17])
+    lens = zo.static_lengths(h)
+    assert list(lens[:4]) == [1, 2, 3, 4] and lens[4:].min() >= 11
+    cb = zo.build_codebook(np.stack([h, np.zeros(256, np.uint64)]), zo.POLICY_STATIC)
+    assert cb.modes == [zo.HUFF, zo.RAW] and np.array_equal(cb.lengths[0], lens)
+
+
+def test_static_dictionary_codes_a_tensor_with_unseen_symbols():
+    a = _random_tensor(zo.BF16, 20000, 1)
+    b = _random_tensor(zo.BF16, 20000, 2).copy()
+    ha = zo.histogram(zo.BF16, a, 20000)
+    unseen = np.flatnonzero(ha[0] == 0)
+    b.view(np.uint16)[:50] = (unseen[:50].astype(np.uint16) << 7)      # exponents the dictionary never saw
+    cb = zo.build_codebook(ha, zo.POLICY_STATIC)
+    cont = zo.compress(zo.BF16, b, 20000, 4096, cb)
+    assert np.array_equal(zo.decompress(cont, b.size), b)
+    hb = zo.histogram(zo.BF16, b, 20000)
+    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == int((hb[0].astype(np.int64) * cb.lengths[0]).sum())
+
+
+def test_dictionary_replacement_rule():
+    """Sec. 3.3: a dictionary stays while the ratio holds and is replaced when it gets worse; the first tensor
+    after a (re)build sets the baseline."""
+    h = np.stack([_hist_of([100, 50, 20, 5]), _hist_of([10] * 256)])
+    d = zo.StaticDictionary(h, 0.05)
+    assert d.observe(1000, 700) is False and d.baseline == 0.7
+    assert d.observe(1000, 734) is False         # 0.734 <= 0.7 * 1.05
+    assert d.observe(1000, 736) is True
+    assert d.observe(2000, 1400) is False        # ratios, not sizes, are compared
+    assert d.observe(1000, 600) is False         # better than the baseline never triggers
+    d.rebuild(h)
+    assert d.baseline is None and d.n_rebuilds == 1
+    assert d.observe(1000, 900) is False and d.baseline == 0.9
+    assert zo.StaticDictionary(h, 0.0).observe(10, 7) is False
+    d0 = zo.StaticDictionary(h, 0.0)
+    d0.observe(10, 7)
+    assert d0.observe(10, 7) is False and d0.observe(1000, 701) is True
+
+
 def test_damaged_container_is_rejected():
     data = _random_tensor(zo.BF16, 3000, 9)
     cb = zo.build_codebook(zo.histogram(zo.BF16, data, 3000), zo.POLICY_AUTO)
