@@ -59,7 +59,8 @@
  *       each stream, cut into 32 equal subchunks that are concatenated bit by
  *       bit; each chunk payload starts on a 16-byte boundary.
  *   R6  AUTO policy: a stream is Huffman-coded iff
- *       64 * sum(count*len) <= 63 * 8 * n_syms, otherwise stored raw.
+ *       64 * sum(count*len) <= 63 * 8 * n_syms, otherwise stored raw.  A stream
+ *       without symbols is stored raw under every policy and with every codebook.
  *   R11 A stream of scale bytes (E8M0 or E4M3 scales, one "element" per byte)
  *       uses the same two-stream container: the bytes at odd offsets are the
  *       symbols of stream 0, the bytes at even offsets those of stream 1, so
@@ -458,12 +459,14 @@ static void set_bit(uint8_t *piece, uint64_t pos)
  * (len ignored for RAW).  Returns the container size, or a negative error:
  * -1 bad argument, -2 out of memory, -3 capacity too small, -4 a symbol has no code. */
 int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk_bytes,
-                    const int mode[2], const uint8_t len[2][256], uint8_t *out, uint64_t cap)
+                    const int mode_in[2], const uint8_t len[2][256], uint8_t *out, uint64_t cap)
 {
     int g = zo_group(fmt);
     if (!g || !valid_chunk_bytes(chunk_bytes)) return -1;
     if (fmt == ZO_FP4_E2M1 && (n_elems & 1)) return -1;
     uint64_t ns = zo_n_syms(fmt, n_elems);
+    /* a stream without symbols is stored raw (reading R6), also when the codebook comes from another tensor */
+    int mode[2] = {ns ? mode_in[0] : ZO_RAW, ns ? mode_in[1] : ZO_RAW};
     uint32_t nc = n_chunks_of(ns, chunk_bytes);
     uint64_t cs = chunk_bytes / 2, sub = cs / ZO_SUBS;
 

@@ -901,10 +901,17 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
             ++n;
         }
         B.n_tensors = n; B.total_chunks = (uint32_t)total;
-        const uint32_t want = std::max<uint32_t>((uint32_t)((total + shape.warps - 1) / shape.warps), 1);
+        uint32_t with_chunks = 0;
+        for (uint32_t i = 0; i < n; ++i) with_chunks += B.item[i].n_chunks != 0;
+        // enough blocks for one chunk per warp, and (many small tensors, say the K/V pages of a step) for one
+        // tensor per block, so that their tables are built side by side
+        const uint32_t want = std::max<uint32_t>({(uint32_t)((total + shape.warps - 1) / shape.warps), with_chunks, 1u});
         const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
-        // up to 8 ranges per block, none shorter than 16 chunks per warp (a range costs a table build)
+        // up to 8 ranges per block, none shorter than 16 chunks per warp (a range costs a table build), but not
+        // fewer than there are tensors as long as that stays within 8 per block
         B.n_ranges = grid * (uint32_t)std::min<uint64_t>(8, std::max<uint64_t>(1, total / ((uint64_t)grid * shape.warps * 16)));
+        B.n_ranges = std::max<uint32_t>(B.n_ranges, std::min<uint32_t>(with_chunks, 8 * grid));
+        B.n_ranges = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(B.n_ranges, total));
         // the ranges are handed out through the ticket word of the control block
         if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
         cudaError_t e = cudaSuccess;

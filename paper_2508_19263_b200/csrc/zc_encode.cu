@@ -2,6 +2,8 @@
 // zc_compress_batch, zc_compress_noalloc, zc_device_status.
 #include "zc_device.cuh"
 
+#include <cstring>
+#include <unordered_map>
 #include <vector>
 
 namespace zc {
@@ -21,8 +23,8 @@ struct EncItem {
     uint64_t input_bytes, n_syms, n_elems;
     uint32_t n_chunks;
     uint32_t first_batch;                        // batches of all earlier tensors of the launch
-    uint32_t index;                              // position in the caller's arrays (counters, tables, error reports)
-    uint32_t pad;
+    uint32_t index;                              // position in the caller's arrays (counters, error reports)
+    uint32_t table;                              // its code tables among the uploaded ones (tensors may share a codebook)
     Layout lay;
 };
 
@@ -255,6 +257,26 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         long long lb_base = 0;
         unsigned long long* lb_flags = nullptr;
         uint32_t lb_b = 0, idle = 0;
+        // Loads tensor t's code tables into the slot after the newest one, once every worker has posted the last
+        // batch that was packed with the table that is there now; false when that is not yet the case.
+        auto load_next_slot = [&](const uint32_t t, const uint32_t placed_now) -> bool {
+            const uint32_t nslot = (tab_slot + 1) % kTabSlots;
+            const uint32_t last = nslot == 0 ? slot_last0 : nslot == 1 ? slot_last1 : nslot == 2 ? slot_last2 : slot_last3;
+            if (placed_now < last) return false;
+            uint32_t* tab = tabs + nslot * tab_words;
+            uint32_t hs = 0;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                if (!is_huff(s)) continue;
+                const uint32_t* src;
+                if constexpr (N_ITEMS == 1) src = P.table.enc[s]; else src = C.tables[item(t).table].enc[s];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) tab[256 * hs + lane + 32 * i] = src[lane + 32 * i];
+                ++hs;
+            }
+            __syncwarp();
+            return true;
+        };
         for (;;) {
             bool did = false;
             // batches worker 0 handed out itself since the last look: they use the newest table slot
@@ -335,27 +357,12 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                     const EncItem& I = item(t);
                     cbase = (g - I.first_batch) * n_workers;
                     if (n_huff && t != tab_tensor) {
-                        // another tensor: its table goes to the next slot, once every worker has posted the last
-                        // batch that was packed with the table that is there now
-                        const uint32_t nslot = (tab_slot + 1) % kTabSlots;
-                        const uint32_t last = nslot == 0 ? slot_last0 : nslot == 1 ? slot_last1 : nslot == 2 ? slot_last2 : slot_last3;
-                        if (placed + (lb_on ? 1u : 0u) < last) {
-                            publish = false;                     // not yet: look back some more first
-                        } else {
-                            uint32_t* tab = tabs + nslot * tab_words;
-                            uint32_t hs = 0;
-#pragma unroll
-                            for (int s = 0; s < 2; ++s) {
-                                if (!is_huff(s)) continue;
-                                const uint32_t* src;
-                                if constexpr (N_ITEMS == 1) src = P.table.enc[s]; else src = C.tables[I.index].enc[s];
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) tab[256 * hs + lane + 32 * i] = src[lane + 32 * i];
-                                ++hs;
-                            }
-                            tab_slot = nslot;
+                        // another tensor: its table goes to the next slot
+                        if (load_next_slot(t, placed + (lb_on ? 1u : 0u))) {
+                            tab_slot = (tab_slot + 1) % kTabSlots;
                             tab_tensor = t;
-                            __syncwarp();
+                        } else {
+                            publish = false;                     // not yet: look back some more first
                         }
                     }
                     if (publish && g == I.first_batch) {
@@ -822,7 +829,7 @@ void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const
 }
 
 void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const void* d_in, const void* d_base, void* d_out,
-               uint32_t first_batch, uint32_t index)
+               uint32_t first_batch, uint32_t index, uint32_t table)
 {
     it.in = (const uint8_t*)d_in;
     it.base = (const uint8_t*)d_base;
@@ -831,7 +838,7 @@ void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const vo
     it.n_chunks = p->n_chunks;
     it.first_batch = first_batch;
     it.index = index;
-    it.pad = 0;
+    it.table = table;
     it.lay = make_layout(*p, mode);
 }
 
@@ -870,16 +877,17 @@ cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const E
     return e;
 }
 
-// Workspace of a batched call: control block | counters[n] | tables[n] | look-back words[batches]
-struct BatchLayout { size_t counters, tables, flags, total; };
+// Workspace of a batched call: control block | counters[n] | look-back words[batches] | tables[n].  Everything
+// before the tables starts from zero (one clear), the tables are uploaded.
+struct BatchLayout { size_t counters, flags, tables, total; };
 
 BatchLayout batch_layout(uint32_t n_tensors, uint64_t total_batches)
 {
     BatchLayout L{};
     L.counters = kControlBytes;
-    L.tables = (size_t)round_up(L.counters + sizeof(TensorCounters) * (uint64_t)n_tensors, 256);
-    L.flags = (size_t)round_up(L.tables + sizeof(EncTables) * (uint64_t)n_tensors, 256);
-    L.total = (size_t)round_up(L.flags + 8ull * total_batches, 256);
+    L.flags = (size_t)round_up(L.counters + sizeof(TensorCounters) * (uint64_t)n_tensors, 256);
+    L.tables = (size_t)round_up(L.flags + 8ull * total_batches, 256);
+    L.total = (size_t)round_up(L.tables + sizeof(EncTables) * (uint64_t)n_tensors, 256);
     return L;
 }
 
@@ -928,7 +936,7 @@ zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const voi
     P.c.tables = nullptr;
     P.c.n_tensors = 1;
     P.c.total_batches = (uint32_t)((p->n_chunks + (uint64_t)sh.workers - 1) / sh.workers);
-    fill_item(P.item[0], p, mode, d_in, d_base, d_out, 0, 0);
+    fill_item(P.item[0], p, mode, d_in, d_base, d_out, 0, 0, 0);
     fill_tables(P.table, cb);
 
     if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * P.c.total_batches, st) != cudaSuccess) return ZC_E_CUDA;
@@ -986,25 +994,41 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
     uint8_t* ws = (uint8_t*)d_workspace;
     const zc_plan_t* p0 = plans[0];
 
-    // control block, counters and look-back words start from zero; the tables are uploaded in one copy
+    // control block, counters and look-back words start from zero
     if (cudaMemsetAsync(ws, 0, L.tables, st) != cudaSuccess) return ZC_E_CUDA;
-    if (cudaMemsetAsync(ws + L.flags, 0, L.total - L.flags, st) != cudaSuccess) return ZC_E_CUDA;
+    // the code tables are uploaded in one copy, one per distinct codebook (the K/V pages of a step share theirs)
     static thread_local std::vector<EncTables> h_tables;
-    h_tables.resize(n_tensors);
-    for (uint32_t t = 0; t < n_tensors; ++t) fill_tables(h_tables[t], codebooks[t]);
-    if (cudaMemcpyAsync(ws + L.tables, h_tables.data(), sizeof(EncTables) * (size_t)n_tensors, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    static thread_local std::vector<uint32_t> table_of;          // per tensor: its tables among the uploaded ones
+    static thread_local std::vector<uint8_t> table_wide;         // per uploaded table: 1 + wide slots wanted, per mode pair
+    static thread_local std::unordered_map<const zc_codebook_t*, uint32_t> seen;
+    h_tables.clear(); table_wide.clear(); seen.clear();
+    table_of.resize(n_tensors);
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        auto found = seen.find(codebooks[t]);
+        if (found == seen.end()) {
+            found = seen.emplace(codebooks[t], (uint32_t)h_tables.size()).first;
+            h_tables.emplace_back();
+            fill_tables(h_tables.back(), codebooks[t]);
+            const uint32_t m[2] = {codebooks[t]->mode[0], codebooks[t]->mode[1]};
+            table_wide.push_back(wants_wide_slots(codebooks[t], m) ? 1 : 0);
+        }
+        table_of[t] = found->second;
+    }
+    if (cudaMemcpyAsync(ws + L.tables, h_tables.data(), sizeof(EncTables) * h_tables.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return ZC_E_CUDA;
 
     // one launch per combination of stream modes and slot size (the kernel's shared-memory layout depends on
     // them) and per kEncBatchMax tensors of it
     static thread_local EncParamsT<(int)kEncBatchMax> P;
     uint64_t flag_base = 0;
+    bool first_launch = true;
     static thread_local std::vector<uint8_t> group;              // per tensor: mode0 | mode1 << 1 | wide << 2
     group.resize(n_tensors);
     for (uint32_t t = 0; t < n_tensors; ++t) {
         const bool any = plans[t]->n_syms != 0;                  // an empty tensor: both streams raw
         const uint32_t m[2] = {any ? codebooks[t]->mode[0] : (uint32_t)ZC_MODE_RAW, any ? codebooks[t]->mode[1] : (uint32_t)ZC_MODE_RAW};
-        group[t] = (uint8_t)(m[0] | (m[1] << 1) | (wants_wide_slots(codebooks[t], m) ? 4u : 0u));
+        const bool wide = (m[0] == ZC_MODE_HUFF || m[1] == ZC_MODE_HUFF) && table_wide[table_of[t]];
+        group[t] = (uint8_t)(m[0] | (m[1] << 1) | (wide ? 4u : 0u));
     }
     for (uint32_t combo = 0; combo < 8; ++combo) {
         const uint32_t mode[2] = {combo & 1u, (combo >> 1) & 1u};
@@ -1023,7 +1047,7 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
                 if (!in_combo(t)) continue;
                 const uint64_t nb = (plans[t]->n_chunks + (uint64_t)sh.workers - 1) / sh.workers;
                 if (batches + nb >= (1ull << 32)) break;
-                fill_item(P.item[n], plans[t], mode, d_in[t], d_base ? d_base[t] : nullptr, d_out[t], (uint32_t)batches, t);
+                fill_item(P.item[n], plans[t], mode, d_in[t], d_base ? d_base[t] : nullptr, d_out[t], (uint32_t)batches, t, table_of[t]);
                 batches += nb;
                 ++n;
             }
@@ -1038,22 +1062,28 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
             P.c.n_tensors = n;
             P.c.total_batches = (uint32_t)batches;
             flag_base += batches;
-            // the ticket counter restarts for every launch
-            if (cudaMemsetAsync(&((Control*)ws)->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
+            // the ticket counter restarts for every launch (the first one finds it cleared)
+            if (!first_launch && cudaMemsetAsync(&((Control*)ws)->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
+            first_launch = false;
             if (launch_encode<(int)kEncBatchMax>(P, p0->format, sh, st) != cudaSuccess) return ZC_E_CUDA;
         }
     }
 
     if (h_out_bytes) {
-        static thread_local std::vector<TensorCounters> h_counters;
-        h_counters.resize(n_tensors);
-        Control h;
-        if (cudaMemcpyAsync(&h, ws, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
-        if (cudaMemcpyAsync(h_counters.data(), ws + L.counters, sizeof(TensorCounters) * (size_t)n_tensors, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-            return ZC_E_CUDA;
+        // control block and counters lie next to each other: one copy
+        static thread_local std::vector<uint8_t> h_state;
+        const size_t bytes = L.counters + sizeof(TensorCounters) * (size_t)n_tensors;
+        h_state.resize(bytes);
+        if (cudaMemcpyAsync(h_state.data(), ws, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZC_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return ZC_E_CUDA;
+        Control h;
+        std::memcpy(&h, h_state.data(), sizeof(Control));
         if (h.status & 0xFF) return (zc_status)(h.status & 0xFF);
-        for (uint32_t t = 0; t < n_tensors; ++t) h_out_bytes[t] = h_counters[t].total16;
+        for (uint32_t t = 0; t < n_tensors; ++t) {
+            TensorCounters tc;
+            std::memcpy(&tc, h_state.data() + L.counters + sizeof(TensorCounters) * (size_t)t, sizeof(tc));
+            h_out_bytes[t] = tc.total16;
+        }
     }
     return ZC_OK;
 }

@@ -165,6 +165,45 @@ def test_batched_encoder_many_small_tensors_and_the_batched_decoder_after_it():
         assert np.array_equal(back[: p.input_bytes].cpu().numpy(), data[: p.input_bytes])
 
 
+@pytest.mark.parametrize("fmt", [zc.FMT_BF16, zc.FMT_FP8_E4M3])
+def test_batched_encoder_with_codebooks_shared_between_tensors(fmt):
+    """Pages of a K/V cache share their dictionaries (Sec. 3.3): three static codebooks serve 40 tensors, a few
+    tensors bring their own; every container equals the oracle's with the same code."""
+    chunk_bytes = 4096
+    rng = np.random.default_rng(3)
+    G = zo.group(fmt)
+    sizes = [int(v) * 2 * G for v in rng.integers(1, 12000, 40)] + [0, 2 * G]
+    datas = [_weights(fmt, n, 500 + i) for i, n in enumerate(sizes)]
+    plans = [zc.plan(fmt, n, chunk_bytes) for n in sizes]
+    hists = [zo.histogram(fmt, d, n) for d, n in zip(datas, sizes)]
+    shared = [zc.build_codebook(plans[k], hists[k], zc.POLICY_STATIC) for k in range(3)]
+    oshared = [zo.build_codebook(hists[k], zo.POLICY_STATIC) for k in range(3)]
+    cbs, ocbs = [], []
+    for i in range(len(sizes)):
+        if i % 7 == 6:                                               # its own codebook
+            cbs.append(zc.build_codebook(plans[i], hists[i], zc.POLICY_AUTO))
+            ocbs.append(zo.build_codebook(hists[i], zo.POLICY_AUTO))
+        else:
+            cbs.append(shared[i % 3])
+            ocbs.append(oshared[i % 3])
+    d_ins = [_to_dev(d) for d in datas]
+    d_outs = [torch.full((p.max_compressed_bytes,), 0xA5, dtype=torch.uint8, device=DEV) for p in plans]
+    batch = zc.CompressBatch(plans, d_ins, d_outs)
+    batch.set_codebooks(cbs)
+    ws = torch.full((batch.workspace_bytes,), 0x5A, dtype=torch.uint8, device=DEV)
+    for _ in range(2):
+        got = zc.compress_batch(batch, ws)
+        for n, data, ocb, out, nbytes in zip(sizes, datas, ocbs, d_outs, got):
+            want = zo.compress(fmt, data, n, chunk_bytes, ocb)
+            assert nbytes == want.size and np.array_equal(out[:nbytes].cpu().numpy(), want)
+    backs = [torch.full((p.input_bytes + 16,), 0xEE, dtype=torch.uint8, device=DEV) for p in plans]
+    dws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    zc.decompress_batch(zc.DecompressBatch(plans, d_outs, got, backs), dws)
+    assert zc.batch_status(dws) == (zc.OK, None)
+    for p, data, back in zip(plans, datas, backs):
+        assert np.array_equal(back[: p.input_bytes].cpu().numpy(), data[: p.input_bytes])
+
+
 def test_batched_encoder_reports_a_symbol_without_code_and_its_tensor():
     fmt, chunk_bytes = zc.FMT_BF16, 4096
     sizes = [30000, 50000, 20000]

@@ -586,6 +586,10 @@ def test_static_dictionary_codes_a_tensor_with_unseen_symbols():
     assert np.array_equal(zo.decompress(cont, b.size), b)
     hb = zo.histogram(zo.BF16, b, 20000)
     assert zo.parse_header(cont)["streams"][0]["payload_bits"] == int((hb[0].astype(np.int64) * cb.lengths[0]).sum())
+    # a tensor without elements is all header, whatever the dictionary's modes say
+    empty = zo.compress(zo.BF16, np.zeros(0, np.uint8), 0, 4096, cb)
+    assert empty.size == 128 and [st["mode"] for st in zo.parse_header(empty)["streams"]] == [zo.RAW, zo.RAW]
+    assert zo.decompress(empty, 0).size == 0
 
 
 def test_dictionary_replacement_rule():
