@@ -79,6 +79,9 @@ def workload_specs(name: str):
         # delta checkpoints (Sec. 3.1 / 4.1): the XOR of two consecutive BF16 checkpoints of the config-2 stack is
         # coded; the earlier checkpoint is a second resident input of every call
         return wl.BF16, wl.llama8b_stack(2) if name.startswith("next2") else wl.llama8b_stack(2, n_layers=2, include_embedding=False)
+    if name == "next4_fp8_e5m2":
+        # config 3's stack in the other FP8 format (Sec. 3.2 names E5M2, Sec. 4.2 leaves it out): cast without scales
+        return wl.FP8_E5M2, wl.llama8b_stack(3)
     if name == "small_bf16":
         return wl.BF16, wl.llama8b_stack(2, n_layers=2, include_embedding=False)
     if name == "small_fp8":

@@ -85,9 +85,13 @@ typedef enum zc_format {
     ZC_FMT_BF16 = 1,            /* u16 little-endian: sign 15, exponent 14..7, mantissa 6..0 */
     ZC_FMT_FP8_E4M3 = 2,        /* u8: sign 7, exponent 6..3, mantissa 2..0 */
     ZC_FMT_FP4_E2M1 = 3,        /* two per byte, element 2i in bits 3..0: sign 3, exponent 2..1, mantissa 0 */
-    ZC_FMT_SCALE_U8 = 4         /* a stream of scale bytes (E8M0 / E4M3 block scales of FP4 tensors, Sec. 3.4 and 4.4):
+    ZC_FMT_SCALE_U8 = 4,        /* a stream of scale bytes (E8M0 / E4M3 block scales of FP4 tensors, Sec. 3.4 and 4.4):
                                    one element per byte; the bytes at odd offsets are the symbols of stream 0, the
                                    bytes at even offsets those of stream 1 (a missing last odd byte counts as 0) */
+    ZC_FMT_FP8_E5M2 = 5         /* u8: sign 7, exponent 6..2, mantissa 1..0 (Sec. 3.2).  Five exponent bits do not
+                                   pair into byte symbols, so the coded field is the upper four exponent bits
+                                   (bits 6..3); sign, lowest exponent bit and mantissa form the other field.
+                                   Bit for bit the split of E4M3; the container records format 5 */
 } zc_format;
 
 typedef enum zc_policy {

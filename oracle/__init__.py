@@ -16,7 +16,7 @@ from dataclasses import dataclass
 
 import numpy as np
 
-BF16, FP8_E4M3, FP4_E2M1, SCALE_U8 = 1, 2, 3, 4
+BF16, FP8_E4M3, FP4_E2M1, SCALE_U8, FP8_E5M2 = 1, 2, 3, 4, 5
 RAW, HUFF = 0, 1
 POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL, POLICY_STATIC = 0, 1, 2, 3
 L_MAX = 12
@@ -48,6 +48,8 @@ def lib():
         L.zo_bf16_value.argtypes = [C.c_uint16]
         L.zo_e4m3_value.restype = C.c_double
         L.zo_e4m3_value.argtypes = [C.c_uint8]
+        L.zo_e5m2_value.restype = C.c_double
+        L.zo_e5m2_value.argtypes = [C.c_uint8]
         L.zo_e2m1_value.restype = C.c_double
         L.zo_e2m1_value.argtypes = [C.c_uint8]
         L.zo_group.restype = C.c_int
@@ -105,6 +107,10 @@ def bf16_value(bits: int) -> float:
 
 def e4m3_value(bits: int) -> float:
     return lib().zo_e4m3_value(bits)
+
+
+def e5m2_value(bits: int) -> float:
+    return lib().zo_e5m2_value(bits)
 
 
 def e2m1_value(nibble: int) -> float:

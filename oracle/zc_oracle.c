@@ -74,6 +74,13 @@
  *       where the baseline is that quotient for the first tensor coded after the
  *       dictionary was built and the tolerance is the caller's (the paper gives
  *       no number).
+ *   R13 FP8 E5M2 (sign 7, exponent 6..2, mantissa 1..0; Sec. 3.2 names the format,
+ *       Sec. 4.2 leaves it out because its fields do not align to bytes): the
+ *       exponent field of the codec is the upper four exponent bits (bits 6..3),
+ *       the other field is sign, lowest exponent bit and mantissa
+ *       ((sign << 3) | bits 2..0); two elements per symbol as for E4M3.  The
+ *       lowest exponent bit goes with the poorly compressible bits; what is
+ *       coded is the part of the exponent that byte symbols can carry.
  *
  * Container layout (little-endian, every section 16-byte aligned):
  *   header 128 B:
@@ -101,7 +108,7 @@
 #include <string.h>
 #include <math.h>
 
-enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3, ZO_SCALE_U8 = 4 };
+enum { ZO_BF16 = 1, ZO_FP8_E4M3 = 2, ZO_FP4_E2M1 = 3, ZO_SCALE_U8 = 4, ZO_FP8_E5M2 = 5 };
 enum { ZO_RAW = 0, ZO_HUFF = 1 };
 enum { ZO_POLICY_AUTO = 0, ZO_POLICY_HUFF_ALL = 1, ZO_POLICY_RAW_ALL = 2, ZO_POLICY_STATIC = 3 };
 enum { ZO_LMAX = 12, ZO_SUBS = 32, ZO_HEADER = 128 };
@@ -132,6 +139,17 @@ double zo_e4m3_value(uint8_t x)
     return s ? -v : v;
 }
 
+/* FP8 E5M2: bias 15, e = 31 is infinity (m = 0) or NaN, e = 0 subnormal (Sec. 3.2). */
+double zo_e5m2_value(uint8_t x)
+{
+    int s = x >> 7, e = (x >> 2) & 0x1F, m = x & 3;
+    double v;
+    if (e == 31) v = m ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)m / 4.0, -14);
+    else v = ldexp(1.0 + (double)m / 4.0, e - 15);
+    return s ? -v : v;
+}
+
 /* FP4 E2M1: bias 1, values 0, .5, 1, 1.5, 2, 3, 4, 6 (Sec. 3.4). */
 double zo_e2m1_value(uint8_t nib)
 {
@@ -153,6 +171,7 @@ int zo_group(int fmt)
     case ZO_FP8_E4M3: return 2;
     case ZO_FP4_E2M1: return 4;
     case ZO_SCALE_U8: return 2;
+    case ZO_FP8_E5M2: return 2;
     default: return 0;
     }
 }
@@ -170,6 +189,7 @@ uint64_t zo_input_bytes(int fmt, uint64_t n_elems)
     case ZO_FP8_E4M3: return n_elems;
     case ZO_FP4_E2M1: return (n_elems + 1) / 2;
     case ZO_SCALE_U8: return n_elems;
+    case ZO_FP8_E5M2: return n_elems;
     default: return 0;
     }
 }
@@ -189,6 +209,11 @@ static void element_fields(int fmt, const uint8_t *in, uint64_t i, unsigned *e, 
         unsigned x = in[i];
         *e = (x >> 3) & 0xF;
         *sm = ((x >> 7) << 3) | (x & 7);
+    } else if (fmt == ZO_FP8_E5M2) {             /* R13: exponent bits 4..1 | sign, exponent bit 0, mantissa */
+        unsigned x = in[i];
+        unsigned s = x >> 7, ex = (x >> 2) & 0x1F, m = x & 3;
+        *e = ex >> 1;
+        *sm = (s << 3) | ((ex & 1) << 2) | m;
     } else {
         unsigned b = in[i / 2];
         unsigned x = (i & 1) ? (b >> 4) : (b & 0xF);
@@ -248,6 +273,9 @@ void zo_merge(int fmt, const uint8_t *s0, const uint8_t *s1, uint64_t n_elems, u
             out[2 * el + 1] = (uint8_t)(x >> 8);
         } else if (fmt == ZO_FP8_E4M3) {
             out[el] = (uint8_t)(((sm >> 3) << 7) | (e << 3) | (sm & 7));
+        } else if (fmt == ZO_FP8_E5M2) {
+            unsigned ex = (e << 1) | ((sm >> 2) & 1);
+            out[el] = (uint8_t)(((sm >> 3) << 7) | (ex << 2) | (sm & 3));
         } else {
             unsigned x = ((sm >> 1) << 3) | (e << 1) | (sm & 1);
             out[el / 2] |= (uint8_t)((el & 1) ? (x << 4) : x);

@@ -18,7 +18,7 @@ import torch
 
 from . import build as _build
 
-FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1, FMT_SCALE_U8 = 1, 2, 3, 4
+FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1, FMT_SCALE_U8, FMT_FP8_E5M2 = 1, 2, 3, 4, 5
 POLICY_AUTO, POLICY_HUFF_ALL, POLICY_RAW_ALL, POLICY_STATIC = 0, 1, 2, 3
 MODE_RAW, MODE_HUFF = 0, 1
 (OK, E_INVALID_ARG, E_UNSUPPORTED, E_BUFFER_TOO_SMALL, E_CORRUPT, E_CUDA, E_NOMEM, E_DEVICE_TIMEOUT, E_NO_CODE,

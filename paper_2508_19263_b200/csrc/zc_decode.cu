@@ -843,7 +843,7 @@ zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t co
     else launch(decode_kernel<F, 1>);
     switch (p->format) {
     case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
-    case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
     case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
     default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
     }
@@ -935,7 +935,7 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
     }
         switch (p0->format) {
         case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
-        case ZC_FMT_FP8_E4M3: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
+        case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
         case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
     default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
         }

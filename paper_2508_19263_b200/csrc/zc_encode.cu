@@ -869,7 +869,7 @@ cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const E
     else launch(encode_kernel<F, N_ITEMS, false, false>);
     switch (format) {
     case ZC_FMT_BF16: ZC_ENC_CASE(ZC_FMT_BF16) break;
-    case ZC_FMT_FP8_E4M3: ZC_ENC_CASE(ZC_FMT_FP8_E4M3) break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_ENC_CASE(ZC_FMT_FP8_E4M3) break;
     case ZC_FMT_SCALE_U8: ZC_ENC_CASE(ZC_FMT_SCALE_U8) break;
     default: ZC_ENC_CASE(ZC_FMT_FP4_E2M1) break;
     }

@@ -236,7 +236,7 @@ zc_status zc_histogram_xor(const zc_plan_t* p, const void* d_in, const void* d_b
     };
     switch (p->format) {
     case ZC_FMT_BF16: launch(hist_kernel<ZC_FMT_BF16>); break;
-    case ZC_FMT_FP8_E4M3: launch(hist_kernel<ZC_FMT_FP8_E4M3>); break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: launch(hist_kernel<ZC_FMT_FP8_E4M3>); break;
     case ZC_FMT_SCALE_U8: launch(hist_kernel<ZC_FMT_SCALE_U8>); break;
     default: launch(hist_kernel<ZC_FMT_FP4_E2M1>); break;
     }
@@ -292,7 +292,7 @@ zc_status zc_histogram_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pla
         };
         switch (plans[0]->format) {
         case ZC_FMT_BF16: launch(hist_batch_kernel<ZC_FMT_BF16>); break;
-        case ZC_FMT_FP8_E4M3: launch(hist_batch_kernel<ZC_FMT_FP8_E4M3>); break;
+        case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: launch(hist_batch_kernel<ZC_FMT_FP8_E4M3>); break;
         case ZC_FMT_SCALE_U8: launch(hist_batch_kernel<ZC_FMT_SCALE_U8>); break;
         default: launch(hist_batch_kernel<ZC_FMT_FP4_E2M1>); break;
         }

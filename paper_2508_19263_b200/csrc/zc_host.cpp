@@ -24,6 +24,7 @@ uint32_t group_of(uint32_t fmt)
     case ZC_FMT_FP8_E4M3: return 2;
     case ZC_FMT_FP4_E2M1: return 4;
     case ZC_FMT_SCALE_U8: return 2;
+    case ZC_FMT_FP8_E5M2: return 2;
     default: return 0;
     }
 }
@@ -440,7 +441,7 @@ zc_status zc_test_split16(zc_format fmt, const uint8_t* h_in16, uint8_t* h_e8, u
     std::memcpy(in, h_in16, 16);
     switch (fmt) {
     case ZC_FMT_BF16: split16<ZC_FMT_BF16>(in, e, sm); break;
-    case ZC_FMT_FP8_E4M3: split16<ZC_FMT_FP8_E4M3>(in, e, sm); break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: split16<ZC_FMT_FP8_E4M3>(in, e, sm); break;
     case ZC_FMT_FP4_E2M1: split16<ZC_FMT_FP4_E2M1>(in, e, sm); break;
     case ZC_FMT_SCALE_U8: split16<ZC_FMT_SCALE_U8>(in, e, sm); break;
     default: return ZC_E_UNSUPPORTED;
@@ -458,7 +459,7 @@ zc_status zc_test_merge16(zc_format fmt, const uint8_t* h_e8, const uint8_t* h_s
     std::memcpy(sm, h_sm8, 8);
     switch (fmt) {
     case ZC_FMT_BF16: merge16<ZC_FMT_BF16>(e, sm, out); break;
-    case ZC_FMT_FP8_E4M3: merge16<ZC_FMT_FP8_E4M3>(e, sm, out); break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: merge16<ZC_FMT_FP8_E4M3>(e, sm, out); break;
     case ZC_FMT_FP4_E2M1: merge16<ZC_FMT_FP4_E2M1>(e, sm, out); break;
     case ZC_FMT_SCALE_U8: merge16<ZC_FMT_SCALE_U8>(e, sm, out); break;
     default: return ZC_E_UNSUPPORTED;

@@ -22,8 +22,8 @@ from typing import Iterator, List, Optional, Tuple
 
 import torch
 
-BF16, FP8_E4M3, FP4_E2M1, SCALE_U8 = 1, 2, 3, 4
-FORMAT_NAMES = {BF16: "bf16", FP8_E4M3: "fp8_e4m3", FP4_E2M1: "fp4_e2m1"}
+BF16, FP8_E4M3, FP4_E2M1, SCALE_U8, FP8_E5M2 = 1, 2, 3, 4, 5
+FORMAT_NAMES = {BF16: "bf16", FP8_E4M3: "fp8_e4m3", FP4_E2M1: "fp4_e2m1", FP8_E5M2: "fp8_e5m2"}
 
 
 def _gen(seed: int, device) -> torch.Generator:
@@ -116,6 +116,8 @@ def make_weight(spec: TensorSpec, fmt: int, device) -> Tuple[torch.Tensor, int, 
     if fmt == FP8_E4M3:
         scale = (x.abs().amax(dim=-1, keepdim=True) / 448.0).clamp_(min=1e-30)
         return to_e4m3_bytes(x, scale), spec.n_elems, scale.reshape(-1)
+    if fmt == FP8_E5M2:                          # the wide-range FP8 format: cast as it is (RNE), no scale
+        return x.to(torch.float8_e5m2).view(torch.uint8).reshape(-1), spec.n_elems, None
     if fmt == FP4_E2M1:
         packed, scales = to_mxfp4_bytes(x)
         return packed, spec.n_elems, scales

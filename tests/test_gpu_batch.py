@@ -12,7 +12,7 @@ from paper_2508_19263_b200 import binding as zc
 from test_gpu_parity import _weights
 
 pytestmark = pytest.mark.gpu
-FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8]
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8, zc.FMT_FP8_E5M2]
 DEV = "cuda"
 
 

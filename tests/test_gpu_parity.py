@@ -11,7 +11,7 @@ from paper_2508_19263_b200 import binding as zc
 from paper_2508_19263_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
-FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8]
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8, zc.FMT_FP8_E5M2]
 DEV = "cuda"
 
 
@@ -66,6 +66,9 @@ def _weights(fmt, n, seed):
         x = rng.standard_normal(n).astype(np.float32)
         x = x / (np.abs(x).max() / 448.0)
         return torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(-1).copy()
+    if fmt == zc.FMT_FP8_E5M2:
+        x = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+        return x.to(torch.float8_e5m2).view(torch.uint8).numpy().reshape(-1).copy()
     v = rng.choice(16, size=n, p=np.array([6, 5, 4, 3, 2, 1, 1, 1, 6, 5, 4, 3, 2, 1, 1, 1]) / 46.0).astype(np.uint8)
     return (v[0::2] | (v[1::2] << 4)).astype(np.uint8)
 

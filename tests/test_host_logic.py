@@ -11,7 +11,7 @@ from paper_2508_19263_b200 import binding as zc
 from paper_2508_19263_b200 import build as zbuild
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8]
+FORMATS = [zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8, zc.FMT_FP8_E5M2]
 
 
 def test_library_exports_every_declared_symbol():
@@ -27,7 +27,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_enums_match_the_oracle_s_numbering():
-    assert (zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8) == (zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8)
+    assert (zc.FMT_BF16, zc.FMT_FP8_E4M3, zc.FMT_FP4_E2M1, zc.FMT_SCALE_U8, zc.FMT_FP8_E5M2) == \
+        (zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8, zo.FP8_E5M2)
     assert (zc.POLICY_AUTO, zc.POLICY_HUFF_ALL, zc.POLICY_RAW_ALL, zc.POLICY_STATIC) == \
         (zo.POLICY_AUTO, zo.POLICY_HUFF_ALL, zo.POLICY_RAW_ALL, zo.POLICY_STATIC)
     assert (zc.MODE_RAW, zc.MODE_HUFF) == (zo.RAW, zo.HUFF)
@@ -187,7 +188,7 @@ def test_word_level_split_and_merge_match_oracle(fmt):
         for bit in range(8):
             x = np.zeros(16, np.uint8); x[b] = 1 << bit
             cases.append(x)
-    n_elems = {zc.FMT_BF16: 8, zc.FMT_FP8_E4M3: 16, zc.FMT_FP4_E2M1: 32, zc.FMT_SCALE_U8: 16}[fmt]
+    n_elems = {zc.FMT_BF16: 8, zc.FMT_FP8_E4M3: 16, zc.FMT_FP4_E2M1: 32, zc.FMT_SCALE_U8: 16, zc.FMT_FP8_E5M2: 16}[fmt]
     for x in cases:
         e, sm = zc.test_split16(fmt, x)
         we, wsm = zo.split(fmt, x, n_elems)

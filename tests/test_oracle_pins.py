@@ -16,7 +16,7 @@ import torch
 import oracle as zo
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-FORMATS = [zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8]
+FORMATS = [zo.BF16, zo.FP8_E4M3, zo.FP4_E2M1, zo.SCALE_U8, zo.FP8_E5M2]
 
 
 # --------------------------------------------------------------------------------------------
@@ -68,6 +68,40 @@ def test_e4m3_values_match_torch_for_all_patterns():
     ok = ~np.isnan(ref)
     assert np.array_equal(ref[ok], got[ok])
     assert got[0x7E] == 448.0 and np.nanmax(got) == 448.0
+
+
+def test_e5m2_values_match_torch_for_all_patterns():
+    bits = np.arange(256, dtype=np.uint8)
+    ref = torch.from_numpy(bits.copy()).view(torch.float8_e5m2).to(torch.float64).numpy()
+    got = np.array([zo.e5m2_value(int(b)) for b in bits])
+    assert np.array_equal(np.isnan(ref), np.isnan(got))
+    ok = ~np.isnan(ref)
+    assert np.array_equal(ref[ok], got[ok])
+    assert got[0x7B] == 57344.0 and got[0x7C] == np.inf and got[0x01] == 2.0 ** -16
+
+
+def test_split_fields_rebuild_the_value_e5m2():
+    """E5M2 (Sec. 3.2): the coded field holds the upper four exponent bits, the other field sign, lowest exponent
+    bit and mantissa; read back that way the two fields give the element's value for every pattern."""
+    bits = np.arange(256, dtype=np.uint8)
+    data = np.stack([bits, bits[::-1]], axis=1).reshape(-1)
+    hi, rest = zo.split(zo.FP8_E5M2, data, data.size)
+    ref = torch.from_numpy(data.copy()).view(torch.float8_e5m2).to(torch.float64).numpy()
+    for half, sl in ((0, slice(0, None, 2)), (1, slice(1, None, 2))):
+        e_hi = ((hi >> (4 * half)) & 0xF).astype(np.int64)
+        f = (rest >> (4 * half)) & 0xF
+        s = f >> 3
+        ee = 2 * e_hi + ((f >> 2) & 1)
+        m = (f & 3).astype(np.float64)
+        val = np.where(ee == 0, np.ldexp(m / 4.0, -14), np.ldexp(1.0 + m / 4.0, ee - 15))
+        val = np.where(s == 1, -val, val)
+        r = ref[sl]
+        ok = np.isfinite(r)
+        assert np.array_equal(val[ok], r[ok])
+        assert (ee[~ok] == 31).all()
+    # 1.0 = 0 01111 00 (0x3C) and -2^-14 = 1 00001 00 (0x84): upper exponent bits 7 and 0, rest 0100 and 1100
+    hi, rest = zo.split(zo.FP8_E5M2, np.array([0x3C, 0x84], np.uint8), 2)
+    assert (int(hi[0]), int(rest[0])) == (0x07, 0xC4)
 
 
 def test_e2m1_value_set():
@@ -418,6 +452,9 @@ def _random_tensor(fmt, n, seed, skew=True):
         x = rng.standard_normal(n).astype(np.float32)
         x = np.clip(x / (np.abs(x).max() / 448.0), -448, 448) if n else x
         return torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(-1).copy()
+    if fmt == zo.FP8_E5M2:
+        x = (rng.standard_normal(n) * 0.02).astype(np.float32)
+        return torch.from_numpy(x).to(torch.float8_e5m2).view(torch.uint8).numpy().reshape(-1).copy()
     v = rng.choice(16, size=n, p=np.array([6, 5, 4, 3, 2, 1, 1, 1, 6, 5, 4, 3, 2, 1, 1, 1]) / 46.0).astype(np.uint8)
     return (v[0::2] | (v[1::2] << 4)).astype(np.uint8)
 
