@@ -567,8 +567,9 @@ def run_ours(args):
         e2e = {"value": whole_job_gbs(world, U, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": U, "d2h_bytes_per_step": C + n_t * 4096,
                "ms_per_step": ms_e2e,
                "groups": len(gb) if args.batch else n_t,
-               "note": "host tensor -> H2D -> histogram -> codebook -> compress -> D2H container; decoded tensor stays on the device; "
-                       "pipelined over groups of tensors on three streams"}
+               "note": ("host tensor -> H2D -> compress with the static dictionaries -> D2H container" if static else
+                        "host tensor -> H2D -> histogram -> codebook -> compress -> D2H container")
+                       + "; decoded tensor stays on the device; pipelined over groups of tensors on three streams"}
         del h_in, h_out
     except Exception as ex:  # pinned host memory for the whole stack may be unavailable
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "error": str(ex)[:200]}
