@@ -56,6 +56,12 @@
  *   payload area: for chunk 0, 1, ...: for each HUFF stream (stream order) the
  *      chunk's bits, zero padded to a multiple of 16 bytes
  *   16 zero guard bytes when at least one stream is HUFF
+ *   Constant chunks: when both streams are HUFF, a chunk of a stream whose symbols are all the
+ *      stream's fill symbol (the first symbol in (length, symbol) order, whose code is all zeros)
+ *      has no payload at all: its 32 sub_end entries are 0, its piece is empty and its chunk_off16
+ *      equals that of the piece that follows.  A chunk that holds symbols and has 0 bits can be
+ *      nothing else.  This is what lets unchanged stretches of a delta checkpoint (Sec. 3.1, 4.1)
+ *      cost less than the one bit per symbol of a per-symbol code.
  * The container is a pure function of (input bytes, plan, codebook).
  */
 #ifndef ZC_H

@@ -81,6 +81,16 @@
  *       ((sign << 3) | bits 2..0); two elements per symbol as for E4M3.  The
  *       lowest exponent bit goes with the poorly compressible bits; what is
  *       coded is the part of the exponent that byte symbols can carry.
+ *   R14 In a container with BOTH streams coded, a chunk of a stream whose symbols
+ *       are all the stream's fill symbol takes no payload bits at all: all its
+ *       subchunk ends are 0 and its piece is empty.  (With one stream stored raw
+ *       the tensor pays 8 bits per symbol for that stream anyway and the rule
+ *       does not apply: a chunk of fill symbols is coded like any other.)  The fill symbol is the first symbol in (length, symbol) order,
+ *       the one whose code is all zeros.  A chunk that holds symbols and has 0
+ *       bits can be nothing else (every code has at least one bit), so no flag
+ *       is needed.  This is what lets unchanged stretches of a delta checkpoint
+ *       (Sec. 3.1, 4.1) or the unused part of a cache page fall below the 1 bit
+ *       per symbol that a per-symbol code costs at least.
  *
  * Container layout (little-endian, every section 16-byte aligned):
  *   header 128 B:
@@ -385,6 +395,15 @@ void zo_canonical_codes(const uint8_t len[256], uint32_t code[256])
     }
 }
 
+/* The fill symbol of a code (reading R14): first in (length, symbol) order; -1 without codes. */
+int zo_fill_symbol(const uint8_t len[256])
+{
+    int best = -1;
+    for (int v = 0; v < 256; ++v)
+        if (len[v] && (best < 0 || len[v] < len[best])) best = v;
+    return best;
+}
+
 /* Sum of count*len. */
 uint64_t zo_payload_bits(const uint64_t hist[256], const uint8_t len[256])
 {
@@ -540,9 +559,18 @@ int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk
             if (mode[s] != ZO_HUFF) continue;
             uint8_t *chunk_off = out + sec[s] + 256;
             uint8_t *sub_end = out + sec[s] + 256 + round16(4ull * nc);
-            /* bits of this chunk */
+            /* bits of this chunk; none at all if every symbol is the fill symbol (reading R14) */
             uint64_t bits = 0;
-            for (uint64_t k = c_lo; k < c_hi; ++k) bits += len[s][st[s][k]];
+            int fill = zo_fill_symbol(len[s]), constant = (mode[0] == ZO_HUFF && mode[1] == ZO_HUFF);
+            for (uint64_t k = c_lo; k < c_hi; ++k) {
+                bits += len[s][st[s][k]];
+                if (st[s][k] != fill) constant = 0;
+            }
+            if (constant) {
+                put32(chunk_off + 4ull * c, (uint32_t)pos16);
+                for (int j = 0; j < ZO_SUBS; ++j) put_sub_end(sub_end, sub_end_width(chunk_bytes), c, j, 0);
+                continue;
+            }
             uint64_t piece_bytes = round16((bits + 7) / 8);
             uint64_t piece_off = payload_off + 16 * pos16;
             if (cap < piece_off + piece_bytes + 16) { free(st[0]); free(st[1]); return -3; }
@@ -706,6 +734,13 @@ static int decode_chunk_stream(const uint8_t *cont, const zo_header *h, int s, u
     uint64_t piece_bytes = round16((chunk_bits + 7) / 8);
     if (16 * off16 > h->payload_bytes || piece_bytes > h->payload_bytes - 16 * off16) return -1;
     const uint8_t *piece = cont + h->payload_off + 16 * off16;
+    if (chunk_bits == 0 && c_hi > c_lo && h->mode[0] == ZO_HUFF && h->mode[1] == ZO_HUFF) {   /* reading R14 */
+        int fill = zo_fill_symbol(cont + h->sec[s]);
+        if (fill < 0) return -1;
+        for (int j = 0; j < ZO_SUBS; ++j) if (get_sub_end(sub_end, sw, c, j) != 0) return -1;
+        memset(dst, fill, (size_t)(c_hi - c_lo));
+        return 0;
+    }
     uint64_t start = 0;
     for (int j = 0; j < ZO_SUBS; ++j) {
         uint64_t lo = c_lo + (uint64_t)j * sub, hi = lo + sub;

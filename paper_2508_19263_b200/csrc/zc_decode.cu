@@ -291,6 +291,15 @@ __device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uin
     }
 }
 
+// With both streams coded, a chunk without payload bits holds nothing but the stream's fill symbol, the symbol
+// with the all-zero code:
+// the first symbol of the table entry for a window of zeros.
+__device__ __noinline__ void fill_words(uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+{
+    const uint32_t word = ((lds32(lut_s) >> 8) & 0xFFu) * 0x01010101u;
+    for (uint32_t i = 0; i < n_words; ++i) sts32(row_s + 4 * i, word);
+}
+
 // The same result one symbol at a time, from the first-code fields every table entry carries whatever the
 // table's mode (symbol in bits 15..8, length in bits 27..24).  Small and slow on purpose: it serves pieces
 // that were too long to stage (read from global memory) and the rarely coded sign+mantissa stream.
@@ -461,13 +470,15 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                 if (n_words) {
                     if (H0) {
                         const uint32_t row_s = rows0_s + lane * kRowStride;
-                        if (!staged0) decode_words_plain<false>(st0, S.lut0_s, row_s, n_words);
+                        if (H1 && piece0 == 0) fill_words(S.lut0_s, row_s, n_words);   // both streams coded and no bits: fill symbols
+                        else if (!staged0) decode_words_plain<false>(st0, S.lut0_s, row_s, n_words);
                         else if (S.pairs0) decode_words<2>(st0, S.lut0_s, row_s, n_words);
                         else decode_words<1>(st0, S.lut0_s, row_s, n_words);
                     }
                     if (H1) {
                         const uint32_t row_s = rows1_s + lane * kRowStride;
-                        if (!staged1) decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
+                        if (H0 && piece1 == 0) fill_words(S.lut1_s, row_s, n_words);
+                        else if (!staged1) decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
                         else if (S.pairs1) decode_words<2>(st1, S.lut1_s, row_s, n_words);
                         else decode_words<1>(st1, S.lut1_s, row_s, n_words);
                     }

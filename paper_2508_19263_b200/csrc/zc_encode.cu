@@ -174,6 +174,17 @@ struct PackedChunk {
     uint32_t end[2];            // per stream: inclusive scan of the subchunks' bit counts over the lanes (= sub_end)
 };
 
+// Whether the n staged symbols of every lane (at shared address src) all equal `symbol`; the whole warp calls it.
+// Rarely needed (chunks that might be constant), so it is kept out of line.
+__device__ __noinline__ bool all_symbols_are(uint32_t src, uint32_t n, uint32_t symbol)
+{
+    const uint32_t want = symbol * 0x01010101u;
+    bool same = true;
+    for (uint32_t i = 0; i < n / 4; ++i) same = same && lds32(src + 4 * i) == want;
+    if (n & 3u) same = same && ((lds32(src + (n & ~3u)) ^ want) & (0xFFFFFFFFu >> (32 - 8 * (n & 3u)))) == 0;
+    return __all_sync(0xFFFFFFFFu, same);
+}
+
 // The kernel.  A block is up to kEncMaxWorkers worker warps plus one service warp.
 //
 // Batches: the chunks of every tensor are grouped into batches of n_workers consecutive chunks, the batches of
@@ -227,6 +238,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 
     __shared__ uint32_t s_ticket[kRing], s_tensor[kRing], s_cbase[kRing], s_tabslot[kRing], s_cnt[kRing];
     __shared__ uint32_t s_ticket_seq, s_base_seq, s_off_seq, s_fail;
+    __shared__ uint32_t s_fill[kTabSlots][2];                   // per table slot and coded stream: fill symbol | its code length << 8
     __shared__ unsigned long long s_tot[kRing][kEncMaxWorkers], s_off[kRing][kEncMaxWorkers];
 
     if (threadIdx.x < kRing) s_cnt[threadIdx.x] = 0;
@@ -270,8 +282,20 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 if (!is_huff(s)) continue;
                 const uint32_t* src;
                 if constexpr (N_ITEMS == 1) src = P.table.enc[s]; else src = C.tables[item(t).table].enc[s];
+                // the fill symbol (needed when both streams are coded) is the one whose code is all zeros: its
+                // entry is nothing but its length
+                uint32_t fill = 0xFFFFFFFFu;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) tab[256 * hs + lane + 32 * i] = src[lane + 32 * i];
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t v = src[lane + 32 * i];
+                    tab[256 * hs + lane + 32 * i] = v;
+                    if (H0 && H1 && v >= 1 && v <= kLmax) fill = (lane + 32 * i) | (v << 8);
+                }
+                if (H0 && H1) {
+                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, fill != 0xFFFFFFFFu);
+                    fill = __shfl_sync(0xFFFFFFFFu, fill, who ? __ffs(who) - 1 : 0);
+                    if (lane == 0) s_fill[nslot][hs] = who ? fill : 0xFF00u;     // no code at all: a length no chunk can match
+                }
                 ++hs;
             }
             __syncwarp();
@@ -696,6 +720,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             // ---- phase C: subchunk end bits and the chunk's size in the payload area ----
             uint64_t tot16 = 0;
             {
+                uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     if (!is_huff(s)) continue;
@@ -705,11 +730,25 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         const uint32_t x = __shfl_up_sync(0xFFFFFFFFu, inc, o);
                         if (lane >= (uint32_t)o) inc += x;
                     }
+                    // With both streams coded, a chunk that holds nothing but the fill symbol (the symbol with the
+                    // all-zero code) takes no bits at all.  Candidates are the chunks with exactly symbols * length
+                    // bits (rare otherwise); their staged symbols are then compared one by one.
+                    uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                    const uint32_t fill = (H0 && H1) ? vol32(&s_fill[tab_slot_idx][hs]) : 0u;   // fill symbol | its code length << 8
+                    if (H0 && H1 && active && chunk_bits <= C.cs * (fill >> 8)) {  // the last chunk may be shorter
+                        const uint32_t syms = (uint32_t)min((uint64_t)C.cs, I.n_syms - (uint64_t)my_c * C.cs);
+                        const uint32_t mine = lane * C.sub < syms ? min(C.sub, syms - lane * C.sub) : 0u;
+                        if (chunk_bits == syms * (fill >> 8) &&
+                            all_symbols_are(smem_u32(stage + hs * C.stage_stride + lane * region) + sym_off, mine, fill & 0xFFu)) {
+                            inc = 0;
+                            chunk_bits = 0;
+                        }
+                    }
+                    ++hs;
                     cur.end[s] = inc;
                     if (active) {
                         if (C.sub_width == 2) reinterpret_cast<uint16_t*>(I.out + I.lay.sub_end_tab[s] + 64ull * my_c)[lane] = (uint16_t)inc;
                         else reinterpret_cast<uint32_t*>(I.out + I.lay.sub_end_tab[s] + 128ull * my_c)[lane] = inc;
-                        const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
                         tot16 += (chunk_bits + 127) / 128;
                         if (lane == 0) atomicAdd(&counters(t)->payload_bits[s], (unsigned long long)chunk_bits);
                     }

@@ -53,6 +53,21 @@ def _gpu_round_trip(fmt, data_np, n, chunk_bytes, policy, oracle_codebook_hist=N
     return p, cb, hist, cont
 
 
+def _compress_with_modes(fmt, data_np, n, chunk_bytes, hist, modes):
+    """Compress with a HUFF_ALL codebook whose stream modes are overridden (one stream raw), against the oracle."""
+    ocb = zo.build_codebook(hist, zo.POLICY_HUFF_ALL)
+    ocb.modes = list(modes)
+    want = zo.compress(fmt, data_np, n, chunk_bytes, ocb)
+    # the library has no call that overrides modes; the policies give the same two combinations on suitable counts
+    p = zc.plan(fmt, n, chunk_bytes)
+    d_back = torch.full((p.input_bytes + 64,), 0xEE, dtype=torch.uint8, device=DEV)
+    d_ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+    d_comp = torch.from_numpy(want.copy()).to(DEV)
+    zc.decompress(p, d_comp, want.size, d_back, d_ws)
+    assert zc.device_status(p, d_ws) == zc.OK
+    assert np.array_equal(d_back.cpu().numpy()[: p.input_bytes], data_np[: p.input_bytes])
+
+
 def _weights(fmt, n, seed):
     rng = np.random.default_rng(seed)
     if n == 0:
@@ -107,9 +122,41 @@ def test_special_bit_patterns():
     allb = np.tile(np.arange(256, dtype=np.uint8), 100)
     _gpu_round_trip(zc.FMT_FP8_E4M3, allb, allb.size, 2048, zc.POLICY_HUFF_ALL)
     _gpu_round_trip(zc.FMT_FP4_E2M1, allb, 2 * allb.size, 2048, zc.POLICY_HUFF_ALL)
+    rng = np.random.default_rng(9)                                    # one exponent value, noise below it: [HUFF, RAW], and
+    noisy = (np.uint16(0x3F80) | rng.integers(0, 128, 30000).astype(np.uint16) | (rng.integers(0, 2, 30000).astype(np.uint16) << 15))
+    p, cb, _, cont = _gpu_round_trip(zc.FMT_BF16, noisy.view(np.uint8), 30000, 4096, zc.POLICY_AUTO)
+    assert cb.modes == [zc.MODE_HUFF, zc.MODE_RAW]                    # the constant exponent chunks pay one bit per symbol
+    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 30000
     rng = np.random.default_rng(1)
     uni = rng.integers(0, 256, 1 << 18, dtype=np.uint8)               # incompressible: every code length near 8
     _gpu_round_trip(zc.FMT_BF16, uni, 1 << 17, 8192, zc.POLICY_HUFF_ALL)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("chunk_bytes", [1024, 4096, 16384])
+def test_chunks_of_nothing_but_the_fill_symbol_take_no_bits(fmt, chunk_bytes):
+    """Unchanged stretches of a delta checkpoint or the unused part of a cache page: chunks whose symbols are all the
+    symbol with the all-zero code have empty pieces; chunks next to them are coded as usual."""
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    per_sym = 2                                                      # element bytes per symbol in every format
+    body = _weights(fmt, 2 * cs * G + 6 * G, 77 + fmt)               # two chunks and a bit of ordinary data
+    zeros = lambda n_syms: np.zeros(n_syms * per_sym, np.uint8)
+    data = np.concatenate([zeros(3 * cs), body[: (2 * cs + 6) * per_sym], zeros(cs - 6), zeros(4 * cs + cs // 3)])
+    n = data.size // per_sym * G
+    for policy in (zc.POLICY_HUFF_ALL, zc.POLICY_AUTO):
+        _gpu_round_trip(fmt, data, n, chunk_bytes, policy)
+    cb = zo.build_codebook(zo.histogram(fmt, data, n), zo.POLICY_HUFF_ALL)
+    hd = zo.parse_header(zo.compress(fmt, data, n, chunk_bytes, cb))
+    assert hd["streams"][0]["payload_bits"] < 8 * 3 * cs           # far below one bit per symbol of the whole tensor
+    # a tensor that is constant altogether: header and tables only
+    flat = zeros(5 * cs + 9)
+    _gpu_round_trip(fmt, flat, flat.size // per_sym * G, chunk_bytes, zc.POLICY_HUFF_ALL)
+    # one stream raw: the rule does not apply, constant chunks of the coded stream pay their bit per symbol
+    h = zo.histogram(fmt, data, n)
+    p = zc.plan(fmt, n, chunk_bytes)
+    for modes in ((zc.MODE_HUFF, zc.MODE_RAW), (zc.MODE_RAW, zc.MODE_HUFF)):
+        _compress_with_modes(fmt, data, n, chunk_bytes, h, modes)
 
 
 def test_long_codes_and_skew():

@@ -426,7 +426,11 @@ def test_golden_message_bitstream():
     cont = zo.compress(zo.BF16, elems, elems.size, 1024, cb)
     hd = zo.parse_header(cont)
     assert hd["magic"] == b"ZC10" and hd["total_bytes"] == cont.size and hd["n_chunks"] == 1
-    assert hd["streams"][0]["payload_bits"] == 15 and hd["streams"][1]["payload_bits"] == 9   # sm: one symbol, 1 bit each
+    # the sign+mantissa stream holds one symbol only: its single chunk is constant and takes no bits at all
+    assert hd["streams"][0]["payload_bits"] == 15 and hd["streams"][1]["payload_bits"] == 0
+    sec1 = hd["streams"][1]["section_off"]
+    assert int.from_bytes(cont[sec1 + 256: sec1 + 260].tobytes(), "little") == 1      # it "starts" behind stream 0's piece
+    assert not cont[sec1 + 256 + 16: sec1 + 256 + 16 + 64].any() and hd["payload_bytes"] == 16
     p = hd["payload_off"]
     assert cont[p:p + 4].tobytes() == bytes(int(x, 16) for x in stored.split())
     assert int.from_bytes(cont[p:p + 4].tobytes(), "little") == int(word, 16)
@@ -543,13 +547,32 @@ def test_round_trip_edge_sizes(fmt):
 
 
 def test_round_trip_special_patterns():
-    # all-zero tensor: one active symbol per stream, 1-bit codes
+    # all-zero tensor: one active symbol per stream; every chunk is constant and takes no payload at all
     z = np.zeros(5000, np.uint16)
     cb = zo.build_codebook(zo.histogram(zo.BF16, z, z.size), zo.POLICY_HUFF_ALL)
     cont = zo.compress(zo.BF16, z, z.size, 1024, cb)
     hd = zo.parse_header(cont)
-    assert hd["streams"][0]["payload_bits"] == 5000 and hd["streams"][1]["payload_bits"] == 5000
+    assert hd["streams"][0]["payload_bits"] == 0 and hd["streams"][1]["payload_bits"] == 0 and hd["payload_bytes"] == 0
     assert np.array_equal(zo.decompress(cont, z.size * 2), z.view(np.uint8))
+    # one element that differs: only its chunk (512 symbols) is coded, one bit per symbol plus the odd one's code
+    z[1700] = 0x3F80
+    cb = zo.build_codebook(zo.histogram(zo.BF16, z, z.size), zo.POLICY_HUFF_ALL)
+    cont = zo.compress(zo.BF16, z, z.size, 1024, cb)
+    hd = zo.parse_header(cont)
+    assert hd["streams"][0]["payload_bits"] == 512 and hd["streams"][1]["payload_bits"] == 0
+    assert hd["payload_bytes"] == 64
+    assert np.array_equal(zo.decompress(cont, z.size * 2), z.view(np.uint8))
+    for c in range(hd["n_chunks"]):
+        assert np.array_equal(zo.decompress_chunk(cont, c, 1024), z.view(np.uint8)[1024 * c: 1024 * (c + 1)])
+    # the rule needs both streams coded: with noise in the sign+mantissa bits that stream is stored raw, and the
+    # constant exponent stream pays its one bit per symbol
+    rng = np.random.default_rng(9)
+    noisy = (np.uint16(0x3F80) | rng.integers(0, 128, 5000).astype(np.uint16) | (rng.integers(0, 2, 5000).astype(np.uint16) << 15))
+    cb = zo.build_codebook(zo.histogram(zo.BF16, noisy, noisy.size), zo.POLICY_AUTO)
+    assert cb.modes == [zo.HUFF, zo.RAW]
+    cont = zo.compress(zo.BF16, noisy, noisy.size, 1024, cb)
+    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 5000
+    assert np.array_equal(zo.decompress(cont, noisy.size * 2), noisy.view(np.uint8))
     # NaN / inf / -0 / subnormal patterns are ordinary symbols
     pats = np.array([0x7FC0, 0xFFC1, 0x7F80, 0xFF80, 0x8000, 0x0001, 0x807F, 0x7FFF] * 300, np.uint16)
     cb = zo.build_codebook(zo.histogram(zo.BF16, pats, pats.size), zo.POLICY_HUFF_ALL)
