@@ -652,6 +652,24 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
             __syncwarp();
 
+            // Warm the L2 for the batch one round of tickets ahead (whichever block gets it; it may lie in one of
+            // the next tensors): the loads of phase A are the longest wait of a turn.  One 128-byte line per lane
+            // and 4 KiB of chunk.
+            {
+                uint32_t g2 = vol32(&s_ticket[it % kRing]) + gridDim.x, t2 = t;
+                if (N_ITEMS > 1)
+                    for (uint32_t hop = 0; hop < 4 && t2 + 1 < C.n_tensors && g2 >= P.item[N_ITEMS > 1 ? t2 + 1 : 0].first_batch; ++hop) ++t2;
+                const EncItem& I2 = item(t2);
+                const uint64_t c2 = (uint64_t)(g2 - I2.first_batch) * n_workers + warp;
+                if (g2 < C.total_batches && c2 < I2.n_chunks) {
+                    const uint64_t lo = c2 * C.chunk_bytes;
+                    for (uint32_t o = 128 * lane; o < C.chunk_bytes; o += 4096)
+                        if (lo + o < I2.input_bytes) {
+                            asm volatile("prefetch.global.L2 [%0];" :: "l"(I2.in + lo + o));
+                            if (I2.base) asm volatile("prefetch.global.L2 [%0];" :: "l"(I2.base + lo + o));
+                        }
+                }
+            }
 
             // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
             if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
