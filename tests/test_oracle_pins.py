@@ -137,7 +137,7 @@ def test_split_fields_rebuild_the_value_fp8_and_grouping():
         r = ref[sl]
         ok = ~np.isnan(r)
         assert np.array_equal(val[ok], r[ok])
-    # the survey's hand vector: bytes 7E 08 -> exponent symbol 0x1F, sign+mantissa symbol 0x06
+    # a hand vector: bytes 7E 08 -> exponent symbol 0x1F, sign+mantissa symbol 0x06
     e, sm = zo.split(zo.FP8_E4M3, np.array([0x7E, 0x08], np.uint8), 2)
     assert (int(e[0]), int(sm[0])) == (0x1F, 0x06)
 
