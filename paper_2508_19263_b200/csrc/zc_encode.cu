@@ -840,11 +840,13 @@ zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* ou
     // pack slots per lane region: first as many resident blocks of 8 worker warps per SM as possible (up to 3),
     // then as many slots (up to 3) as that number of blocks leaves room for
     s.n_slots = 1;
-    uint32_t best_blocks = 0;
+    uint32_t best_score = 0;
     for (uint32_t ns = 1; ns <= 3; ++ns) {
         const size_t block = fixed + (size_t)kEncMaxWorkers * std::max<uint32_t>(n_huff, 1) * kSubs * (ns * s.slot_bytes + p->syms_per_sub + 4);
         const uint32_t blocks = (uint32_t)std::min<size_t>((kMaxSmem + 1024) / (block + 2048 + 1024), 3);
-        if (blocks >= best_blocks && blocks > 0) { best_blocks = blocks; s.n_slots = ns; }
+        // a second slot is worth a resident block (with one slot every turn waits for its look-back), a third is not
+        const uint32_t score = blocks * std::min<uint32_t>(ns, 2) * 4 + ns;
+        if (blocks > 0 && score >= best_score) { best_score = score; s.n_slots = ns; }
     }
     s.region_bytes = s.n_slots * s.slot_bytes + p->syms_per_sub + 4;
     s.stage_stride = kSubs * s.region_bytes;
