@@ -10,6 +10,12 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # a fresh checkout has no built libraries (they are kept out of the history): build them once, in-tree
+    from paper_2508_19263_b200 import build as zbuild
+    if not os.path.exists(zbuild.LIB):
+        zbuild.build_library()
+    import oracle
+    oracle.build()
 
 
 def pytest_collection_modifyitems(config, items):
