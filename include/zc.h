@@ -290,7 +290,8 @@ zc_status zc_decompress_chunks(const zc_plan_t* plan, const void* d_comp, size_t
  * each (one launch per combination of stream modes that occurs and per 256 tensors of it).
  * n_tensors        number of tensors (0 returns ZC_OK and launches nothing)
  * plans            host array of n_tensors plans; all must have the same format and chunk_bytes
- * codebooks        host array, one codebook per tensor
+ * codebooks        host array, one codebook per tensor; tensors may share one (the pages of a K/V cache
+ *                  coded with one dictionary): its tables are then uploaded once
  * d_in             host array of DEVICE pointers (16-byte aligned): the tensors' element bytes
  * d_out            host array of DEVICE pointers (16-byte aligned): d_out[t] receives container t
  * out_capacity     host array: out_capacity[t] >= zc_max_compressed_bytes(plans[t])
