@@ -861,19 +861,12 @@ zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* ou
     return ZC_OK;
 }
 
-// Wide pack slots (12 bits per symbol) for code tables whose codes are long on average: with the symbol
-// probabilities the code lengths imply (2^-length), the expected length is above 6.5 bits.  Shorter codes get
-// slots of 8 bits per symbol and the slow path for the rare subchunk that needs more.
+// Wide pack slots (12 bits per symbol) for code tables whose codes are long on average (decided per stream when
+// the codebook is built).  Shorter codes get slots of 8 bits per symbol and the slow path for the rare subchunk
+// that needs more.
 bool wants_wide_slots(const zc_codebook_t* cb, const uint32_t mode[2])
 {
-    for (int s = 0; s < 2; ++s) {
-        if (mode[s] != ZC_MODE_HUFF) continue;
-        uint64_t acc = 0;                        // sum of length * 2^(12 - length)
-        for (int v = 0; v < 256; ++v)
-            if (cb->len[s][v]) acc += (uint64_t)cb->len[s][v] << (kLmax - cb->len[s][v]);
-        if (2 * acc > 13ull << kLmax) return true;
-    }
-    return false;
+    return (mode[0] == ZC_MODE_HUFF && cb->wide[0]) || (mode[1] == ZC_MODE_HUFF && cb->wide[1]);
 }
 
 void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const EncShape& sh)
@@ -903,9 +896,8 @@ void fill_item(EncItem& it, const zc_plan_t* p, const uint32_t mode[2], const vo
 
 void fill_tables(EncTables& T, const zc_codebook_t* cb)
 {
-    for (int s = 0; s < 2; ++s)
-        for (int v = 0; v < 256; ++v)
-            T.enc[s][v] = cb->len[s][v] ? (cb->code[s][v] << (32 - cb->len[s][v])) | cb->len[s][v] : 16u;
+    static_assert(sizeof(T.enc) == sizeof(cb->enc), "table layout");
+    std::memcpy(T.enc, cb->enc, sizeof(T.enc));
 }
 
 template <int N_ITEMS>

@@ -196,6 +196,7 @@ zc_status zc_build_codebook(const zc_plan_t* plan, const uint64_t* h_hist, zc_po
             mode = ZC_MODE_HUFF;
         cb->mode[s] = mode;
     }
+    finish_codebook(cb);
     *out = cb;
     return ZC_OK;
 }

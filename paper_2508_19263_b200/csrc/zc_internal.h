@@ -41,9 +41,27 @@ struct zc_codebook_s {
     uint32_t mode[2];
     uint8_t len[2][256];
     uint32_t code[2][256];     // right-aligned canonical code values
+    // derived once when the codebook is built, so that a compress call only copies them:
+    uint32_t enc[2][256];      // the encoder's table entry of every symbol: code << (32 - length) | length; 16: no code
+    uint8_t wide[2];           // the stream's codes are long on average: the encoder uses 12-bit pack slots
 };
 
 namespace zc {
+// Fills the derived fields of a codebook (call after len[] and code[] are final).
+// wide: with the symbol probabilities the code lengths imply (2^-length) the expected length is above 6.5 bits.
+inline void finish_codebook(zc_codebook_s* cb)
+{
+    for (int s = 0; s < 2; ++s) {
+        uint64_t acc = 0;                        // sum of length * 2^(12 - length)
+        for (int v = 0; v < 256; ++v) {
+            const uint32_t l = cb->len[s][v];
+            cb->enc[s][v] = l ? (cb->code[s][v] << (32 - l)) | l : 16u;
+            if (l) acc += (uint64_t)l << (12 - l);
+        }
+        cb->wide[s] = 2 * acc > (13ull << 12) ? 1 : 0;
+    }
+}
+
 
 // Bytes of one sub_end entry: chunks of at most 8 KiB hold fewer than 65536 bits, so 16 bits are enough.
 inline uint32_t sub_end_width(uint32_t chunk_bytes) { return chunk_bytes <= 8192 ? 2u : 4u; }
