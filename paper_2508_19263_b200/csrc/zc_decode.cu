@@ -918,10 +918,10 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         // tensor per block, so that their tables are built side by side
         const uint32_t want = std::max<uint32_t>({(uint32_t)((total + shape.warps - 1) / shape.warps), with_chunks, 1u});
         const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
-        // up to 8 ranges per block, none shorter than 16 chunks per warp (a range costs a table build), but not
-        // fewer than there are tensors as long as that stays within 8 per block
+        // up to 8 ranges per block, none shorter than 16 chunks per warp (a range costs a table build); with fewer
+        // tensors than blocks, one range per tensor at least
         B.n_ranges = grid * (uint32_t)std::min<uint64_t>(8, std::max<uint64_t>(1, total / ((uint64_t)grid * shape.warps * 16)));
-        B.n_ranges = std::max<uint32_t>(B.n_ranges, std::min<uint32_t>(with_chunks, 8 * grid));
+        if (with_chunks <= grid) B.n_ranges = std::max<uint32_t>(B.n_ranges, with_chunks);
         B.n_ranges = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(B.n_ranges, total));
         // the ranges are handed out through the ticket word of the control block
         if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
