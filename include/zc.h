@@ -302,6 +302,8 @@ zc_status zc_decompress_chunks(const zc_plan_t* plan, const void* d_comp, size_t
  *                  null the call is asynchronous (sizes are in the headers; status via
  *                  zc_batch_status)
  * The arrays are read before the call returns; the caller keeps ownership of everything.
+ * (Large sets of code tables travel through a pinned host staging buffer that the library keeps
+ * per calling thread; no device memory is allocated.)
  * Errors: INVALID_ARG (null or misaligned pointers, mixed formats or chunk sizes),
  * BUFFER_TOO_SMALL (an output or the workspace), UNSUPPORTED, CUDA, and the device status
  * (NO_CODE, DEVICE_TIMEOUT) when synchronous. */

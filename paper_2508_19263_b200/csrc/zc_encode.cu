@@ -942,6 +942,47 @@ BatchLayout batch_layout(uint32_t n_tensors, uint64_t total_batches)
     return L;
 }
 
+// Host-to-device copy of the code tables of a batched call.  A large copy from pageable memory holds the host
+// until the stream has drained, which would make an asynchronous call wait for the previous call's kernel; so
+// the tables go through a pinned staging buffer, one per calling thread, that is reused once the previous copy
+// out of it has been done (an event says so).  The buffer is never freed (a thread's last CUDA calls may come
+// after the runtime has shut down).  Without pinned memory the copy falls back to the pageable one.
+struct TableStage { void* ptr = nullptr; size_t cap = 0; cudaEvent_t done = nullptr; int device = -1; };
+
+cudaError_t upload_tables(void* d_dst, const void* h_src, size_t bytes, cudaStream_t st)
+{
+    static thread_local TableStage stage;
+    if (bytes <= 48 * 1024)                      // small copies leave the caller's memory at once anyway
+        return cudaMemcpyAsync(d_dst, h_src, bytes, cudaMemcpyHostToDevice, st);
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return cudaErrorUnknown;
+    if (stage.done) {
+        if (cudaEventSynchronize(stage.done) != cudaSuccess) return cudaErrorUnknown;
+        if (stage.device != device) { cudaEventDestroy(stage.done); stage.done = nullptr; }
+    }
+    if (stage.cap < bytes) {
+        if (stage.ptr) cudaFreeHost(stage.ptr);
+        stage.ptr = nullptr;
+        stage.cap = 0;
+        const size_t want = (size_t)round_up(bytes, 1u << 18);
+        if (cudaHostAlloc(&stage.ptr, want, cudaHostAllocPortable) == cudaSuccess) stage.cap = want;
+        else { stage.ptr = nullptr; (void)cudaGetLastError(); }
+    }
+    if (!stage.ptr) return cudaMemcpyAsync(d_dst, h_src, bytes, cudaMemcpyHostToDevice, st);
+    if (!stage.done) {
+        if (cudaEventCreateWithFlags(&stage.done, cudaEventDisableTiming) != cudaSuccess) {
+            stage.done = nullptr;
+            (void)cudaGetLastError();
+            return cudaMemcpyAsync(d_dst, h_src, bytes, cudaMemcpyHostToDevice, st);
+        }
+        stage.device = device;
+    }
+    std::memcpy(stage.ptr, h_src, bytes);
+    const cudaError_t e = cudaMemcpyAsync(d_dst, stage.ptr, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return e;
+    return cudaEventRecord(stage.done, st);
+}
+
 // Upper bound of the batches a tensor is cut into, whatever the modes of its streams turn out to be.
 uint64_t max_batches_of(const zc_plan_t* p)
 {
@@ -1065,8 +1106,7 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
         }
         table_of[t] = found->second;
     }
-    if (cudaMemcpyAsync(ws + L.tables, h_tables.data(), sizeof(EncTables) * h_tables.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return ZC_E_CUDA;
+    if (upload_tables(ws + L.tables, h_tables.data(), sizeof(EncTables) * h_tables.size(), st) != cudaSuccess) return ZC_E_CUDA;
 
     // one launch per combination of stream modes and slot size (the kernel's shared-memory layout depends on
     // them) and per kEncBatchMax tensors of it
