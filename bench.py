@@ -400,7 +400,9 @@ def run_ours(args):
             sel = [tensors[i] for i in idx]
             eb = zc.CompressBatch([t["plan"] for t in sel], [t["in"] for t in sel], [t["comp"] for t in sel],
                                   [t["base"] for t in sel] if delta else None)
-            step_groups.append({"idx": idx, "enc": eb, "ws": torch.empty(eb.workspace_bytes, dtype=torch.uint8, device=dev)})
+            hb = zc.HistogramBatch([t["plan"] for t in sel], [t["in"] for t in sel], [t["base"] for t in sel] if delta else None)
+            step_groups.append({"idx": idx, "enc": eb, "hist": hb, "ev": torch.cuda.Event(),
+                                "ws": torch.empty(eb.workspace_bytes, dtype=torch.uint8, device=dev)})
 
     def step():
         # histogram of every tensor, then codebook / compress / decompress per tensor: the host builds the
@@ -414,11 +416,18 @@ def run_ours(args):
                     raise SystemExit(f"dictionary {i % 2} no longer fits tensor {t['name']}")
             zc.decompress_batch(dec_batch, batch_ws, stream=stream)
             return
-        phase_hist()
         if args.batch:
+            # group by group: the counts of a group come back while the GPU counts the next one, and the host builds
+            # a group's codebooks while the GPU is still busy with histograms or with the group before
             hh = h_hist.numpy()
             for g in step_groups:
                 lo, hi = g["idx"][0], g["idx"][-1] + 1
+                zc.histogram_batch(g["hist"], d_hist[lo:hi], stream=stream)
+                h_hist[lo:hi].copy_(d_hist[lo:hi], non_blocking=True)
+                g["ev"].record(stream)
+            for g in step_groups:
+                lo, hi = g["idx"][0], g["idx"][-1] + 1
+                g["ev"].synchronize()
                 cbs = zc.build_codebooks([tensors[i]["plan"] for i in g["idx"]], hh[lo:hi], zc.POLICY_AUTO)
                 for i, cb in zip(g["idx"], cbs):
                     tensors[i]["cb"] = cb
@@ -426,6 +435,7 @@ def run_ours(args):
                 zc.compress_batch(g["enc"], g["ws"], sync=False, stream=stream)
             zc.decompress_batch(dec_batch, batch_ws, stream=stream)
             return
+        phase_hist()
         hh = h_hist.numpy()
         fork()
         for i, t in enumerate(tensors):
@@ -648,7 +658,8 @@ def run_ours(args):
                               "sign_mantissa_stream_payload": st_bits[1] / (8 * n_syms),
                               "paper_context": "abstract: up to 62% (BF16) / 83% (FP8) total"},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": ((n_enc_launch if static else n_hist_launch + n_enc_launch_step) + n_dec_launch) * args.steps,
+        "gpu_launches": ((n_enc_launch if static else (len(step_groups) if args.batch else n_hist_launch) + n_enc_launch_step)
+                         + n_dec_launch) * args.steps,
     }
     print(json.dumps(line))
     if dist is not None:
