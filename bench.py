@@ -396,7 +396,7 @@ def run_ours(args):
     # the step compresses in a few groups: the host builds the codebooks of the next group while the GPU encodes
     step_groups = []
     if args.batch and not static:
-        for idx in split_groups(max(1, min(4, n_t // 8))):
+        for idx in split_groups(max(1, min(4, n_t // 2))):
             sel = [tensors[i] for i in idx]
             eb = zc.CompressBatch([t["plan"] for t in sel], [t["in"] for t in sel], [t["comp"] for t in sel],
                                   [t["base"] for t in sel] if delta else None)
