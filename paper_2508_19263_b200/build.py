@@ -1,15 +1,22 @@
-"""Builds libzc.so (host logic + sm_100a kernels) in-tree with nvcc."""
+"""Builds libzc.so (host logic + sm_100a kernels) in-tree with nvcc.
+
+Every source is compiled to an object file of its own (in parallel, and only when it or a header is newer than
+its object), then the objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libzc.so")
+OBJDIR = os.path.join(HERE, "build")
 SOURCES = ["zc_host.cpp", "zc_hist.cu", "zc_encode.cu", "zc_decode.cu"]
 HEADERS = ["zc_internal.h", "zc_bits.cuh", "zc_device.cuh"]
+ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 
 def _nvcc() -> str:
@@ -19,28 +26,56 @@ def _nvcc() -> str:
     return "nvcc"
 
 
+def _header_time() -> float:
+    deps = [os.path.join(CSRC, f) for f in HEADERS]
+    deps += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE)]
+    return max(os.path.getmtime(d) for d in deps)
+
+
 def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
-    deps += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE)]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return _header_time() > t or any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def extra_flags() -> list:
+    """Extra compiler flags from the environment (ZC_NVCC_FLAGS, space separated), e.g. -DZC_DEBUG_CHECKS=1."""
+    return os.environ.get("ZC_NVCC_FLAGS", "").split()
+
+
+def build_library(force: bool = False, verbose: bool = False, lib: str = LIB, flags=None, objdir: str = OBJDIR) -> str:
     """Compile for sm_100a only.  Returns the path of the shared object."""
-    if not force and not is_stale():
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-I", INCLUDE, "-shared", "-Xcompiler", "-fPIC,-pthread", "-o", tmp]
+    flags = extra_flags() if flags is None else list(flags)
+    if lib == LIB and not flags and not force and not is_stale():
+        return lib
+    os.makedirs(objdir, exist_ok=True)
+    stamp = os.path.join(objdir, "flags.txt")
+    old_flags = open(stamp).read() if os.path.exists(stamp) else None
+    if old_flags != " ".join(flags):
+        force = True
+    hdr_t = _header_time()
+    common = [_nvcc(), *ARCH, "-lineinfo", "-O3", "-std=c++17", "-I", INCLUDE, "-Xcompiler", "-fPIC,-pthread", *flags]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, f) for f in SOURCES]
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+        common += ["-Xptxas", "-v"]
+
+    def compile_one(src: str) -> str:
+        path = os.path.join(CSRC, src)
+        obj = os.path.join(objdir, src + ".o")
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(path), hdr_t):
+            tmp = obj + f".tmp{os.getpid()}"
+            subprocess.check_call(common + ["-c", path, "-o", tmp])
+            os.replace(tmp, obj)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
+    with open(stamp, "w") as f:
+        f.write(" ".join(flags))
+    tmp = lib + f".tmp{os.getpid()}"
+    subprocess.check_call([_nvcc(), *ARCH, "-shared", "-Xcompiler", "-fPIC,-pthread", "-o", tmp] + objs)
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

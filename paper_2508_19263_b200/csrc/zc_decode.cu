@@ -89,8 +89,9 @@ __device__ __forceinline__ CodeBook codebook_views(uint32_t* scratch)
 }
 
 // Fills the table of one stream and decides how many symbols every lookup yields (returned in *per_lookup).
-//   entry bits  7..0  bits the lookup consumes      15..8 first symbol     23..16 second symbol
-//              27..24 length of the first code       31   "only the first symbol is valid" (2-symbol mode)
+//   two-symbol mode   entry bits  7..0  bits the lookup consumes      15..8 first symbol     23..16 second symbol
+//                                27..24 length of the first code       31   "only the first symbol is valid"
+//   one-symbol mode   entry bits  7..0  length of the code              31..24 the symbol
 // Two-symbol mode: a lookup normally yields the two symbols whose codes start the 12-bit window; when the two
 // codes together are longer than 12 bits the entry carries the first one and bit 31, and the decoder fetches
 // the second with one more lookup.  That mode is chosen when such pairs are rare (estimated from the code
@@ -171,8 +172,9 @@ __device__ bool build_lut(uint32_t my_len, uint32_t* lut, uint16_t* single, uint
     for (uint32_t idx = tid; idx < kLutEntries; idx += blockDim.x) {
         const uint32_t e1 = single[idx];
         const uint32_t l1 = e1 >> 8, s1 = e1 & 0xFF;
-        uint32_t e = l1 | (s1 << 8) | (l1 << 24);
+        uint32_t e = l1 | (s1 << 24);                             // one-symbol mode: length | symbol << 24
         if (mode == 2) {
+            e = l1 | (s1 << 8) | (l1 << 24);
             const uint32_t e2 = single[(idx << l1) & (kLutEntries - 1)];
             const uint32_t l2 = e2 >> 8, s2 = e2 & 0xFF;
             if (l1 + l2 <= kLmax) e = (l1 + l2) | (s1 << 8) | (s2 << 16) | (l1 << 24);
@@ -195,130 +197,137 @@ __device__ __forceinline__ uint32_t load_sub_end(const uint8_t* tab, uint32_t wi
     return reinterpret_cast<const uint32_t*>(tab + 128ull * chunk)[lane];
 }
 
-struct LaneStream {
-    uint32_t hi, lo;        // bit buffer: the next bit is the top bit of hi; bits below `valid` are zero
-    uint32_t valid;         // number of valid bits in the buffer
-    uint32_t ptr_s;         // shared address of the next payload word (piece staged in shared memory)
-    const uint32_t* ptr_g;  // or its global address (piece read from global memory)
-};
+// A lane's place in its chunk's piece is one number, the bit position `pos`.  Piece staged in shared memory: pos
+// counts from shared address 0 (8 * byte address of the slot + bit in the piece), so a window costs a shift, a mask,
+// two loads and a funnel shift, and nothing else has to be kept between lookups (no pointer, no count of valid
+// bits, no second buffer word).  Piece read from global memory: pos counts from the start of the piece and the
+// word index is clamped to `lim`, the last place from which two words can be read.
+// Bounds of the staged form: a lane starts inside its piece (checked against the tables before the chunk is
+// decoded) and consumes at most 12 bits per symbol, so it reads less than 1.5 * sub + 16 bytes past the piece
+// whatever the payload bits are; the block's shared memory ends with that much slack behind the last warp's
+// slot.  With a valid container a lane reads at most 16 bytes past its piece (covered by the copy); with a
+// damaged payload it decodes garbage in bounds and the consumed-bits check after the chunk reports the damage.
+constexpr uint32_t kPosMask = (1u << 21) - 1;            // bits of pos that hold the position (8 * 256 KiB)
 
-// Point the lane at bit `start` of the chunk's piece.
-template <bool STAGED>
-__device__ __forceinline__ void lane_begin(LaneStream& st, uint32_t pay_s, const uint32_t* __restrict__ pay_g, uint32_t start)
+__device__ __forceinline__ uint32_t window_s(uint32_t pos)
 {
-    const uint32_t w = start >> 5;
+    const uint32_t a = (pos >> 3) & (kPosMask >> 3 & ~3u);
     uint32_t w0, w1;
-    if (STAGED) { w0 = lds32(pay_s + 4 * w); w1 = lds32(pay_s + 4 * w + 4); st.ptr_s = pay_s + 4 * w + 8; }
-    else { w0 = __ldg(pay_g + w); w1 = __ldg(pay_g + w + 1); st.ptr_g = pay_g + w + 2; }
-    st.hi = __funnelshift_l(w1, w0, start);
-    st.lo = __funnelshift_l(0, w1, start);
-    st.valid = 64 - (start & 31);
+    asm volatile("ld.shared.u32 %0, [%2];\n\tld.shared.u32 %1, [%2+4];" : "=r"(w0), "=r"(w1) : "r"(a));
+    return __funnelshift_l(w1, w0, pos);                        // the shift takes the low 5 bits of pos
+}
+__device__ __forceinline__ uint32_t window_g(const uint32_t* __restrict__ pay, uint32_t pos, uint32_t lim)
+{
+    const uint32_t w = min((pos & kPosMask) >> 5, lim);
+    return __funnelshift_l(__ldg(pay + w + 1), __ldg(pay + w), pos);
+}
+__device__ __forceinline__ uint32_t lut_peek(uint32_t win, uint32_t lut_s)
+{
+    return lds32(lut_s + 4u * (win >> (32 - kLmax)));           // window = top 12 bits; scaled by the address add
+}
+// pos + low byte of x, in one multiply-add-like instruction off the integer ALU pipe
+__device__ __forceinline__ uint32_t add_low_byte(uint32_t pos, uint32_t x) { return __dp4a(x, 1u, pos); }
+
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
 }
 
-// Top the 64-bit buffer up with one word when 32 bits or fewer are left: at least 33 are valid afterwards,
-// enough for two lookups of at most 12 bits each.
-template <bool STAGED>
-__device__ __forceinline__ void lane_refill(LaneStream& st)
-{
-    const bool need = st.valid <= 32;
-    uint32_t word = 0;
-    if (STAGED) { if (need) word = lds32(st.ptr_s); st.ptr_s += need ? 4 : 0; }
-    else { if (need) word = __ldg(st.ptr_g); st.ptr_g += need ? 1 : 0; }
-    st.hi |= __funnelshift_rc(word, 0, st.valid);               // word >> valid (0 when valid == 32)
-    st.lo |= __funnelshift_rc(0, word, st.valid);               // word << (32 - valid)
-    st.valid += need ? 32 : 0;
-}
-
-__device__ __forceinline__ uint32_t lane_peek(const LaneStream& st, uint32_t lut_s)
-{
-    return lds32(lut_s + 4u * (st.hi >> (32 - kLmax)));         // window = top 12 bits; scaled by the address add
-}
-__device__ __forceinline__ void lane_consume(LaneStream& st, uint32_t n)    // n < 32 in its low 5 bits
-{
-    st.hi = __funnelshift_l(st.lo, st.hi, n);
-    st.lo = __funnelshift_l(0, st.lo, n);
-}
-
-// Decode n_words words of 4 symbols into the lane's row from a piece staged in shared memory.
-// K = symbols per lookup (1 or 2).
-// One-symbol mode: top up, two lookups, top up, two lookups.  Two-symbol mode: top up, two lookups; a lookup
-// whose second code did not fit the window (bit 31 of the entry, rare by construction of the mode) tops up
-// again and takes the second symbol from the next window.
+// Decode one word of 4 symbols from a piece staged in shared memory.  K = symbols per lookup (1 or 2).
+// A window of 32 bits serves two lookups of at most 12 bits each.
+// Two-symbol mode: entry = bits | first symbol << 8 | second symbol << 16 | first length << 24 | flag << 31.  A
+// lookup whose second code did not fit the window carries the flag (rare by construction of the mode) and
+// consumes its first code only, so the two lookups still end on a code boundary, one symbol short (two if both
+// carry the flag); the missing symbols come from a fresh window.
+// One-symbol mode: entry = length | symbol << 24, so that `pos += entry` advances the position and leaves the
+// symbol in bits the position does not use.
 template <int K>
-__device__ __forceinline__ void decode_words(LaneStream& st, uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+__device__ __forceinline__ uint32_t decode_word(uint32_t& pos, uint32_t lut_s)
 {
-    for (uint32_t i = 0; i < n_words; ++i) {
-        uint32_t word;
-        if (K == 2) {
-            lane_refill<true>(st);
-            uint32_t pair[2];
-            uint32_t used = 0;                                    // bits consumed since the last update of st.valid
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t e = lane_peek(st, lut_s);
-                lane_consume(st, e);
-                used += e;                                        // low byte = bits; the sum of two stays below 256
-                if ((int)e < 0) {
-                    st.valid -= used & 0xFF;
-                    used = 0;
-                    lane_refill<true>(st);
-                    const uint32_t f = lane_peek(st, lut_s);
-                    const uint32_t l = (f >> 24) & 15;
-                    lane_consume(st, l);
-                    st.valid -= l;
-                    e = (e & 0xFF00u) | ((f & 0xFF00u) << 8);
-                }
-                pair[h] = e;
+    uint32_t win = window_s(pos);
+    if (K == 2) {
+        const uint32_t e0 = lut_peek(win, lut_s);
+        const uint32_t e1 = lut_peek(__funnelshift_l(0, win, e0), lut_s);   // consume: low 5 bits of the entry
+        pos = add_low_byte(pos, e0 + e1);                        // the sum of two bit counts stays below 256
+        if ((int)(e0 | e1) < 0) {
+            win = window_s(pos);
+            const uint32_t f = lut_peek(win, lut_s), lf = (f >> 24) & 15;
+            pos += lf;
+            if ((int)(e0 & e1) < 0) {                            // both: first symbols of e0, e1, f and of one more lookup
+                const uint32_t g = lut_peek(__funnelshift_l(0, win, lf), lut_s);
+                pos += (g >> 24) & 15;
+                return __byte_perm(__byte_perm(e0, e1, 0x0051), __byte_perm(f, g, 0x0051), 0x5410);
             }
-            st.valid -= used & 0xFF;
-            word = __byte_perm(pair[0], pair[1], 0x6521);
-        } else {
-            lane_refill<true>(st);
-            const uint32_t a = lane_peek(st, lut_s);
-            lane_consume(st, a);
-            const uint32_t b = lane_peek(st, lut_s);
-            lane_consume(st, b);
-            st.valid -= (a + b) & 0xFF;
-            lane_refill<true>(st);
-            const uint32_t c = lane_peek(st, lut_s);
-            lane_consume(st, c);
-            const uint32_t d = lane_peek(st, lut_s);
-            lane_consume(st, d);
-            st.valid -= (c + d) & 0xFF;
-            word = __byte_perm(__byte_perm(a, b, 0x0051), __byte_perm(c, d, 0x0051), 0x5410);
+            // e0 short: e0's first, e1's two; e1 short: e0's two, e1's first; then f's first
+            return __byte_perm(__byte_perm(e0, e1, (int)e0 < 0 ? 0x0651 : 0x0521), f, 0x5210);
         }
-        sts32(row_s + 4 * i, word);
+        return __byte_perm(e0, e1, 0x6521);
+    }
+    const uint32_t a = lut_peek(win, lut_s);
+    const uint32_t b = lut_peek(__funnelshift_l(0, win, a), lut_s);
+    pos += a + b;
+    win = window_s(pos);
+    const uint32_t c = lut_peek(win, lut_s);
+    const uint32_t d = lut_peek(__funnelshift_l(0, win, c), lut_s);
+    pos += c + d;
+    return __byte_perm(__byte_perm(a, b, 0x0073), __byte_perm(c, d, 0x0073), 0x5410);
+}
+
+// Decoded symbols of a round, per coded stream and warp: lane L owns PPL quads (16 symbols = 16 bytes each);
+// its quad q lives in 16-byte slot L * PPL + (q ^ f(L)), f(L) = (L >> (3 - log2 PPL)) & (PPL - 1).  With this
+// placement both the writers (32 lanes, same q, one 16-byte store each) and the readers of the merge (lane l
+// reads quad l % PPL of row l / PPL + i * 32 / PPL) touch eight different 16-byte bank groups per quarter warp:
+// no bank conflicts on either side, one store per 16 symbols and one load per merged part.
+template <int K, int PPL, bool FULL>
+__device__ __forceinline__ void decode_round(uint32_t& pos, uint32_t lut_s, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
+{
+#pragma unroll
+    for (int q = 0; q < PPL; ++q) {
+        if (!FULL && (uint32_t)q >= n_quads) break;
+        const uint32_t w0 = decode_word<K>(pos, lut_s);
+        const uint32_t w1 = decode_word<K>(pos, lut_s);
+        const uint32_t w2 = decode_word<K>(pos, lut_s);
+        const uint32_t w3 = decode_word<K>(pos, lut_s);
+        sts128(wr_s + 16 * ((uint32_t)q ^ fw), w0, w1, w2, w3);
     }
 }
 
 // With both streams coded, a chunk without payload bits holds nothing but the stream's fill symbol, the symbol
-// with the all-zero code:
-// the first symbol of the table entry for a window of zeros.
-__device__ __noinline__ void fill_words(uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+// with the all-zero code: the first symbol of the table entry for a window of zeros.
+__device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
 {
-    const uint32_t word = ((lds32(lut_s) >> 8) & 0xFFu) * 0x01010101u;
-    for (uint32_t i = 0; i < n_words; ++i) sts32(row_s + 4 * i, word);
+    const uint32_t e = lds32(lut_s);
+    const uint32_t word = (pairs ? (e >> 8) & 0xFFu : e >> 24) * 0x01010101u;
+    for (uint32_t q = 0; q < n_quads; ++q) sts128(wr_s + 16 * (q ^ fw), word, word, word, word);
 }
 
-// The same result one symbol at a time, from the first-code fields every table entry carries whatever the
-// table's mode (symbol in bits 15..8, length in bits 27..24).  Small and slow on purpose: it serves pieces
-// that were too long to stage (read from global memory) and the rarely coded sign+mantissa stream.
-template <bool STAGED>
-__device__ __forceinline__ void decode_words_plain(LaneStream& st, uint32_t lut_s, uint32_t row_s, uint32_t n_words)
+// The same result as decode_round one symbol at a time, from the first code of every table entry (two-symbol
+// tables: symbol in bits 15..8, length in bits 27..24; one-symbol tables: symbol in bits 31..24, length in bits
+// 3..0), reading the piece from global memory.  Small and slow on purpose: it serves pieces that were too long
+// to stage.  Returns the new position.
+__device__ __noinline__ uint32_t decode_quads_global(uint32_t pos, const uint32_t* __restrict__ pay, uint32_t lut_s, uint32_t pairs,
+                                                     uint32_t wr_s, uint32_t fw, uint32_t n_quads, uint32_t lim)
 {
-    for (uint32_t i = 0; i < n_words; ++i) {
-        uint32_t word = 0;
+    for (uint32_t i = 0; i < 4 * n_quads; ++i) {
+        uint32_t word = 0, win = 0;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            if ((k & 1) == 0) lane_refill<STAGED>(st);
-            const uint32_t e = lane_peek(st, lut_s);
-            const uint32_t l = (e >> 24) & 15;
-            lane_consume(st, l);
-            st.valid -= l;
-            word |= ((e >> 8) & 0xFF) << (8 * k);
+            if ((k & 1) == 0) win = window_g(pay, pos, lim);
+            const uint32_t e = lut_peek(win, lut_s);
+            const uint32_t l = pairs ? (e >> 24) & 15 : e & 15, sy = pairs ? (e >> 8) & 0xFF : e >> 24;
+            win = __funnelshift_l(0, win, l);
+            pos += l;
+            word |= sy << (8 * k);
         }
-        sts32(row_s + 4 * i, word);
+        sts32(wr_s + 16 * ((i >> 2) ^ fw) + 4 * (i & 3), word);
     }
+    return pos;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -332,6 +341,8 @@ struct DecShared {                   // what the block's prologue leaves for the
     unsigned long long payload_off, payload_bytes;
 };
 
+template <bool V> struct BoolTag { static constexpr bool value = V; };
+
 // PPL = 16-symbol parts each lane merges per round = R / 16, R in {16, 32, 64}.
 template <int FMT, int PPL, bool H0, bool H1, bool XOR>
 __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShared& S, uint8_t* pool, uint64_t* bar,
@@ -340,8 +351,8 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                                                uint32_t& parity0, uint32_t& parity1)
 {
     constexpr uint32_t R = 16 * PPL;
-    constexpr uint32_t kRowStride = R + 4;                     // bytes; the padding spreads the lanes' rows over the banks
-    constexpr uint32_t kRowsBytes = 32 * kRowStride;           // one stream's rows of a warp (multiple of 16)
+    constexpr uint32_t kLog = PPL == 4 ? 2 : PPL == 2 ? 1 : 0;
+    constexpr uint32_t kRowsBytes = 512 * PPL;                 // one stream's decoded symbols of a warp and round
     constexpr uint32_t kHuff = (H0 ? 1u : 0u) + (H1 ? 1u : 0u);
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;
@@ -349,19 +360,28 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
     const uint8_t* sec0 = P.comp + S.sec0;
     const uint8_t* sec1 = P.comp + S.sec1;
     const uint8_t* payload = P.comp + S.payload_off;
+    const uint64_t payload16 = S.payload_bytes >> 4;
 
-    // pool: rows of stream 0 (if coded), rows of stream 1 (if coded), then one staging slot per coded stream
+    // pool: symbols of stream 0 (if coded), of stream 1 (if coded), then one staging slot per coded stream
     constexpr uint32_t rows1_off = H0 ? kRowsBytes : 0;
     constexpr uint32_t slots_off = rows1_off + (H1 ? kRowsBytes : 0);
     const uint32_t slot_room = P.pool_bytes > slots_off ? P.pool_bytes - slots_off : 0u;
     const uint32_t slot_bytes = kHuff ? (slot_room / (kHuff ? kHuff : 1)) & ~15u : 0u;
     const uint32_t rows0_s = smem_u32(pool), rows1_s = rows0_s + rows1_off;
     const uint32_t slot0_s = rows0_s + slots_off, slot1_s = slot0_s + (H0 ? slot_bytes : 0);
+    // where this lane writes its quads and reads the parts it merges (see decode_round)
+    const uint32_t fw = (lane >> (3 - kLog)) & (PPL - 1);
+    const uint32_t wr_off = 16 * PPL * lane;
+    const uint32_t rl = lane / PPL, rq = lane % PPL;
+    const uint32_t rd_off = 16 * (rl * PPL + (rq ^ ((rl >> (3 - kLog)) & (PPL - 1))));   // part i: + 512 * i
     uint32_t err = 0;
 
     // this lane's parts of a round: part i covers symbols k_lane + i * k_step (+ round offset) of the chunk
-    const uint32_t k_lane = (lane / PPL) * P.sub + (lane % PPL) * 16, k_step = (32 / PPL) * P.sub;
-    const uint32_t row_lane = (lane / PPL) * kRowStride + (lane % PPL) * 16, row_step = (32 / PPL) * kRowStride;
+    const uint32_t k_lane = rl * P.sub + rq * 16, k_step = (32 / PPL) * P.sub;
+    const uint32_t n_rounds = P.sub / R;
+    // every chunk but possibly the last one is complete
+    const uint32_t n_full = ((uint64_t)P.n_chunks * P.cs == P.n_syms && (uint64_t)P.n_chunks * P.chunk_bytes == P.input_bytes)
+                                ? P.n_chunks : P.n_chunks - 1;
 
     uint32_t nx_end0 = first_end0, nx_off0 = first_off0, nx_end1 = 0, nx_off1 = 0;
     if (H1 && c < c_end) {
@@ -370,42 +390,37 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
     }
 
     for (; c < c_end; c += step) {
-        const uint64_t c_lo = (uint64_t)c * P.cs;
-        const uint32_t c_syms = (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
-        const uint64_t out_lo = 2 * c_lo;                       // two element bytes per symbol in every format
-        const uint32_t out_bytes = (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - out_lo);
-        const uint32_t lo_sym = lane * P.sub;
-        const uint32_t n_my = lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u;
-
         // ---- where my subchunk starts and where the chunk's pieces are; check, then stage ----
-        LaneStream st0{0, 0, 0, 0, nullptr}, st1{0, 0, 0, 0, nullptr};
+        uint32_t pos0 = 0, pos1 = 0, lim0 = 0, lim1 = 0, end0 = 0, end1 = 0;
         uint32_t start0 = 0, start1 = 0, piece0 = 0, piece1 = 0;
         const uint32_t* pay0_g = nullptr;
         const uint32_t* pay1_g = nullptr;
         bool staged0 = false, staged1 = false, ok = true;
         if (H0) {
-            const uint32_t my_end = nx_end0, off16 = nx_off0;
-            start0 = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
+            const uint32_t off16 = nx_off0;
+            end0 = nx_end0;
+            start0 = __shfl_up_sync(0xFFFFFFFFu, end0, 1);
             if (lane == 0) start0 = 0;
-            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
+            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end0, 31);
             piece0 = ((chunk_bits + 127) / 128) * 16;
-            ok = ok && start0 <= my_end && my_end - start0 <= n_my * kLmax && 16ull * off16 + piece0 <= S.payload_bytes;
+            ok = ok && start0 <= end0 && end0 - start0 <= P.sub * kLmax && (uint64_t)off16 + piece0 / 16 <= payload16;
             pay0_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
         }
         if (H1) {
-            const uint32_t my_end = nx_end1, off16 = nx_off1;
-            start1 = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
+            const uint32_t off16 = nx_off1;
+            end1 = nx_end1;
+            start1 = __shfl_up_sync(0xFFFFFFFFu, end1, 1);
             if (lane == 0) start1 = 0;
-            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, my_end, 31);
+            const uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, end1, 31);
             piece1 = ((chunk_bits + 127) / 128) * 16;
-            ok = ok && start1 <= my_end && my_end - start1 <= n_my * kLmax && 16ull * off16 + piece1 <= S.payload_bytes;
+            ok = ok && start1 <= end1 && end1 - start1 <= P.sub * kLmax && (uint64_t)off16 + piece1 / 16 <= payload16;
             pay1_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
         }
         if (kHuff && !__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; break; }
         // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
         if (H0 && piece0 + 16 <= slot_bytes) {
             staged0 = true;
-            if (lane == 0) {
+            if (lane == 0 && !probe_skip(3)) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[0], piece0 + 16);
                 bulk_g2s(pool + slots_off, pay0_g, piece0 + 16, &bar[0]);
@@ -413,7 +428,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         }
         if (H1 && piece1 + 16 <= slot_bytes) {
             staged1 = true;
-            if (lane == 0) {
+            if (lane == 0 && !probe_skip(3)) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[1], piece1 + 16);
                 bulk_g2s(pool + slots_off + (H0 ? slot_bytes : 0), pay1_g, piece1 + 16, &bar[1]);
@@ -430,98 +445,120 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
             }
         }
 
-        const uint8_t* raw0 = sec0 + c_lo + k_lane;             // my first part's bytes in a raw stream
-        const uint8_t* raw1 = sec1 + c_lo + k_lane;
-        uint8_t* dst_lane = P.out + out_lo + 2 * k_lane;
-        const uint32_t n_rounds = P.sub / R;
-        bool waited = false;
-        for (uint32_t r = 0; r < n_rounds; ++r) {
-            if (r * R >= c_syms) break;                          // lane 0 has the most symbols; nothing left
-            // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
-            uint4 pre[PPL];
+        // ---- the chunk itself; FULL: a complete chunk, every lane has P.sub symbols ----
+        auto body = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
+            const uint64_t c_lo = (uint64_t)c * P.cs;
+            const uint32_t c_syms = FULL ? P.cs : (uint32_t)min((uint64_t)P.cs, P.n_syms - c_lo);
+            const uint32_t out_bytes = FULL ? P.chunk_bytes : (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - 2 * c_lo);
+            const uint32_t lo_sym = lane * P.sub;
+            const uint32_t n_my = FULL ? P.sub : (lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u);
+            const uint8_t* raw0 = sec0 + c_lo + k_lane;             // my first part's bytes in a raw stream
+            const uint8_t* raw1 = sec1 + c_lo + k_lane;
+            uint8_t* dst_lane = P.out + 2 * c_lo + 2 * k_lane;      // two element bytes per symbol in every format
+            for (uint32_t r = 0; r < n_rounds; ++r) {
+                if (!FULL && r * R >= c_syms) break;                // lane 0 has the most symbols; nothing left
+                // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
+                uint4 pre[PPL];
 #pragma unroll
-            for (int i = 0; i < PPL; ++i) {
-                pre[i] = make_uint4(0, 0, 0, 0);
-                if (!H1 && k_lane + i * k_step + r * R < c_syms) pre[i] = ld_nc_v4(raw1 + i * k_step + r * R);
-            }
-            if (kHuff && !waited) {
-                waited = true;
-                if (H0 && staged0) {
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait(&bar[0], parity0)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                    parity0 ^= 1;
+                for (int i = 0; i < PPL; ++i) {
+                    pre[i] = make_uint4(0, 0, 0, 0);
+                    if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms) && !probe_skip(2)) pre[i] = ld_nc_v4(raw1 + i * k_step + r * R);
                 }
-                if (H1 && staged1) {
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait(&bar[1], parity1)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                    parity1 ^= 1;
+                if (kHuff && r == 0) {
+                    if (H0 && staged0 && !probe_skip(3)) {
+                        uint32_t spins = 0;
+                        while (!mbar_try_wait(&bar[0], parity0)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                        parity0 ^= 1;
+                    }
+                    if (H1 && staged1 && !probe_skip(3)) {
+                        uint32_t spins = 0;
+                        while (!mbar_try_wait(&bar[1], parity1)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                        parity1 ^= 1;
+                    }
+                    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                    // staged: positions count from shared address 0; from global memory: from the piece, and the last
+                    // readable word pair ends with the guard (piece + 16 bytes)
+                    if (H0) { pos0 = staged0 ? 8 * slot0_s + start0 : start0; lim0 = piece0 / 4 + 2; }
+                    if (H1) { pos1 = staged1 ? 8 * slot1_s + start1 : start1; lim1 = piece1 / 4 + 2; }
                 }
-                if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                if (n_my) {
-                    if (H0) { if (staged0) lane_begin<true>(st0, slot0_s, nullptr, start0); else lane_begin<false>(st0, 0, pay0_g, start0); }
-                    if (H1) { if (staged1) lane_begin<true>(st1, slot1_s, nullptr, start1); else lane_begin<false>(st1, 0, pay1_g, start1); }
+                // ---- every lane decodes R symbols of its subchunk ----
+                if (kHuff) {
+                    const uint32_t done = r * R;
+                    // a ragged end decodes up to 15 symbols too many (from the bits that follow); they are not used
+                    const uint32_t n_quads = FULL ? (uint32_t)PPL : (n_my > done ? (min(R, n_my - done) + 15) / 16 : 0u);
+                    if (n_quads && !probe_skip(0)) {
+                        if (H0) {
+                            const uint32_t wr_s = rows0_s + wr_off;
+                            if (H1 && piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // both streams coded and no bits: fill symbols
+                            else if (!staged0) pos0 = decode_quads_global(pos0, pay0_g, S.lut0_s, S.pairs0, wr_s, fw, n_quads, lim0);
+                            else if (S.pairs0) decode_round<2, PPL, FULL>(pos0, S.lut0_s, wr_s, fw, n_quads);
+                            else decode_round<1, PPL, FULL>(pos0, S.lut0_s, wr_s, fw, n_quads);
+                        }
+                        if (H1) {
+                            const uint32_t wr_s = rows1_s + wr_off;
+                            if (H0 && piece1 == 0) fill_quads(S.lut1_s, S.pairs1, wr_s, fw, n_quads);
+                            else if (!staged1) pos1 = decode_quads_global(pos1, pay1_g, S.lut1_s, S.pairs1, wr_s, fw, n_quads, lim1);
+                            else if (S.pairs1) decode_round<2, PPL, FULL>(pos1, S.lut1_s, wr_s, fw, n_quads);
+                            else decode_round<1, PPL, FULL>(pos1, S.lut1_s, wr_s, fw, n_quads);
+                        }
+                    }
+                    __syncwarp();
                 }
-            }
-            // ---- every lane decodes R symbols of its subchunk ----
-            if (kHuff) {
-                const uint32_t done = r * R;
-                const uint32_t target = n_my > done ? min(R, n_my - done) : 0u;
-                const uint32_t n_words = (target + 3) / 4;      // a ragged last word decodes up to 3 symbols too many
-                if (n_words) {
+                // ---- cooperative merge: a part covers 16 symbols = 32 output bytes ----
+#pragma unroll
+                for (int i = 0; i < PPL; ++i) {
+                    const uint32_t k = k_lane + i * k_step + r * R;
+                    if ((!FULL && k >= c_syms) || probe_skip(1)) continue;
+                    uint32_t e[4], m[4];
                     if (H0) {
-                        const uint32_t row_s = rows0_s + lane * kRowStride;
-                        if (H1 && piece0 == 0) fill_words(S.lut0_s, row_s, n_words);   // both streams coded and no bits: fill symbols
-                        else if (!staged0) decode_words_plain<false>(st0, S.lut0_s, row_s, n_words);
-                        else if (S.pairs0) decode_words<2>(st0, S.lut0_s, row_s, n_words);
-                        else decode_words<1>(st0, S.lut0_s, row_s, n_words);
+                        const uint4 v = lds128(rows0_s + rd_off + 512 * i);
+                        e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
+                    } else {
+                        const uint4 v = ld_nc_v4(raw0 + i * k_step + r * R);
+                        e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
                     }
                     if (H1) {
-                        const uint32_t row_s = rows1_s + lane * kRowStride;
-                        if (H0 && piece1 == 0) fill_words(S.lut1_s, row_s, n_words);
-                        else if (!staged1) decode_words_plain<false>(st1, S.lut1_s, row_s, n_words);
-                        else if (S.pairs1) decode_words<2>(st1, S.lut1_s, row_s, n_words);
-                        else decode_words<1>(st1, S.lut1_s, row_s, n_words);
+                        const uint4 v = lds128(rows1_s + rd_off + 512 * i);
+                        m[0] = v.x; m[1] = v.y; m[2] = v.z; m[3] = v.w;
+                    } else { m[0] = pre[i].x; m[1] = pre[i].y; m[2] = pre[i].z; m[3] = pre[i].w; }
+                    uint32_t o[8];
+                    merge16<FMT>(e, m, o);
+                    merge16<FMT>(e + 2, m + 2, o + 4);
+                    uint8_t* dst = dst_lane + 2 * (i * k_step + r * R);
+                    if (XOR && P.base) {                              // delta form: XOR the base tensor back in
+                        const uint64_t off = (uint64_t)(dst - P.out);
+                        const uint4 b0 = load16_guarded(P.base, off, P.input_bytes), b1 = load16_guarded(P.base, off + 16, P.input_bytes);
+                        o[0] ^= b0.x; o[1] ^= b0.y; o[2] ^= b0.z; o[3] ^= b0.w;
+                        o[4] ^= b1.x; o[5] ^= b1.y; o[6] ^= b1.z; o[7] ^= b1.w;
+                    }
+                    if (FULL || 2 * k + 32 <= out_bytes) {
+                        st_cs_v8(dst, o);
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < 32; ++t)
+                            if (2 * k + t < out_bytes) dst[t] = (uint8_t)(o[t >> 2] >> (8 * (t & 3)));
                     }
                 }
-                __syncwarp();
+                if (kHuff) __syncwarp();
             }
-            // ---- cooperative merge: a part covers 16 symbols = 32 output bytes ----
-#pragma unroll
-            for (int i = 0; i < PPL; ++i) {
-                const uint32_t k = k_lane + i * k_step + r * R;
-                if (k >= c_syms) continue;
-                uint32_t e[4], m[4];
+            if (err) return;
+            // Every lane must have consumed exactly the bits of its subchunk (a ragged end decodes up to fifteen
+            // symbols too many).  Anything else means the payload does not belong to the tables.
+            if (kHuff) {
+                bool good = true;
                 if (H0) {
-                    const uint32_t a = rows0_s + row_lane + i * row_step;
-                    e[0] = lds32(a); e[1] = lds32(a + 4); e[2] = lds32(a + 8); e[3] = lds32(a + 12);
-                } else {
-                    const uint4 v = ld_nc_v4(raw0 + i * k_step + r * R);
-                    e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
+                    const uint32_t used = (pos0 & kPosMask) - (staged0 ? 8 * slot0_s : 0u);
+                    good = good && (FULL ? used == end0 : used - end0 <= 15 * kLmax);
                 }
                 if (H1) {
-                    const uint32_t a = rows1_s + row_lane + i * row_step;
-                    m[0] = lds32(a); m[1] = lds32(a + 4); m[2] = lds32(a + 8); m[3] = lds32(a + 12);
-                } else { m[0] = pre[i].x; m[1] = pre[i].y; m[2] = pre[i].z; m[3] = pre[i].w; }
-                uint32_t o[8];
-                merge16<FMT>(e, m, o);
-                merge16<FMT>(e + 2, m + 2, o + 4);
-                uint8_t* dst = dst_lane + 2 * (i * k_step + r * R);
-                if (XOR && P.base) {                              // delta form: XOR the base tensor back in
-                    const uint64_t off = (uint64_t)(dst - P.out);
-                    const uint4 b0 = load16_guarded(P.base, off, P.input_bytes), b1 = load16_guarded(P.base, off + 16, P.input_bytes);
-                    o[0] ^= b0.x; o[1] ^= b0.y; o[2] ^= b0.z; o[3] ^= b0.w;
-                    o[4] ^= b1.x; o[5] ^= b1.y; o[6] ^= b1.z; o[7] ^= b1.w;
+                    const uint32_t used = (pos1 & kPosMask) - (staged1 ? 8 * slot1_s : 0u);
+                    good = good && (FULL ? used == end1 : used - end1 <= 15 * kLmax);
                 }
-                if (2 * k + 32 <= out_bytes) {
-                    st_cs_v8(dst, o);
-                } else {
-#pragma unroll
-                    for (int t = 0; t < 32; ++t)
-                        if (2 * k + t < out_bytes) dst[t] = (uint8_t)(o[t >> 2] >> (8 * (t & 3)));
-                }
+                if (!__all_sync(0xFFFFFFFFu, good) && !probe_skip(0)) err = ZC_E_CORRUPT;
             }
-            if (kHuff) __syncwarp();
-        }
+        };
+        if (c < n_full) body(BoolTag<true>{}); else body(BoolTag<false>{});
         if (err) break;
     }
     if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) {
@@ -765,11 +802,13 @@ zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
     s.ppl = (p->syms_per_sub % 64 == 0) ? 4 : (p->syms_per_sub % 32 == 0) ? 2 : 1;
     // scale bytes and deltas have both streams coded as a rule, plain tensors one (the other one is raw)
     const uint32_t coded = (both_coded || p->format == ZC_FMT_SCALE_U8) ? 2 : 1;
-    const uint32_t rows_bytes = 32 * (16 * s.ppl + 4);
+    const uint32_t rows_bytes = 512 * s.ppl;
     // per warp: the coded streams' rows plus room to stage, per coded stream, a piece as large as the raw chunk
     // stream; pieces that do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
     s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32), 2 * rows_bytes);
-    const size_t fixed = kDecFixedSmem + 512 /* static shared */;
+    // slack behind the last slot: what a lane can read past its piece when the payload is damaged (see window_s)
+    const size_t slack = (size_t)round_up(p->syms_per_sub + p->syms_per_sub / 2 + 16, 16);
+    const size_t fixed = kDecFixedSmem + 512 /* static shared */ + slack;
     size_t per_warp = 16 + s.pool_bytes;
     s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     if (s.warps < 8) {               // large chunks: stage less
@@ -780,7 +819,7 @@ zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
     // the table build uses 8 KiB of the pools and 256 threads
     while (s.warps * (size_t)s.pool_bytes < 8192) ++s.warps;
     if (s.warps < 8 || s.warps > kDecMaxWarps) return ZC_E_UNSUPPORTED;
-    s.smem = kDecFixedSmem + s.warps * per_warp;
+    s.smem = kDecFixedSmem + s.warps * per_warp + slack;
     *out = s;
     return ZC_OK;
 }
@@ -925,6 +964,7 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         B.n_ranges = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(B.n_ranges, total));
         // the ranges are handed out through the ticket word of the control block
         if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
+        probe_upload(st);
         cudaError_t e = cudaSuccess;
         auto launch = [&](auto kern) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
