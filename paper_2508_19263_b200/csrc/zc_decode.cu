@@ -46,7 +46,7 @@ struct DecBatchParams {
 
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
 constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
-constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
+constexpr uint32_t kDecMaxWarps = 24;              // 768 threads: 85 registers per thread fit the register file
 constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
@@ -207,18 +207,34 @@ __device__ __forceinline__ uint32_t load_sub_end(const uint8_t* tab, uint32_t wi
 // whatever the payload bits are; the block's shared memory ends with that much slack behind the last warp's
 // slot.  With a valid container a lane reads at most 16 bytes past its piece (covered by the copy); with a
 // damaged payload it decodes garbage in bounds and the consumed-bits check after the chunk reports the damage.
-constexpr uint32_t kPosMask = (1u << 21) - 1;            // bits of pos that hold the position (8 * 256 KiB)
 
-__device__ __forceinline__ uint32_t window_s(uint32_t pos)
+// The two payload words a lane's windows come from, kept in registers between lookups: w0, w1 = the aligned
+// words that hold bits [32 i, 32 i + 64) of shared memory, next = 32 (i + 1), with i = pos / 32.  A lane consumes at
+// most 24 bits between two windows, so pos crosses at most one word boundary: then w1 moves to w0 and one word
+// is loaded (a predicated load in which only the lanes that crossed take part: about one word per 32 bits of
+// payload instead of two words per window).
+#define ZC_LANE_BITS uint32_t &pos, uint32_t &w0, uint32_t &w1, uint32_t &next
+#define ZC_LANE_ARGS pos, w0, w1, next
+
+__device__ __forceinline__ void lane_start(ZC_LANE_BITS, uint32_t at)
 {
-    const uint32_t a = (pos >> 3) & (kPosMask >> 3 & ~3u);
-    uint32_t w0, w1;
+    const uint32_t a = (at >> 3) & ~3u;
+    pos = at;
     asm volatile("ld.shared.u32 %0, [%2];\n\tld.shared.u32 %1, [%2+4];" : "=r"(w0), "=r"(w1) : "r"(a));
+    next = (at & ~31u) + 32;
+}
+__device__ __forceinline__ uint32_t window_s(ZC_LANE_BITS)
+{
+    const bool cross = pos >= next;
+    const uint32_t w2 = lds32_if(cross, (next >> 3) + 4);
+    w0 = cross ? w1 : w0;
+    w1 = cross ? w2 : w1;
+    next += cross ? 32u : 0u;
     return __funnelshift_l(w1, w0, pos);                        // the shift takes the low 5 bits of pos
 }
 __device__ __forceinline__ uint32_t window_g(const uint32_t* __restrict__ pay, uint32_t pos, uint32_t lim)
 {
-    const uint32_t w = min((pos & kPosMask) >> 5, lim);
+    const uint32_t w = min(pos >> 5, lim);
     return __funnelshift_l(__ldg(pay + w + 1), __ldg(pay + w), pos);
 }
 __device__ __forceinline__ uint32_t lut_peek(uint32_t win, uint32_t lut_s)
@@ -248,15 +264,15 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
 // One-symbol mode: entry = length | symbol << 24, so that `pos += entry` advances the position and leaves the
 // symbol in bits the position does not use.
 template <int K>
-__device__ __forceinline__ uint32_t decode_word(uint32_t& pos, uint32_t lut_s)
+__device__ __forceinline__ uint32_t decode_word(ZC_LANE_BITS, uint32_t lut_s)
 {
-    uint32_t win = window_s(pos);
+    uint32_t win = window_s(ZC_LANE_ARGS);
     if (K == 2) {
         const uint32_t e0 = lut_peek(win, lut_s);
         const uint32_t e1 = lut_peek(__funnelshift_l(0, win, e0), lut_s);   // consume: low 5 bits of the entry
-        pos = add_low_byte(pos, e0 + e1);                        // the sum of two bit counts stays below 256
+        pos = add_low_byte(pos, e0 + e1);                    // the sum of two bit counts stays below 256
         if ((int)(e0 | e1) < 0) {
-            win = window_s(pos);
+            win = window_s(ZC_LANE_ARGS);
             const uint32_t f = lut_peek(win, lut_s), lf = (f >> 24) & 15;
             pos += lf;
             if ((int)(e0 & e1) < 0) {                            // both: first symbols of e0, e1, f and of one more lookup
@@ -270,13 +286,13 @@ __device__ __forceinline__ uint32_t decode_word(uint32_t& pos, uint32_t lut_s)
         return __byte_perm(e0, e1, 0x6521);
     }
     const uint32_t a = lut_peek(win, lut_s);
-    const uint32_t b = lut_peek(__funnelshift_l(0, win, a), lut_s);
-    pos += a + b;
-    win = window_s(pos);
+    const uint32_t bb = lut_peek(__funnelshift_l(0, win, a), lut_s);
+    pos = add_low_byte(pos, a + bb);
+    win = window_s(ZC_LANE_ARGS);
     const uint32_t c = lut_peek(win, lut_s);
     const uint32_t d = lut_peek(__funnelshift_l(0, win, c), lut_s);
-    pos += c + d;
-    return __byte_perm(__byte_perm(a, b, 0x0073), __byte_perm(c, d, 0x0073), 0x5410);
+    pos = add_low_byte(pos, c + d);
+    return __byte_perm(__byte_perm(a, bb, 0x0073), __byte_perm(c, d, 0x0073), 0x5410);
 }
 
 // Decoded symbols of a round, per coded stream and warp: lane L owns PPL quads (16 symbols = 16 bytes each);
@@ -285,16 +301,16 @@ __device__ __forceinline__ uint32_t decode_word(uint32_t& pos, uint32_t lut_s)
 // reads quad l % PPL of row l / PPL + i * 32 / PPL) touch eight different 16-byte bank groups per quarter warp:
 // no bank conflicts on either side, one store per 16 symbols and one load per merged part.
 template <int K, int PPL, bool FULL>
-__device__ __forceinline__ void decode_round(uint32_t& pos, uint32_t lut_s, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
+__device__ __forceinline__ void decode_round(ZC_LANE_BITS, uint32_t lut_s, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
 {
 #pragma unroll
     for (int q = 0; q < PPL; ++q) {
         if (!FULL && (uint32_t)q >= n_quads) break;
-        const uint32_t w0 = decode_word<K>(pos, lut_s);
-        const uint32_t w1 = decode_word<K>(pos, lut_s);
-        const uint32_t w2 = decode_word<K>(pos, lut_s);
-        const uint32_t w3 = decode_word<K>(pos, lut_s);
-        sts128(wr_s + 16 * ((uint32_t)q ^ fw), w0, w1, w2, w3);
+        const uint32_t s0 = decode_word<K>(ZC_LANE_ARGS, lut_s);
+        const uint32_t s1 = decode_word<K>(ZC_LANE_ARGS, lut_s);
+        const uint32_t s2 = decode_word<K>(ZC_LANE_ARGS, lut_s);
+        const uint32_t s3 = decode_word<K>(ZC_LANE_ARGS, lut_s);
+        sts128(wr_s + 16 * ((uint32_t)q ^ fw), s0, s1, s2, s3);
     }
 }
 
@@ -389,13 +405,17 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[c];
     }
 
-    for (; c < c_end; c += step) {
-        // ---- where my subchunk starts and where the chunk's pieces are; check, then stage ----
-        uint32_t pos0 = 0, pos1 = 0, lim0 = 0, lim1 = 0, end0 = 0, end1 = 0;
-        uint32_t start0 = 0, start1 = 0, piece0 = 0, piece1 = 0;
-        const uint32_t* pay0_g = nullptr;
-        const uint32_t* pay1_g = nullptr;
-        bool staged0 = false, staged1 = false, ok = true;
+    // The pieces of one chunk at a time live in the warp's staging slots.  A chunk's pieces are requested as soon
+    // as the chunk before it has been decoded (the slots are free then), so the copy runs while that chunk is
+    // merged and written.  State of the chunk whose pieces are in the slots or on their way:
+    uint32_t end0 = 0, end1 = 0, start0 = 0, start1 = 0, piece0 = 0, piece1 = 0;
+    const uint32_t* pay0_g = nullptr;
+    const uint32_t* pay1_g = nullptr;
+    bool staged0 = false, staged1 = false, flying0 = false, flying1 = false;
+    // Takes the table entries in nx_* (of chunk `cc`), checks them, starts the copies, and requests the entries
+    // of the chunk after it.
+    auto prepare = [&](const uint32_t cc) {
+        bool ok = true;
         if (H0) {
             const uint32_t off16 = nx_off0;
             end0 = nx_end0;
@@ -416,36 +436,37 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
             ok = ok && start1 <= end1 && end1 - start1 <= P.sub * kLmax && (uint64_t)off16 + piece1 / 16 <= payload16;
             pay1_g = reinterpret_cast<const uint32_t*>(payload + 16ull * off16);
         }
-        if (kHuff && !__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; break; }
+        staged0 = staged1 = false;
+        if (kHuff && !__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; return; }
         // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
         if (H0 && piece0 + 16 <= slot_bytes) {
-            staged0 = true;
-            if (lane == 0 && !probe_skip(3)) {
+            staged0 = flying0 = true;
+            if (lane == 0) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[0], piece0 + 16);
                 bulk_g2s(pool + slots_off, pay0_g, piece0 + 16, &bar[0]);
             }
         }
         if (H1 && piece1 + 16 <= slot_bytes) {
-            staged1 = true;
-            if (lane == 0 && !probe_skip(3)) {
+            staged1 = flying1 = true;
+            if (lane == 0) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[1], piece1 + 16);
                 bulk_g2s(pool + slots_off + (H0 ? slot_bytes : 0), pay1_g, piece1 + 16, &bar[1]);
             }
         }
-        // request the next chunk's table entries now; they are consumed in the next iteration
-        {
-            const uint32_t cn = c + step;
-            if (cn < c_end) {
-                if (H0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
-                          nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
-                if (H1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
-                          nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[cn]; }
-            }
+        const uint32_t cn = cc + step;
+        if (cn < c_end) {
+            if (H0) { nx_end0 = load_sub_end(sec0 + tab_sub, sub_w, cn, lane);
+                      nx_off0 = reinterpret_cast<const uint32_t*>(sec0 + tab_chunk)[cn]; }
+            if (H1) { nx_end1 = load_sub_end(sec1 + tab_sub, sub_w, cn, lane);
+                      nx_off1 = reinterpret_cast<const uint32_t*>(sec1 + tab_chunk)[cn]; }
         }
+    };
+    if (c < c_end) prepare(c);
 
-        // ---- the chunk itself; FULL: a complete chunk, every lane has P.sub symbols ----
+    for (; c < c_end && !err; c += step) {
+        // ---- the chunk; FULL: a complete chunk, every lane has P.sub symbols ----
         auto body = [&](auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
             const uint64_t c_lo = (uint64_t)c * P.cs;
@@ -453,11 +474,13 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
             const uint32_t out_bytes = FULL ? P.chunk_bytes : (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - 2 * c_lo);
             const uint32_t lo_sym = lane * P.sub;
             const uint32_t n_my = FULL ? P.sub : (lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u);
+            const uint32_t last_r = FULL ? n_rounds - 1 : (c_syms - 1) / R;   // lane 0 has the most symbols
             const uint8_t* raw0 = sec0 + c_lo + k_lane;             // my first part's bytes in a raw stream
             const uint8_t* raw1 = sec1 + c_lo + k_lane;
             uint8_t* dst_lane = P.out + 2 * c_lo + 2 * k_lane;      // two element bytes per symbol in every format
-            for (uint32_t r = 0; r < n_rounds; ++r) {
-                if (!FULL && r * R >= c_syms) break;                // lane 0 has the most symbols; nothing left
+            uint32_t pos0 = 0, pos1 = 0, w00 = 0, w01 = 0, w10 = 0, w11 = 0, next0 = 0, next1 = 0;
+            uint32_t lim0 = 0, lim1 = 0;
+            for (uint32_t r = 0; r <= last_r; ++r) {
                 // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
                 uint4 pre[PPL];
 #pragma unroll
@@ -466,21 +489,18 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms) && !probe_skip(2)) pre[i] = ld_nc_v4(raw1 + i * k_step + r * R);
                 }
                 if (kHuff && r == 0) {
-                    if (H0 && staged0 && !probe_skip(3)) {
-                        uint32_t spins = 0;
-                        while (!mbar_try_wait(&bar[0], parity0)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                        parity0 ^= 1;
+                    if (H0 && staged0) {
+                        if (mbar_wait(&bar[0], parity0)) parity0 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
-                    if (H1 && staged1 && !probe_skip(3)) {
-                        uint32_t spins = 0;
-                        while (!mbar_try_wait(&bar[1], parity1)) if (++spins > kSpinLimit) { err = ZC_E_DEVICE_TIMEOUT; break; }
-                        parity1 ^= 1;
+                    if (H1 && staged1) {
+                        if (mbar_wait(&bar[1], parity1)) parity1 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
-                    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; break; }
+                    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; return; }
+                    flying0 = flying1 = false;
                     // staged: positions count from shared address 0; from global memory: from the piece, and the last
                     // readable word pair ends with the guard (piece + 16 bytes)
-                    if (H0) { pos0 = staged0 ? 8 * slot0_s + start0 : start0; lim0 = piece0 / 4 + 2; }
-                    if (H1) { pos1 = staged1 ? 8 * slot1_s + start1 : start1; lim1 = piece1 / 4 + 2; }
+                    if (H0) { if (staged0) lane_start(pos0, w00, w01, next0, 8 * slot0_s + start0); else pos0 = start0; lim0 = piece0 / 4 + 2; }
+                    if (H1) { if (staged1) lane_start(pos1, w10, w11, next1, 8 * slot1_s + start1); else pos1 = start1; lim1 = piece1 / 4 + 2; }
                 }
                 // ---- every lane decodes R symbols of its subchunk ----
                 if (kHuff) {
@@ -492,18 +512,34 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                             const uint32_t wr_s = rows0_s + wr_off;
                             if (H1 && piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // both streams coded and no bits: fill symbols
                             else if (!staged0) pos0 = decode_quads_global(pos0, pay0_g, S.lut0_s, S.pairs0, wr_s, fw, n_quads, lim0);
-                            else if (S.pairs0) decode_round<2, PPL, FULL>(pos0, S.lut0_s, wr_s, fw, n_quads);
-                            else decode_round<1, PPL, FULL>(pos0, S.lut0_s, wr_s, fw, n_quads);
+                            else if (S.pairs0) decode_round<2, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wr_s, fw, n_quads);
+                            else decode_round<1, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wr_s, fw, n_quads);
                         }
                         if (H1) {
                             const uint32_t wr_s = rows1_s + wr_off;
                             if (H0 && piece1 == 0) fill_quads(S.lut1_s, S.pairs1, wr_s, fw, n_quads);
                             else if (!staged1) pos1 = decode_quads_global(pos1, pay1_g, S.lut1_s, S.pairs1, wr_s, fw, n_quads, lim1);
-                            else if (S.pairs1) decode_round<2, PPL, FULL>(pos1, S.lut1_s, wr_s, fw, n_quads);
-                            else decode_round<1, PPL, FULL>(pos1, S.lut1_s, wr_s, fw, n_quads);
+                            else if (S.pairs1) decode_round<2, PPL, FULL>(pos1, w10, w11, next1, S.lut1_s, wr_s, fw, n_quads);
+                            else decode_round<1, PPL, FULL>(pos1, w10, w11, next1, S.lut1_s, wr_s, fw, n_quads);
                         }
                     }
                     __syncwarp();
+                    if (r == last_r) {
+                        // Every lane must have consumed exactly the bits of its subchunk (a ragged end decodes up to
+                        // fifteen symbols too many).  Anything else means the payload does not belong to the tables.
+                        bool good = true;
+                        if (H0) {
+                            const uint32_t used = pos0 - (staged0 ? 8 * slot0_s : 0u);
+                            good = good && (FULL ? used == end0 : used - end0 <= 15 * kLmax);
+                        }
+                        if (H1) {
+                            const uint32_t used = pos1 - (staged1 ? 8 * slot1_s : 0u);
+                            good = good && (FULL ? used == end1 : used - end1 <= 15 * kLmax);
+                        }
+                        if (!__all_sync(0xFFFFFFFFu, good) && !probe_skip(0)) err = ZC_E_CORRUPT;
+                        // the slots are free: the next chunk's pieces travel while this round is merged and written
+                        if (!err && c + step < c_end) prepare(c + step);
+                    }
                 }
                 // ---- cooperative merge: a part covers 16 symbols = 32 output bytes ----
 #pragma unroll
@@ -542,30 +578,12 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                 }
                 if (kHuff) __syncwarp();
             }
-            if (err) return;
-            // Every lane must have consumed exactly the bits of its subchunk (a ragged end decodes up to fifteen
-            // symbols too many).  Anything else means the payload does not belong to the tables.
-            if (kHuff) {
-                bool good = true;
-                if (H0) {
-                    const uint32_t used = (pos0 & kPosMask) - (staged0 ? 8 * slot0_s : 0u);
-                    good = good && (FULL ? used == end0 : used - end0 <= 15 * kLmax);
-                }
-                if (H1) {
-                    const uint32_t used = (pos1 & kPosMask) - (staged1 ? 8 * slot1_s : 0u);
-                    good = good && (FULL ? used == end1 : used - end1 <= 15 * kLmax);
-                }
-                if (!__all_sync(0xFFFFFFFFu, good) && !probe_skip(0)) err = ZC_E_CORRUPT;
-            }
         };
         if (c < n_full) body(BoolTag<true>{}); else body(BoolTag<false>{});
-        if (err) break;
     }
-    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) {
-        // give copies in flight one more bounded chance to land before the block leaves
-        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0 ^ 1); ++spins) {}
-        for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1 ^ 1); ++spins) {}
-    }
+    // a copy that was started and not waited for (the loop ended early) must land before the block may leave
+    if (flying0) for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0); ++spins) {}
+    if (flying1) for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1); ++spins) {}
     return err;
 }
 

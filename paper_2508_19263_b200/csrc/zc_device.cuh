@@ -99,6 +99,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+// Bounded wait for a phase of an mbarrier; false when the wait gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    for (uint32_t spins = 0; spins <= kSpinLimit; ++spins)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
 // Bulk asynchronous copy global -> shared of this CTA, completion counted in bytes on an mbarrier.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
 {
