@@ -46,7 +46,7 @@ struct DecBatchParams {
 
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
 constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
-constexpr uint32_t kDecMaxWarps = 24;              // 768 threads: 85 registers per thread fit the register file
+constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
 constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
@@ -482,12 +482,10 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
             uint32_t lim0 = 0, lim1 = 0;
             for (uint32_t r = 0; r <= last_r; ++r) {
                 // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
-                uint4 pre[PPL];
 #pragma unroll
-                for (int i = 0; i < PPL; ++i) {
-                    pre[i] = make_uint4(0, 0, 0, 0);
-                    if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms) && !probe_skip(2)) pre[i] = ld_nc_v4(raw1 + i * k_step + r * R);
-                }
+                for (int i = 0; i < PPL; ++i)
+                    if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms) && !probe_skip(2))
+                        asm volatile("prefetch.global.L2 [%0];" :: "l"(raw1 + i * k_step + r * R));
                 if (kHuff && r == 0) {
                     if (H0 && staged0) {
                         if (mbar_wait(&bar[0], parity0)) parity0 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
@@ -557,7 +555,10 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     if (H1) {
                         const uint4 v = lds128(rows1_s + rd_off + 512 * i);
                         m[0] = v.x; m[1] = v.y; m[2] = v.z; m[3] = v.w;
-                    } else { m[0] = pre[i].x; m[1] = pre[i].y; m[2] = pre[i].z; m[3] = pre[i].w; }
+                    } else {
+                        const uint4 v = ld_nc_v4(raw1 + i * k_step + r * R);
+                        m[0] = v.x; m[1] = v.y; m[2] = v.z; m[3] = v.w;
+                    }
                     uint32_t o[8];
                     merge16<FMT>(e, m, o);
                     merge16<FMT>(e + 2, m + 2, o + 4);
