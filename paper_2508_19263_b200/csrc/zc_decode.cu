@@ -474,7 +474,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
             const uint32_t out_bytes = FULL ? P.chunk_bytes : (uint32_t)min((uint64_t)P.chunk_bytes, P.input_bytes - 2 * c_lo);
             const uint32_t lo_sym = lane * P.sub;
             const uint32_t n_my = FULL ? P.sub : (lo_sym < c_syms ? min(P.sub, c_syms - lo_sym) : 0u);
-            const uint32_t last_r = FULL ? n_rounds - 1 : (c_syms - 1) / R;   // lane 0 has the most symbols
+            const uint32_t last_r = FULL ? n_rounds - 1 : (min(c_syms, P.sub) - 1) / R;   // lane 0 has the most symbols
             const uint8_t* raw0 = sec0 + c_lo + k_lane;             // my first part's bytes in a raw stream
             const uint8_t* raw1 = sec1 + c_lo + k_lane;
             uint8_t* dst_lane = P.out + 2 * c_lo + 2 * k_lane;      // two element bytes per symbol in every format

@@ -166,6 +166,7 @@ constexpr uint32_t kRing = 8;                // batches of a block whose bookkee
 constexpr uint32_t kTabSlots = 4;            // code tables (of the tensors the last batches belong to) alive at the same time
 constexpr uint32_t kNoTensor = 0xFFFFFFFFu;  // "no more batches"
 constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
+constexpr int kLookWide = 8;                 // look-back rounds cover 32 * kLookWide predecessors
 
 // What a worker warp keeps about a chunk between packing it and copying it out.
 struct PackedChunk {
@@ -339,21 +340,35 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 if (lb_on) {
                     bool done = !n_huff || lb_b == 0;
                     if (!done) {
-                        // one round of the look-back: 32 predecessors at a time, newest first, up to the first
-                        // one that already knows its prefix
-                        const long long idx = lb_base - lane;
-                        unsigned long long f = kFlagPrefix;      // before batch 0: prefix 0
-                        if (idx >= 0) f = ld_flag(&lb_flags[idx]);
-                        const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (f >> 62) != 0);
-                        const uint32_t prefix = __ballot_sync(0xFFFFFFFFu, (f >> 62) == 2);
-                        const uint32_t first_prefix = prefix ? (uint32_t)__ffs(prefix) - 1 : 32u;
-                        const uint32_t need = first_prefix == 32 ? 0xFFFFFFFFu : (0xFFFFFFFFu >> (31 - first_prefix));
-                        if ((ready & need) == need) {
-                            unsigned long long x = (lane <= first_prefix || first_prefix == 32) ? (f & kFlagValue) : 0;
+                        // One round of the look-back: kLookWide * 32 predecessors at a time, newest first, up to the
+                        // first one that already knows its prefix.  All loads of a round are in flight together, so a
+                        // round costs one trip to the L2 however wide it is; it has to be wider than the number of
+                        // batches in flight (one per resident block), or the prefixes of a turn form a chain of
+                        // rounds from block to block.
+                        unsigned long long f[kLookWide];
+#pragma unroll
+                        for (int k = 0; k < kLookWide; ++k) {
+                            const long long idx = lb_base - 32 * k - lane;
+                            f[k] = idx >= 0 ? ld_flag(&lb_flags[idx]) : kFlagPrefix;      // before batch 0: prefix 0
+                        }
+                        unsigned long long x = 0;
+                        bool found = false, stuck = false;
+#pragma unroll
+                        for (int k = 0; k < kLookWide; ++k) {
+                            if (found || stuck) continue;
+                            const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (f[k] >> 62) != 0);
+                            const uint32_t prefix = __ballot_sync(0xFFFFFFFFu, (f[k] >> 62) == 2);
+                            const uint32_t first_prefix = prefix ? (uint32_t)__ffs(prefix) - 1 : 32u;
+                            const uint32_t need = first_prefix == 32 ? 0xFFFFFFFFu : (0xFFFFFFFFu >> (31 - first_prefix));
+                            if ((ready & need) != need) { stuck = true; continue; }
+                            if (lane <= first_prefix || first_prefix == 32) x += f[k] & kFlagValue;
+                            found = first_prefix != 32;
+                        }
+                        if (!stuck) {
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
                             lb_sum += x;
-                            if (first_prefix != 32) done = true; else lb_base -= 32;
+                            if (found) done = true; else lb_base -= 32 * kLookWide;
                             did = true;
                         }
                     }
@@ -563,7 +578,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 pc.end[1] = n_pend == 1 ? q0.end[1] : n_pend == 2 ? q1.end[1] : q2.end[1];
                 // its slot: the slots are used round-robin, so it lies n_pend steps behind the current one
                 const uint32_t sl = (slot_idx + n_slots * 4 - n_pend) % n_slots;
-                if (pc.c != kNoChunk)
+                if (pc.c != kNoChunk && !probe_skip(10))
                     copy_out(pc, sl * C.slot_bytes, *reinterpret_cast<const volatile unsigned long long*>(&s_off[j % kRing][warp]));
             }
             --n_pend;
@@ -617,7 +632,8 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             uint32_t g = lane;
             uint32_t off = stage_off(lane);                             // running offset (constant-step case)
             auto off_at = [&](const uint32_t g_, const uint32_t i) { return step ? off + i * step : stage_off(g_); };
-            if (I.base) {
+            if (probe_skip(8)) {
+            } else if (I.base) {
                 // delta form: the chunk of the base tensor is read alongside and XOR-ed in (two pairs of loads in flight)
                 const uint8_t* base_c = I.base + 2 * c_lo;
                 auto x4 = [](const uint4 a, const uint4 b) { return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w); };
@@ -652,6 +668,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
             __syncwarp();
 
+            if (!probe_skip(11))
             // Warm the L2 for the batch one round of tickets ahead (whichever block gets it; it may lie in one of
             // the next tensors): the loads of phase A are the longest wait of a turn.  One 128-byte line per lane
             // and 4 KiB of chunk.
@@ -724,7 +741,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 for (int s = 0; s < 2; ++s) {
                     if (!is_huff(s)) continue;
                     // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
-                    my_bits[s] = pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
+                    my_bits[s] = probe_skip(9) ? 100u : pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
                     // more than the slot holds: the bits beyond it do not survive the next staging
                     oversize |= my_bits[s] > 8 * C.slot_bytes;
                     ++hs;
@@ -903,6 +920,7 @@ void fill_tables(EncTables& T, const zc_codebook_t* cb)
 template <int N_ITEMS>
 cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const EncShape& sh, cudaStream_t st)
 {
+    probe_upload(st);
     const uint32_t want = std::max<uint32_t>(P.c.total_batches, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * sh.per_sm);
     cudaError_t e = cudaSuccess;
