@@ -15,7 +15,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libzc.so")
 OBJDIR = os.path.join(HERE, "build")
 SOURCES = ["zc_host.cpp", "zc_hist.cu", "zc_encode.cu", "zc_decode.cu"]
-HEADERS = ["zc_internal.h", "zc_bits.cuh", "zc_device.cuh"]
+HEADERS = ["zc_internal.h", "zc_bits.cuh", "zc_device.cuh", "zc_encode_rows.cuh"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

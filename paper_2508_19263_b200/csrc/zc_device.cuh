@@ -126,7 +126,26 @@ inline void probe_upload(cudaStream_t st)
     const uint32_t v = e ? (uint32_t)strtoul(e, nullptr, 0) : 0u;
     cudaMemcpyToSymbolAsync(g_probe_bits, &v, sizeof(v), 0, cudaMemcpyHostToDevice, st);
 }
+// cycle counters a kernel adds up (slot k: sum, slot 32 + k: number of samples)
+static __device__ unsigned long long g_probe_stats[64];
+__device__ __forceinline__ long long probe_clock() { return clock64(); }
+struct ProbeAcc {
+    long long sum[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    uint32_t n[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    __device__ __forceinline__ void add(int k, long long v) { sum[k] += v; ++n[k]; }
+    __device__ __forceinline__ void flush()
+    {
+#pragma unroll
+        for (int k = 0; k < 10; ++k)
+            if (n[k]) { atomicAdd(&g_probe_stats[k], (unsigned long long)sum[k]); atomicAdd(&g_probe_stats[32 + k], (unsigned long long)n[k]); }
+    }
+};
 #else
+__device__ __forceinline__ long long probe_clock() { return 0; }
+struct ProbeAcc {
+    __device__ __forceinline__ void add(int, long long) {}
+    __device__ __forceinline__ void flush() {}
+};
 __device__ __forceinline__ constexpr bool probe_skip(uint32_t) { return false; }
 inline void probe_upload(cudaStream_t) {}
 #endif

@@ -166,7 +166,7 @@ constexpr uint32_t kRing = 8;                // batches of a block whose bookkee
 constexpr uint32_t kTabSlots = 4;            // code tables (of the tensors the last batches belong to) alive at the same time
 constexpr uint32_t kNoTensor = 0xFFFFFFFFu;  // "no more batches"
 constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
-constexpr int kLookWide = 8;                 // look-back rounds cover 32 * kLookWide predecessors
+constexpr int kLookWide = 1;                 // look-back rounds cover 32 * kLookWide predecessors
 
 // What a worker warp keeps about a chunk between packing it and copying it out.
 struct PackedChunk {
@@ -242,6 +242,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
     __shared__ uint32_t s_fill[kTabSlots][2];                   // per table slot and coded stream: fill symbol | its code length << 8
     __shared__ unsigned long long s_tot[kRing][kEncMaxWorkers], s_off[kRing][kEncMaxWorkers];
 
+    ProbeAcc pr;
     if (threadIdx.x < kRing) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) {
         s_fail = 0; s_off_seq = 0; s_base_seq = 0;
@@ -270,6 +271,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         long long lb_base = 0;
         unsigned long long* lb_flags = nullptr;
         uint32_t lb_b = 0, idle = 0;
+        long long pr_t0 = 0, pr_last = 0, pr_polls = 0;
         // Loads tensor t's code tables into the slot after the newest one, once every worker has posted the last
         // batch that was packed with the table that is there now; false when that is not yet the case.
         auto load_next_slot = [&](const uint32_t t, const uint32_t placed_now) -> bool {
@@ -318,6 +320,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             if (placed < real) {
                 const uint32_t r = placed % kRing;
                 if (!lb_on && vol32(&s_cnt[r]) == n_workers) {   // every worker has posted a size (0 without a chunk)
+                    pr_t0 = probe_clock();
                     __threadfence_block();
                     if (lane == 0) s_cnt[r] = 0;
                     lb_v = lane < n_workers ? *reinterpret_cast<const volatile unsigned long long*>(&s_tot[r][lane]) : 0ull;
@@ -339,6 +342,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 }
                 if (lb_on) {
                     bool done = !n_huff || lb_b == 0;
+                    ++pr_polls;
                     if (!done) {
                         // One round of the look-back: kLookWide * 32 predecessors at a time, newest first, up to the
                         // first one that already knows its prefix.  All loads of a round are in flight together, so a
@@ -378,6 +382,8 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         __threadfence_block();
                         __syncwarp();
                         if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = placed + 1;
+                        if (lane == 0) { const long long now = probe_clock(); pr.add(0, now - pr_t0); pr.add(1, pr_polls); if (pr_last) pr.add(2, now - pr_last); pr_last = now; }
+                        pr_polls = 0;
                         ++placed;
                         lb_on = false;
                         did = true;
@@ -466,12 +472,16 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         // Chunks this warp has completely written, per tensor; added to the tensor's counter (behind a fence)
         // when the warp moves on to another tensor or leaves.  Whoever completes a tensor writes its header.
         uint32_t acc_t = kNoTensor, acc_n = 0;
+        unsigned long long acc_bits0 = 0, acc_bits1 = 0;           // lane 0: payload bits of those chunks, per stream
         auto flush_acc = [&]() {
             if (acc_n == 0) return;
             __threadfence();
             __syncwarp();
             if (lane == 0) {
                 TensorCounters* tc = counters(acc_t);
+                if (H0) atomicAdd(&tc->payload_bits[0], acc_bits0);
+                if (H1) atomicAdd(&tc->payload_bits[1], acc_bits1);
+                __threadfence();
                 const uint32_t before = atomicAdd(&tc->done, acc_n);
                 if (before + acc_n == item(acc_t).n_chunks) {
                     __threadfence();
@@ -479,10 +489,12 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 }
             }
             acc_n = 0;
+            acc_bits0 = acc_bits1 = 0;
         };
-        auto chunk_done = [&](const uint32_t t) {
+        auto chunk_done = [&](const uint32_t t, const uint32_t bits0, const uint32_t bits1) {
             if (t != acc_t) { flush_acc(); acc_t = t; }
             ++acc_n;
+            acc_bits0 += bits0; acc_bits1 += bits1;
         };
 
         // ---- copy-out of a packed chunk: every lane moves its bits to their final position in the piece ----
@@ -558,7 +570,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             // the warp that owns the last chunk knows the size of the whole payload area
             if (lane == 0 && pc.c == I.n_chunks - 1) counters(pc.t)->total16 = piece_off16;
             __syncwarp();
-            chunk_done(pc.t);
+            chunk_done(pc.t, H0 ? __shfl_sync(0xFFFFFFFFu, pc.end[0], 31) : 0u, H1 ? __shfl_sync(0xFFFFFFFFu, pc.end[1], 31) : 0u);
         };
 
         uint32_t bad = 0;                                           // 1 + tensor in which a symbol had no code
@@ -569,7 +581,9 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         // waits until the oldest pending batch is placed and copies this warp's chunk of it out
         auto flush_oldest = [&](const uint32_t it) -> bool {
             const uint32_t j = it - n_pend;                         // the batch in question
+            const long long pr_w = probe_clock();
             if (!wait_seq(&s_off_seq, j + 1)) return false;
+            if (lane == 0) pr.add(9, probe_clock() - pr_w);       // of which: waiting for the placement
             if (n_huff) {
                 PackedChunk pc;
                 pc.c = n_pend == 1 ? q0.c : n_pend == 2 ? q1.c : q2.c;
@@ -586,7 +600,10 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         };
         bool failed = false;
         for (uint32_t it = 0;; ++it) {
+            const long long pr_a = probe_clock();
             if (!wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
+            const long long pr_b = probe_clock();
+            if (lane == 0) pr.add(4, pr_b - pr_a);
             const uint32_t t = vol32(&s_tensor[it % kRing]);
             if (t == kNoTensor) {
                 while (n_pend && !failed) failed = !flush_oldest(it);
@@ -689,7 +706,11 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
 
             // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
+            const long long pr_c = probe_clock();
+            if (lane == 0) pr.add(5, pr_c - pr_b);                // phase A
             if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
+            const long long pr_d = probe_clock();
+            if (lane == 0) pr.add(6, pr_d - pr_c);                // wait for the placement + copy-out
 
             // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
             const uint32_t lo_sym = lane * C.sub;
@@ -748,6 +769,8 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 }
             }
 
+            const long long pr_e = probe_clock();
+            if (lane == 0) pr.add(7, pr_e - pr_d);                // pack
             // the ticket of the next batch (see above)
             uint32_t next_ticket = 0;
             if (threadIdx.x == 0) next_ticket = atomicAdd(&C.ctl->ticket, 1u);
@@ -785,7 +808,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         if (C.sub_width == 2) reinterpret_cast<uint16_t*>(I.out + I.lay.sub_end_tab[s] + 64ull * my_c)[lane] = (uint16_t)inc;
                         else reinterpret_cast<uint32_t*>(I.out + I.lay.sub_end_tab[s] + 128ull * my_c)[lane] = inc;
                         tot16 += (chunk_bits + 127) / 128;
-                        if (lane == 0) atomicAdd(&counters(t)->payload_bits[s], (unsigned long long)chunk_bits);
                     }
                 }
             }
@@ -806,8 +828,9 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 if (same) *reinterpret_cast<volatile uint32_t*>(&s_base_seq) = it + 2;
                 *reinterpret_cast<volatile uint32_t*>(&s_ticket_seq) = it + 2;   // after s_base_seq: the service warp reads it first
             }
-            if (!n_huff && active) chunk_done(t);                   // nothing to copy out: the chunk is complete
+            if (!n_huff && active) chunk_done(t, 0, 0);             // nothing to copy out: the chunk is complete
 
+            if (lane == 0) pr.add(8, probe_clock() - pr_e);      // ticket + phase C
             q2 = q1; q1 = q0; q0 = cur;
             ++n_pend;
             slot_idx = last_slot ? 0 : slot_idx + 1;
@@ -836,15 +859,85 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         flush_acc();
         if (bad && raise_status(C.ctl, 0, ZC_E_NO_CODE)) C.ctl->failed = item(bad - 1).index + 1;
     }
+    if (lane == 0) pr.flush();
     __syncthreads();
     if (s_fail && threadIdx.x == 0) raise_status(C.ctl, 0, ZC_E_DEVICE_TIMEOUT);
 }
 
 }  // namespace zc
 
+#include "zc_encode_rows.cuh"
+
 using namespace zc;
 
 namespace {
+
+// Chunk size from which on encode_kernel is used instead of the row encoder (which can take chunks up to 8 KiB).
+// ZC_ROW_ENCODER_BELOW overrides it (bytes; 0 turns the row encoder off, 8193 gives it everything it can take).
+uint32_t row_kernel_limit()
+{
+    static const uint32_t limit = [] {
+        const char* e = getenv("ZC_ROW_ENCODER_BELOW");
+        return e ? std::min<uint32_t>((uint32_t)strtoul(e, nullptr, 0), 8193u) : 4096u;
+    }();
+    return limit;
+}
+
+// Launch shape of the row encoder for a plan, or workers == 0 when the plan is not for it (large chunks, no coded
+// stream).
+RowShape row_shape(const zc_plan_t* p, uint32_t n_huff)
+{
+    RowShape s{};
+    // Measured on one B200 (fractions of the HBM roofline, encode_kernel -> this kernel): 1 KiB chunks 16 -> 22 %,
+    // 2 KiB 29 -> 32 %, 4 KiB 49 -> 46 %, 8 KiB 49 -> 41 %: it takes the chunks below 4 KiB.
+    if (n_huff == 0 || p->chunk_bytes >= row_kernel_limit()) return s;
+    const uint32_t row = p->chunk_bytes / 32;
+    s.row_stride = row + 16;
+    s.in_bytes = 32 * s.row_stride;
+    s.pack1_bytes = n_huff == 2 ? (uint32_t)round_up(32ull * (p->syms_per_sub + p->syms_per_sub / 2 + 4), 16) : 0;
+    const uint32_t max_piece = n_huff * (uint32_t)round_up((uint64_t)p->syms_per_chunk * kLmax / 8, 16);
+    s.ring_bytes = 4096;
+    while (s.ring_bytes < max_piece) s.ring_bytes *= 2;
+    // One input buffer per warp: more warps fit, and with about two dozen of them the SM has enough to do while a
+    // warp waits for its next chunk.  (Two buffers, the next chunk travelling while this one is packed, leave room
+    // for 16 warps at 4 KiB chunks, which measured slower.)
+    s.n_buf = 1;
+    const size_t per_warp = s.n_buf * (size_t)s.in_bytes + s.pack1_bytes + s.ring_bytes;
+    const size_t fixed = (size_t)4 * kTabSlots * 256 * n_huff + 12288 /* static shared and reserve */;
+    s.workers = (uint32_t)std::min<size_t>(kRowMaxWorkers, (kMaxSmem - fixed) / per_warp);
+    if (s.workers < 4) { s.workers = 0; return s; }
+    s.smem = (size_t)4 * kTabSlots * 256 * n_huff + s.workers * per_warp;
+    return s;
+}
+
+template <int N_ITEMS>
+cudaError_t launch_encode_rows(const EncParamsT<N_ITEMS>& P, uint32_t format, const RowShape& sh, const zc_plan_t* p0, cudaStream_t st)
+{
+    RowParams RP{sh.row_stride, sh.in_bytes, sh.pack1_bytes, sh.ring_bytes, p0->chunk_bytes / 512, sh.n_buf};
+    const uint32_t want = std::max<uint32_t>(P.c.total_batches, 1);
+    const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
+    probe_upload(st);
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kern) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
+        if (e != cudaSuccess) return;
+        kern<<<grid, (sh.workers + 2) * 32, sh.smem, st>>>(P, RP);
+        e = cudaGetLastError();
+    };
+    const bool h0 = P.c.mode[0] == ZC_MODE_HUFF, h1 = P.c.mode[1] == ZC_MODE_HUFF;
+#define ZC_ENC_CASE(F)                                                                  \
+    if (h0 && h1) launch(encode_rows_kernel<F, N_ITEMS, true, true>);                  \
+    else if (h0) launch(encode_rows_kernel<F, N_ITEMS, true, false>);                  \
+    else launch(encode_rows_kernel<F, N_ITEMS, false, true>);
+    switch (format) {
+    case ZC_FMT_BF16: ZC_ENC_CASE(ZC_FMT_BF16) break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_ENC_CASE(ZC_FMT_FP8_E4M3) break;
+    case ZC_FMT_SCALE_U8: ZC_ENC_CASE(ZC_FMT_SCALE_U8) break;
+    default: ZC_ENC_CASE(ZC_FMT_FP4_E2M1) break;
+    }
+#undef ZC_ENC_CASE
+    return e;
+}
 
 // Shared-memory shape of a launch for given chunk geometry, number of coded streams and slot size.
 struct EncShape { uint32_t n_slots, slot_bytes, region_bytes, stage_stride, workers, per_sm; size_t smem; };
@@ -1006,7 +1099,12 @@ uint64_t max_batches_of(const zc_plan_t* p)
 {
     EncShape sh;
     if (enc_shape(p, 2, true, &sh) != ZC_OK) return p->n_chunks;
-    return (p->n_chunks + (uint64_t)sh.workers - 1) / sh.workers;
+    uint64_t workers = sh.workers;
+    for (uint32_t n_huff = 1; n_huff <= 2; ++n_huff) {
+        const RowShape rs = row_shape(p, n_huff);
+        if (rs.workers) workers = std::min<uint64_t>(workers, rs.workers);
+    }
+    return (p->n_chunks + workers - 1) / workers;
 }
 
 }  // namespace
@@ -1036,6 +1134,8 @@ zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const voi
     EncShape sh;
     const zc_status ss = enc_shape(p, n_huff, wants_wide_slots(cb, mode), &sh);
     if (ss != ZC_OK) return ss;
+    const RowShape rows = d_base ? RowShape{} : row_shape(p, n_huff);
+    if (rows.workers) sh.workers = rows.workers;                 // chunks per batch
 
     static thread_local EncParamsT<1> P;
     P.c = EncCommon{};
@@ -1050,7 +1150,7 @@ zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const voi
     fill_tables(P.table, cb);
 
     if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * P.c.total_batches, st) != cudaSuccess) return ZC_E_CUDA;
-    if (launch_encode<1>(P, p->format, sh, st) != cudaSuccess) return ZC_E_CUDA;
+    if ((rows.workers ? launch_encode_rows<1>(P, p->format, rows, p, st) : launch_encode<1>(P, p->format, sh, st)) != cudaSuccess) return ZC_E_CUDA;
 
     if (h_out_bytes) {
         Control h;
@@ -1146,6 +1246,10 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
         EncShape sh;
         const zc_status ss = enc_shape(p0, n_huff, (combo & 4u) != 0, &sh);
         if (ss != ZC_OK) return ss;
+        bool any_base = false;
+        if (d_base) for (uint32_t i = 0; i < n_tensors; ++i) any_base = any_base || d_base[i] != nullptr;
+        const RowShape rows = any_base ? RowShape{} : row_shape(p0, n_huff);
+        if (rows.workers) sh.workers = rows.workers;
         uint32_t t = 0;
         while (t < n_tensors) {
             P.c = EncCommon{};
@@ -1174,7 +1278,8 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
             // the ticket counter restarts for every launch (the first one finds it cleared)
             if (!first_launch && cudaMemsetAsync(&((Control*)ws)->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
             first_launch = false;
-            if (launch_encode<(int)kEncBatchMax>(P, p0->format, sh, st) != cudaSuccess) return ZC_E_CUDA;
+            if ((rows.workers ? launch_encode_rows<(int)kEncBatchMax>(P, p0->format, rows, p0, st)
+                              : launch_encode<(int)kEncBatchMax>(P, p0->format, sh, st)) != cudaSuccess) return ZC_E_CUDA;
         }
     }
 
@@ -1234,6 +1339,15 @@ zc_status zc_compress_noalloc(const zc_plan_t* p, const zc_codebook_t* cb, const
     // zc_compress clears the control block and the look-back words it uses before launching
     return zc_compress(p, cb, d_in, d_out, out_capacity, scratch, h_out_bytes, cuda_stream);
 }
+
+#ifdef ZC_PROBE
+void zc_probe_stats(unsigned long long* out, int clear)
+{
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_probe_stats, sizeof(g_probe_stats));
+    if (clear) { unsigned long long z[64] = {0}; cudaMemcpyToSymbol(g_probe_stats, z, sizeof(z)); }
+}
+#endif
 
 zc_status zc_device_status(const zc_plan_t* p, const void* d_workspace, void* cuda_stream)
 {
