@@ -26,6 +26,7 @@ constexpr uint32_t kRowRing = 16;            // batches of a block whose bookkee
                                              // batches wait for their place, and a worker sends what has been placed at every turn)
 constexpr uint32_t kRowSleep = 400;          // nanoseconds a waiting warp sleeps between two looks: polling costs issue slots the
                                              // packing warps need
+constexpr uint32_t kRowAhead = 2;            // batches dealt out beyond the newest one a worker has begun
 constexpr int kRowLook = 5;                  // look-back rounds cover 32 * kRowLook predecessors: more than the resident blocks
 
 struct RowShape {
@@ -185,7 +186,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             //      behind this ticket waits for its batch to be packed.  Packed batches may wait for their place up
             //      to five deep.  A batch only ever waits for batches with smaller tickets, which blocks that are
             //      running hold: the scheme does not depend on every block of the grid being resident. ----
-            if (!ended && handed < uni32(&s_lead) + 2 && handed < uni32(&s_off_seq) + 6) {
+            if (!ended && handed < uni32(&s_lead) + kRowAhead && handed < uni32(&s_off_seq) + 6) {
                 if (ticket_state == 0) {
                     if (lane == 0) ticket = atomicAdd(&C.ctl->ticket, 1u);   // used one turn of the loop later
                     ticket_state = 1;
@@ -510,9 +511,10 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
         uint32_t requested = 0;                                   // batches whose input has been requested
         for (uint32_t it = 0;; ++it) {
             const long long pr_a = probe_clock();
-            if (!wait_seq(&s_base_seq, it + 1)) { failed = true; if (lane == 0) C.ctl->pad[1] = 200 + 1000 * it; break; }
+            // (a batch whose input has been requested has been seen already; no second wait, and above all no memory
+            // fence while the asynchronous copies are in flight: the fence would wait for them)
+            if (requested <= it && !wait_seq(&s_base_seq, it + 1)) { failed = true; if (lane == 0) C.ctl->pad[1] = 200 + 1000 * it; break; }
             if (lane == 0 && vol32(&s_lead) < it + 1) atomicMax(&s_lead, it + 1);
-            send_placed(it);
             const uint32_t t = vol32(&s_tensor[it % kRowRing]);
             if (t == kNoTensor) {
                 // everything this warp packed must leave before the block's shared memory goes away
@@ -738,10 +740,8 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                     piece_word += piece_words;
                 }
             }
-            if (lane == 0) pr.add(6, probe_clock() - pr_f);         // move into the piece
-            // one buffer: the rows are free now, the next batch's input travels while this warp posts, sends and waits
-            __syncwarp();
-            if (RP.n_buf == 1 && uni32(&s_base_seq) >= it + 2) { __threadfence_block(); request(it + 1); requested = it + 2; }
+            const long long pr_post = probe_clock();
+            if (lane == 0) pr.add(6, pr_post - pr_f);                // move into the piece
             // what the lanes wrote must be visible to the bulk copy that reads it
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -752,6 +752,16 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                 __threadfence_block();
                 atomicAdd(&s_cnt[r], 1u);
             }
+            // pieces of earlier batches that have been placed leave now (before the next input is requested: the
+            // fences on this path would wait for the copies in flight)
+            __syncwarp();
+            const long long pr_g = probe_clock();
+            send_placed(it);
+            const long long pr_h = probe_clock();
+            if (lane == 0) { pr.add(0, pr_g - pr_post); pr.add(3, pr_h - pr_g); }
+            // one buffer: the rows are free now, the next batch's input travels while this warp waits
+            if (RP.n_buf == 1 && uni32(&s_base_seq) >= it + 2) { __threadfence_block(); request(it + 1); requested = it + 2; }
+            if (lane == 0) pr.add(2, probe_clock() - pr_h);
         }
         if (lane == 0) {
             flush_acc();
