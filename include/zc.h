@@ -160,10 +160,13 @@ typedef struct zc_stats_t {
  * fmt         element format
  * n_elems     number of elements (0 is valid and gives a header-only container);
  *             must be even for FP4
- * chunk_bytes uncompressed element bytes per chunk: a multiple of 1024 in [1 KiB, 256 KiB]
+ * chunk_bytes uncompressed element bytes per chunk: a multiple of 1024 in [1 KiB, ZC_MAX_CHUNK_BYTES]
+ *             (64 KiB: what the kernels can hold of a chunk in shared memory with both streams coded;
+ *             the container format itself has room for chunks of up to 256 KiB)
  * out         receives a new plan (host object; destroy with zc_plan_destroy)
  * Errors: INVALID_ARG (null out, bad chunk_bytes, odd FP4 count, more than 2^32-1 chunks),
  *         UNSUPPORTED (format), NOMEM. */
+#define ZC_MAX_CHUNK_BYTES 65536u
 zc_status zc_plan(zc_format fmt, uint64_t n_elems, uint32_t chunk_bytes, zc_plan_t** out);
 void zc_plan_destroy(zc_plan_t* plan);
 zc_status zc_plan_get_info(const zc_plan_t* plan, zc_plan_info* out);

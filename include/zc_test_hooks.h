@@ -16,6 +16,26 @@ extern "C" {
 zc_status zc_test_split16(zc_format fmt, const uint8_t* h_in16, uint8_t* h_e8, uint8_t* h_sm8);
 /* Inverse: 8 + 8 symbols (host) -> 16 element bytes (host). */
 zc_status zc_test_merge16(zc_format fmt, const uint8_t* h_e8, const uint8_t* h_sm8, uint8_t* h_out16);
+
+/* ---- bounded waits (no counterpart in the paper: failure handling of this library) ----------
+ * Every wait inside a kernel (for another block's look-back word, for a batch inside a block,
+ * for the bulk copy of a chunk's piece) gives up after a number of polls and the call reports
+ * ZC_E_DEVICE_TIMEOUT.  These switches let a test reach that branch without hanging or faulting
+ * anything: the kernels return by themselves.  They change process-wide settings; a test puts
+ * them back (polls = 0 restores the default limit, 0 turns a stall off).
+ *   zc_test_set_wait_limit  polls after which a device-side wait gives up
+ *   zc_test_stall_encoder   zc_compress hands out its batches from this number on, so batch 0 is
+ *                           never packed and every look-back waits for a word nobody posts
+ *   zc_test_stall_decoder   the decoder does not start the copies of the pieces it waits for */
+/* Launch shapes (host arithmetic only, no GPU): worker warps per block the encoder would use for a plan
+ * with n_coded Huffman-coded streams (0..2) and narrow or wide pack slots, and warps per block of the
+ * decoder with one or both streams coded.  0 = the kernels cannot take this plan.  A test checks that
+ * every chunk size zc_plan accepts gives at least one. */
+uint32_t zc_test_encoder_workers(const zc_plan_t* plan, uint32_t n_coded, uint32_t wide_slots);
+uint32_t zc_test_decoder_warps(const zc_plan_t* plan, uint32_t both_coded);
+void zc_test_set_wait_limit(uint32_t polls);
+void zc_test_stall_encoder(uint32_t first_ticket);
+void zc_test_stall_decoder(uint32_t on);
 #ifdef __cplusplus
 }
 #endif

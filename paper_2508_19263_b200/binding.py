@@ -139,6 +139,13 @@ def _load():
     L.zc_test_split16.argtypes = [C.c_int, vp, vp, vp]
     L.zc_test_merge16.restype = C.c_int
     L.zc_test_merge16.argtypes = [C.c_int, vp, vp, vp]
+    L.zc_test_encoder_workers.restype = C.c_uint32
+    L.zc_test_encoder_workers.argtypes = [vp, C.c_uint32, C.c_uint32]
+    L.zc_test_decoder_warps.restype = C.c_uint32
+    L.zc_test_decoder_warps.argtypes = [vp, C.c_uint32]
+    for name in ("zc_test_set_wait_limit", "zc_test_stall_encoder", "zc_test_stall_decoder"):
+        getattr(L, name).restype = None
+        getattr(L, name).argtypes = [C.c_uint32]
     return L
 
 
@@ -481,3 +488,26 @@ def test_merge16(fmt: int, e8: np.ndarray, sm8: np.ndarray):
 
 test_split16.__test__ = False
 test_merge16.__test__ = False
+
+
+def test_set_wait_limit(polls: int) -> None:
+    """zc_test_set_wait_limit (0 restores the default)."""
+    _lib.zc_test_set_wait_limit(polls)
+
+
+def test_stall_encoder(first_ticket: int) -> None:
+    """zc_test_stall_encoder (0 turns the stall off)."""
+    _lib.zc_test_stall_encoder(first_ticket)
+
+
+def test_stall_decoder(on: bool) -> None:
+    """zc_test_stall_decoder."""
+    _lib.zc_test_stall_decoder(1 if on else 0)
+
+
+def test_encoder_workers(p: Plan, n_coded: int, wide_slots: bool) -> int:
+    return int(_lib.zc_test_encoder_workers(p._h, n_coded, 1 if wide_slots else 0))
+
+
+def test_decoder_warps(p: Plan, both_coded: bool) -> int:
+    return int(_lib.zc_test_decoder_warps(p._h, 1 if both_coded else 0))

@@ -23,6 +23,8 @@ struct DecParams {
     uint32_t pool_bytes;     // per-warp shared memory: symbol rows first, the rest stages compressed pieces
     uint32_t c_begin, c_end; // chunks the launch decodes (zc_decompress: all of them)
     uint32_t spec;           // the container is long enough to read stream 0's tables before the header is checked
+    uint32_t spin_limit;     // polls after which a wait for a staged piece gives up
+    uint32_t skip_copy;      // test hook: the copies of the pieces are not started
     unsigned long long call_id;
 };
 
@@ -41,6 +43,7 @@ struct DecBatchParams {
     unsigned long long call_id;
     uint32_t cs, sub, chunk_bytes, format, group, pool_bytes;
     uint32_t n_tensors, total_chunks, tensor_base, n_ranges;
+    uint32_t spin_limit, skip_copy;
     DecItem item[kDecBatchMax];
 };
 
@@ -441,7 +444,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
         if (H0 && piece0 + 16 <= slot_bytes) {
             staged0 = flying0 = true;
-            if (lane == 0) {
+            if (lane == 0 && !P.skip_copy) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[0], piece0 + 16);
                 bulk_g2s(pool + slots_off, pay0_g, piece0 + 16, &bar[0]);
@@ -449,7 +452,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         }
         if (H1 && piece1 + 16 <= slot_bytes) {
             staged1 = flying1 = true;
-            if (lane == 0) {
+            if (lane == 0 && !P.skip_copy) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(&bar[1], piece1 + 16);
                 bulk_g2s(pool + slots_off + (H0 ? slot_bytes : 0), pay1_g, piece1 + 16, &bar[1]);
@@ -488,10 +491,10 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                         asm volatile("prefetch.global.L2 [%0];" :: "l"(raw1 + i * k_step + r * R));
                 if (kHuff && r == 0) {
                     if (H0 && staged0) {
-                        if (mbar_wait(&bar[0], parity0)) parity0 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
+                        if (mbar_wait(&bar[0], parity0, P.spin_limit)) parity0 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
                     if (H1 && staged1) {
-                        if (mbar_wait(&bar[1], parity1)) parity1 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
+                        if (mbar_wait(&bar[1], parity1, P.spin_limit)) parity1 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
                     if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; return; }
                     flying0 = flying1 = false;
@@ -583,8 +586,8 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         if (c < n_full) body(BoolTag<true>{}); else body(BoolTag<false>{});
     }
     // a copy that was started and not waited for (the loop ended early) must land before the block may leave
-    if (flying0) for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[0], parity0); ++spins) {}
-    if (flying1) for (uint32_t spins = 0; spins < kSpinLimit && !mbar_try_wait(&bar[1], parity1); ++spins) {}
+    if (flying0 && !P.skip_copy) mbar_wait(&bar[0], parity0, P.spin_limit);
+    if (flying1 && !P.skip_copy) mbar_wait(&bar[1], parity1, P.spin_limit);
     return err;
 }
 
@@ -753,6 +756,7 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
         P.n_syms = B.item[t].n_syms; P.n_elems = B.item[t].n_elems; P.n_chunks = B.item[t].n_chunks;
         P.cs = B.cs; P.sub = B.sub; P.chunk_bytes = B.chunk_bytes; P.format = B.format; P.group = B.group;
         P.pool_bytes = B.pool_bytes; P.call_id = B.call_id; P.c_begin = 0; P.c_end = P.n_chunks;
+        P.spin_limit = B.spin_limit; P.skip_copy = B.skip_copy;
         const uint64_t tables = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * (P.chunk_bytes <= 8192 ? 2u : 4u) * P.n_chunks;
         P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
         __syncthreads();                                         // everybody is done with the previous tensor's tables
@@ -852,6 +856,13 @@ unsigned long long new_call_id()
 
 }  // namespace
 
+uint32_t zc_test_decoder_warps(const zc_plan_t* p, uint32_t both_coded)
+{
+    DecShape sh;
+    if (!p || dec_shape(p, both_coded != 0, &sh) != ZC_OK) return 0;
+    return sh.warps;
+}
+
 zc_status zc_decompress(const zc_plan_t* p, const void* d_comp, size_t comp_bytes, void* d_out, void* d_workspace,
                         void* cuda_stream)
 {
@@ -894,6 +905,7 @@ zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t co
     P.call_id = new_call_id();
     P.spec = comp_bytes >= kHeaderBytes + table_section_bytes(p->n_chunks, p->chunk_bytes) ? 1u : 0u;
     P.pool_bytes = shape.pool_bytes;
+    P.spin_limit = test_knobs().spin_limit; P.skip_copy = test_knobs().skip_copy;
     const uint32_t warps = shape.warps, ppl = shape.ppl;
     const size_t smem = shape.smem;
     // at least one block even for an empty range: the header is still checked
@@ -955,6 +967,7 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         B.cs = p0->syms_per_chunk; B.sub = p0->syms_per_sub; B.chunk_bytes = p0->chunk_bytes;
         B.format = p0->format; B.group = p0->group; B.pool_bytes = shape.pool_bytes;
         B.tensor_base = base;
+        B.spin_limit = test_knobs().spin_limit; B.skip_copy = test_knobs().skip_copy;
         uint32_t n = 0;
         uint64_t total = 0;
         // as many tensors as fit one launch: at most kDecBatchMax, fewer than 2^32 chunks together

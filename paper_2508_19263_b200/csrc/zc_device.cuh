@@ -11,7 +11,6 @@
 
 namespace zc {
 
-constexpr uint32_t kSpinLimit = 1u << 22;     // bounded waits: look-back and mbarrier
 constexpr uint32_t kLutEntries = 1u << kLmax;
 constexpr size_t kMaxSmem = 227 * 1024;       // usable shared memory per block on sm_100
 
@@ -100,9 +99,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait for a phase of an mbarrier; false when the wait gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t spin_limit)
 {
-    for (uint32_t spins = 0; spins <= kSpinLimit; ++spins)
+    for (uint32_t spins = 0; spins <= spin_limit; ++spins)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

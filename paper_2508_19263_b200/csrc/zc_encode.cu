@@ -50,6 +50,7 @@ struct EncCommon {
     uint32_t stage_step;                         // staging offset between a lane's consecutive groups (256 symbols apart)
                                                  // when that is a constant, i.e. sub divides 256; else 0
     uint32_t n_tensors, total_batches;
+    uint32_t spin_limit;                         // polls after which a bounded wait gives up
 };
 
 template <int N_ITEMS> struct EncParamsT;
@@ -450,7 +451,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             if (ended && placed == handed - 1) break;
             if (vol32(&s_fail)) break;
             if (did) { idle = 0; continue; }
-            if (++idle > kSpinLimit) { s_fail = 1; break; }
+            if (++idle > C.spin_limit) { s_fail = 1; break; }
             __nanosleep(1000);                                   // nothing to do right now: leave the issue slots to the workers
         }
     } else {
@@ -459,7 +460,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         // when the wait gives up.
         auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
             bool ok = false;
-            for (uint32_t n = 0; n < kSpinLimit; ++n) {
+            for (uint32_t n = 0; n < C.spin_limit; ++n) {
                 if (vol32(word) >= target) { ok = true; break; }
                 if (vol32(&s_fail)) break;
                 if (n > 64) __nanosleep(40);
@@ -986,6 +987,7 @@ void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const
     c.mode[0] = mode[0]; c.mode[1] = mode[1];
     c.n_slots = sh.n_slots; c.slot_bytes = sh.slot_bytes; c.region_bytes = sh.region_bytes; c.stage_stride = sh.stage_stride;
     c.sub_width = sub_end_width(p->chunk_bytes);
+    c.spin_limit = test_knobs().spin_limit;
     c.sub_magic = (uint32_t)(((1ull << 32) + p->syms_per_sub - 1) / p->syms_per_sub);
     c.stage_step = 256 % p->syms_per_sub == 0 ? (256 / p->syms_per_sub) * sh.region_bytes : 0;
 }
@@ -1111,6 +1113,13 @@ uint64_t max_batches_of(const zc_plan_t* p)
 
 extern "C" {
 
+uint32_t zc_test_encoder_workers(const zc_plan_t* p, uint32_t n_coded, uint32_t wide_slots)
+{
+    EncShape sh;
+    if (!p || n_coded > 2 || enc_shape(p, n_coded, wide_slots != 0, &sh) != ZC_OK) return 0;
+    return sh.workers;
+}
+
 zc_status zc_compress(const zc_plan_t* p, const zc_codebook_t* cb, const void* d_in, void* d_out, size_t out_capacity,
                       void* d_workspace, uint64_t* h_out_bytes, void* cuda_stream)
 {
@@ -1150,6 +1159,11 @@ zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const voi
     fill_tables(P.table, cb);
 
     if (cudaMemsetAsync(d_workspace, 0, kControlBytes + 8ull * P.c.total_batches, st) != cudaSuccess) return ZC_E_CUDA;
+    if (test_knobs().first_ticket) {             // test hook: the tickets start late, batch 0 is never packed
+        static uint32_t first;
+        first = test_knobs().first_ticket;
+        if (cudaMemcpyAsync(&((Control*)d_workspace)->ticket, &first, sizeof(first), cudaMemcpyHostToDevice, st) != cudaSuccess) return ZC_E_CUDA;
+    }
     if ((rows.workers ? launch_encode_rows<1>(P, p->format, rows, p, st) : launch_encode<1>(P, p->format, sh, st)) != cudaSuccess) return ZC_E_CUDA;
 
     if (h_out_bytes) {
@@ -1239,7 +1253,15 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
         const bool wide = (m[0] == ZC_MODE_HUFF || m[1] == ZC_MODE_HUFF) && table_wide[table_of[t]];
         group[t] = (uint8_t)(m[0] | (m[1] << 1) | (wide ? 4u : 0u));
     }
+    // the launch shapes of the combinations that occur, checked before anything is launched
+    bool combo_used[8] = {false, false, false, false, false, false, false, false};
+    for (uint32_t t = 0; t < n_tensors; ++t) combo_used[group[t]] = true;
     for (uint32_t combo = 0; combo < 8; ++combo) {
+        EncShape sh;
+        if (combo_used[combo] && enc_shape(p0, (combo & 1u) + ((combo >> 1) & 1u), (combo & 4u) != 0, &sh) != ZC_OK) return ZC_E_UNSUPPORTED;
+    }
+    for (uint32_t combo = 0; combo < 8; ++combo) {
+        if (!combo_used[combo]) continue;
         const uint32_t mode[2] = {combo & 1u, (combo >> 1) & 1u};
         const uint32_t n_huff = (mode[0] == ZC_MODE_HUFF) + (mode[1] == ZC_MODE_HUFF);
         auto in_combo = [&](uint32_t t) { return group[t] == combo; };

@@ -253,7 +253,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             if (ended && agg_posted == handed - 1) break;
             if (uni32(&s_fail)) break;
             if (did) { idle = 0; continue; }
-            if (++idle > kSpinLimit) { s_fail = 1; dbg_where = 100 + 1000 * agg_posted + 100000 * handed; break; }
+            if (++idle > C.spin_limit) { s_fail = 1; dbg_where = 100 + 1000 * agg_posted + 100000 * handed; break; }
             __nanosleep(kRowSleep);
         }
         if (dbg_where && lane == 0) C.ctl->pad[0] = dbg_where;
@@ -393,7 +393,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             }
             if (uni32(&s_fail)) break;
             if (did) { idle = 0; continue; }
-            if (++idle > kSpinLimit) { s_fail = 1; dbg_where = 500 + (lb_on ? 10 : 0) + 1000 * placed; break; }
+            if (++idle > C.spin_limit) { s_fail = 1; dbg_where = 500 + (lb_on ? 10 : 0) + 1000 * placed; break; }
             __nanosleep(kRowSleep);
         }
         if (dbg_where && lane == 0) C.ctl->pad[3] = dbg_where;
@@ -401,7 +401,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
         // =========================== a worker warp ===========================
         auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
             bool ok = false;
-            for (uint32_t n = 0; n < kSpinLimit; ++n) {
+            for (uint32_t n = 0; n < C.spin_limit; ++n) {
                 if (vol32(word) >= target) { ok = true; break; }
                 if (vol32(&s_fail)) break;
                 if (n > 2) __nanosleep(kRowSleep);
@@ -518,7 +518,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             const uint32_t t = vol32(&s_tensor[it % kRowRing]);
             if (t == kNoTensor) {
                 // everything this warp packed must leave before the block's shared memory goes away
-                for (uint32_t n = 0; n < kSpinLimit && sent < it; ++n) {
+                for (uint32_t n = 0; n < C.spin_limit && sent < it; ++n) {
                     send_placed(it);
                     if (sent < it) { if (uni32(&s_fail)) break; __nanosleep(200); }
                 }
@@ -664,7 +664,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             uint32_t roff = ring_head;
             if (need) {
                 bool room = false;
-                for (uint32_t n = 0; n < kSpinLimit; ++n) {
+                for (uint32_t n = 0; n < C.spin_limit; ++n) {
                     if (ring_used + need <= ring_units) { room = true; break; }
                     // pieces that have been sent are free as soon as their copies have read them
                     send_placed(it);

@@ -114,14 +114,26 @@ uint64_t cost_bits(const uint64_t hist[256], const uint8_t len[256])
 
 }  // namespace
 
+namespace zc {
+TestKnobs& test_knobs()
+{
+    static TestKnobs k{kDefaultSpinLimit, 0, 0};
+    return k;
+}
+}  // namespace zc
+
 extern "C" {
+
+void zc_test_set_wait_limit(uint32_t polls) { test_knobs().spin_limit = polls ? polls : kDefaultSpinLimit; }
+void zc_test_stall_encoder(uint32_t first_ticket) { test_knobs().first_ticket = first_ticket; }
+void zc_test_stall_decoder(uint32_t on) { test_knobs().skip_copy = on ? 1u : 0u; }
 
 zc_status zc_plan(zc_format fmt, uint64_t n_elems, uint32_t chunk_bytes, zc_plan_t** out)
 {
     if (!out) return ZC_E_INVALID_ARG;
     const uint32_t g = group_of((uint32_t)fmt);
     if (!g) return ZC_E_UNSUPPORTED;
-    if (chunk_bytes < 1024 || chunk_bytes > 262144 || chunk_bytes % 1024) return ZC_E_INVALID_ARG;
+    if (chunk_bytes < 1024 || chunk_bytes > ZC_MAX_CHUNK_BYTES || chunk_bytes % 1024) return ZC_E_INVALID_ARG;
     if (fmt == ZC_FMT_FP4_E2M1 && (n_elems & 1)) return ZC_E_INVALID_ARG;
     if (n_elems > (1ull << 40)) return ZC_E_INVALID_ARG;
     zc_plan_s* p = new (std::nothrow) zc_plan_s;

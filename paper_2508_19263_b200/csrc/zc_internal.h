@@ -112,4 +112,13 @@ struct Control {
 };
 constexpr size_t kControlBytes = 256;
 
+// What the test hooks (zc_test_hooks.h) can change; the product path never writes these.
+struct TestKnobs {
+    uint32_t spin_limit;     // polls after which a bounded wait on the device gives up
+    uint32_t first_ticket;   // first batch the encoder hands out (not 0: batch 0 is never packed, so every look-back stalls)
+    uint32_t skip_copy;      // the decoder does not start the copies of the pieces it then waits for
+};
+TestKnobs& test_knobs();
+constexpr uint32_t kDefaultSpinLimit = 1u << 22;
+
 }  // namespace zc

@@ -382,3 +382,45 @@ def test_batched_calls_at_bench_size_on_sampled_chunks():
     assert zc.batch_status(ws) == (zc.OK, None)
     for b, x in zip(d_backs, d_ins):
         assert torch.equal(b, x)
+
+
+@pytest.mark.parametrize("fmt", [zc.FMT_BF16, zc.FMT_FP8_E4M3])
+@pytest.mark.parametrize("chunk_bytes", [2048, 4096, 65536])
+def test_whole_containers_at_bench_size_equal_the_oracle_s(fmt, chunk_bytes):
+    """Tensors of the size class the benchmark times, in one batched call that crosses tensor boundaries: every byte
+    of every container against the oracle (not a sample).  The large tensor has thousands of batches, far more
+    than blocks run at a time, so its chunks are placed through many rounds of the look-back; the ragged one ends
+    in the middle of a chunk."""
+    G = zo.group(fmt)
+    sizes = [(24 << 20) * G, (3 << 20) * G + 1234 * G + 2 * G, 0, (7 << 20) * G]     # 48 MiB, 6 MiB + a bit, nothing, 14 MiB of BF16
+    g = torch.Generator(device=DEV); g.manual_seed(7 + chunk_bytes)
+    d_ins, plans, datas = [], [], []
+    for i, n in enumerate(sizes):
+        x = torch.randn(max(n, 16), generator=g, device=DEV) * (0.02 / (1 + i))
+        if fmt == zc.FMT_BF16:
+            b = x.to(torch.bfloat16).view(torch.uint8)[: 2 * n]
+        else:
+            b = (x / (x.abs().max() / 448)).clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)[:n]
+        d_ins.append(b.contiguous() if n else torch.zeros(16, dtype=torch.uint8, device=DEV))
+        datas.append(b.cpu().numpy().copy() if n else np.zeros(0, np.uint8))
+        plans.append(zc.plan(fmt, n, chunk_bytes))
+    n_t = len(plans)
+    d_hists = torch.zeros((n_t, 2, 256), dtype=torch.int64, device=DEV)
+    zc.histogram_batch(zc.HistogramBatch(plans, d_ins), d_hists)
+    hists = d_hists.cpu().numpy().astype(np.uint64)
+    cbs = zc.build_codebooks(plans, hists, zc.POLICY_AUTO)
+    d_outs = [torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=DEV) for p in plans]
+    enc = zc.CompressBatch(plans, d_ins, d_outs)
+    enc.set_codebooks(cbs)
+    ws = torch.empty(enc.workspace_bytes, dtype=torch.uint8, device=DEV)
+    got_sizes = zc.compress_batch(enc, ws)
+    for t in range(n_t):
+        assert np.array_equal(hists[t], zo.histogram(fmt, datas[t], sizes[t]))
+        want = zo.compress(fmt, datas[t], sizes[t], chunk_bytes, zo.build_codebook(hists[t], zo.POLICY_AUTO))
+        assert got_sizes[t] == want.size
+        assert np.array_equal(d_outs[t][: got_sizes[t]].cpu().numpy(), want), f"container of tensor {t} differs"
+    d_backs = [torch.empty(max(p.input_bytes, 16), dtype=torch.uint8, device=DEV) for p in plans]
+    zc.decompress_batch(zc.DecompressBatch(plans, d_outs, got_sizes, d_backs), ws)
+    assert zc.batch_status(ws) == (zc.OK, None)
+    for p, b, x in zip(plans, d_backs, d_ins):
+        assert torch.equal(b[: p.input_bytes], x[: p.input_bytes])

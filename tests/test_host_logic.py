@@ -37,7 +37,7 @@ def test_enums_match_the_oracle_s_numbering():
 @pytest.mark.parametrize("fmt", FORMATS)
 def test_plan_geometry(fmt):
     for n in [0, 2, 6, 1000, 4096, 65536 * 3 + 10, 1 << 24]:
-        for cb in [1024, 8192, 65536, 262144]:
+        for cb in [1024, 8192, 32768, 65536]:
             p = zc.plan(fmt, n, cb)
             assert p.n_syms == zo.n_syms(fmt, n)
             assert p.input_bytes == zo.input_bytes(fmt, n)
@@ -48,8 +48,20 @@ def test_plan_geometry(fmt):
             assert p.workspace_bytes >= 256 + 8 * p.n_chunks and p.workspace_bytes % 256 == 0
 
 
+def test_every_accepted_chunk_size_has_a_launch_shape():
+    """Whatever zc_plan accepts, the encoder (any number of coded streams, narrow and wide pack slots) and the
+    decoder (one or both streams coded) have a launch shape for; beyond the limit the plan itself is refused."""
+    for cb in range(1024, 65536 + 1, 1024):
+        p = zc.plan(zc.FMT_BF16, 1 << 20, cb)
+        for n_coded in (0, 1, 2):
+            for wide in (False, True):
+                assert zc.test_encoder_workers(p, n_coded, wide) >= 1, (cb, n_coded, wide)
+        for both in (False, True):
+            assert zc.test_decoder_warps(p, both) >= 8, (cb, both)
+
+
 def test_plan_rejects_bad_arguments():
-    for cb in [0, 512, 1000, 1025, 262144 + 1024, 1 << 20]:
+    for cb in [0, 512, 1000, 1025, 65536 + 1024, 131072, 262144, 1 << 20]:
         with pytest.raises(zc.ZcError) as e:
             zc.plan(zc.FMT_BF16, 100, cb)
         assert e.value.status == zc.E_INVALID_ARG
