@@ -69,12 +69,21 @@ def workload_specs(name: str):
         # the E8M0 block scales of the same stack as byte streams (config 4 stores them raw; coding them is
         # what the paper's FP4 result rests on, Sec. 3.4 / 4.4): 225 streams, 234.5 MB
         return wl.SCALE_U8, wl.llama8b_stack(4)
+    if name in ("cfg5_kv_bf16_all", "cfg5_kv_fp8_all"):
+        # config 5 in full: K and V of all 32 layers, [8, 8, 32768, 128] each (34.4 GB in BF16, 17.2 GB in FP8)
+        fmt = wl.BF16 if "bf16" in name else wl.FP8_E4M3
+        return fmt, [wl.TensorSpec(f"kv.{l}.{'kv'[w]}", (8, 8, 32768, 128), 0.0, 10 * l + w) for l in range(32) for w in range(2)]
     if name in ("cfg5_kv_bf16", "cfg5_kv_fp8", "next3_kv_bf16_static", "next3_kv_fp8_static"):
         # K/V cache tensors [8, 8, 32768, 128]; a subset of the 32 layers keeps the run short (K and V of 4 layers).
         # The *_static workloads code them the way Sec. 3.3 describes the run-time use: with dictionaries computed
         # ahead of time (from layer 0's K and V), no histogram pass and no codebook build in the step
         fmt = wl.BF16 if "bf16" in name else wl.FP8_E4M3
         return fmt, [wl.TensorSpec(f"kv.{l}.{'kv'[w]}", (8, 8, 32768, 128), 0.0, 10 * l + w) for l in range(4) for w in range(2)]
+    if name in ("next2_bf16_delta_frozen", "small_bf16_delta_frozen"):
+        # the same pair of checkpoints with a stated share of the weights left untouched (frozen layers and rows, the
+        # state Sec. 3.1 describes for a fine-tuning run that has converged): unchanged stretches XOR to zero, their
+        # chunks are constant and cost no payload bits
+        return wl.BF16, wl.llama8b_stack(2) if name.startswith("next2") else wl.llama8b_stack(2, n_layers=2, include_embedding=False)
     if name in ("next2_bf16_delta", "small_bf16_delta"):
         # delta checkpoints (Sec. 3.1 / 4.1): the XOR of two consecutive BF16 checkpoints of the config-2 stack is
         # coded; the earlier checkpoint is a second resident input of every call
@@ -153,7 +162,7 @@ def oracle_sample(fmt, specs, device, delta=False):
     out, total = [], 0
     for spec in specs:
         if delta:
-            cur, base, n = wl.checkpoint_pair(spec, device)
+            cur, base, n = wl.checkpoint_pair(spec, device, frozen_rows=wl.frozen_rows_of(spec) if delta == "frozen" else 0.0)
             t = cur ^ base
         elif spec.name.startswith("kv."):
             t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, device)
@@ -192,13 +201,53 @@ def oracle_step(fmt, sample, chunk_bytes, static_cb=None):
     return t_h, t_e, t_d, cbytes
 
 
+def cpu_model() -> str:
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.lower().startswith("model name"):
+                return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def _oracle_job(job):
+    fmt, data, n, chunk_bytes = job
+    return oracle_step(fmt, [("slice", data, n)], chunk_bytes)[3]
+
+
+def oracle_all_cores(fmt, sample, chunk_bytes):
+    """The oracle on every core the process may use: the sample is cut into row slices, every slice is compressed
+    and decompressed as a tensor of its own by one of N worker processes (N = cores of the affinity mask).
+    Returns (GB/s of the whole path, N, slices)."""
+    import multiprocessing as mp
+    import oracle as zo
+    cores = len(os.sched_getaffinity(0))
+    per = zo.input_bytes(fmt, zo.group(fmt) * 2) // 2 or 1          # bytes per symbol pair unit: slices stay whole symbols
+    jobs = []
+    for name, data, n in sample:
+        pieces = max(1, min(4 * cores // max(len(sample), 1), data.size // (1 << 20)))
+        step = (data.size // pieces) // 64 * 64
+        for k in range(pieces):
+            lo = k * step
+            hi = data.size if k == pieces - 1 else lo + step
+            part = data[lo:hi]
+            jobs.append((fmt, part, part.size * n // data.size if data.size else 0, chunk_bytes))
+    total = sum(j[1].size for j in jobs)
+    ctx = mp.get_context("fork")
+    t0 = time.perf_counter()
+    with ctx.Pool(cores) as pool:
+        pool.map(_oracle_job, jobs, chunksize=1)
+    return total / (time.perf_counter() - t0) / 1e9, cores, len(jobs)
+
+
 def run_reference(args):
     """--impl reference: the paper ships no code, so the reference arm is the CPU oracle as it stands."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     fmt, specs = workload_specs(args.workload)
-    sample, total = oracle_sample(fmt, specs, "cpu", args.workload.endswith("_delta"))
+    sample, total = oracle_sample(fmt, specs, "cpu", ("frozen" if args.workload.endswith("_frozen") else True) if "_delta" in args.workload else False)
     chunk_bytes = args.chunk_kib * 1024
     static_cb = oracle_static_codebook(fmt, sample) if args.workload.endswith("_static") else None
     for _ in range(min(args.warmup, 1)):
@@ -253,19 +302,11 @@ def whole_job_gbs(world: int, bytes_per_rank: int, ms: float) -> float:
 # the CUDA path
 # --------------------------------------------------------------------------------------------
 
-def run_ours(args):
+def measure(args, ctx):
+    """One workload through the CUDA path: returns the JSON line as a dict (rank 0) or None (other ranks)."""
     from paper_2508_19263_b200 import binding as zc
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist_mod.init_process_group("nccl", device_id=dev)
-        dist = dist_mod
+    rank, world, dev, dist = ctx["rank"], ctx["world"], ctx["dev"], ctx["dist"]
 
     def barrier():
         torch.cuda.synchronize()
@@ -281,14 +322,15 @@ def run_ours(args):
 
     # ---- resident inputs, plans, output buffers ----
     tensors = []
-    delta = args.workload.endswith("_delta")
+    delta = "_delta" in args.workload
+    frozen = args.workload.endswith("_delta_frozen")
     static = args.workload.endswith("_static")
     if static and not args.batch:
         raise SystemExit("the *_static workloads use the batched calls")
     for spec in specs:
         base_t = None
         if delta:
-            t, base_t, n = wl.checkpoint_pair(spec, dev)
+            t, base_t, n = wl.checkpoint_pair(spec, dev, frozen_rows=wl.frozen_rows_of(spec) if frozen else 0.0)
         elif spec.name.startswith("kv."):
             t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, dev)
         else:
@@ -585,9 +627,7 @@ def run_ours(args):
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "error": str(ex)[:200]}
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
 
     peak, peak_src = measured_peaks()
     gbs = lambda nbytes, ms: nbytes / ms / 1e6
@@ -627,16 +667,24 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": (U + C) / (n_dec_launch if dom_name == "decode_kernel" else n_enc_launch),
                 "traffic": (NCU_DRAM_BYTES_PER_INPUT_BYTE[dom_name] * U / (n_dec_launch if dom_name == "decode_kernel" else n_enc_launch)
                             if args.workload == "cfg2_bf16_llama8b" and args.chunk_kib == 4 and args.batch else None),
-                "traffic_source": "ncu dram__bytes_read+write of the two-layer BF16 stack (profiles/), scaled by input bytes per launch"}
+                "traffic_source": "from profiles/ (ncu dram__bytes_read+write of the two-layer BF16 stack, scaled by input bytes per launch), not measured in this run"}
 
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only) ----
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        sample, total = oracle_sample(fmt, specs, dev, delta)
+        sample, total = oracle_sample(fmt, specs, dev, ('frozen' if frozen else True) if delta else False)
         t_h, t_e, t_d, cb_sample = oracle_step(fmt, sample, chunk_bytes, oracle_static_codebook(fmt, sample) if static else None)
         cpu = {"value": total / (t_h + t_e + t_d) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {len(sample)} tensors of {args.workload}, {total} bytes",
-               "decode_gbs": total / t_d / 1e9, "encode_gbs": total / t_e / 1e9, "histogram_codebook_gbs": (total / t_h / 1e9 if not static else None)}
+               "decode_gbs": total / t_d / 1e9, "encode_gbs": total / t_e / 1e9, "histogram_codebook_gbs": (total / t_h / 1e9 if not static else None),
+               "cpu_model": cpu_model()}
+        if not static and not delta:
+            try:
+                all_gbs, n_cores, n_slices = oracle_all_cores(fmt, sample, chunk_bytes)
+                cpu["all_cores"] = {"value": all_gbs, "unit": UNIT, "cores": n_cores,
+                                    "sample": f"the same sample cut into {n_slices} row slices, each compressed and decompressed as a tensor of its own by one of {n_cores} worker processes"}
+            except Exception as ex:
+                cpu["all_cores"] = {"value": None, "error": str(ex)[:200]}
 
     # compression ratios next to the paper's (context): exponent stream, sign+mantissa stream, total
     st_bits = [0, 0]
@@ -661,7 +709,112 @@ def run_ours(args):
         "gpu_launches": ((n_enc_launch if static else (len(step_groups) if args.batch else n_hist_launch) + n_enc_launch_step)
                          + n_dec_launch) * args.steps,
     }
-    print(json.dumps(line))
+    return line
+
+
+# Workloads reported next to the headline (key, workload, chunk KiB): the other configurations the paper's
+# method is measured on, the larger chunk sizes, and the rows that follow the headline path.
+PER_WORKLOAD = [
+    ("cfg3_fp8_llama8b", "cfg3_fp8_llama8b", 4),
+    ("cfg5_kv_bf16_32layers", "cfg5_kv_bf16_all", 4),
+    ("cfg5_kv_fp8_32layers", "cfg5_kv_fp8_all", 4),
+    ("cfg4_fp4_llama8b", "cfg4_fp4_llama8b", 4),
+    ("cfg4_fp4_scales", "cfg4_fp4_scales", 4),
+    ("cfg2_bf16_llama8b_chunk16k", "cfg2_bf16_llama8b", 16),
+    ("cfg2_bf16_llama8b_chunk64k", "cfg2_bf16_llama8b", 64),
+    ("cfg3_fp8_llama8b_chunk16k", "cfg3_fp8_llama8b", 16),
+    ("cfg3_fp8_llama8b_chunk64k", "cfg3_fp8_llama8b", 64),
+    ("next2_bf16_delta", "next2_bf16_delta", 4),
+    ("next2_bf16_delta_frozen", "next2_bf16_delta_frozen", 4),
+    ("next3_kv_bf16_static", "next3_kv_bf16_static", 4),
+    ("next4_fp8_e5m2", "next4_fp8_e5m2", 4),
+]
+
+
+def summary_of(line):
+    """What per_workload keeps of a workload's line."""
+    out = {"workload": line["config"]["workload"], "chunk_kib": line["config"]["chunk_kib"], "tensors": line["config"]["tensors"],
+           "uncompressed_bytes": line["config"]["uncompressed_bytes"], "compressed_bytes": line["config"]["compressed_bytes"],
+           "container_ratio": line["compression_ratio"]["total_container"],
+           "exponent_stream_ratio": line["compression_ratio"]["exponent_stream_payload"],
+           "sign_mantissa_stream_ratio": line["compression_ratio"]["sign_mantissa_stream_payload"],
+           "step_ms": line["ms_per_step"], "step_gbs": line["value"], "round_trip": "byte-identical"}
+    for leg in ("decode", "encode", "histogram"):
+        out[leg] = {k: line[leg][k] for k in ("ms", "value", "hbm_gbs", "frac_of_measured_peak", "frac_of_nominal_8TBs")}
+    if line.get("extra"):
+        out.update(line["extra"])
+    return out
+
+
+def config1_latency(ctx):
+    """Config 1 (one 1024 x 1024 FP8 E4M3 tensor, 64 KiB chunks): a latency case, microseconds per call."""
+    from paper_2508_19263_b200 import binding as zc
+    dev = ctx["dev"]
+    d_in, n = wl.config1_tensor(dev)
+    p = zc.plan(wl.FP8_E4M3, n, 65536)
+    d_hist = torch.zeros((2, 256), dtype=torch.int64, device=dev)
+    d_out = torch.empty(p.max_compressed_bytes, dtype=torch.uint8, device=dev)
+    d_back = torch.empty(p.input_bytes, dtype=torch.uint8, device=dev)
+    d_ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=dev)
+    hist = zc.histogram(p, d_in, d_hist).cpu().numpy().astype(np.uint64)
+    cb = zc.build_codebook(p, hist, zc.POLICY_HUFF_ALL)          # the config codes both streams
+    nbytes = zc.compress(p, cb, d_in, d_out, d_ws)
+    zc.decompress(p, d_out, nbytes, d_back, d_ws)
+    if zc.device_status(p, d_ws) != zc.OK or not torch.equal(d_back, d_in[: p.input_bytes]):
+        raise SystemExit("config 1 round trip mismatch")
+
+    def timed_us(fn, reps=200):
+        for _ in range(10):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    return {"workload": "cfg1_fp8_1024x1024", "chunk_kib": 64, "policy": "huff_all", "uncompressed_bytes": p.input_bytes,
+            "compressed_bytes": nbytes, "container_ratio": nbytes / p.input_bytes, "round_trip": "byte-identical",
+            "histogram_us": timed_us(lambda: zc.histogram(p, d_in, d_hist)),
+            "encode_us": timed_us(lambda: zc.compress(p, cb, d_in, d_out, d_ws, sync=False)),
+            "decode_us": timed_us(lambda: zc.decompress(p, d_out, nbytes, d_back, d_ws)),
+            "note": "asynchronous calls back to back on one stream, CUDA events; 16 chunks: a latency case, not a bandwidth case"}
+
+
+def run_ours(args):
+    import copy
+    import gc
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    ctx = {"rank": rank, "world": world, "dev": dev, "dist": dist}
+    line = measure(args, ctx)
+    # the other workloads, device-resident legs only, one after the other (single GPU, default workload only)
+    if world == 1 and args.per_workload and args.workload == "cfg2_bf16_llama8b" and args.chunk_kib == 4 and args.batch:
+        per = {}
+        for key, name, ck in PER_WORKLOAD:
+            gc.collect(); torch.cuda.empty_cache()
+            sub = copy.copy(args)
+            sub.workload, sub.chunk_kib, sub.steps, sub.warmup = name, ck, 3, 2
+            sub.no_e2e, sub.no_cpu_baseline = True, True
+            try:
+                per[key] = summary_of(measure(sub, ctx))
+            except SystemExit as ex:
+                per[key] = {"workload": name, "chunk_kib": ck, "error": str(ex)[:200]}
+        gc.collect(); torch.cuda.empty_cache()
+        per["cfg1_fp8_1024x1024_chunk64k"] = config1_latency(ctx)
+        line["per_workload"] = per
+    if rank == 0:
+        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
@@ -680,6 +833,8 @@ def main():
                     help="1: the batched entry points (all tensors of the stack per call); 0: one call per tensor")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used for profiler captures)")
+    ap.add_argument("--per-workload", type=int, default=1, choices=[0, 1],
+                    help="1: after the headline workload, time the other configurations and add them as per_workload")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

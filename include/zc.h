@@ -255,7 +255,12 @@ zc_status zc_compress(const zc_plan_t* plan, const zc_codebook_t* cb, const void
  *
  * First call on a device: the library looks up the device address of its scratch array once
  * per device (with that device current) and remembers it.  Make that first call outside of
- * any stream capture.
+ * any stream capture.  Host threads may make it at the same time.  The remembered address
+ * does not survive cudaDeviceReset: do not reset a device between calls.
+ *
+ * Asynchronous form (h_out_bytes == NULL): the caller holds no workspace pointer to read the
+ * device status from (a symbol without code, a wait that gave up); zc_noalloc_status reads it
+ * from the built-in array of the current device after waiting for the stream.
  *
  * Sharing: all calls on one device use the same scratch array.  Each call clears the part it
  * needs before use, so stale contents of an earlier call never matter, but two calls whose
@@ -266,6 +271,9 @@ zc_status zc_compress(const zc_plan_t* plan, const zc_codebook_t* cb, const void
 #define ZC_NOALLOC_SCRATCH_BYTES (256u + 8u * ZC_NOALLOC_MAX_CHUNKS)
 zc_status zc_compress_noalloc(const zc_plan_t* plan, const zc_codebook_t* cb, const void* d_in, void* d_out,
                               size_t out_capacity, uint64_t* h_out_bytes, void* cuda_stream);
+/* Status word of the last zc_compress_noalloc call on the current device (waits for the stream):
+ * ZC_OK, ZC_E_NO_CODE, ZC_E_DEVICE_TIMEOUT, or ZC_E_CUDA. */
+zc_status zc_noalloc_status(void* cuda_stream);
 
 /* ---- decompress (Sec. 3.1: chunks decode independently, in parallel) ------------------------
  * d_comp      device, a container made for the same plan; comp_bytes = bytes available

@@ -139,6 +139,8 @@ def _load():
     L.zc_test_split16.argtypes = [C.c_int, vp, vp, vp]
     L.zc_test_merge16.restype = C.c_int
     L.zc_test_merge16.argtypes = [C.c_int, vp, vp, vp]
+    L.zc_noalloc_status.restype = C.c_int
+    L.zc_noalloc_status.argtypes = [vp]
     L.zc_test_encoder_workers.restype = C.c_uint32
     L.zc_test_encoder_workers.argtypes = [vp, C.c_uint32, C.c_uint32]
     L.zc_test_decoder_warps.restype = C.c_uint32
@@ -366,6 +368,11 @@ def compress_noalloc(p: Plan, cb: Codebook, d_in: torch.Tensor, d_out: torch.Ten
                                   C.byref(n) if sync else None, _stream_ptr(stream))
     _check(st, "zc_compress_noalloc")
     return n.value if sync else None
+
+
+def noalloc_status(stream=None) -> int:
+    """zc_noalloc_status: device status of the last compress_noalloc call on the current device."""
+    return int(_lib.zc_noalloc_status(_stream_ptr(stream)))
 
 
 def decompress(p: Plan, d_comp: torch.Tensor, comp_bytes: int, d_out: torch.Tensor, d_workspace: torch.Tensor,

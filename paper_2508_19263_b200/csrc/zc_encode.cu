@@ -2,6 +2,7 @@
 // zc_compress_batch, zc_compress_noalloc, zc_device_status.
 #include "zc_device.cuh"
 
+#include <atomic>
 #include <cstring>
 #include <unordered_map>
 #include <vector>
@@ -1333,19 +1334,20 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[ZC_NOALLOC_SCRA
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::atomic<void*> g_noalloc_ptr[kMaxDevices];
 
-// Device address of the scratch array on the current device; looked up once per device.
+// Device address of the scratch array on the current device; looked up once per device (two host threads that
+// make the first call together both look it up and store the same address).
 zc_status noalloc_scratch(void** out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ZC_E_CUDA;
-    if (!g_noalloc_ptr[dev]) {
-        void* ptr = nullptr;
+    void* ptr = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return ZC_E_CUDA;
-        g_noalloc_ptr[dev] = ptr;
+        g_noalloc_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_noalloc_ptr[dev];
+    *out = ptr;
     return ZC_OK;
 }
 }  // namespace
@@ -1370,6 +1372,18 @@ void zc_probe_stats(unsigned long long* out, int clear)
     if (clear) { unsigned long long z[64] = {0}; cudaMemcpyToSymbol(g_probe_stats, z, sizeof(z)); }
 }
 #endif
+
+zc_status zc_noalloc_status(void* cuda_stream)
+{
+    void* scratch = nullptr;
+    const zc_status st = noalloc_scratch(&scratch);
+    if (st != ZC_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long word[2] = {0, 0};            // status, call id
+    if (cudaMemcpyAsync(word, scratch, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return ZC_E_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return ZC_E_CUDA;
+    return (word[0] >> 8) == word[1] ? (zc_status)(word[0] & 0xFF) : ZC_OK;
+}
 
 zc_status zc_device_status(const zc_plan_t* p, const void* d_workspace, void* cuda_stream)
 {

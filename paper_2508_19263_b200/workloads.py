@@ -127,14 +127,29 @@ def make_weight(spec: TensorSpec, fmt: int, device) -> Tuple[torch.Tensor, int, 
     raise ValueError(fmt)
 
 
-def checkpoint_pair(spec: TensorSpec, device, rel_step: float = 0.03) -> Tuple[torch.Tensor, torch.Tensor, int]:
+def checkpoint_pair(spec: TensorSpec, device, rel_step: float = 0.03, frozen_rows: float = 0.0) -> Tuple[torch.Tensor, torch.Tensor, int]:
     """Two consecutive BF16 checkpoints of one weight tensor: the earlier one is the tensor of `make_weight`, the
     later one is every weight moved by a relative step N(0, rel_step^2) (seed + 7) before the BF16 cast, so that
-    most exponents and the upper mantissa bits stay the same.  Returns (later bytes, earlier bytes, n_elems)."""
+    most exponents and the upper mantissa bits stay the same.  frozen_rows: share of the leading rows (first
+    dimension) that the step leaves untouched (1.0: a frozen tensor, the later checkpoint equals the earlier one).
+    Returns (later bytes, earlier bytes, n_elems)."""
     x = _randn(spec.shape, spec.std, spec.seed, device)
     base = to_bf16_bytes(x)
-    x.mul_(1.0 + rel_step * torch.randn(spec.shape, generator=_gen(spec.seed + 7, device), device=device, dtype=torch.float32))
+    step = 1.0 + rel_step * torch.randn(spec.shape, generator=_gen(spec.seed + 7, device), device=device, dtype=torch.float32)
+    keep = int(round(frozen_rows * spec.shape[0]))
+    if keep:
+        step[:keep] = 1.0
+    x.mul_(step)
     return to_bf16_bytes(x), base, spec.n_elems
+
+
+def frozen_rows_of(spec: TensorSpec) -> float:
+    """The *_delta_frozen workloads: the tensors of the even layers did not change at all, in all other tensors the
+    first half of the rows did not change (three quarters of the weights are untouched in all)."""
+    parts = spec.name.split(".")
+    if parts[0] == "layers" and int(parts[1]) % 2 == 0:
+        return 1.0
+    return 0.5
 
 
 def config1_tensor(device) -> Tuple[torch.Tensor, int]:

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as zo
 from paper_2508_19263_b200 import binding as zc
 from paper_2508_19263_b200 import workloads as wl
 
@@ -28,6 +29,14 @@ def _compress_both_ways(fmt, d_in, n, chunk_bytes, policy):
     n_new = zc.compress_noalloc(p, cb, d_in, d_new)
     assert n_new == n_ref
     assert torch.equal(d_new[:n_new], d_ref[:n_ref])              # integer work: bit-exact, no tolerance
+    # the CPU oracle writes the same container
+    want = zo.compress(fmt, d_in.cpu().numpy(), n, chunk_bytes, zo.build_codebook(hist, policy))
+    assert n_new == want.size and np.array_equal(d_new[:n_new].cpu().numpy(), want)
+    # the asynchronous form: nothing comes back with the call, the status is read from the built-in scratch
+    d_async = torch.full((p.max_compressed_bytes,), 0x33, dtype=torch.uint8, device=DEV)
+    assert zc.compress_noalloc(p, cb, d_in, d_async, sync=False) is None
+    assert zc.noalloc_status() == zc.OK
+    assert torch.equal(d_async[:n_new], d_new[:n_new])
     # and the container decodes back to the input
     d_back = torch.empty(p.input_bytes, dtype=torch.uint8, device=DEV)
     zc.decompress(p, d_new, n_new, d_back, d_ws)
