@@ -81,16 +81,17 @@
  *       ((sign << 3) | bits 2..0); two elements per symbol as for E4M3.  The
  *       lowest exponent bit goes with the poorly compressible bits; what is
  *       coded is the part of the exponent that byte symbols can carry.
- *   R14 In a container with BOTH streams coded, a chunk of a stream whose symbols
- *       are all the stream's fill symbol takes no payload bits at all: all its
- *       subchunk ends are 0 and its piece is empty.  (With one stream stored raw
- *       the tensor pays 8 bits per symbol for that stream anyway and the rule
- *       does not apply: a chunk of fill symbols is coded like any other.)  The fill symbol is the first symbol in (length, symbol) order,
- *       the one whose code is all zeros.  A chunk that holds symbols and has 0
- *       bits can be nothing else (every code has at least one bit), so no flag
- *       is needed.  This is what lets unchanged stretches of a delta checkpoint
- *       (Sec. 3.1, 4.1) or the unused part of a cache page fall below the 1 bit
- *       per symbol that a per-symbol code costs at least.
+ *   R14 A chunk of a Huffman-coded stream whose symbols are all the stream's fill
+ *       symbol takes no payload bits at all: all its subchunk ends are 0 and its
+ *       piece is empty, whatever the mode of the other stream.  The fill symbol is
+ *       the first symbol in (length, symbol) order, the one whose code is all
+ *       zeros.  A chunk that holds symbols and has 0 bits can be nothing else
+ *       (every code has at least one bit), so no flag is needed.  This is what
+ *       lets unchanged stretches of a delta checkpoint (Sec. 3.1, 4.1: the
+ *       reported exponent ratio of 0.07 is below the 0.125 that one bit per byte
+ *       symbol allows) or the constant exponents of an unused part of a cache
+ *       page fall below the 1 bit per symbol that a per-symbol code costs at
+ *       least.
  *
  * Container layout (little-endian, every section 16-byte aligned):
  *   header 128 B:
@@ -561,7 +562,7 @@ int64_t zo_compress(int fmt, const uint8_t *in, uint64_t n_elems, uint32_t chunk
             uint8_t *sub_end = out + sec[s] + 256 + round16(4ull * nc);
             /* bits of this chunk; none at all if every symbol is the fill symbol (reading R14) */
             uint64_t bits = 0;
-            int fill = zo_fill_symbol(len[s]), constant = (mode[0] == ZO_HUFF && mode[1] == ZO_HUFF);
+            int fill = zo_fill_symbol(len[s]), constant = 1;
             for (uint64_t k = c_lo; k < c_hi; ++k) {
                 bits += len[s][st[s][k]];
                 if (st[s][k] != fill) constant = 0;
@@ -734,7 +735,7 @@ static int decode_chunk_stream(const uint8_t *cont, const zo_header *h, int s, u
     uint64_t piece_bytes = round16((chunk_bits + 7) / 8);
     if (16 * off16 > h->payload_bytes || piece_bytes > h->payload_bytes - 16 * off16) return -1;
     const uint8_t *piece = cont + h->payload_off + 16 * off16;
-    if (chunk_bits == 0 && c_hi > c_lo && h->mode[0] == ZO_HUFF && h->mode[1] == ZO_HUFF) {   /* reading R14 */
+    if (chunk_bits == 0 && c_hi > c_lo) {   /* reading R14 */
         int fill = zo_fill_symbol(cont + h->sec[s]);
         if (fill < 0) return -1;
         for (int j = 0; j < ZO_SUBS; ++j) if (get_sub_end(sub_end, sw, c, j) != 0) return -1;

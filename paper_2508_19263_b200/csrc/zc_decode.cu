@@ -317,8 +317,8 @@ __device__ __forceinline__ void decode_round(ZC_LANE_BITS, uint32_t lut_s, uint3
     }
 }
 
-// With both streams coded, a chunk without payload bits holds nothing but the stream's fill symbol, the symbol
-// with the all-zero code: the first symbol of the table entry for a window of zeros.
+// A chunk without payload bits holds nothing but the stream's fill symbol, the symbol with the all-zero code:
+// the first symbol of the table entry for a window of zeros.
 __device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
 {
     const uint32_t e = lds32(lut_s);
@@ -511,14 +511,14 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     if (n_quads && !probe_skip(0)) {
                         if (H0) {
                             const uint32_t wr_s = rows0_s + wr_off;
-                            if (H1 && piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // both streams coded and no bits: fill symbols
+                            if (piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // a chunk without bits: nothing but the fill symbol
                             else if (!staged0) pos0 = decode_quads_global(pos0, pay0_g, S.lut0_s, S.pairs0, wr_s, fw, n_quads, lim0);
                             else if (S.pairs0) decode_round<2, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wr_s, fw, n_quads);
                             else decode_round<1, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wr_s, fw, n_quads);
                         }
                         if (H1) {
                             const uint32_t wr_s = rows1_s + wr_off;
-                            if (H0 && piece1 == 0) fill_quads(S.lut1_s, S.pairs1, wr_s, fw, n_quads);
+                            if (piece1 == 0) fill_quads(S.lut1_s, S.pairs1, wr_s, fw, n_quads);
                             else if (!staged1) pos1 = decode_quads_global(pos1, pay1_g, S.lut1_s, S.pairs1, wr_s, fw, n_quads, lim1);
                             else if (S.pairs1) decode_round<2, PPL, FULL>(pos1, w10, w11, next1, S.lut1_s, wr_s, fw, n_quads);
                             else decode_round<1, PPL, FULL>(pos1, w10, w11, next1, S.lut1_s, wr_s, fw, n_quads);

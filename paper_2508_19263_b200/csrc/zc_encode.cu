@@ -294,9 +294,9 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 for (int i = 0; i < 8; ++i) {
                     const uint32_t v = src[lane + 32 * i];
                     tab[256 * hs + lane + 32 * i] = v;
-                    if (H0 && H1 && v >= 1 && v <= kLmax) fill = (lane + 32 * i) | (v << 8);
+                    if (v >= 1 && v <= kLmax) fill = (lane + 32 * i) | (v << 8);
                 }
-                if (H0 && H1) {
+                {
                     const uint32_t who = __ballot_sync(0xFFFFFFFFu, fill != 0xFFFFFFFFu);
                     fill = __shfl_sync(0xFFFFFFFFu, fill, who ? __ffs(who) - 1 : 0);
                     if (lane == 0) s_fill[nslot][hs] = who ? fill : 0xFF00u;     // no code at all: a length no chunk can match
@@ -790,12 +790,12 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         const uint32_t x = __shfl_up_sync(0xFFFFFFFFu, inc, o);
                         if (lane >= (uint32_t)o) inc += x;
                     }
-                    // With both streams coded, a chunk that holds nothing but the fill symbol (the symbol with the
-                    // all-zero code) takes no bits at all.  Candidates are the chunks with exactly symbols * length
+                    // A chunk that holds nothing but the fill symbol (the symbol with the all-zero code) takes no bits
+                    // at all.  Candidates are the chunks with exactly symbols * length
                     // bits (rare otherwise); their staged symbols are then compared one by one.
                     uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                    const uint32_t fill = (H0 && H1) ? vol32(&s_fill[tab_slot_idx][hs]) : 0u;   // fill symbol | its code length << 8
-                    if (H0 && H1 && active && chunk_bits <= C.cs * (fill >> 8)) {  // the last chunk may be shorter
+                    const uint32_t fill = vol32(&s_fill[tab_slot_idx][hs]);   // fill symbol | its code length << 8
+                    if (active && chunk_bits <= C.cs * (fill >> 8)) {  // the last chunk may be shorter
                         const uint32_t syms = (uint32_t)min((uint64_t)C.cs, I.n_syms - (uint64_t)my_c * C.cs);
                         const uint32_t mine = lane * C.sub < syms ? min(C.sub, syms - lane * C.sub) : 0u;
                         if (chunk_bits == syms * (fill >> 8) &&

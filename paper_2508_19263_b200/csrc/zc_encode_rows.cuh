@@ -150,9 +150,9 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                 for (int i = 0; i < 8; ++i) {
                     const uint32_t v = src[lane + 32 * i];
                     tab[256 * hs + lane + 32 * i] = v;
-                    if (H0 && H1 && v >= 1 && v <= kLmax) fill = (lane + 32 * i) | (v << 8);
+                    if (v >= 1 && v <= kLmax) fill = (lane + 32 * i) | (v << 8);
                 }
-                if (H0 && H1) {
+                {
                     const uint32_t who = __ballot_sync(0xFFFFFFFFu, fill != 0xFFFFFFFFu);
                     fill = __shfl_sync(0xFFFFFFFFu, fill, who ? __ffs(who) - 1 : 0);
                     if (lane == 0) s_fill[nslot][hs] = who ? fill : 0xFF00u;
@@ -635,13 +635,13 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                         if (lane >= (uint32_t)o) inc += x;
                     }
                     uint32_t chunk_bits = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                    // With both streams coded, a chunk that holds nothing but the fill symbol (the symbol with the
-                    // all-zero code, the shortest one) takes no bits at all.  Such a chunk has exactly symbols * length
-                    // bits (rare otherwise), and all of them are zero: every other code has a one somewhere.
-                    if (H0 && H1) {
+                    // A chunk that holds nothing but the fill symbol (the symbol with the all-zero code, the shortest
+                    // one) takes no bits at all.  Such a chunk has exactly symbols * length bits (rare otherwise), and
+                    // all of them are zero: every other code has a one somewhere.
+                    {
                         const uint32_t fill_len = vol32(&s_fill[tab_slot_idx][hs]) >> 8;
                         if (active && chunk_bits == c_syms * fill_len) {
-                            const uint32_t src = s == 0 ? row_s : p1_s;
+                            const uint32_t src = (s == 1 && H0) ? p1_s : row_s;
                             uint32_t any = 0;
                             for (uint32_t i = 0; i < (my_bits[s] + 31) / 32; ++i) any |= lds32(src + 4 * i);
                             if (!__any_sync(0xFFFFFFFFu, any != 0)) { inc = 0; chunk_bits = 0; }

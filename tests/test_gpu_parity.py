@@ -125,8 +125,8 @@ def test_special_bit_patterns():
     rng = np.random.default_rng(9)                                    # one exponent value, noise below it: [HUFF, RAW], and
     noisy = (np.uint16(0x3F80) | rng.integers(0, 128, 30000).astype(np.uint16) | (rng.integers(0, 2, 30000).astype(np.uint16) << 15))
     p, cb, _, cont = _gpu_round_trip(zc.FMT_BF16, noisy.view(np.uint8), 30000, 4096, zc.POLICY_AUTO)
-    assert cb.modes == [zc.MODE_HUFF, zc.MODE_RAW]                    # the constant exponent chunks pay one bit per symbol
-    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 30000
+    assert cb.modes == [zc.MODE_HUFF, zc.MODE_RAW]                    # the constant exponent chunks cost nothing
+    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 0
     rng = np.random.default_rng(1)
     uni = rng.integers(0, 256, 1 << 18, dtype=np.uint8)               # incompressible: every code length near 8
     _gpu_round_trip(zc.FMT_BF16, uni, 1 << 17, 8192, zc.POLICY_HUFF_ALL)
@@ -152,7 +152,7 @@ def test_chunks_of_nothing_but_the_fill_symbol_take_no_bits(fmt, chunk_bytes):
     # a tensor that is constant altogether: header and tables only
     flat = zeros(5 * cs + 9)
     _gpu_round_trip(fmt, flat, flat.size // per_sym * G, chunk_bytes, zc.POLICY_HUFF_ALL)
-    # one stream raw: the rule does not apply, constant chunks of the coded stream pay their bit per symbol
+    # one stream raw: the coded stream's constant chunks cost nothing all the same
     h = zo.histogram(fmt, data, n)
     p = zc.plan(fmt, n, chunk_bytes)
     for modes in ((zc.MODE_HUFF, zc.MODE_RAW), (zc.MODE_RAW, zc.MODE_HUFF)):

@@ -564,14 +564,21 @@ def test_round_trip_special_patterns():
     assert np.array_equal(zo.decompress(cont, z.size * 2), z.view(np.uint8))
     for c in range(hd["n_chunks"]):
         assert np.array_equal(zo.decompress_chunk(cont, c, 1024), z.view(np.uint8)[1024 * c: 1024 * (c + 1)])
-    # the rule needs both streams coded: with noise in the sign+mantissa bits that stream is stored raw, and the
-    # constant exponent stream pays its one bit per symbol
+    # the rule is per stream: with noise in the sign+mantissa bits that stream is stored raw, and the constant
+    # exponent stream still costs nothing
     rng = np.random.default_rng(9)
     noisy = (np.uint16(0x3F80) | rng.integers(0, 128, 5000).astype(np.uint16) | (rng.integers(0, 2, 5000).astype(np.uint16) << 15))
     cb = zo.build_codebook(zo.histogram(zo.BF16, noisy, noisy.size), zo.POLICY_AUTO)
     assert cb.modes == [zo.HUFF, zo.RAW]
     cont = zo.compress(zo.BF16, noisy, noisy.size, 1024, cb)
-    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 5000
+    hd = zo.parse_header(cont)
+    assert hd["streams"][0]["payload_bits"] == 0 and hd["payload_bytes"] == 0
+    # one chunk with another exponent in it: that chunk alone pays (one bit per symbol, two for the odd symbol)
+    noisy[2000] = np.uint16(0x4000) | (noisy[2000] & np.uint16(0x807F))
+    cb = zo.build_codebook(zo.histogram(zo.BF16, noisy, noisy.size), zo.POLICY_AUTO)
+    assert cb.modes == [zo.HUFF, zo.RAW]
+    cont = zo.compress(zo.BF16, noisy, noisy.size, 1024, cb)
+    assert zo.parse_header(cont)["streams"][0]["payload_bits"] == 512
     assert np.array_equal(zo.decompress(cont, noisy.size * 2), noisy.view(np.uint8))
     # NaN / inf / -0 / subnormal patterns are ordinary symbols
     pats = np.array([0x7FC0, 0xFFC1, 0x7F80, 0xFF80, 0x8000, 0x0001, 0x807F, 0x7FFF] * 300, np.uint16)
