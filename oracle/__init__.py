@@ -119,6 +119,26 @@ def e2m1_value(nibble: int) -> float:
 
 # ---- geometry -------------------------------------------------------------------------------
 
+def e5m2_element_fields(data):
+    """FP8 E5M2 split the way Sec. 3.2 states it: the 5 exponent bits of every element on one side, the sign and
+    the 2 mantissa bits on the other ((sign << 2) | mantissa), one symbol per element.  Returns two uint8 arrays."""
+    x = _bytes(data)
+    return ((x >> 2) & 0x1F).astype(np.uint8), (((x >> 7) << 2) | (x & 3)).astype(np.uint8)
+
+
+def e5m2_element_payload_bits(data, L: int = L_MAX):
+    """Payload bits of an E5M2 tensor coded per element with that split (an optimal prefix code per stream, length
+    limit L, stored at its field width when the code does not save 1/64: the AUTO rule with 5- and 3-bit raw
+    symbols).  Returns (exponent bits, sign+mantissa bits).  Plain arithmetic on the two histograms."""
+    out = []
+    for syms, width in zip(e5m2_element_fields(data), (5, 3)):
+        hist = np.bincount(syms, minlength=256).astype(np.uint64)
+        coded = payload_bits(hist, code_lengths(hist, L)) if syms.size else 0
+        raw = width * int(syms.size)
+        out.append(coded if 64 * coded <= 63 * raw else raw)
+    return tuple(out)
+
+
 def group(fmt: int) -> int:
     return lib().zo_group(fmt)
 

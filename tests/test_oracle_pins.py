@@ -592,6 +592,76 @@ def test_round_trip_special_patterns():
     assert np.array_equal(zo.decompress(cont, allb.size), allb)
 
 
+@pytest.mark.parametrize("chunk_bytes", [1024, 8192, 16384])
+def test_container_bound_is_met_by_a_constructed_worst_case(chunk_bytes):
+    """The capacity bound against a container that is as large as the format allows: a dictionary made on a steep
+    histogram gives some symbols 12-bit codes, and a tensor of whole chunks made of nothing but those symbols (in
+    both streams, both coded) fills every piece to 12 bits per symbol.  Its size, worked out here from the layout
+    (header, two table sections, pieces, guard), must be exactly the bound; anything else stays below it."""
+    steep = np.ones((2, 256), np.uint64)
+    steep[:, :20] = (np.uint64(1) << np.arange(40, 20, -1, dtype=np.uint64))      # twenty heavy symbols push the rest to the limit
+    cb = zo.build_codebook(steep, zo.POLICY_HUFF_ALL)
+    assert cb.modes == [zo.HUFF, zo.HUFF]
+    long0 = np.flatnonzero(cb.lengths[0] == 12)
+    long1 = np.flatnonzero(cb.lengths[1] == 12)
+    assert long0.size >= 2 and long1.size >= 2
+    n_chunks, cs = 5, chunk_bytes // 2
+    n = n_chunks * cs                                                # BF16: one element per symbol, whole chunks
+    rng = np.random.default_rng(4)
+    e = long0[rng.integers(0, long0.size, n)].astype(np.uint16)      # exponent symbols
+    sm = long1[rng.integers(0, long1.size, n)].astype(np.uint16)     # sign+mantissa symbols
+    data = ((e << 7) | (sm & 0x7F) | ((sm >> 7) << 15)).astype(np.uint16).view(np.uint8)
+    s0, s1 = zo.split(zo.BF16, data, n)
+    assert np.array_equal(s0, e.astype(np.uint8)) and np.array_equal(s1, sm.astype(np.uint8))
+    cont = zo.compress(zo.BF16, data, n, chunk_bytes, cb)
+    width = 2 if chunk_bytes <= 8192 else 4
+    tables = 256 + ((4 * n_chunks + 15) // 16) * 16 + 32 * width * n_chunks
+    piece = ((cs * 12 // 8 + 15) // 16) * 16
+    want = 128 + 2 * tables + 2 * n_chunks * piece + 16
+    assert cont.size == want
+    assert zo.container_bound(zo.BF16, n, chunk_bytes) == want
+    assert np.array_equal(zo.decompress(cont, data.size), data)
+    # a ragged tensor and ordinary data stay below the bound
+    assert zo.container_bound(zo.BF16, n + 7, chunk_bytes) >= want
+
+
+def test_e5m2_split_as_the_paper_states_it():
+    """Sec. 3.2: E5M2 gives 5 bits to the exponent and the rest to sign and mantissa.  The per-element fields rebuild
+    the value of every one of the 256 patterns (torch's float8_e5m2 is the independent reference), and on Gaussian
+    weights the per-element code of the full exponent beats the byte-symbol reading that codes its upper four
+    bits (the format id the kernels serve)."""
+    pats = np.arange(256, dtype=np.uint8)
+    e5, sm3 = zo.e5m2_element_fields(pats)
+    assert e5.max() == 31 and sm3.max() == 7
+    ref = torch.from_numpy(pats.copy()).view(torch.float8_e5m2).to(torch.float32).numpy()
+    for x in range(256):
+        s, m, e = int(sm3[x]) >> 2, int(sm3[x]) & 3, int(e5[x])
+        if e == 31:
+            val = float("inf") if m == 0 else float("nan")
+        elif e == 0:
+            val = m / 4.0 * 2.0 ** -14
+        else:
+            val = (1 + m / 4.0) * 2.0 ** (e - 15)
+        val = -val if s else val
+        assert (np.isnan(val) and np.isnan(ref[x])) or val == ref[x], x
+    # hand vector: 0x3C = +1.0 (exponent 15, mantissa 0), 0xC2 = -(2 + 1) = -3.0 (exponent 16, mantissa 2)
+    e5, sm3 = zo.e5m2_element_fields(np.array([0x3C, 0xC2], np.uint8))
+    assert list(e5) == [15, 16] and list(sm3) == [0, 6]
+    assert zo.e5m2_value(0x3C) == 1.0 and zo.e5m2_value(0xC2) == -3.0
+    # ratios on synthetic weights
+    rng = np.random.default_rng(12)
+    w = torch.from_numpy((rng.standard_normal(1 << 20) * 0.02).astype(np.float32)).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    be, bs = zo.e5m2_element_payload_bits(w)
+    exact = (be + bs) / (8 * w.size)
+    h = zo.histogram(zo.FP8_E5M2, w, w.size)
+    cb = zo.build_codebook(h, zo.POLICY_AUTO)
+    bits = [zo.payload_bits(h[s], cb.lengths[s]) if cb.modes[s] == zo.HUFF else 8 * int(h[s].sum()) for s in range(2)]
+    grouped = sum(bits) / (8 * w.size)
+    assert exact < grouped < 1.0
+    assert 0.60 < exact < 0.75 and 0.65 < grouped < 0.80
+    print(f"E5M2 payload ratios: exponent/mantissa split per element {exact:.4f}, byte symbols of the upper exponent bits {grouped:.4f}")
+
+
 def test_static_dictionary_from_another_tensor():
     """A code built on one tensor encodes another (Sec. 3.3 precomputed dictionaries) as long as it
     covers its symbols; a symbol without a code is an error, not silent damage."""
