@@ -487,7 +487,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                 // ---- raw sign+mantissa bytes of this round go to registers before the decoding starts ----
 #pragma unroll
                 for (int i = 0; i < PPL; ++i)
-                    if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms) && !probe_skip(2))
+                    if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms))
                         asm volatile("prefetch.global.L2 [%0];" :: "l"(raw1 + i * k_step + r * R));
                 if (kHuff && r == 0) {
                     if (H0 && staged0) {
@@ -508,7 +508,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     const uint32_t done = r * R;
                     // a ragged end decodes up to 15 symbols too many (from the bits that follow); they are not used
                     const uint32_t n_quads = FULL ? (uint32_t)PPL : (n_my > done ? (min(R, n_my - done) + 15) / 16 : 0u);
-                    if (n_quads && !probe_skip(0)) {
+                    if (n_quads) {
                         if (H0) {
                             const uint32_t wr_s = rows0_s + wr_off;
                             if (piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // a chunk without bits: nothing but the fill symbol
@@ -537,7 +537,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                             const uint32_t used = pos1 - (staged1 ? 8 * slot1_s : 0u);
                             good = good && (FULL ? used == end1 : used - end1 <= 15 * kLmax);
                         }
-                        if (!__all_sync(0xFFFFFFFFu, good) && !probe_skip(0)) err = ZC_E_CORRUPT;
+                        if (!__all_sync(0xFFFFFFFFu, good)) err = ZC_E_CORRUPT;
                         // the slots are free: the next chunk's pieces travel while this round is merged and written
                         if (!err && c + step < c_end) prepare(c + step);
                     }
@@ -546,7 +546,7 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
 #pragma unroll
                 for (int i = 0; i < PPL; ++i) {
                     const uint32_t k = k_lane + i * k_step + r * R;
-                    if ((!FULL && k >= c_syms) || probe_skip(1)) continue;
+                    if ((!FULL && k >= c_syms)) continue;
                     uint32_t e[4], m[4];
                     if (H0) {
                         const uint4 v = lds128(rows0_s + rd_off + 512 * i);
@@ -996,7 +996,6 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         B.n_ranges = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(B.n_ranges, total));
         // the ranges are handed out through the ticket word of the control block
         if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
-        probe_upload(st);
         cudaError_t e = cudaSuccess;
         auto launch = [&](auto kern) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);

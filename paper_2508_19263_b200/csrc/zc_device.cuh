@@ -4,7 +4,6 @@
 #include <stdint.h>
 
 #include <algorithm>
-#include <cstdlib>
 
 #include "zc_bits.cuh"
 #include "zc_internal.h"
@@ -112,42 +111,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-
-// Development probe (compiled only with -DZC_PROBE): a word of switches read from the environment variable
-// ZC_PROBE_BITS at every launch, with which a kernel skips parts of its work so that their cost can be measured.
-// The product build has none of it: probe_skip() is the constant false there.
-#ifdef ZC_PROBE
-static __constant__ uint32_t g_probe_bits;
-__device__ __forceinline__ bool probe_skip(uint32_t bit) { return (g_probe_bits >> bit) & 1u; }
-inline void probe_upload(cudaStream_t st)
-{
-    const char* e = getenv("ZC_PROBE_BITS");
-    const uint32_t v = e ? (uint32_t)strtoul(e, nullptr, 0) : 0u;
-    cudaMemcpyToSymbolAsync(g_probe_bits, &v, sizeof(v), 0, cudaMemcpyHostToDevice, st);
-}
-// cycle counters a kernel adds up (slot k: sum, slot 32 + k: number of samples)
-static __device__ unsigned long long g_probe_stats[64];
-__device__ __forceinline__ long long probe_clock() { return clock64(); }
-struct ProbeAcc {
-    long long sum[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-    uint32_t n[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-    __device__ __forceinline__ void add(int k, long long v) { sum[k] += v; ++n[k]; }
-    __device__ __forceinline__ void flush()
-    {
-#pragma unroll
-        for (int k = 0; k < 10; ++k)
-            if (n[k]) { atomicAdd(&g_probe_stats[k], (unsigned long long)sum[k]); atomicAdd(&g_probe_stats[32 + k], (unsigned long long)n[k]); }
-    }
-};
-#else
-__device__ __forceinline__ long long probe_clock() { return 0; }
-struct ProbeAcc {
-    __device__ __forceinline__ void add(int, long long) {}
-    __device__ __forceinline__ void flush() {}
-};
-__device__ __forceinline__ constexpr bool probe_skip(uint32_t) { return false; }
-inline void probe_upload(cudaStream_t) {}
-#endif
 
 inline int sm_count()
 {

@@ -244,7 +244,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
     __shared__ uint32_t s_fill[kTabSlots][2];                   // per table slot and coded stream: fill symbol | its code length << 8
     __shared__ unsigned long long s_tot[kRing][kEncMaxWorkers], s_off[kRing][kEncMaxWorkers];
 
-    ProbeAcc pr;
     if (threadIdx.x < kRing) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) {
         s_fail = 0; s_off_seq = 0; s_base_seq = 0;
@@ -273,7 +272,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         long long lb_base = 0;
         unsigned long long* lb_flags = nullptr;
         uint32_t lb_b = 0, idle = 0;
-        long long pr_t0 = 0, pr_last = 0, pr_polls = 0;
         // Loads tensor t's code tables into the slot after the newest one, once every worker has posted the last
         // batch that was packed with the table that is there now; false when that is not yet the case.
         auto load_next_slot = [&](const uint32_t t, const uint32_t placed_now) -> bool {
@@ -322,7 +320,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             if (placed < real) {
                 const uint32_t r = placed % kRing;
                 if (!lb_on && vol32(&s_cnt[r]) == n_workers) {   // every worker has posted a size (0 without a chunk)
-                    pr_t0 = probe_clock();
                     __threadfence_block();
                     if (lane == 0) s_cnt[r] = 0;
                     lb_v = lane < n_workers ? *reinterpret_cast<const volatile unsigned long long*>(&s_tot[r][lane]) : 0ull;
@@ -344,7 +341,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 }
                 if (lb_on) {
                     bool done = !n_huff || lb_b == 0;
-                    ++pr_polls;
                     if (!done) {
                         // One round of the look-back: kLookWide * 32 predecessors at a time, newest first, up to the
                         // first one that already knows its prefix.  All loads of a round are in flight together, so a
@@ -384,8 +380,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                         __threadfence_block();
                         __syncwarp();
                         if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = placed + 1;
-                        if (lane == 0) { const long long now = probe_clock(); pr.add(0, now - pr_t0); pr.add(1, pr_polls); if (pr_last) pr.add(2, now - pr_last); pr_last = now; }
-                        pr_polls = 0;
                         ++placed;
                         lb_on = false;
                         did = true;
@@ -583,9 +577,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         // waits until the oldest pending batch is placed and copies this warp's chunk of it out
         auto flush_oldest = [&](const uint32_t it) -> bool {
             const uint32_t j = it - n_pend;                         // the batch in question
-            const long long pr_w = probe_clock();
             if (!wait_seq(&s_off_seq, j + 1)) return false;
-            if (lane == 0) pr.add(9, probe_clock() - pr_w);       // of which: waiting for the placement
             if (n_huff) {
                 PackedChunk pc;
                 pc.c = n_pend == 1 ? q0.c : n_pend == 2 ? q1.c : q2.c;
@@ -594,7 +586,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 pc.end[1] = n_pend == 1 ? q0.end[1] : n_pend == 2 ? q1.end[1] : q2.end[1];
                 // its slot: the slots are used round-robin, so it lies n_pend steps behind the current one
                 const uint32_t sl = (slot_idx + n_slots * 4 - n_pend) % n_slots;
-                if (pc.c != kNoChunk && !probe_skip(10))
+                if (pc.c != kNoChunk)
                     copy_out(pc, sl * C.slot_bytes, *reinterpret_cast<const volatile unsigned long long*>(&s_off[j % kRing][warp]));
             }
             --n_pend;
@@ -602,10 +594,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         };
         bool failed = false;
         for (uint32_t it = 0;; ++it) {
-            const long long pr_a = probe_clock();
             if (!wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
-            const long long pr_b = probe_clock();
-            if (lane == 0) pr.add(4, pr_b - pr_a);
             const uint32_t t = vol32(&s_tensor[it % kRing]);
             if (t == kNoTensor) {
                 while (n_pend && !failed) failed = !flush_oldest(it);
@@ -651,8 +640,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             uint32_t g = lane;
             uint32_t off = stage_off(lane);                             // running offset (constant-step case)
             auto off_at = [&](const uint32_t g_, const uint32_t i) { return step ? off + i * step : stage_off(g_); };
-            if (probe_skip(8)) {
-            } else if (I.base) {
+            if (I.base) {
                 // delta form: the chunk of the base tensor is read alongside and XOR-ed in (two pairs of loads in flight)
                 const uint8_t* base_c = I.base + 2 * c_lo;
                 auto x4 = [](const uint4 a, const uint4 b) { return make_uint4(a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w); };
@@ -687,7 +675,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
             __syncwarp();
 
-            if (!probe_skip(11))
             // Warm the L2 for the batch one round of tickets ahead (whichever block gets it; it may lie in one of
             // the next tensors): the loads of phase A are the longest wait of a turn.  One 128-byte line per lane
             // and 4 KiB of chunk.
@@ -708,11 +695,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
 
             // the chunk that was packed into this slot n_slots batches ago must leave before this one is packed
-            const long long pr_c = probe_clock();
-            if (lane == 0) pr.add(5, pr_c - pr_b);                // phase A
             if (n_pend == n_slots && !flush_oldest(it)) { failed = true; break; }
-            const long long pr_d = probe_clock();
-            if (lane == 0) pr.add(6, pr_d - pr_c);                // wait for the placement + copy-out
 
             // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
             const uint32_t lo_sym = lane * C.sub;
@@ -764,15 +747,13 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 for (int s = 0; s < 2; ++s) {
                     if (!is_huff(s)) continue;
                     // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
-                    my_bits[s] = probe_skip(9) ? 100u : pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
+                    my_bits[s] = pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
                     // more than the slot holds: the bits beyond it do not survive the next staging
                     oversize |= my_bits[s] > 8 * C.slot_bytes;
                     ++hs;
                 }
             }
 
-            const long long pr_e = probe_clock();
-            if (lane == 0) pr.add(7, pr_e - pr_d);                // pack
             // the ticket of the next batch (see above)
             uint32_t next_ticket = 0;
             if (threadIdx.x == 0) next_ticket = atomicAdd(&C.ctl->ticket, 1u);
@@ -832,7 +813,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             }
             if (!n_huff && active) chunk_done(t, 0, 0);             // nothing to copy out: the chunk is complete
 
-            if (lane == 0) pr.add(8, probe_clock() - pr_e);      // ticket + phase C
             q2 = q1; q1 = q0; q0 = cur;
             ++n_pend;
             slot_idx = last_slot ? 0 : slot_idx + 1;
@@ -861,7 +841,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
         flush_acc();
         if (bad && raise_status(C.ctl, 0, ZC_E_NO_CODE)) C.ctl->failed = item(bad - 1).index + 1;
     }
-    if (lane == 0) pr.flush();
     __syncthreads();
     if (s_fail && threadIdx.x == 0) raise_status(C.ctl, 0, ZC_E_DEVICE_TIMEOUT);
 }
@@ -918,7 +897,6 @@ cudaError_t launch_encode_rows(const EncParamsT<N_ITEMS>& P, uint32_t format, co
     RowParams RP{sh.row_stride, sh.in_bytes, sh.pack1_bytes, sh.ring_bytes, p0->chunk_bytes / 512, sh.n_buf};
     const uint32_t want = std::max<uint32_t>(P.c.total_batches, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
-    probe_upload(st);
     cudaError_t e = cudaSuccess;
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
@@ -1016,7 +994,6 @@ void fill_tables(EncTables& T, const zc_codebook_t* cb)
 template <int N_ITEMS>
 cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const EncShape& sh, cudaStream_t st)
 {
-    probe_upload(st);
     const uint32_t want = std::max<uint32_t>(P.c.total_batches, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count() * sh.per_sm);
     cudaError_t e = cudaSuccess;
@@ -1363,15 +1340,6 @@ zc_status zc_compress_noalloc(const zc_plan_t* p, const zc_codebook_t* cb, const
     // zc_compress clears the control block and the look-back words it uses before launching
     return zc_compress(p, cb, d_in, d_out, out_capacity, scratch, h_out_bytes, cuda_stream);
 }
-
-#ifdef ZC_PROBE
-void zc_probe_stats(unsigned long long* out, int clear)
-{
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_probe_stats, sizeof(g_probe_stats));
-    if (clear) { unsigned long long z[64] = {0}; cudaMemcpyToSymbol(g_probe_stats, z, sizeof(z)); }
-}
-#endif
 
 zc_status zc_noalloc_status(void* cuda_stream)
 {

@@ -107,7 +107,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
     __shared__ uint32_t s_agg_seq;                              // batches of this block whose size has been published
     __shared__ uint32_t s_lead;                                 // batches of this block that some worker has begun
 
-    ProbeAcc pr;
     if (threadIdx.x < kRowRing) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) { s_fail = 0; s_base_seq = 0; s_off_seq = 0; s_agg_seq = 0; s_lead = 0; }
     __syncthreads();
@@ -128,7 +127,7 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                 if (item(t).n_chunks == 0) write_header(C, item(t), counters(t));
 
         uint32_t handed = 0, agg_posted = 0;
-        uint32_t tcur = 0, dbg_where = 0, idle = 0;
+        uint32_t tcur = 0, idle = 0;
         uint32_t tab_tensor = kNoTensor, tab_slot = 0;
         uint32_t slot_last0 = 0, slot_last1 = 0, slot_last2 = 0, slot_last3 = 0;   // 1 + last batch that used slot k
         bool ended = false;
@@ -253,17 +252,16 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             if (ended && agg_posted == handed - 1) break;
             if (uni32(&s_fail)) break;
             if (did) { idle = 0; continue; }
-            if (++idle > C.spin_limit) { s_fail = 1; dbg_where = 100 + 1000 * agg_posted + 100000 * handed; break; }
+            if (++idle > C.spin_limit) { s_fail = 1; break; }
             __nanosleep(kRowSleep);
         }
-        if (dbg_where && lane == 0) C.ctl->pad[0] = dbg_where;
     } else if (warp == n_workers + 1) {
         // =========================== the placer warp ===========================
         // Finds where the block's batches go.  It keeps a cursor into the tensor's row of look-back words: cur_sum =
         // size of all batches below cur_pos.  The cursor moves forward over other blocks' batches as their sizes
         // appear, whether or not this block's own batch is packed yet, so that a batch is placed the moment the
         // cursor stands at it.  The cursor starts with a look-back from the block's first batch in the tensor.
-        uint32_t placed = 0, idle = 0, dbg_where = 0;
+        uint32_t placed = 0, idle = 0;
         bool lb_on = false;
         unsigned long long lb_sum = 0;
         long long lb_base = 0;
@@ -272,7 +270,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
         uint32_t cur_t = kNoTensor, cur_pos = 0, cur_n = 0;       // the cursor: tensor, next batch, batches of the tensor
         unsigned long long cur_sum = 0;
         unsigned long long* cur_flags = nullptr;
-        long long pr_t1 = 0, pr_last = 0;
         for (;;) {
             bool did = false;
             const uint32_t agg_posted = uni32(&s_agg_seq);
@@ -281,7 +278,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                 const uint32_t r = placed % kRowRing;
                 const uint32_t tj = vol32(&s_tensor[r]);
                 const uint32_t bj = vol32(&s_ticket[r]) - item(tj).first_batch;
-                if (probe_skip(12)) { cur_t = tj; cur_pos = bj; cur_sum = 0; cur_flags = C.flags + item(tj).first_batch; cur_n = 0; }
                 if (cur_t != tj && !lb_on) {
                     lb_t = tj;
                     lb_flags = C.flags + item(tj).first_batch;   // the look-back stays inside the tensor
@@ -331,7 +327,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                     }
                 }
                 if (cur_t == tj && cur_pos == bj) {
-                    pr_t1 = probe_clock();
                     const uint32_t v = lane < n_workers ? vol32(&s_tot[r][lane]) : 0u;
                     uint32_t inc = v;
 #pragma unroll
@@ -348,7 +343,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                     if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_off_seq) = placed + 1;
                     cur_sum += own;
                     ++cur_pos;
-                    if (lane == 0) { const long long now = probe_clock(); pr.add(1, now - pr_t1); if (pr_last) pr.add(2, now - pr_last); pr_last = now; }
                     ++placed;
                     did = true;
                 }
@@ -393,10 +387,9 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             }
             if (uni32(&s_fail)) break;
             if (did) { idle = 0; continue; }
-            if (++idle > C.spin_limit) { s_fail = 1; dbg_where = 500 + (lb_on ? 10 : 0) + 1000 * placed; break; }
+            if (++idle > C.spin_limit) { s_fail = 1; break; }
             __nanosleep(kRowSleep);
         }
-        if (dbg_where && lane == 0) C.ctl->pad[3] = dbg_where;
     } else {
         // =========================== a worker warp ===========================
         auto wait_seq = [&](const uint32_t* word, const uint32_t target) -> bool {
@@ -510,10 +503,9 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
         };
         uint32_t requested = 0;                                   // batches whose input has been requested
         for (uint32_t it = 0;; ++it) {
-            const long long pr_a = probe_clock();
             // (a batch whose input has been requested has been seen already; no second wait, and above all no memory
             // fence while the asynchronous copies are in flight: the fence would wait for them)
-            if (requested <= it && !wait_seq(&s_base_seq, it + 1)) { failed = true; if (lane == 0) C.ctl->pad[1] = 200 + 1000 * it; break; }
+            if (requested <= it && !wait_seq(&s_base_seq, it + 1)) { failed = true; break; }
             if (lane == 0 && vol32(&s_lead) < it + 1) atomicMax(&s_lead, it + 1);
             const uint32_t t = vol32(&s_tensor[it % kRowRing]);
             if (t == kNoTensor) {
@@ -526,11 +518,8 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                 break;
             }
             if (requested <= it) { request(it); requested = it + 1; }
-            const long long pr_b = probe_clock();
             cp_async_wait_all();
             __syncwarp();
-            const long long pr_c = probe_clock();
-            if (lane == 0) { pr.add(4, pr_b - pr_a); pr.add(5, pr_c - pr_b); }
             // two buffers: the next batch's input travels while this one is packed (if it has been dealt out already)
             if (RP.n_buf == 2 && uni32(&s_base_seq) >= it + 2) { __threadfence_block(); request(it + 1); requested = it + 2; }
 
@@ -619,8 +608,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             if (H1) my_bits[1] = 8 * (w1 - ((H0 && H1) ? p1_s : row_s)) + nb1;
             __syncwarp();
 
-            const long long pr_d = probe_clock();
-            if (lane == 0) pr.add(7, pr_d - pr_c);                   // request + pack
             // ---- subchunk end bits and the sizes of the chunk's pieces ----
             uint32_t end[2] = {0, 0}, piece16[2] = {0, 0}, cbits[2] = {0, 0};
             {
@@ -658,8 +645,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             }
             const uint32_t need = piece16[0] + piece16[1];
 
-            const long long pr_e = probe_clock();
-            if (lane == 0) pr.add(8, pr_e - pr_d);                   // end bits
             // ---- room in the ring: give back what the service warp has sent off, wait if that is not enough ----
             uint32_t roff = ring_head;
             if (need) {
@@ -678,12 +663,10 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                     if (uni32(&s_fail)) break;
                     __nanosleep(kRowSleep);
                 }
-                if (!room) { failed = true; if (lane == 0) C.ctl->pad[2] = 300 + 1000 * it; break; }
+                if (!room) { failed = true; break; }
                 ring_head = (ring_head + need) % ring_units;
                 ring_used += need;
             }
-            const long long pr_f = probe_clock();
-            if (lane == 0) pr.add(9, pr_f - pr_e);                   // ring room
             // ---- every lane moves its bits to their place in the piece ----
             {
                 uint32_t piece_word = 4 * roff;                                   // first word of the piece in the ring
@@ -740,8 +723,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
                     piece_word += piece_words;
                 }
             }
-            const long long pr_post = probe_clock();
-            if (lane == 0) pr.add(6, pr_post - pr_f);                // move into the piece
             // what the lanes wrote must be visible to the bulk copy that reads it
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -755,13 +736,9 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
             // pieces of earlier batches that have been placed leave now (before the next input is requested: the
             // fences on this path would wait for the copies in flight)
             __syncwarp();
-            const long long pr_g = probe_clock();
             send_placed(it);
-            const long long pr_h = probe_clock();
-            if (lane == 0) { pr.add(0, pr_g - pr_post); pr.add(3, pr_h - pr_g); }
             // one buffer: the rows are free now, the next batch's input travels while this warp waits
             if (RP.n_buf == 1 && uni32(&s_base_seq) >= it + 2) { __threadfence_block(); request(it + 1); requested = it + 2; }
-            if (lane == 0) pr.add(2, probe_clock() - pr_h);
         }
         if (lane == 0) {
             flush_acc();
@@ -770,7 +747,6 @@ encode_rows_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P, const __grid_c
         if (failed) s_fail = 1;
         if (bad && raise_status(C.ctl, 0, ZC_E_NO_CODE)) C.ctl->failed = item(bad - 1).index + 1;
     }
-    if (lane == 0) pr.flush();
     __syncthreads();
     if (s_fail && threadIdx.x == 0) raise_status(C.ctl, 0, ZC_E_DEVICE_TIMEOUT);
 }
