@@ -25,6 +25,7 @@ struct DecParams {
     uint32_t spec;           // the container is long enough to read stream 0's tables before the header is checked
     uint32_t spin_limit;     // polls after which a wait for a staged piece gives up
     uint32_t skip_copy;      // test hook: the copies of the pieces are not started
+    uint32_t sliced;         // large chunks: pieces are staged slice by slice and lane by lane (see run_chunks)
     unsigned long long call_id;
 };
 
@@ -43,7 +44,7 @@ struct DecBatchParams {
     unsigned long long call_id;
     uint32_t cs, sub, chunk_bytes, format, group, pool_bytes;
     uint32_t n_tensors, total_chunks, tensor_base, n_ranges;
-    uint32_t spin_limit, skip_copy;
+    uint32_t spin_limit, skip_copy, sliced;
     DecItem item[kDecBatchMax];
 };
 
@@ -51,6 +52,9 @@ constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 
 constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
 constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
 constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
+constexpr uint32_t kSliceSyms = 128;               // symbols a lane decodes from one slice of its subchunk
+constexpr uint32_t kSliceBytes = 256;              // copied per slice: 15 bytes of alignment + 128 * 12 bits + the window's look-ahead fit
+constexpr uint32_t kSliceSlot = 272;               // a lane's slot
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
@@ -358,6 +362,7 @@ struct DecShared {                   // what the block's prologue leaves for the
     uint32_t pairs0, pairs1;         // the stream's table yields two symbols per lookup
     unsigned long long sec0, sec1;   // byte offsets of the streams' sections
     unsigned long long payload_off, payload_bytes;
+    uint32_t pool_bytes;             // bytes of this warp's pool
 };
 
 template <bool V> struct BoolTag { static constexpr bool value = V; };
@@ -384,10 +389,19 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
     // pool: symbols of stream 0 (if coded), of stream 1 (if coded), then one staging slot per coded stream
     constexpr uint32_t rows1_off = H0 ? kRowsBytes : 0;
     constexpr uint32_t slots_off = rows1_off + (H1 ? kRowsBytes : 0);
-    const uint32_t slot_room = P.pool_bytes > slots_off ? P.pool_bytes - slots_off : 0u;
+    const uint32_t slot_room = S.pool_bytes > slots_off ? S.pool_bytes - slots_off : 0u;
     const uint32_t slot_bytes = kHuff ? (slot_room / (kHuff ? kHuff : 1)) & ~15u : 0u;
     const uint32_t rows0_s = smem_u32(pool), rows1_s = rows0_s + rows1_off;
-    const uint32_t slot0_s = rows0_s + slots_off, slot1_s = slot0_s + (H0 ? slot_bytes : 0);
+    // A piece that does not fit its slot is staged in slices instead, lane by lane (where the geometry allows:
+    // subchunks of a multiple of kSliceSyms symbols, slots of at least 32 lane slots): the stream's slot becomes 32
+    // lane slots of kSliceSlot bytes, and every kSliceSyms symbols each lane copies the next kSliceBytes of its own
+    // subchunk there.  The copy is waited for on the spot, so this is slower than staging the piece as a whole,
+    // and much faster than decoding it from global memory.
+    const bool can_slice = P.sliced && slot_bytes >= 32 * kSliceSlot;
+    const uint32_t base0_s = rows0_s + slots_off, base1_s = base0_s + (H0 ? slot_bytes : 0u);
+    uint32_t slot0_s = base0_s, slot1_s = base1_s;
+    bool sliced0 = false, sliced1 = false;
+    constexpr uint32_t kRoundsPerSlice = kSliceSyms / R;
     // where this lane writes its quads and reads the parts it merges (see decode_round)
     const uint32_t fw = (lane >> (3 - kLog)) & (PPL - 1);
     const uint32_t wr_off = 16 * PPL * lane;
@@ -415,6 +429,34 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
     const uint32_t* pay0_g = nullptr;
     const uint32_t* pay1_g = nullptr;
     bool staged0 = false, staged1 = false, flying0 = false, flying1 = false;
+    // Sliced pieces: bits of the piece before the current slice (rel), position at the slice's start (org), and the
+    // slice that is on its way: its bytes per lane (by), where it starts in the piece (at), bytes of the whole warp (tot).
+    uint32_t rel0 = 0, rel1 = 0, org0 = 0, org1 = 0;
+    uint32_t by0 = 0, by1 = 0, at0 = 0, at1 = 0, tot0 = 0, tot1 = 0;
+    // Every lane fetches the next slice of its own subchunk, from bit rel of the piece on: 16-byte aligned, long
+    // enough for kSliceSyms symbols of 12 bits plus the window's look-ahead, not past the piece's guard (with a
+    // damaged payload a lane may have run past its piece: the copy still stays inside piece + guard).  The copies
+    // are waited for when the slice is needed; until then the warp merges and writes the symbols it has.
+    auto issue_slices = [&](const bool more0, const bool more1) {
+        by0 = by1 = 0;
+        at0 = min(16 * (rel0 >> 7), piece0); at1 = min(16 * (rel1 >> 7), piece1);
+        if (H0 && sliced0 && more0) by0 = min(kSliceBytes, piece0 + 16 - at0);
+        if (H1 && sliced1 && more1) by1 = min(kSliceBytes, piece1 + 16 - at1);
+        tot0 = H0 ? __reduce_add_sync(0xFFFFFFFFu, by0) : 0u;
+        tot1 = H1 ? __reduce_add_sync(0xFFFFFFFFu, by1) : 0u;
+        __syncwarp();                                            // every lane is done with the previous slices
+        if (tot0) flying0 = true;
+        if (tot1) flying1 = true;
+        if (P.skip_copy) return;
+        if (lane == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (tot0) mbar_expect_tx(&bar[0], tot0);
+            if (tot1) mbar_expect_tx(&bar[1], tot1);
+        }
+        __syncwarp();
+        if (by0) bulk_g2s_addr(slot0_s, reinterpret_cast<const uint8_t*>(pay0_g) + at0, by0, &bar[0]);
+        if (by1) bulk_g2s_addr(slot1_s, reinterpret_cast<const uint8_t*>(pay1_g) + at1, by1, &bar[1]);
+    };
     // Takes the table entries in nx_* (of chunk `cc`), checks them, starts the copies, and requests the entries
     // of the chunk after it.
     auto prepare = [&](const uint32_t cc) {
@@ -442,6 +484,16 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
         staged0 = staged1 = false;
         if (kHuff && !__all_sync(0xFFFFFFFFu, ok)) { err = ZC_E_CORRUPT; return; }
         // the copy takes 16 bytes more than the piece (the next piece or the guard), so window peeks stay inside
+        sliced0 = H0 && can_slice && piece0 + 16 > slot_bytes;
+        sliced1 = H1 && can_slice && piece1 + 16 > slot_bytes;
+        slot0_s = base0_s + (sliced0 ? lane * kSliceSlot : 0u);
+        slot1_s = base1_s + (sliced1 ? lane * kSliceSlot : 0u);
+        if (sliced0) staged0 = true;
+        if (sliced1) staged1 = true;
+        if (sliced0 || sliced1) {
+            rel0 = start0; rel1 = start1;
+            issue_slices(end0 > start0, end1 > start1);          // lanes that have bits at all
+        }
         if (H0 && piece0 + 16 <= slot_bytes) {
             staged0 = flying0 = true;
             if (lane == 0 && !P.skip_copy) {
@@ -489,19 +541,30 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                 for (int i = 0; i < PPL; ++i)
                     if (!H1 && (FULL || k_lane + i * k_step + r * R < c_syms))
                         asm volatile("prefetch.global.L2 [%0];" :: "l"(raw1 + i * k_step + r * R));
+                if (kHuff && (sliced0 || sliced1) && r % kRoundsPerSlice == 0) {
+                    // the slice requested after the previous one was used up (or, for the chunk's first one, while
+                    // the chunk before was merged) is needed now
+                    if (tot0) { if (mbar_wait(&bar[0], parity0, P.spin_limit)) { parity0 ^= 1; flying0 = false; } else err = ZC_E_DEVICE_TIMEOUT; }
+                    if (tot1) { if (mbar_wait(&bar[1], parity1, P.spin_limit)) { parity1 ^= 1; flying1 = false; } else err = ZC_E_DEVICE_TIMEOUT; }
+                    if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; return; }
+                    if (by0) { org0 = 8 * slot0_s + min(rel0 - 8 * at0, 127u); lane_start(pos0, w00, w01, next0, org0); }
+                    if (by1) { org1 = 8 * slot1_s + min(rel1 - 8 * at1, 127u); lane_start(pos1, w10, w11, next1, org1); }
+                    tot0 = tot1 = 0;
+                }
                 if (kHuff && r == 0) {
-                    if (H0 && staged0) {
+                    if (H0 && staged0 && !sliced0) {
                         if (mbar_wait(&bar[0], parity0, P.spin_limit)) parity0 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
-                    if (H1 && staged1) {
+                    if (H1 && staged1 && !sliced1) {
                         if (mbar_wait(&bar[1], parity1, P.spin_limit)) parity1 ^= 1; else err = ZC_E_DEVICE_TIMEOUT;
                     }
                     if (__any_sync(0xFFFFFFFFu, err == ZC_E_DEVICE_TIMEOUT)) { err = ZC_E_DEVICE_TIMEOUT; return; }
-                    flying0 = flying1 = false;
+                    if (!sliced0) flying0 = false;
+                    if (!sliced1) flying1 = false;
                     // staged: positions count from shared address 0; from global memory: from the piece, and the last
                     // readable word pair ends with the guard (piece + 16 bytes)
-                    if (H0) { if (staged0) lane_start(pos0, w00, w01, next0, 8 * slot0_s + start0); else pos0 = start0; lim0 = piece0 / 4 + 2; }
-                    if (H1) { if (staged1) lane_start(pos1, w10, w11, next1, 8 * slot1_s + start1); else pos1 = start1; lim1 = piece1 / 4 + 2; }
+                    if (H0 && !sliced0) { if (staged0) lane_start(pos0, w00, w01, next0, 8 * slot0_s + start0); else pos0 = start0; lim0 = piece0 / 4 + 2; }
+                    if (H1 && !sliced1) { if (staged1) lane_start(pos1, w10, w11, next1, 8 * slot1_s + start1); else pos1 = start1; lim1 = piece1 / 4 + 2; }
                 }
                 // ---- every lane decodes R symbols of its subchunk ----
                 if (kHuff) {
@@ -525,16 +588,21 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                         }
                     }
                     __syncwarp();
+                    if ((sliced0 || sliced1) && (r + 1) % kRoundsPerSlice == 0 && r < last_r) {
+                        if (sliced0) { rel0 += pos0 - org0; org0 = pos0; }
+                        if (sliced1) { rel1 += pos1 - org1; org1 = pos1; }
+                        issue_slices(n_my > (r + 1) * R, n_my > (r + 1) * R);
+                    }
                     if (r == last_r) {
                         // Every lane must have consumed exactly the bits of its subchunk (a ragged end decodes up to
                         // fifteen symbols too many).  Anything else means the payload does not belong to the tables.
                         bool good = true;
                         if (H0) {
-                            const uint32_t used = pos0 - (staged0 ? 8 * slot0_s : 0u);
+                            const uint32_t used = sliced0 ? rel0 + pos0 - org0 : pos0 - (staged0 ? 8 * slot0_s : 0u);
                             good = good && (FULL ? used == end0 : used - end0 <= 15 * kLmax);
                         }
                         if (H1) {
-                            const uint32_t used = pos1 - (staged1 ? 8 * slot1_s : 0u);
+                            const uint32_t used = sliced1 ? rel1 + pos1 - org1 : pos1 - (staged1 ? 8 * slot1_s : 0u);
                             good = good && (FULL ? used == end1 : used - end1 <= 15 * kLmax);
                         }
                         if (!__all_sync(0xFFFFFFFFu, good)) err = ZC_E_CORRUPT;
@@ -626,10 +694,12 @@ __device__ __forceinline__ DecSmem carve_smem(uint8_t* smem, uint32_t pool_bytes
 // together (the header check and the table build are block-wide).  Returns a zc_status, the same in every
 // thread for the block-wide checks.
 template <int FMT, int PPL, bool XOR>
-__device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem& M, const uint32_t c0, const uint32_t c_end,
-                                               const uint32_t step, uint32_t& parity0, uint32_t& parity1)
+__device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem& M, const uint32_t chunk_base, const uint32_t c_end,
+                                               const uint32_t block_index, const uint32_t n_blocks, uint32_t& parity0, uint32_t& parity1)
 {
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    // chunk chunk_base + k goes to block (k / n_warps) % n_blocks, warp k % n_warps
+    uint32_t c0 = chunk_base + block_index * n_warps + warp, step = n_blocks * n_warps;
     const uint32_t sub_w = P.chunk_bytes <= 8192 ? 2u : 4u;     // bytes per sub_end entry
     const uint64_t tab_chunk = 256, tab_sub = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull);
     // Nearly every container has stream 0 coded, its table section right behind the header.  Its code lengths
@@ -705,7 +775,28 @@ __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem
         if (!tables_ok) return ZC_E_CORRUPT;
     }
 
+    // Large chunks with both streams coded: a warp's pool was sized for one coded stream's lane slots (the plan
+    // does not say how many streams a container codes); fewer warps then share the block's pools, each with room
+    // for both, and the chunks are dealt to those warps only.
+    uint8_t* pool = M.pool;
+    uint32_t pool_bytes = P.pool_bytes;
+    if (P.sliced && huff0 && huff1) {
+        const uint32_t need = 2 * (512 * PPL + 32 * kSliceSlot);
+        if (need > P.pool_bytes) {
+            const uint32_t active = max(1u, n_warps * P.pool_bytes / need);
+            pool = M.pools + (size_t)min(warp, active - 1) * need;
+            pool_bytes = need;
+            c0 = warp < active ? chunk_base + block_index * active + warp : c_end;
+            step = n_blocks * active;
+            spec_end = spec_off = 0;
+            if (c0 < c_end) {
+                spec_end = load_sub_end(P.comp + kHeaderBytes + tab_sub, sub_w, c0, lane);
+                spec_off = reinterpret_cast<const uint32_t*>(P.comp + kHeaderBytes + tab_chunk)[c0];
+            }
+        }
+    }
     DecShared S;
+    S.pool_bytes = pool_bytes;
     S.lut0_s = smem_u32(M.lut0); S.lut1_s = smem_u32(M.lut1);
     S.pairs0 = huff0 && s_per_lookup[0] == 2;
     S.pairs1 = huff1 && s_per_lookup[1] == 2;
@@ -716,10 +807,10 @@ __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem
         first_end0 = load_sub_end(P.comp + S.sec0 + tab_sub, sub_w, c0, lane);
         first_off0 = reinterpret_cast<const uint32_t*>(P.comp + S.sec0 + tab_chunk)[c0];
     }
-    if (huff0 && !huff1) return run_chunks<FMT, PPL, true, false, XOR>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
-    if (!huff0 && !huff1) return run_chunks<FMT, PPL, false, false, XOR>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
-    if (huff0) return run_chunks<FMT, PPL, true, true, XOR>(P, S, M.pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
-    return run_chunks<FMT, PPL, false, true, XOR>(P, S, M.pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+    if (huff0 && !huff1) return run_chunks<FMT, PPL, true, false, XOR>(P, S, pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    if (!huff0 && !huff1) return run_chunks<FMT, PPL, false, false, XOR>(P, S, pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
+    if (huff0) return run_chunks<FMT, PPL, true, true, XOR>(P, S, pool, M.bar, first_end0, first_off0, c0, c_end, step, parity0, parity1);
+    return run_chunks<FMT, PPL, false, true, XOR>(P, S, pool, M.bar, 0, 0, c0, c_end, step, parity0, parity1);
 }
 
 // One tensor per launch: the warps of all blocks take the chunks in turn.
@@ -728,11 +819,10 @@ __global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
 decode_kernel(const __grid_constant__ DecParams P)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const DecSmem M = carve_smem(smem, P.pool_bytes);
     if (P.ctl && blockIdx.x == 0 && threadIdx.x == 0) P.ctl->call_id = P.call_id;
     uint32_t parity0 = 0, parity1 = 0;
-    const uint32_t err = decode_one<FMT, PPL, false>(P, M, P.c_begin + blockIdx.x * n_warps + warp, P.c_end, gridDim.x * n_warps, parity0, parity1);
+    const uint32_t err = decode_one<FMT, PPL, false>(P, M, P.c_begin, P.c_end, blockIdx.x, gridDim.x, parity0, parity1);
     if (err) raise_status(P.ctl, P.call_id, err);
 }
 
@@ -744,7 +834,6 @@ __global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
 decode_batch_kernel(const __grid_constant__ DecBatchParams B)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    const uint32_t warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const DecSmem M = carve_smem(smem, B.pool_bytes);
     if (blockIdx.x == 0 && threadIdx.x == 0 && B.tensor_base == 0) B.ctl->call_id = B.call_id;
     uint32_t parity0 = 0, parity1 = 0;
@@ -756,11 +845,11 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
         P.n_syms = B.item[t].n_syms; P.n_elems = B.item[t].n_elems; P.n_chunks = B.item[t].n_chunks;
         P.cs = B.cs; P.sub = B.sub; P.chunk_bytes = B.chunk_bytes; P.format = B.format; P.group = B.group;
         P.pool_bytes = B.pool_bytes; P.call_id = B.call_id; P.c_begin = 0; P.c_end = P.n_chunks;
-        P.spin_limit = B.spin_limit; P.skip_copy = B.skip_copy;
+        P.spin_limit = B.spin_limit; P.skip_copy = B.skip_copy; P.sliced = B.sliced;
         const uint64_t tables = 256 + (((uint64_t)4 * P.n_chunks + 15) & ~15ull) + 32ull * (P.chunk_bytes <= 8192 ? 2u : 4u) * P.n_chunks;
         P.spec = P.comp_bytes >= kHeaderBytes + tables ? 1u : 0u;
         __syncthreads();                                         // everybody is done with the previous tensor's tables
-        const uint32_t err = decode_one<FMT, PPL, XOR>(P, M, seg_lo + warp, seg_hi, n_warps, parity0, parity1);
+        const uint32_t err = decode_one<FMT, PPL, XOR>(P, M, seg_lo, seg_hi, 0, 1, parity0, parity1);
         if (err && raise_status(B.ctl, B.call_id, err)) B.ctl->failed = B.tensor_base + t + 1;
     };
 
@@ -815,7 +904,7 @@ extern "C" {
 namespace {
 
 // Launch shape for a plan: symbols per round and lane, per-warp pool, warps per block, shared memory.
-struct DecShape { uint32_t ppl, pool_bytes, warps; size_t smem; };
+struct DecShape { uint32_t ppl, pool_bytes, warps, sliced; size_t smem; };
 
 // both_coded: expect both streams to be Huffman-coded (scale bytes, deltas) instead of one
 zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
@@ -828,14 +917,18 @@ zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
     const uint32_t rows_bytes = 512 * s.ppl;
     // per warp: the coded streams' rows plus room to stage, per coded stream, a piece as large as the raw chunk
     // stream; pieces that do not fit (or chunks above 16 KiB of symbols) are read from global memory instead
+    s.sliced = p->syms_per_sub % kSliceSyms == 0 ? 1u : 0u;   // pieces beyond their slot can be staged slice by slice
     s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + std::min<uint32_t>(p->syms_per_chunk, 16384) + 32), 2 * rows_bytes);
+    // chunks above 16 KiB: whole pieces would leave room for a dozen warps at most; lane slots for sliced pieces
+    // are enough, and more warps decode
+    if (s.sliced && p->syms_per_chunk > 8192) s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + 32 * kSliceSlot), 2 * rows_bytes);
     // slack behind the last slot: what a lane can read past its piece when the payload is damaged (see window_s)
     const size_t slack = (size_t)round_up(p->syms_per_sub + p->syms_per_sub / 2 + 16, 16);
     const size_t fixed = kDecFixedSmem + 512 /* static shared */ + slack;
     size_t per_warp = 16 + s.pool_bytes;
     s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     if (s.warps < 8) {               // large chunks: stage less
-        s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + 4096 + 32), 2 * rows_bytes);
+        s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + 32 * kSliceSlot), 2 * rows_bytes);   // room for the lane slots of sliced pieces
         per_warp = 16 + s.pool_bytes;
         s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
     }
@@ -905,7 +998,7 @@ zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t co
     P.call_id = new_call_id();
     P.spec = comp_bytes >= kHeaderBytes + table_section_bytes(p->n_chunks, p->chunk_bytes) ? 1u : 0u;
     P.pool_bytes = shape.pool_bytes;
-    P.spin_limit = test_knobs().spin_limit; P.skip_copy = test_knobs().skip_copy;
+    P.spin_limit = test_knobs().spin_limit; P.skip_copy = test_knobs().skip_copy; P.sliced = shape.sliced;
     const uint32_t warps = shape.warps, ppl = shape.ppl;
     const size_t smem = shape.smem;
     // at least one block even for an empty range: the header is still checked
@@ -967,7 +1060,7 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         B.cs = p0->syms_per_chunk; B.sub = p0->syms_per_sub; B.chunk_bytes = p0->chunk_bytes;
         B.format = p0->format; B.group = p0->group; B.pool_bytes = shape.pool_bytes;
         B.tensor_base = base;
-        B.spin_limit = test_knobs().spin_limit; B.skip_copy = test_knobs().skip_copy;
+        B.spin_limit = test_knobs().spin_limit; B.skip_copy = test_knobs().skip_copy; B.sliced = shape.sliced;
         uint32_t n = 0;
         uint64_t total = 0;
         // as many tensors as fit one launch: at most kDecBatchMax, fewer than 2^32 chunks together

@@ -112,6 +112,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 }
 
 
+// the same with the destination given as a shared address
+__device__ __forceinline__ void bulk_g2s_addr(uint32_t dst_s, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst_s), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 inline int sm_count()
 {
     static int cached = 0;
