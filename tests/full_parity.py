@@ -55,7 +55,8 @@ def run(workload, chunk_kib, procs, limit):
     fmt, specs = bench.workload_specs(workload)
     if workload.endswith("_static"):
         raise SystemExit("the *_static workloads share dictionaries between tensors: see tests/test_gpu_kv_dictionary.py")
-    delta = workload.endswith("_delta")          # the XOR with the earlier checkpoint is what is coded
+    delta = "_delta" in workload                 # the XOR with the earlier checkpoint is what is coded
+    frozen = workload.endswith("_delta_frozen")  # ... with a share of the rows left untouched
     if limit:
         specs = specs[:limit]
     chunk_bytes = chunk_kib * 1024
@@ -112,7 +113,7 @@ def run(workload, chunk_kib, procs, limit):
             for spec in specs:
                 base = None
                 if delta:
-                    t, base, n = wl.checkpoint_pair(spec, dev)
+                    t, base, n = wl.checkpoint_pair(spec, dev, frozen_rows=wl.frozen_rows_of(spec) if frozen else 0.0)
                 elif spec.name.startswith("kv."):
                     t, n = wl.kv_cache_tensor(fmt, spec.seed // 10, spec.seed % 10, dev)
                 else:
