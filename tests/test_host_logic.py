@@ -300,3 +300,22 @@ def test_threaded_codebook_builder_matches_the_single_one():
                     a, b = many[t].get(s), one.get(s)
                     assert a[0] == b[0] and np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
     assert zc.build_codebooks([], np.zeros((0, 2, 256), np.uint64)) == []
+
+
+def test_codebook_builder_against_the_oracle_s_on_a_million_histograms(tmp_path):
+    """tests/codebook_fuzz.c, one process per core: ties, Fibonacci, powers of two, counts near 2^33, ...
+
+    ZC_FUZZ_HISTOGRAMS sets the total (default 10^6, or 125 000 per core where fewer than 8 cores are available)."""
+    import subprocess
+    exe = str(tmp_path / "codebook_fuzz")
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "codebook_fuzz.c")
+    subprocess.check_call(["gcc", "-O2", "-std=c99", "-Wall", "-o", exe, src, "-ldl"])
+    cores = len(os.sched_getaffinity(0))
+    total = int(os.environ.get("ZC_FUZZ_HISTOGRAMS", min(1_000_000, 125_000 * cores)))
+    per = -(-total // cores)
+    procs = [subprocess.Popen([exe, zbuild.build_library(), zo.build(), str(per), str(1000 + i)],
+                              stdout=subprocess.PIPE, text=True) for i in range(cores)]
+    outs = [p.communicate()[0] for p in procs]
+    for p, out in zip(procs, outs):
+        assert p.returncode == 0 and out.startswith("ok "), out[-2000:]
+    assert sum(int(o.split()[1]) for o in outs) >= total
