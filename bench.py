@@ -41,8 +41,8 @@ ORACLE_SAMPLE_BYTES = int(os.environ.get("ZC_ORACLE_SAMPLE_BYTES", 768 << 20))  
 # stack of 872.4 MB, 4 KiB chunks, batched kernels); traffic grows in proportion to the input, so the figure for a
 # launch over the whole stack is this ratio times its input bytes.  The write part is undercounted in a capture
 # because some of the output is still in L2 when the kernel ends.
-NCU_DRAM_BYTES_PER_INPUT_BYTE = {"decode_kernel": 1408.5e6 / 872415232.0,
-                                 "encode_kernel": 1408.9e6 / 872415232.0}
+NCU_DRAM_BYTES_PER_INPUT_BYTE = {"decode_kernel": (607251968.0 + 827155200.0) / 872415232.0,
+                                 "encode_kernel": (872882944.0 + 535107840.0) / 872415232.0}
 
 
 def measured_peaks():
