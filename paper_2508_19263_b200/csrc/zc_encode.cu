@@ -619,6 +619,20 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 const uint32_t k = 8 * g_, j = __umulhi(k, C.sub_magic);
                 return j * region + (k - j * C.sub);
             };
+            // A complete chunk of nothing but a coded stream's fill symbol takes no bits and need not be packed.  With both
+            // streams coded (delta checkpoints: stretches of unchanged weights are such chunks in both streams) every
+            // staged word is compared with the fill symbol on the way, one logic operation per word; with one coded
+            // stream such chunks are rare and are found after packing (phase C), so that path pays nothing here.
+            constexpr bool kSpotConstant = H0 && H1;
+            const uint32_t tab_slot_idx = vol32(&s_tabslot[it % kRing]);
+            uint32_t fill4[2] = {0, 0}, differs[2] = {1, 1};
+            if (kSpotConstant) {
+#pragma unroll
+                for (int hs = 0; hs < 2; ++hs) {
+                    fill4[hs] = (vol32(&s_fill[tab_slot_idx][hs]) & 0xFFu) * 0x01010101u;
+                    differs[hs] = 0;
+                }
+            }
             auto stage_group = [&](const uint4 x, const uint32_t g_, const uint32_t off) {
                 const uint32_t w[4] = {x.x, x.y, x.z, x.w};
                 uint32_t sy[2][2];
@@ -631,6 +645,7 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                     } else {
                         sts32(sym_s + hs * C.stage_stride + off, sy[s][0]);
                         sts32(sym_s + hs * C.stage_stride + off + 4, sy[s][1]);
+                        if (kSpotConstant) differs[hs] |= (sy[s][0] ^ fill4[hs]) | (sy[s][1] ^ fill4[hs]);
                         ++hs;
                     }
                 }
@@ -700,7 +715,6 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
             // ---- phase B: every lane packs the codes of its subchunk into its pack slot, from bit 0 ----
             const uint32_t lo_sym = lane * C.sub;
             const uint32_t n_my = lo_sym < c_syms ? min(C.sub, c_syms - lo_sym) : 0u;
-            const uint32_t tab_slot_idx = vol32(&s_tabslot[it % kRing]);
             const uint32_t tab_slot_s = smem_u32(tabs + tab_slot_idx * tab_words);
             // batches below this ticket belong to the same tensor
             const uint32_t t_end = (N_ITEMS > 1 && t + 1 < C.n_tensors) ? P.item[N_ITEMS > 1 ? t + 1 : 0].first_batch : C.total_batches;
@@ -746,8 +760,11 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     if (!is_huff(s)) continue;
+                    // nothing but the fill symbol (which has a code): no bits, nothing to pack
+                    const bool constant = kSpotConstant && __all_sync(0xFFFFFFFFu, differs[hs] == 0) && active &&
+                                          c_syms == C.cs && (vol32(&s_fill[tab_slot_idx][hs]) >> 8) <= kLmax;
                     // anything beyond a slot other than the last one would overwrite an older chunk in the next slot
-                    my_bits[s] = pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
+                    my_bits[s] = constant ? 0u : pack(hs, slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes);
                     // more than the slot holds: the bits beyond it do not survive the next staging
                     oversize |= my_bits[s] > 8 * C.slot_bytes;
                     ++hs;
