@@ -51,6 +51,11 @@ struct DecBatchParams {
 constexpr uint32_t kLutBytes = kLutEntries * 4;       // one decode table: 4096 entries of 4 bytes
 constexpr uint32_t kScratchBytes = 1280;           // code bookkeeping of build_lut (258 words)
 constexpr uint32_t kDecMaxWarps = 28;              // 896 threads: 72 registers per thread fit the register file
+// Launches that expect both streams to be coded (scale bytes, deltas) keep two bit readers per lane going and stage two
+// pieces per warp: fewer warps fit the shared memory anyway, and the kernels built for them get more registers.
+constexpr uint32_t kDecMaxWarpsBoth = 20;          // 640 threads: 96 registers per thread
+template <int FMT, bool XOR>
+constexpr uint32_t dec_block_warps() { return (XOR || FMT == ZC_FMT_SCALE_U8) ? kDecMaxWarpsBoth : kDecMaxWarps; }
 constexpr uint32_t kDecFixedSmem = 2 * kLutBytes + kScratchBytes;
 constexpr uint32_t kSliceSyms = 128;               // symbols a lane decodes from one slice of its subchunk
 constexpr uint32_t kSliceBytes = 256;              // copied per slice: 15 bytes of alignment + 128 * 12 bits + the window's look-ahead fit
@@ -321,6 +326,64 @@ __device__ __forceinline__ void decode_round(ZC_LANE_BITS, uint32_t lut_s, uint3
     }
 }
 
+// Two coded streams: the same words, decoded for both streams side by side.  A lane's two bit readers are independent
+// chains of dependent operations (window -> lookup -> shift -> lookup); issued alternately, one chain's shared-memory
+// latency is covered by the other's arithmetic.  word_first makes the window and the two lookups that every word
+// needs; word_second finishes the word: two more lookups from a second window in one-symbol mode, the rare extra
+// lookups of short pair entries in two-symbol mode.  Together they compute exactly what decode_word computes.
+template <int K>
+__device__ __forceinline__ void word_first(ZC_LANE_BITS, uint32_t lut_s, uint32_t& x, uint32_t& y)
+{
+    const uint32_t win = window_s(ZC_LANE_ARGS);
+    x = lut_peek(win, lut_s);
+    y = lut_peek(__funnelshift_l(0, win, x), lut_s);
+    pos = add_low_byte(pos, x + y);
+}
+template <int K>
+__device__ __forceinline__ uint32_t word_second(ZC_LANE_BITS, uint32_t lut_s, const uint32_t e0, const uint32_t e1)
+{
+    if (K == 2) {
+        if ((int)(e0 | e1) < 0) {
+            const uint32_t win = window_s(ZC_LANE_ARGS);
+            const uint32_t f = lut_peek(win, lut_s), lf = (f >> 24) & 15;
+            pos += lf;
+            if ((int)(e0 & e1) < 0) {
+                const uint32_t g = lut_peek(__funnelshift_l(0, win, lf), lut_s);
+                pos += (g >> 24) & 15;
+                return __byte_perm(__byte_perm(e0, e1, 0x0051), __byte_perm(f, g, 0x0051), 0x5410);
+            }
+            return __byte_perm(__byte_perm(e0, e1, (int)e0 < 0 ? 0x0651 : 0x0521), f, 0x5210);
+        }
+        return __byte_perm(e0, e1, 0x6521);
+    }
+    const uint32_t win = window_s(ZC_LANE_ARGS);
+    const uint32_t c = lut_peek(win, lut_s);
+    const uint32_t d = lut_peek(__funnelshift_l(0, win, c), lut_s);
+    pos = add_low_byte(pos, c + d);
+    return __byte_perm(__byte_perm(e0, e1, 0x0073), __byte_perm(c, d, 0x0073), 0x5410);
+}
+template <int K0, int K1, int PPL, bool FULL>
+__device__ __forceinline__ void decode_round2(uint32_t& posa, uint32_t& wa0, uint32_t& wa1, uint32_t& nexta, uint32_t luta_s, uint32_t wra_s,
+                                              uint32_t& posb, uint32_t& wb0, uint32_t& wb1, uint32_t& nextb, uint32_t lutb_s, uint32_t wrb_s,
+                                              uint32_t fw, uint32_t n_quads)
+{
+#pragma unroll
+    for (int q = 0; q < PPL; ++q) {
+        if (!FULL && (uint32_t)q >= n_quads) break;
+        uint32_t a[4], b[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t ax, ay, bx, by;
+            word_first<K0>(posa, wa0, wa1, nexta, luta_s, ax, ay);
+            word_first<K1>(posb, wb0, wb1, nextb, lutb_s, bx, by);
+            a[j] = word_second<K0>(posa, wa0, wa1, nexta, luta_s, ax, ay);
+            b[j] = word_second<K1>(posb, wb0, wb1, nextb, lutb_s, bx, by);
+        }
+        sts128(wra_s + 16 * ((uint32_t)q ^ fw), a[0], a[1], a[2], a[3]);
+        sts128(wrb_s + 16 * ((uint32_t)q ^ fw), b[0], b[1], b[2], b[3]);
+    }
+}
+
 // A chunk without payload bits holds nothing but the stream's fill symbol, the symbol with the all-zero code:
 // the first symbol of the table entry for a window of zeros.
 __device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
@@ -571,7 +634,19 @@ __device__ __forceinline__ uint32_t run_chunks(const DecParams& P, const DecShar
                     const uint32_t done = r * R;
                     // a ragged end decodes up to 15 symbols too many (from the bits that follow); they are not used
                     const uint32_t n_quads = FULL ? (uint32_t)PPL : (n_my > done ? (min(R, n_my - done) + 15) / 16 : 0u);
-                    if (n_quads) {
+                    // (only in the kernels built for launches that expect two coded streams: they have the registers for it)
+                    constexpr bool kSideBySide = H0 && H1 && (XOR || FMT == ZC_FMT_SCALE_U8);
+                    if (kSideBySide && n_quads && staged0 && staged1 && piece0 != 0 && piece1 != 0) {
+                        // both streams come from staged pieces: their words are decoded side by side
+                        const uint32_t wra_s = rows0_s + wr_off, wrb_s = rows1_s + wr_off;
+                        if (S.pairs0) {
+                            if (S.pairs1) decode_round2<2, 2, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wra_s, pos1, w10, w11, next1, S.lut1_s, wrb_s, fw, n_quads);
+                            else decode_round2<2, 1, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wra_s, pos1, w10, w11, next1, S.lut1_s, wrb_s, fw, n_quads);
+                        } else {
+                            if (S.pairs1) decode_round2<1, 2, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wra_s, pos1, w10, w11, next1, S.lut1_s, wrb_s, fw, n_quads);
+                            else decode_round2<1, 1, PPL, FULL>(pos0, w00, w01, next0, S.lut0_s, wra_s, pos1, w10, w11, next1, S.lut1_s, wrb_s, fw, n_quads);
+                        }
+                    } else if (n_quads) {
                         if (H0) {
                             const uint32_t wr_s = rows0_s + wr_off;
                             if (piece0 == 0) fill_quads(S.lut0_s, S.pairs0, wr_s, fw, n_quads);   // a chunk without bits: nothing but the fill symbol
@@ -815,7 +890,7 @@ __device__ __forceinline__ uint32_t decode_one(const DecParams& P, const DecSmem
 
 // One tensor per launch: the warps of all blocks take the chunks in turn.
 template <int FMT, int PPL>
-__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
+__global__ void __launch_bounds__(dec_block_warps<FMT, false>() * 32, 1)
 decode_kernel(const __grid_constant__ DecParams P)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -830,7 +905,7 @@ decode_kernel(const __grid_constant__ DecParams P)
 // concatenated chunk index space, tensor by tensor; it builds the tables of a tensor once for its whole share.
 // XOR: the launch has base tensors (delta form); a kernel of its own so that the plain form pays nothing for it.
 template <int FMT, int PPL, bool XOR>
-__global__ void __launch_bounds__(kDecMaxWarps * 32, 1)
+__global__ void __launch_bounds__(dec_block_warps<FMT, XOR>() * 32, 1)
 decode_batch_kernel(const __grid_constant__ DecBatchParams B)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -926,15 +1001,16 @@ zc_status dec_shape(const zc_plan_t* p, bool both_coded, DecShape* out)
     const size_t slack = (size_t)round_up(p->syms_per_sub + p->syms_per_sub / 2 + 16, 16);
     const size_t fixed = kDecFixedSmem + 512 /* static shared */ + slack;
     size_t per_warp = 16 + s.pool_bytes;
-    s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
+    const size_t max_warps = coded == 2 ? kDecMaxWarpsBoth : kDecMaxWarps;     // the kernels' launch bounds
+    s.warps = (uint32_t)std::min<size_t>(max_warps, (kMaxSmem - fixed - 1024) / per_warp);
     if (s.warps < 8) {               // large chunks: stage less
         s.pool_bytes = std::max<uint32_t>(coded * (rows_bytes + 32 * kSliceSlot), 2 * rows_bytes);   // room for the lane slots of sliced pieces
         per_warp = 16 + s.pool_bytes;
-        s.warps = (uint32_t)std::min<size_t>(kDecMaxWarps, (kMaxSmem - fixed - 1024) / per_warp);
+        s.warps = (uint32_t)std::min<size_t>(max_warps, (kMaxSmem - fixed - 1024) / per_warp);
     }
     // the table build uses 8 KiB of the pools and 256 threads
     while (s.warps * (size_t)s.pool_bytes < 8192) ++s.warps;
-    if (s.warps < 8 || s.warps > kDecMaxWarps) return ZC_E_UNSUPPORTED;
+    if (s.warps < 8 || s.warps > max_warps) return ZC_E_UNSUPPORTED;
     s.smem = kDecFixedSmem + s.warps * per_warp + slack;
     *out = s;
     return ZC_OK;
