@@ -36,6 +36,12 @@ uint32_t zc_test_decoder_warps(const zc_plan_t* plan, uint32_t both_coded);
 void zc_test_set_wait_limit(uint32_t polls);
 void zc_test_stall_encoder(uint32_t first_ticket);
 void zc_test_stall_decoder(uint32_t on);
+/* Development build of the library (compiled with -DZC_DEBUG_CHECKS=1): every shared-memory and global-memory
+ * access the kernels make through their load/store helpers is checked against the block's shared window and the
+ * buffers of the launch; a violation is counted and the access skipped (no trap, no fault).  This call waits for the
+ * device, stores the number of refused shared accesses in out[0] and of refused global accesses in out[1], clears
+ * the counters and returns 1.  The ordinary build has no checks: it returns 0 and leaves out alone. */
+int zc_test_debug_counts(uint32_t out[2]);
 #ifdef __cplusplus
 }
 #endif

@@ -56,7 +56,8 @@ class DictInfo(C.Structure):
 
 
 def _load():
-    path = _build.LIB
+    # ZC_LIBRARY: another build of the same library (the development build with in-kernel checks), for tests
+    path = os.environ.get("ZC_LIBRARY") or _build.LIB
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing: run paper_2508_19263_b200.build.build_library() "
                           "(or __graft_entry__.build()) first; there is no fallback implementation")
@@ -145,6 +146,8 @@ def _load():
     L.zc_test_encoder_workers.argtypes = [vp, C.c_uint32, C.c_uint32]
     L.zc_test_decoder_warps.restype = C.c_uint32
     L.zc_test_decoder_warps.argtypes = [vp, C.c_uint32]
+    L.zc_test_debug_counts.restype = C.c_int
+    L.zc_test_debug_counts.argtypes = [C.POINTER(C.c_uint32)]
     for name in ("zc_test_set_wait_limit", "zc_test_stall_encoder", "zc_test_stall_decoder"):
         getattr(L, name).restype = None
         getattr(L, name).argtypes = [C.c_uint32]
@@ -510,6 +513,12 @@ def test_stall_encoder(first_ticket: int) -> None:
 def test_stall_decoder(on: bool) -> None:
     """zc_test_stall_decoder."""
     _lib.zc_test_stall_decoder(1 if on else 0)
+
+
+def test_debug_counts():
+    """zc_test_debug_counts: (refused shared accesses, refused global accesses) of a development build, else None."""
+    out = (C.c_uint32 * 2)()
+    return (int(out[0]), int(out[1])) if _lib.zc_test_debug_counts(out) else None
 
 
 def test_encoder_workers(p: Plan, n_coded: int, wide_slots: bool) -> int:

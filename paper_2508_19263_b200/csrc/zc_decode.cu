@@ -63,11 +63,13 @@ constexpr uint32_t kSliceSlot = 272;               // a lane's slot
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
+    if (p) ZC_DBG_SHARED(addr, 4, return);
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}"
                  :: "r"(addr), "r"(v), "r"((uint32_t)p) : "memory");
 }
 __device__ __forceinline__ uint32_t lds32_if(bool p, uint32_t addr)
 {
+    if (p) ZC_DBG_SHARED(addr, 4, return 0);
     uint32_t v;
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\tmov.u32 %0, 0;\n\t@q ld.shared.u32 %0, [%1];\n\t}"
                  : "=r"(v) : "r"(addr), "r"((uint32_t)p));
@@ -230,6 +232,7 @@ __device__ __forceinline__ uint32_t load_sub_end(const uint8_t* tab, uint32_t wi
 
 __device__ __forceinline__ void lane_start(ZC_LANE_BITS, uint32_t at)
 {
+    ZC_DBG_SHARED((at >> 3) & ~3u, 4, return); ZC_DBG_SHARED(((at >> 3) & ~3u) + 4, 4, return);
     const uint32_t a = (at >> 3) & ~3u;
     pos = at;
     asm volatile("ld.shared.u32 %0, [%2];\n\tld.shared.u32 %1, [%2+4];" : "=r"(w0), "=r"(w1) : "r"(a));
@@ -258,10 +261,12 @@ __device__ __forceinline__ uint32_t add_low_byte(uint32_t pos, uint32_t x) { ret
 
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
+    ZC_DBG_SHARED(addr, 16, return);
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
+    ZC_DBG_SHARED(addr, 16, return make_uint4(0, 0, 0, 0));
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
@@ -1025,6 +1030,19 @@ unsigned long long new_call_id()
 
 }  // namespace
 
+}  // extern "C"
+namespace zc {
+void debug_counts_decode(uint32_t out[2])
+{
+#if ZC_DEBUG_CHECKS
+    dbg_read_counts(out);
+#else
+    (void)out;
+#endif
+}
+}  // namespace zc
+extern "C" {
+
 uint32_t zc_test_decoder_warps(const zc_plan_t* p, uint32_t both_coded)
 {
     DecShape sh;
@@ -1084,6 +1102,11 @@ zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t co
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        dbg_set_ranges(st, d_comp, comp_bytes, d_out,
+                       (size_t)std::min<uint64_t>((uint64_t)n_chunks * p->chunk_bytes, p->input_bytes - (uint64_t)first_chunk * p->chunk_bytes),
+                       d_workspace, sizeof(Control));
+#endif
         kern<<<grid, warps * 32, smem, st>>>(P);
         e = cudaGetLastError();
     };
@@ -1169,6 +1192,15 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         auto launch = [&](auto kern) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
             if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+            DbgHull rd, wr;
+            for (uint32_t i = 0; i < n; ++i) {
+                rd.add(B.item[i].comp, B.item[i].comp_bytes);
+                rd.add(B.item[i].base, B.item[i].input_bytes);
+                wr.add(B.item[i].out, B.item[i].input_bytes);
+            }
+            dbg_set_ranges(st, rd.ptr(), rd.bytes(), wr.ptr(), wr.bytes(), d_workspace, sizeof(Control));
+#endif
             kern<<<grid, shape.warps * 32, shape.smem, st>>>(B);
             e = cudaGetLastError();
         };

@@ -100,6 +100,7 @@ __device__ __forceinline__ void st_flag(unsigned long long* p, unsigned long lon
 
 __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 {
+    if (p) ZC_DBG_SHARED(addr, 4, return);
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}"
                  :: "r"(addr), "r"(v), "r"((uint32_t)p) : "memory");
 }
@@ -109,6 +110,7 @@ __device__ __forceinline__ void sts32_if(bool p, uint32_t addr, uint32_t v)
 // pending bits left-aligned.
 __device__ __forceinline__ void put_bits(uint32_t code, uint32_t len, uint32_t& hi, uint32_t& nb, uint32_t& waddr, uint32_t limit)
 {
+    if (nb + len > 31 && waddr < limit) ZC_DBG_SHARED(waddr, 4, return);
     hi |= code >> nb;
     const uint32_t lo = __funnelshift_r(0, code, nb);           // the bits that do not fit: code << (32 - nb), 0 if nb == 0
     const uint32_t n = nb + len;
@@ -908,6 +910,28 @@ RowShape row_shape(const zc_plan_t* p, uint32_t n_huff)
     return s;
 }
 
+#if ZC_DEBUG_CHECKS
+// development build: the address ranges the launch may touch (hulls over the tensors of the launch)
+template <int N_ITEMS>
+void dbg_ranges_of(const EncParamsT<N_ITEMS>& P, cudaStream_t st)
+{
+    DbgHull rd, wr, ws;
+    const uint32_t n = N_ITEMS > 1 ? P.c.n_tensors : 1;
+    for (uint32_t i = 0; i < n; ++i) {
+        const EncItem& it = P.item[i];
+        rd.add(it.in, it.input_bytes);
+        rd.add(it.base, it.input_bytes);
+        // no container is larger than its tables plus 12 bits per symbol of either stream, padding and guard
+        wr.add(it.out, it.lay.payload_off + 3 * it.n_syms + 32ull * it.n_chunks + 64);
+        if (P.c.counters) ws.add(P.c.counters + it.index, sizeof(TensorCounters));
+        if (N_ITEMS > 1 && P.c.tables) ws.add(P.c.tables + it.table, sizeof(EncTables));
+    }
+    ws.add(P.c.ctl, sizeof(Control));
+    ws.add(P.c.flags, 8ull * std::max<uint32_t>(P.c.total_batches, 1));
+    dbg_set_ranges(st, rd.ptr(), rd.bytes(), wr.ptr(), wr.bytes(), ws.ptr(), ws.bytes());
+}
+#endif
+
 template <int N_ITEMS>
 cudaError_t launch_encode_rows(const EncParamsT<N_ITEMS>& P, uint32_t format, const RowShape& sh, const zc_plan_t* p0, cudaStream_t st)
 {
@@ -918,6 +942,9 @@ cudaError_t launch_encode_rows(const EncParamsT<N_ITEMS>& P, uint32_t format, co
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
         if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        dbg_ranges_of(P, st);
+#endif
         kern<<<grid, (sh.workers + 2) * 32, sh.smem, st>>>(P, RP);
         e = cudaGetLastError();
     };
@@ -1017,6 +1044,9 @@ cudaError_t launch_encode(const EncParamsT<N_ITEMS>& P, uint32_t format, const E
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
         if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        dbg_ranges_of(P, st);
+#endif
         kern<<<grid, (sh.workers + 1) * 32, sh.smem, st>>>(P);
         e = cudaGetLastError();
     };
@@ -1105,6 +1135,17 @@ uint64_t max_batches_of(const zc_plan_t* p)
 }
 
 }  // namespace
+
+namespace zc {
+void debug_counts_encode(uint32_t out[2])
+{
+#if ZC_DEBUG_CHECKS
+    dbg_read_counts(out);
+#else
+    (void)out;
+#endif
+}
+}  // namespace zc
 
 extern "C" {
 

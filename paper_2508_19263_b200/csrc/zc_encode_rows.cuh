@@ -46,16 +46,19 @@ struct RowParams {           // appended to the common parameters
 
 __device__ __forceinline__ void cp_async16(uint32_t dst_s, const void* src, uint32_t src_bytes)
 {
+    ZC_DBG_SHARED(dst_s, 16, return); if (src_bytes) ZC_DBG_GLOBAL(src, src_bytes, 16, false, return);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst_s), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src_s, uint32_t bytes)
 {
+    ZC_DBG_GLOBAL(dst, bytes, 16, true, return); ZC_DBG_SHARED(src_s, 16, return); ZC_DBG_SHARED(src_s + bytes - 16, 16, return);
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(dst), "r"(src_s), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint4 lds128e(uint32_t addr)
 {
+    ZC_DBG_SHARED(addr, 16, return make_uint4(0, 0, 0, 0));
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;

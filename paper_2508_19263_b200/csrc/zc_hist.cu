@@ -17,6 +17,7 @@ constexpr int kHistThreads = 512;
 
 __device__ __forceinline__ void red_add1(uint32_t addr)
 {
+    ZC_DBG_SHARED(addr, 4, return);
     asm volatile("red.shared.add.u32 [%0], 1;" :: "r"(addr) : "memory");
 }
 
@@ -207,6 +208,17 @@ hist_batch_kernel(const __grid_constant__ HistBatchParams B)
 
 }  // namespace zc
 
+namespace zc {
+void debug_counts_hist(uint32_t out[2])
+{
+#if ZC_DEBUG_CHECKS
+    dbg_read_counts(out);
+#else
+    (void)out;
+#endif
+}
+}  // namespace zc
+
 using namespace zc;
 
 extern "C" {
@@ -230,6 +242,12 @@ zc_status zc_histogram_xor(const zc_plan_t* p, const void* d_in, const void* d_b
     auto launch = [&](auto kern) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        DbgHull rd;
+        rd.add(d_in, p->input_bytes);
+        rd.add(d_base, p->input_bytes);
+        dbg_set_ranges(st, rd.ptr(), rd.bytes(), d_hist, 2 * 256 * sizeof(uint64_t), nullptr, 0);
+#endif
         kern<<<grid, kHistThreads, smem, st>>>((const uint8_t*)d_in, (const uint8_t*)d_base, p->input_bytes, p->n_syms,
                                                 (unsigned long long*)d_hist);
         e = cudaGetLastError();
@@ -287,6 +305,11 @@ zc_status zc_histogram_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pla
         auto launch = [&](auto kern) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+            DbgHull rd;
+            for (uint32_t i = 0; i < n; ++i) { rd.add(B.item[i].in, B.item[i].input_bytes); rd.add(B.item[i].base, B.item[i].input_bytes); }
+            dbg_set_ranges(st, rd.ptr(), rd.bytes(), B.hist, (size_t)n * 2 * 256 * sizeof(uint64_t), nullptr, 0);
+#endif
             kern<<<grid, kHistThreads, smem, st>>>(B);
             e = cudaGetLastError();
         };

@@ -128,6 +128,20 @@ void zc_test_set_wait_limit(uint32_t polls) { test_knobs().spin_limit = polls ? 
 void zc_test_stall_encoder(uint32_t first_ticket) { test_knobs().first_ticket = first_ticket; }
 void zc_test_stall_decoder(uint32_t on) { test_knobs().skip_copy = on ? 1u : 0u; }
 
+int zc_test_debug_counts(uint32_t out[2])
+{
+#if defined(ZC_DEBUG_CHECKS) && ZC_DEBUG_CHECKS
+    out[0] = out[1] = 0;
+    debug_counts_hist(out);
+    debug_counts_encode(out);
+    debug_counts_decode(out);
+    return 1;
+#else
+    (void)out;
+    return 0;
+#endif
+}
+
 zc_status zc_plan(zc_format fmt, uint64_t n_elems, uint32_t chunk_bytes, zc_plan_t** out)
 {
     if (!out) return ZC_E_INVALID_ARG;

@@ -119,6 +119,11 @@ struct TestKnobs {
     uint32_t skip_copy;      // the decoder does not start the copies of the pieces it then waits for
 };
 TestKnobs& test_knobs();
+// Development build (-DZC_DEBUG_CHECKS=1): each translation unit with kernels adds its counts of refused shared and
+// global accesses to out[0] and out[1] and clears them; in the ordinary build they do nothing.
+void debug_counts_hist(uint32_t out[2]);
+void debug_counts_encode(uint32_t out[2]);
+void debug_counts_decode(uint32_t out[2]);
 constexpr uint32_t kDefaultSpinLimit = 1u << 22;
 
 }  // namespace zc
