@@ -83,12 +83,13 @@ DEBUG_LIB = os.path.join(HERE, "libzc_debug.so")
 
 def build_debug_library(force: bool = False) -> str:
     """The development build: the same sources with -DZC_DEBUG_CHECKS=1 (in-kernel checks of every access the
-    kernels' load/store helpers make), as libzc_debug.so with objects of its own.  Tests only."""
+    kernels' load/store helpers make), as libzc_debug.so with objects of its own; ptxas at -O1, so that it builds
+    in a fraction of the library's time (its speed does not matter).  Tests only."""
     if not force and os.path.exists(DEBUG_LIB):
         t = os.path.getmtime(DEBUG_LIB)
         if _header_time() <= t and all(os.path.getmtime(os.path.join(CSRC, f)) <= t for f in SOURCES):
             return DEBUG_LIB
-    return build_library(force=force, lib=DEBUG_LIB, flags=["-DZC_DEBUG_CHECKS=1"], objdir=OBJDIR + "_debug")
+    return build_library(force=force, lib=DEBUG_LIB, flags=["-DZC_DEBUG_CHECKS=1", "-Xptxas", "-O1"], objdir=OBJDIR + "_debug")
 
 
 if __name__ == "__main__":
