@@ -222,7 +222,8 @@ __device__ __noinline__ bool all_symbols_are(uint32_t src, uint32_t n, uint32_t 
 // H0 / H1: stream 0 / 1 is Huffman-coded (the same for every tensor of a launch; a template parameter so that
 // the code of a raw stream's packing and copy-out does not exist and the kernel stays small).
 template <int FMT, int N_ITEMS, bool H0, bool H1>
-__global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, 3)
+// (with both streams coded the lane regions leave room for two blocks per SM at most: those kernels may use the registers of a third)
+__global__ void __launch_bounds__((kEncMaxWorkers + 1) * 32, (H0 && H1) ? 2 : 3)
 encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -754,10 +755,62 @@ encode_kernel(const __grid_constant__ EncParamsT<N_ITEMS> P)
                 if (seen & 16) bad = t + 1;                             // an entry without a code carries bit 4
                 return 8 * (waddr - w0) + nb;
             };
+            // Both streams at once: two independent accumulators per lane, their table lookups and shifts issued
+            // alternately (one stream's shared-memory latency is covered by the other's arithmetic).
+            auto pack2 = [&](const uint32_t slot_off, const uint32_t room, uint32_t& bits_a, uint32_t& bits_b) {
+                const uint32_t rega = smem_u32(stage + lane * region), regb = rega + C.stage_stride;
+                const uint32_t taba = tab_slot_s, tabb = tab_slot_s + 1024;
+                const uint32_t wa0 = rega + slot_off, lima = wa0 + room, wb0 = regb + slot_off, limb = wb0 + room;
+                uint32_t hia = 0, nba = 0, wa = wa0, hib = 0, nbb = 0, wb = wb0, seen = 0;
+                const uint32_t srca = rega + sym_off, srcb = regb + sym_off;
+                const uint32_t full_words = n_my / 4;
+                for (uint32_t i = 0; i < full_words; ++i) {
+                    const uint32_t fa = lds32(srca + 4 * i), fb = lds32(srcb + 4 * i);
+                    const uint32_t a0 = lds32(taba + 4u * __byte_perm(fa, 0, 0x4440));
+                    const uint32_t b0 = lds32(tabb + 4u * __byte_perm(fb, 0, 0x4440));
+                    const uint32_t a1 = lds32(taba + 4u * __byte_perm(fa, 0, 0x4441));
+                    const uint32_t b1 = lds32(tabb + 4u * __byte_perm(fb, 0, 0x4441));
+                    const uint32_t a2 = lds32(taba + 4u * __byte_perm(fa, 0, 0x4442));
+                    const uint32_t b2 = lds32(tabb + 4u * __byte_perm(fb, 0, 0x4442));
+                    const uint32_t a3 = lds32(taba + 4u * __byte_perm(fa, 0, 0x4443));
+                    const uint32_t b3 = lds32(tabb + 4u * __byte_perm(fb, 0, 0x4443));
+                    seen |= a0 | a1 | a2 | a3 | b0 | b1 | b2 | b3;
+                    put_bits((a0 | __funnelshift_r(a1, 0, a0)) & 0xFFFFFF00u, (a0 + a1) & 31, hia, nba, wa, lima);
+                    put_bits((b0 | __funnelshift_r(b1, 0, b0)) & 0xFFFFFF00u, (b0 + b1) & 31, hib, nbb, wb, limb);
+                    put_bits((a2 | __funnelshift_r(a3, 0, a2)) & 0xFFFFFF00u, (a2 + a3) & 31, hia, nba, wa, lima);
+                    put_bits((b2 | __funnelshift_r(b3, 0, b2)) & 0xFFFFFF00u, (b2 + b3) & 31, hib, nbb, wb, limb);
+                }
+                for (uint32_t i = 4 * full_words; i < n_my; ++i) {      // ragged end of the last chunk
+                    const uint32_t fa = lds32(srca + (i & ~3u)), fb = lds32(srcb + (i & ~3u));
+                    const uint32_t ea = lds32(taba + (((fa >> (8 * (i & 3))) & 0xFF) << 2));
+                    const uint32_t eb = lds32(tabb + (((fb >> (8 * (i & 3))) & 0xFF) << 2));
+                    seen |= ea | eb;
+                    put_bits(ea & 0xFFFFFF00u, ea & 31, hia, nba, wa, lima);
+                    put_bits(eb & 0xFFFFFF00u, eb & 31, hib, nbb, wb, limb);
+                }
+                if (active && wa < lima) sts32(wa, hia);
+                if (active && wb < limb) sts32(wb, hib);
+                if (seen & 16) bad = t + 1;
+                bits_a = 8 * (wa - wa0) + nba;
+                bits_b = 8 * (wb - wb0) + nbb;
+            };
             bool oversize = false;
             uint32_t my_bits[2] = {0, 0};
             const bool last_slot = slot_idx + 1 == n_slots;
-            {
+            bool packed_both = false;
+            if (H0 && H1) {
+                bool constant[2];
+#pragma unroll
+                for (int hs = 0; hs < 2; ++hs)
+                    constant[hs] = kSpotConstant && __all_sync(0xFFFFFFFFu, differs[hs] == 0) && active && c_syms == C.cs &&
+                                   (vol32(&s_fill[tab_slot_idx][hs]) >> 8) <= kLmax;
+                if (!constant[0] && !constant[1]) {
+                    pack2(slot, last_slot ? C.slot_bytes + C.sub : C.slot_bytes, my_bits[0], my_bits[1]);
+                    oversize = my_bits[0] > 8 * C.slot_bytes || my_bits[1] > 8 * C.slot_bytes;
+                    packed_both = true;
+                }
+            }
+            if (!packed_both) {
                 uint32_t hs = 0;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
