@@ -307,6 +307,59 @@ def test_xor_delta_single_calls_match_the_oracle_on_the_xor(fmt, chunk_bytes):
         assert np.array_equal(back[: p.input_bytes], cur[: p.input_bytes]) and (back[p.input_bytes:] == 0xEE).all()
 
 
+def _mixed_delta(fmt, chunk_bytes):
+    """base, current, their XOR and the element count: chunks 0, 3, 5, 8, 10 and the ragged end unchanged; 1-2 mantissa
+    bits only; 4 lowest exponent bit only; 6-7 everything; 9 mantissa bits in its first half."""
+    G = zo.group(fmt)
+    cs = chunk_bytes // 2
+    n_syms = 11 * cs + cs // 3 + 5
+    n = n_syms * G
+    rng = np.random.default_rng(chunk_bytes + fmt)
+    base = _weights(fmt, n, 5 + chunk_bytes)[: 2 * n_syms].copy()
+    delta = np.zeros_like(base)
+    if fmt == zc.FMT_BF16:
+        view, mant, expo, full = delta.view(np.uint16), 0x0003, 0x0080, 0x10000     # sign 15, exponent 14..7, mantissa 6..0
+    else:
+        view, mant, expo, full = delta, 0x03, 0x08, 0x100                             # sign 7, exponent 6..3, mantissa 2..0
+    per_chunk = 2 * cs // view.itemsize
+    def span(c0, c1): return view[c0 * per_chunk: c1 * per_chunk]
+    d = span(1, 3); d[:] = rng.integers(0, mant + 1, d.size) * (rng.random(d.size) < 0.4)
+    d = span(4, 5); d[:] = (rng.random(d.size) < 0.05) * expo
+    d = span(6, 8); d[:] = rng.integers(0, full, d.size) * (rng.random(d.size) < 0.2)
+    d = span(9, 10); d[: d.size // 2] = rng.integers(0, mant + 1, d.size // 2)
+    return base, base ^ delta, delta, n
+
+
+@pytest.mark.parametrize("fmt", [zc.FMT_BF16, zc.FMT_FP8_E4M3])
+@pytest.mark.parametrize("chunk_bytes", [2048, 4096, 16384, 65536])
+def test_xor_delta_with_unchanged_stretches(fmt, chunk_bytes):
+    """A later checkpoint in which whole stretches did not move, stretches where only the low mantissa bits moved (the
+    exponent stream of those chunks is constant, the other stream is not), stretches where only exponent bits
+    moved, ordinary stretches, and an unchanged ragged end: every mix of constant and coded chunks in the two
+    streams, with both streams Huffman-coded."""
+    cs = chunk_bytes // 2
+    base, cur, delta, n = _mixed_delta(fmt, chunk_bytes)
+    p = zc.plan(fmt, n, chunk_bytes)
+    d_cur, d_base = _to_dev(cur), _to_dev(base)
+    hist = zc.histogram(p, d_cur, d_base=d_base).cpu().numpy().astype(np.uint64)
+    assert np.array_equal(hist, zo.histogram(fmt, delta, n))
+    for policy in (zc.POLICY_HUFF_ALL, zc.POLICY_AUTO):
+        cb, ocb = zc.build_codebook(p, hist, policy), zo.build_codebook(hist, policy)
+        d_out = torch.full((p.max_compressed_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+        ws = torch.empty(p.workspace_bytes, dtype=torch.uint8, device=DEV)
+        nbytes = zc.compress(p, cb, d_cur, d_out, ws, d_base=d_base)
+        want = zo.compress(fmt, delta, n, chunk_bytes, ocb)
+        assert nbytes == want.size and np.array_equal(d_out[:nbytes].cpu().numpy(), want)
+        if policy == zc.POLICY_HUFF_ALL:
+            hd = zo.parse_header(want)
+            assert all(st["payload_bits"] < 8 * 4 * cs for st in hd["streams"])      # most chunks of either stream cost nothing
+        d_back = torch.full((p.input_bytes + 32,), 0xEE, dtype=torch.uint8, device=DEV)
+        zc.decompress(p, d_out, nbytes, d_back, ws, d_base=d_base)
+        assert zc.device_status(p, ws) == zc.OK
+        back = d_back.cpu().numpy()
+        assert np.array_equal(back[: p.input_bytes], cur[: p.input_bytes]) and (back[p.input_bytes:] == 0xEE).all()
+
+
 def test_xor_delta_batched_calls():
     fmt, chunk_bytes = zc.FMT_BF16, 4096
     sizes = _sizes(fmt, chunk_bytes)
