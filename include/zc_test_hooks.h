@@ -28,9 +28,10 @@ zc_status zc_test_merge16(zc_format fmt, const uint8_t* h_e8, const uint8_t* h_s
  *                           never packed and every look-back waits for a word nobody posts
  *   zc_test_stall_decoder   the decoder does not start the copies of the pieces it waits for */
 /* Launch shapes (host arithmetic only, no GPU): worker warps per block the encoder would use for a plan
- * with n_coded Huffman-coded streams (0..2) and narrow or wide pack slots, and warps per block of the
- * decoder with one or both streams coded.  0 = the kernels cannot take this plan.  A test checks that
- * every chunk size zc_plan accepts gives at least one. */
+ * with n_coded Huffman-coded streams (0..2) and pack slots of class wide_slots (0: 8 bits per symbol, 1: 12 bits,
+ * 2: one slot of 4 bits per symbol, which the library picks for chunks from 16 KiB whose codes are short), and warps
+ * per block of the decoder with one or both streams coded.  0 = the kernels cannot take this plan.  A test checks
+ * that every chunk size zc_plan accepts gives at least one. */
 uint32_t zc_test_encoder_workers(const zc_plan_t* plan, uint32_t n_coded, uint32_t wide_slots);
 uint32_t zc_test_decoder_warps(const zc_plan_t* plan, uint32_t both_coded);
 void zc_test_set_wait_limit(uint32_t polls);

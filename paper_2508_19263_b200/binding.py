@@ -521,8 +521,9 @@ def test_debug_counts():
     return (int(out[0]), int(out[1])) if _lib.zc_test_debug_counts(out) else None
 
 
-def test_encoder_workers(p: Plan, n_coded: int, wide_slots: bool) -> int:
-    return int(_lib.zc_test_encoder_workers(p._h, n_coded, 1 if wide_slots else 0))
+def test_encoder_workers(p: Plan, n_coded: int, wide_slots: int) -> int:
+    """zc_test_encoder_workers; wide_slots is the slot class 0, 1 or 2."""
+    return int(_lib.zc_test_encoder_workers(p._h, n_coded, int(wide_slots)))
 
 
 def test_decoder_warps(p: Plan, both_coded: bool) -> int:

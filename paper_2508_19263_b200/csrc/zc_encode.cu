@@ -1017,13 +1017,15 @@ cudaError_t launch_encode_rows(const EncParamsT<N_ITEMS>& P, uint32_t format, co
 }
 
 // Shared-memory shape of a launch for given chunk geometry, number of coded streams and slot size.
+constexpr uint32_t kSlotsNarrow = 0, kSlotsWide = 1, kSlotsHalf = 2;    // pack slots of 8 / 12 / 4 bits per symbol
 struct EncShape { uint32_t n_slots, slot_bytes, region_bytes, stage_stride, workers, per_sm; size_t smem; };
 
-zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* out)
+// slots: kSlotsNarrow / kSlotsWide / kSlotsHalf (see slot_class)
+zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, uint32_t slots, EncShape* out)
 {
     EncShape s{};
     const size_t fixed = (size_t)4 * kTabSlots * 256 * std::max<uint32_t>(n_huff, 1);
-    s.slot_bytes = wide ? p->syms_per_sub + p->syms_per_sub / 2 : p->syms_per_sub;
+    s.slot_bytes = slots == kSlotsWide ? p->syms_per_sub + p->syms_per_sub / 2 : p->syms_per_sub;
     // pack slots per lane region: first as many resident blocks of 8 worker warps per SM as possible (up to 3),
     // then as many slots (up to 3) as that number of blocks leaves room for
     s.n_slots = 1;
@@ -1034,6 +1036,15 @@ zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* ou
         // a second slot is worth a resident block (with one slot every turn waits for its look-back), a third is not
         const uint32_t score = blocks * std::min<uint32_t>(ns, 2) * 4 + ns;
         if (blocks > 0 && score >= best_score) { best_score = score; s.n_slots = ns; }
+    }
+    // Long subchunks: lane regions of (slots + 1) * sub bytes leave room for a handful of warps per SM.  One slot of
+    // half a subchunk is enough to be correct (a lane writes at most 1.5 bytes per symbol it has read, so packing from
+    // the start of a region of 1.5 * sub bytes never overtakes the symbols still to be read); a chunk whose bits do
+    // not fit the slot leaves at once instead of waiting up to three turns.  Chosen (slot_class) for code tables that
+    // promise well under 4 bits per symbol: where most chunks overflow the slot every turn waits for its own look-back.
+    if (slots == kSlotsHalf) {
+        s.n_slots = 1;
+        s.slot_bytes = p->syms_per_sub / 2;
     }
     s.region_bytes = s.n_slots * s.slot_bytes + p->syms_per_sub + 4;
     s.stage_stride = kSubs * s.region_bytes;
@@ -1050,10 +1061,14 @@ zc_status enc_shape(const zc_plan_t* p, uint32_t n_huff, bool wide, EncShape* ou
 
 // Wide pack slots (12 bits per symbol) for code tables whose codes are long on average (decided per stream when
 // the codebook is built).  Shorter codes get slots of 8 bits per symbol and the slow path for the rare subchunk
-// that needs more.
-bool wants_wide_slots(const zc_codebook_t* cb, const uint32_t mode[2])
+// that needs more; very short codes in long subchunks get one slot of 4 bits per symbol (enc_shape says why).
+uint32_t slot_class(const zc_plan_t* p, const zc_codebook_t* cb, const uint32_t mode[2])
 {
-    return (mode[0] == ZC_MODE_HUFF && cb->wide[0]) || (mode[1] == ZC_MODE_HUFF && cb->wide[1]);
+    const bool h0 = mode[0] == ZC_MODE_HUFF, h1 = mode[1] == ZC_MODE_HUFF;
+    if ((h0 && cb->wide[0]) || (h1 && cb->wide[1])) return kSlotsWide;
+    // subchunks of 256 symbols and more (chunks from 16 KiB): half-size slots leave room for twice the warps
+    if ((h0 || h1) && p->syms_per_sub >= 256 && (!h0 || cb->brief[0]) && (!h1 || cb->brief[1])) return kSlotsHalf;
+    return kSlotsNarrow;
 }
 
 void fill_common(EncCommon& c, const zc_plan_t* p, const uint32_t mode[2], const EncShape& sh)
@@ -1178,7 +1193,7 @@ cudaError_t upload_tables(void* d_dst, const void* h_src, size_t bytes, cudaStre
 uint64_t max_batches_of(const zc_plan_t* p)
 {
     EncShape sh;
-    if (enc_shape(p, 2, true, &sh) != ZC_OK) return p->n_chunks;
+    if (enc_shape(p, 2, kSlotsWide, &sh) != ZC_OK) return p->n_chunks;
     uint64_t workers = sh.workers;
     for (uint32_t n_huff = 1; n_huff <= 2; ++n_huff) {
         const RowShape rs = row_shape(p, n_huff);
@@ -1205,7 +1220,7 @@ extern "C" {
 uint32_t zc_test_encoder_workers(const zc_plan_t* p, uint32_t n_coded, uint32_t wide_slots)
 {
     EncShape sh;
-    if (!p || n_coded > 2 || enc_shape(p, n_coded, wide_slots != 0, &sh) != ZC_OK) return 0;
+    if (!p || n_coded > 2 || wide_slots > kSlotsHalf || enc_shape(p, n_coded, wide_slots, &sh) != ZC_OK) return 0;
     return sh.workers;
 }
 
@@ -1230,7 +1245,7 @@ zc_status zc_compress_xor(const zc_plan_t* p, const zc_codebook_t* cb, const voi
         n_huff += mode[s] == ZC_MODE_HUFF;
     }
     EncShape sh;
-    const zc_status ss = enc_shape(p, n_huff, wants_wide_slots(cb, mode), &sh);
+    const zc_status ss = enc_shape(p, n_huff, slot_class(p, cb, mode), &sh);
     if (ss != ZC_OK) return ss;
     const RowShape rows = d_base ? RowShape{} : row_shape(p, n_huff);
     if (rows.workers) sh.workers = rows.workers;                 // chunks per batch
@@ -1312,9 +1327,9 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
     // the code tables are uploaded in one copy, one per distinct codebook (the K/V pages of a step share theirs)
     static thread_local std::vector<EncTables> h_tables;
     static thread_local std::vector<uint32_t> table_of;          // per tensor: its tables among the uploaded ones
-    static thread_local std::vector<uint8_t> table_wide;         // per uploaded table: 1 + wide slots wanted, per mode pair
+    static thread_local std::vector<uint8_t> table_slots;        // per uploaded table: the slot class its codes ask for
     static thread_local std::unordered_map<const zc_codebook_t*, uint32_t> seen;
-    h_tables.clear(); table_wide.clear(); seen.clear();
+    h_tables.clear(); table_slots.clear(); seen.clear();
     table_of.resize(n_tensors);
     for (uint32_t t = 0; t < n_tensors; ++t) {
         auto found = seen.find(codebooks[t]);
@@ -1323,7 +1338,7 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
             h_tables.emplace_back();
             fill_tables(h_tables.back(), codebooks[t]);
             const uint32_t m[2] = {codebooks[t]->mode[0], codebooks[t]->mode[1]};
-            table_wide.push_back(wants_wide_slots(codebooks[t], m) ? 1 : 0);
+            table_slots.push_back((uint8_t)slot_class(p0, codebooks[t], m));
         }
         table_of[t] = found->second;
     }
@@ -1334,28 +1349,28 @@ zc_status zc_compress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* plan
     static thread_local EncParamsT<(int)kEncBatchMax> P;
     uint64_t flag_base = 0;
     bool first_launch = true;
-    static thread_local std::vector<uint8_t> group;              // per tensor: mode0 | mode1 << 1 | wide << 2
+    static thread_local std::vector<uint8_t> group;              // per tensor: mode0 | mode1 << 1 | slot class << 2
     group.resize(n_tensors);
     for (uint32_t t = 0; t < n_tensors; ++t) {
         const bool any = plans[t]->n_syms != 0;                  // an empty tensor: both streams raw
         const uint32_t m[2] = {any ? codebooks[t]->mode[0] : (uint32_t)ZC_MODE_RAW, any ? codebooks[t]->mode[1] : (uint32_t)ZC_MODE_RAW};
-        const bool wide = (m[0] == ZC_MODE_HUFF || m[1] == ZC_MODE_HUFF) && table_wide[table_of[t]];
-        group[t] = (uint8_t)(m[0] | (m[1] << 1) | (wide ? 4u : 0u));
+        const uint32_t slots = (m[0] == ZC_MODE_HUFF || m[1] == ZC_MODE_HUFF) ? table_slots[table_of[t]] : kSlotsNarrow;
+        group[t] = (uint8_t)(m[0] | (m[1] << 1) | (slots << 2));
     }
     // the launch shapes of the combinations that occur, checked before anything is launched
-    bool combo_used[8] = {false, false, false, false, false, false, false, false};
+    bool combo_used[12] = {};
     for (uint32_t t = 0; t < n_tensors; ++t) combo_used[group[t]] = true;
-    for (uint32_t combo = 0; combo < 8; ++combo) {
+    for (uint32_t combo = 0; combo < 12; ++combo) {
         EncShape sh;
-        if (combo_used[combo] && enc_shape(p0, (combo & 1u) + ((combo >> 1) & 1u), (combo & 4u) != 0, &sh) != ZC_OK) return ZC_E_UNSUPPORTED;
+        if (combo_used[combo] && enc_shape(p0, (combo & 1u) + ((combo >> 1) & 1u), combo >> 2, &sh) != ZC_OK) return ZC_E_UNSUPPORTED;
     }
-    for (uint32_t combo = 0; combo < 8; ++combo) {
+    for (uint32_t combo = 0; combo < 12; ++combo) {
         if (!combo_used[combo]) continue;
         const uint32_t mode[2] = {combo & 1u, (combo >> 1) & 1u};
         const uint32_t n_huff = (mode[0] == ZC_MODE_HUFF) + (mode[1] == ZC_MODE_HUFF);
         auto in_combo = [&](uint32_t t) { return group[t] == combo; };
         EncShape sh;
-        const zc_status ss = enc_shape(p0, n_huff, (combo & 4u) != 0, &sh);
+        const zc_status ss = enc_shape(p0, n_huff, combo >> 2, &sh);
         if (ss != ZC_OK) return ss;
         bool any_base = false;
         if (d_base) for (uint32_t i = 0; i < n_tensors; ++i) any_base = any_base || d_base[i] != nullptr;

@@ -44,11 +44,13 @@ struct zc_codebook_s {
     // derived once when the codebook is built, so that a compress call only copies them:
     uint32_t enc[2][256];      // the encoder's table entry of every symbol: code << (32 - length) | length; 16: no code
     uint8_t wide[2];           // the stream's codes are long on average: the encoder uses 12-bit pack slots
+    uint8_t brief[2];          // the stream's codes are short on average: half-size pack slots do for long subchunks
 };
 
 namespace zc {
 // Fills the derived fields of a codebook (call after len[] and code[] are final).
-// wide: with the symbol probabilities the code lengths imply (2^-length) the expected length is above 6.5 bits.
+// wide: with the symbol probabilities the code lengths imply (2^-length) the expected length is above 6.5 bits;
+// brief: it is at most 3.25 bits.
 inline void finish_codebook(zc_codebook_s* cb)
 {
     for (int s = 0; s < 2; ++s) {
@@ -59,6 +61,7 @@ inline void finish_codebook(zc_codebook_s* cb)
             if (l) acc += (uint64_t)l << (12 - l);
         }
         cb->wide[s] = 2 * acc > (13ull << 12) ? 1 : 0;
+        cb->brief[s] = 4 * acc <= (13ull << 12) ? 1 : 0;
     }
 }
 

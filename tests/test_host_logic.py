@@ -49,13 +49,16 @@ def test_plan_geometry(fmt):
 
 
 def test_every_accepted_chunk_size_has_a_launch_shape():
-    """Whatever zc_plan accepts, the encoder (any number of coded streams, narrow and wide pack slots) and the
-    decoder (one or both streams coded) have a launch shape for; beyond the limit the plan itself is refused."""
+    """Whatever zc_plan accepts, the encoder (any number of coded streams, every class of pack slots) and the
+    decoder (one or both streams coded) have a launch shape for; beyond the limit the plan itself is refused.
+    Half-size slots never leave room for fewer worker warps than the ordinary ones."""
     for cb in range(1024, 65536 + 1, 1024):
         p = zc.plan(zc.FMT_BF16, 1 << 20, cb)
         for n_coded in (0, 1, 2):
-            for wide in (False, True):
-                assert zc.test_encoder_workers(p, n_coded, wide) >= 1, (cb, n_coded, wide)
+            for slots in (0, 1, 2):
+                assert zc.test_encoder_workers(p, n_coded, slots) >= 1, (cb, n_coded, slots)
+            assert zc.test_encoder_workers(p, n_coded, 2) >= zc.test_encoder_workers(p, n_coded, 0)
+            assert zc.test_encoder_workers(p, n_coded, 3) == 0
         for both in (False, True):
             assert zc.test_decoder_warps(p, both) >= 8, (cb, both)
 
