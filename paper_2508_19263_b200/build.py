@@ -1,7 +1,7 @@
 """Builds libzc.so (host logic + sm_100a kernels) in-tree with nvcc.
 
-Every source is compiled to an object file of its own (in parallel, and only when it or a header is newer than
-its object), then the objects are linked into the shared library.
+Every source is compiled to an object file of its own (the decoder's to one per element format; in parallel, and
+only when it or a header is newer than its object), then the objects are linked into the shared library.
 """
 from __future__ import annotations
 
@@ -15,6 +15,10 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libzc.so")
 OBJDIR = os.path.join(HERE, "build")
 SOURCES = ["zc_host.cpp", "zc_hist.cu", "zc_encode.cu", "zc_decode.cu"]
+# (source, extra flags, object name): the decoder's kernels are compiled one element format per object (ZC_DEC_PART),
+# so that the longest compile of the build runs four ways in parallel
+UNITS = [("zc_host.cpp", [], "zc_host.cpp.o"), ("zc_hist.cu", [], "zc_hist.cu.o"), ("zc_encode.cu", [], "zc_encode.cu.o")] + \
+        [("zc_decode.cu", [f"-DZC_DEC_PART={k}"], f"zc_decode.part{k}.o") for k in (1, 2, 3, 4)]
 HEADERS = ["zc_internal.h", "zc_bits.cuh", "zc_device.cuh", "zc_encode_rows.cuh"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
@@ -59,17 +63,18 @@ def build_library(force: bool = False, verbose: bool = False, lib: str = LIB, fl
     if verbose:
         common += ["-Xptxas", "-v"]
 
-    def compile_one(src: str) -> str:
+    def compile_one(unit) -> str:
+        src, unit_flags, name = unit
         path = os.path.join(CSRC, src)
-        obj = os.path.join(objdir, src + ".o")
+        obj = os.path.join(objdir, name)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(path), hdr_t):
             tmp = obj + f".tmp{os.getpid()}"
-            subprocess.check_call(common + ["-c", path, "-o", tmp])
+            subprocess.check_call(common + unit_flags + ["-c", path, "-o", tmp])
             os.replace(tmp, obj)
         return obj
 
-    with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
-        objs = list(pool.map(compile_one, SOURCES))
+    with ThreadPoolExecutor(max_workers=len(UNITS)) as pool:
+        objs = list(pool.map(compile_one, UNITS))
     with open(stamp, "w") as f:
         f.write(" ".join(flags))
     tmp = lib + f".tmp{os.getpid()}"

@@ -114,7 +114,7 @@ __device__ __forceinline__ CodeBook codebook_views(uint32_t* scratch)
 // symbols per lookup lets a lane assemble words of 4 symbols in registers without any bookkeeping.
 // `single` is a 4096 x u16 scratch table (length << 8 | symbol of the first code of every window).
 // Returns false to all threads if the lengths are not a complete prefix code (or the one-symbol code).
-__device__ bool build_lut(uint32_t my_len, uint32_t* lut, uint16_t* single, uint32_t* scratch, uint32_t* per_lookup)
+static __device__ bool build_lut(uint32_t my_len, uint32_t* lut, uint16_t* single, uint32_t* scratch, uint32_t* per_lookup)
 {
     const CodeBook b = codebook_views(scratch);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -391,7 +391,7 @@ __device__ __forceinline__ void decode_round2(uint32_t& posa, uint32_t& wa0, uin
 
 // A chunk without payload bits holds nothing but the stream's fill symbol, the symbol with the all-zero code:
 // the first symbol of the table entry for a window of zeros.
-__device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
+static __device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t wr_s, uint32_t fw, uint32_t n_quads)
 {
     const uint32_t e = lds32(lut_s);
     const uint32_t word = (pairs ? (e >> 8) & 0xFFu : e >> 24) * 0x01010101u;
@@ -402,7 +402,7 @@ __device__ __noinline__ void fill_quads(uint32_t lut_s, uint32_t pairs, uint32_t
 // tables: symbol in bits 15..8, length in bits 27..24; one-symbol tables: symbol in bits 31..24, length in bits
 // 3..0), reading the piece from global memory.  Small and slow on purpose: it serves pieces that were too long
 // to stage.  Returns the new position.
-__device__ __noinline__ uint32_t decode_quads_global(uint32_t pos, const uint32_t* __restrict__ pay, uint32_t lut_s, uint32_t pairs,
+static __device__ __noinline__ uint32_t decode_quads_global(uint32_t pos, const uint32_t* __restrict__ pay, uint32_t lut_s, uint32_t pairs,
                                                      uint32_t wr_s, uint32_t fw, uint32_t n_quads, uint32_t lim)
 {
     for (uint32_t i = 0; i < 4 * n_quads; ++i) {
@@ -975,7 +975,110 @@ decode_batch_kernel(const __grid_constant__ DecBatchParams B)
     }
 }
 
+
+// ---- launchers, one set per element format -------------------------------------------------------------------
+// The kernels of one format are instantiated where that format's launchers are defined.  This file can be compiled
+// as a whole (ZC_DEC_PART undefined or 0) or in four parts (1: the C ABI and BF16, 2: FP8, 3: scale bytes, 4: FP4), one
+// object each, so that a build compiles the formats side by side.
+#ifndef ZC_DEC_PART
+#define ZC_DEC_PART 0
+#endif
+
+// the buffers of a launch, for the development build's checks
+struct DecRanges { const void* in; size_t in_bytes; const void* out; size_t out_bytes; const void* ws; size_t ws_bytes; };
+
+template <int F>
+cudaError_t dec_launch_single_t(uint32_t ppl, uint32_t grid, uint32_t threads, size_t smem, cudaStream_t st, const DecParams& P,
+                                const DecRanges& R)
+{
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kern) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        dbg_set_ranges(st, R.in, R.in_bytes, R.out, R.out_bytes, R.ws, R.ws_bytes);
+#else
+        (void)R;
+#endif
+        kern<<<grid, threads, smem, st>>>(P);
+        e = cudaGetLastError();
+    };
+    if (ppl == 4) launch(decode_kernel<F, 4>);
+    else if (ppl == 2) launch(decode_kernel<F, 2>);
+    else launch(decode_kernel<F, 1>);
+    return e;
+}
+
+template <int F>
+cudaError_t dec_launch_batch_t(uint32_t ppl, bool any_base, uint32_t grid, uint32_t threads, size_t smem, cudaStream_t st,
+                               const DecBatchParams& B, const DecRanges& R)
+{
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kern) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return;
+#if ZC_DEBUG_CHECKS
+        dbg_set_ranges(st, R.in, R.in_bytes, R.out, R.out_bytes, R.ws, R.ws_bytes);
+#else
+        (void)R;
+#endif
+        kern<<<grid, threads, smem, st>>>(B);
+        e = cudaGetLastError();
+    };
+    if (any_base) {
+        if (ppl == 4) launch(decode_batch_kernel<F, 4, true>);
+        else if (ppl == 2) launch(decode_batch_kernel<F, 2, true>);
+        else launch(decode_batch_kernel<F, 1, true>);
+    } else {
+        if (ppl == 4) launch(decode_batch_kernel<F, 4, false>);
+        else if (ppl == 2) launch(decode_batch_kernel<F, 2, false>);
+        else launch(decode_batch_kernel<F, 1, false>);
+    }
+    return e;
+}
+
+#define ZC_DEC_DECLARE(NAME)                                                                                              \
+    cudaError_t dec_launch_single_##NAME(uint32_t ppl, uint32_t grid, uint32_t threads, size_t smem, cudaStream_t st,     \
+                                         const DecParams& P, const DecRanges& R);                                        \
+    cudaError_t dec_launch_batch_##NAME(uint32_t ppl, bool any_base, uint32_t grid, uint32_t threads, size_t smem,        \
+                                        cudaStream_t st, const DecBatchParams& B, const DecRanges& R);                   \
+    void dec_debug_counts_##NAME(uint32_t out[2]);
+ZC_DEC_DECLARE(bf16)
+ZC_DEC_DECLARE(fp8)
+ZC_DEC_DECLARE(scale)
+ZC_DEC_DECLARE(fp4)
+#undef ZC_DEC_DECLARE
+
+#if ZC_DEBUG_CHECKS
+#define ZC_DEC_COUNTS(out) dbg_read_counts(out)
+#else
+#define ZC_DEC_COUNTS(out) (void)(out)
+#endif
+#define ZC_DEC_DEFINE(NAME, F)                                                                                            \
+    cudaError_t dec_launch_single_##NAME(uint32_t ppl, uint32_t grid, uint32_t threads, size_t smem, cudaStream_t st,     \
+                                         const DecParams& P, const DecRanges& R)                                         \
+    { return dec_launch_single_t<F>(ppl, grid, threads, smem, st, P, R); }                                                \
+    cudaError_t dec_launch_batch_##NAME(uint32_t ppl, bool any_base, uint32_t grid, uint32_t threads, size_t smem,        \
+                                        cudaStream_t st, const DecBatchParams& B, const DecRanges& R)                    \
+    { return dec_launch_batch_t<F>(ppl, any_base, grid, threads, smem, st, B, R); }                                       \
+    void dec_debug_counts_##NAME(uint32_t out[2]) { ZC_DEC_COUNTS(out); }
+#if ZC_DEC_PART == 0 || ZC_DEC_PART == 1
+ZC_DEC_DEFINE(bf16, ZC_FMT_BF16)
+#endif
+#if ZC_DEC_PART == 0 || ZC_DEC_PART == 2
+ZC_DEC_DEFINE(fp8, ZC_FMT_FP8_E4M3)
+#endif
+#if ZC_DEC_PART == 0 || ZC_DEC_PART == 3
+ZC_DEC_DEFINE(scale, ZC_FMT_SCALE_U8)
+#endif
+#if ZC_DEC_PART == 0 || ZC_DEC_PART == 4
+ZC_DEC_DEFINE(fp4, ZC_FMT_FP4_E2M1)
+#endif
+#undef ZC_DEC_DEFINE
+
 }  // namespace zc
+
+#if ZC_DEC_PART <= 1
 
 using namespace zc;
 
@@ -1034,11 +1137,10 @@ unsigned long long new_call_id()
 namespace zc {
 void debug_counts_decode(uint32_t out[2])
 {
-#if ZC_DEBUG_CHECKS
-    dbg_read_counts(out);
-#else
-    (void)out;
-#endif
+    dec_debug_counts_bf16(out);
+    dec_debug_counts_fp8(out);
+    dec_debug_counts_scale(out);
+    dec_debug_counts_fp4(out);
 }
 }  // namespace zc
 extern "C" {
@@ -1098,29 +1200,16 @@ zc_status zc_decompress_chunks(const zc_plan_t* p, const void* d_comp, size_t co
     // at least one block even for an empty range: the header is still checked
     const uint32_t want = std::max<uint32_t>((n_chunks + warps - 1) / warps, 1);
     const uint32_t grid = std::min<uint32_t>(want, (uint32_t)sm_count());
-    cudaError_t e = cudaSuccess;
-    auto launch = [&](auto kern) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return;
-#if ZC_DEBUG_CHECKS
-        dbg_set_ranges(st, d_comp, comp_bytes, d_out,
-                       (size_t)std::min<uint64_t>((uint64_t)n_chunks * p->chunk_bytes, p->input_bytes - (uint64_t)first_chunk * p->chunk_bytes),
-                       d_workspace, sizeof(Control));
-#endif
-        kern<<<grid, warps * 32, smem, st>>>(P);
-        e = cudaGetLastError();
-    };
-#define ZC_DEC_CASE(F)                                                     \
-    if (ppl == 4) launch(decode_kernel<F, 4>);                             \
-    else if (ppl == 2) launch(decode_kernel<F, 2>);                        \
-    else launch(decode_kernel<F, 1>);
+    const DecRanges R{d_comp, comp_bytes, d_out,
+                      (size_t)std::min<uint64_t>((uint64_t)n_chunks * p->chunk_bytes, p->input_bytes - (uint64_t)first_chunk * p->chunk_bytes),
+                      d_workspace, sizeof(Control)};
+    cudaError_t e;
     switch (p->format) {
-    case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
-    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
-    case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
-    default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
+    case ZC_FMT_BF16: e = dec_launch_single_bf16(ppl, grid, warps * 32, smem, st, P, R); break;
+    case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: e = dec_launch_single_fp8(ppl, grid, warps * 32, smem, st, P, R); break;
+    case ZC_FMT_SCALE_U8: e = dec_launch_single_scale(ppl, grid, warps * 32, smem, st, P, R); break;
+    default: e = dec_launch_single_fp4(ppl, grid, warps * 32, smem, st, P, R); break;
     }
-#undef ZC_DEC_CASE
     return e == cudaSuccess ? ZC_OK : ZC_E_CUDA;
 }
 
@@ -1188,41 +1277,25 @@ zc_status zc_decompress_batch_xor(uint32_t n_tensors, const zc_plan_t* const* pl
         B.n_ranges = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(B.n_ranges, total));
         // the ranges are handed out through the ticket word of the control block
         if (cudaMemsetAsync(&B.ctl->ticket, 0, sizeof(uint32_t), st) != cudaSuccess) return ZC_E_CUDA;
-        cudaError_t e = cudaSuccess;
-        auto launch = [&](auto kern) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
-            if (e != cudaSuccess) return;
-#if ZC_DEBUG_CHECKS
-            DbgHull rd, wr;
-            for (uint32_t i = 0; i < n; ++i) {
-                rd.add(B.item[i].comp, B.item[i].comp_bytes);
-                rd.add(B.item[i].base, B.item[i].input_bytes);
-                wr.add(B.item[i].out, B.item[i].input_bytes);
-            }
-            dbg_set_ranges(st, rd.ptr(), rd.bytes(), wr.ptr(), wr.bytes(), d_workspace, sizeof(Control));
-#endif
-            kern<<<grid, shape.warps * 32, shape.smem, st>>>(B);
-            e = cudaGetLastError();
-        };
         bool any_base = false;
         for (uint32_t i = 0; i < n; ++i) any_base = any_base || B.item[i].base != nullptr;
-#define ZC_DEC_CASE(F)                                                                               \
-    if (any_base) {                                                                                  \
-        if (shape.ppl == 4) launch(decode_batch_kernel<F, 4, true>);                                 \
-        else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2, true>);                            \
-        else launch(decode_batch_kernel<F, 1, true>);                                                \
-    } else {                                                                                         \
-        if (shape.ppl == 4) launch(decode_batch_kernel<F, 4, false>);                                \
-        else if (shape.ppl == 2) launch(decode_batch_kernel<F, 2, false>);                           \
-        else launch(decode_batch_kernel<F, 1, false>);                                               \
-    }
-        switch (p0->format) {
-        case ZC_FMT_BF16: ZC_DEC_CASE(ZC_FMT_BF16) break;
-        case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: ZC_DEC_CASE(ZC_FMT_FP8_E4M3) break;
-        case ZC_FMT_SCALE_U8: ZC_DEC_CASE(ZC_FMT_SCALE_U8) break;
-    default: ZC_DEC_CASE(ZC_FMT_FP4_E2M1) break;
+        DecRanges R{nullptr, 0, nullptr, 0, d_workspace, sizeof(Control)};
+#if ZC_DEBUG_CHECKS
+        DbgHull rd, wr;
+        for (uint32_t i = 0; i < n; ++i) {
+            rd.add(B.item[i].comp, B.item[i].comp_bytes);
+            rd.add(B.item[i].base, B.item[i].input_bytes);
+            wr.add(B.item[i].out, B.item[i].input_bytes);
         }
-#undef ZC_DEC_CASE
+        R.in = rd.ptr(); R.in_bytes = rd.bytes(); R.out = wr.ptr(); R.out_bytes = wr.bytes();
+#endif
+        cudaError_t e;
+        switch (p0->format) {
+        case ZC_FMT_BF16: e = dec_launch_batch_bf16(shape.ppl, any_base, grid, shape.warps * 32, shape.smem, st, B, R); break;
+        case ZC_FMT_FP8_E4M3: case ZC_FMT_FP8_E5M2: e = dec_launch_batch_fp8(shape.ppl, any_base, grid, shape.warps * 32, shape.smem, st, B, R); break;
+        case ZC_FMT_SCALE_U8: e = dec_launch_batch_scale(shape.ppl, any_base, grid, shape.warps * 32, shape.smem, st, B, R); break;
+        default: e = dec_launch_batch_fp4(shape.ppl, any_base, grid, shape.warps * 32, shape.smem, st, B, R); break;
+        }
         if (e != cudaSuccess) return ZC_E_CUDA;
         base += n;
     }
@@ -1242,3 +1315,5 @@ zc_status zc_batch_status(const void* d_workspace, uint32_t* h_failed_tensor, vo
 }
 
 }  // extern "C"
+
+#endif  // ZC_DEC_PART <= 1
